@@ -1,0 +1,182 @@
+/*
+ * fff.h -- C ABI of the B200 (sm_100a) library for hard-routed inference of
+ * Fast Feedforward (FFF) networks.
+ *
+ * The library computes FORWARD_I of Algorithm 1 ("FFF forward pass") for a
+ * batch of B independent tokens: every token descends a depth-d balanced
+ * binary tree of single-neuron nodes, taking the right child when the node
+ * output c = sigmoid(<w, x> + b) is >= 1/2 (i.e. when the logit is >= 0) and
+ * the left child otherwise, and is then evaluated by the one leaf network
+ * N_{d,j} it reaches:  y = W2_j act(W1_j x + b1_j) + b2_j.
+ *
+ * Conventions shared by all calls
+ *  - Every pointer is a DEVICE pointer unless its name ends in _host.  Device
+ *    pointers must be 16-byte aligned and belong to the CUDA device that was
+ *    current when the handle was created.  The caller owns every buffer it
+ *    passes in.
+ *  - All tensors are dense and row-major.  One element type per handle: all of
+ *    x, y and the weights are float32 (FFF_DTYPE_F32) or bfloat16
+ *    (FFF_DTYPE_BF16, products accumulated in float32).  Index arrays are
+ *    int32.
+ *  - Node N_{m,n} (level m, position n) is row 2^m - 1 + n of the node arrays;
+ *    its children are N_{m+1,2n} (left) and N_{m+1,2n+1} (right) (Section
+ *    "Algorithm", Definition).  leaf_idx is n of the leaf N_{d,n}: the d
+ *    decisions read from the root as a binary number, 1 = right.
+ *  - `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *    Calls that take a stream only enqueue work on it and return without
+ *    waiting, unless stated otherwise.
+ *  - Every call returns an fff_status_t; nothing throws, aborts or traps.
+ *    Argument errors are detected on the host before anything is launched.
+ *  - A handle serves one forward at a time (its workspace is shared by its
+ *    calls); different handles are independent.
+ *  - Results are bit-reproducible from run to run for fixed inputs.
+ */
+#ifndef FFF_H
+#define FFF_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fff_handle_s *fff_handle_t;
+
+typedef enum {
+    FFF_OK = 0,
+    FFF_ERR_INVALID_ARG = 1,     /* NULL / misaligned pointer, non-positive size, unknown enum, B < 0 */
+    FFF_ERR_UNSUPPORTED = 2,     /* valid request this build cannot serve (e.g. depth > FFF_MAX_DEPTH) */
+    FFF_ERR_ALLOC = 3,           /* device or host allocation failed */
+    FFF_ERR_CUDA = 4,            /* a CUDA runtime call failed */
+    FFF_ERR_DEVICE_TIMEOUT = 5,  /* a bounded device-side wait ran out (read by fff_get_last_status) */
+    FFF_ERR_BAD_HANDLE = 6       /* NULL, destroyed or corrupted handle */
+} fff_status_t;
+
+typedef enum {
+    FFF_ACT_RELU = 0,            /* max(v, 0) */
+    FFF_ACT_GELU = 1             /* v * Phi(v), exact erf form */
+} fff_activation_t;
+
+typedef enum {
+    FFF_DTYPE_F32 = 0,
+    FFF_DTYPE_BF16 = 1           /* bf16 storage, float32 accumulation, y rounded to nearest even */
+} fff_dtype_t;
+
+#define FFF_MAX_DEPTH 20
+
+/* Kernel families a handle may be pinned to with fff_set_path (testing / tuning). */
+typedef enum {
+    FFF_PATH_AUTO = 0,           /* library picks per stage from shapes and B */
+    FFF_PATH_WARP = 1,           /* CUDA-core warp kernels for descent and leaf evaluation */
+    FFF_PATH_TENSOR = 2          /* tensor-core kernels wherever the shapes allow them */
+} fff_path_t;
+
+/*
+ * Create an FFF layer (Section "Algorithm", Definition: a pair <N, L> of
+ * 2^d - 1 node networks of node size 1 and 2^d leaf networks of leaf size l).
+ *
+ *   D, O          dim_I and dim_O, >= 1
+ *   depth         d, 0 <= d <= FFF_MAX_DEPTH; d = 0 is a single leaf, no nodes
+ *   leaf_width    l >= 1
+ *   node_w        [2^d-1, D]   may be NULL iff depth == 0
+ *   node_b        [2^d-1]      NULL = all zero
+ *   leaf_w1       [2^d, l, D]
+ *   leaf_b1       [2^d, l]     NULL = all zero
+ *   leaf_w2       [2^d, O, l]
+ *   leaf_b2       [2^d, O]     NULL = all zero
+ *
+ * The weights are copied (and re-laid-out for the kernels) into memory owned
+ * by the handle before the call returns; the caller's buffers may be freed
+ * afterwards.  The call synchronises the device.  On failure *out is NULL.
+ */
+fff_status_t fff_create(fff_handle_t *out, int D, int O, int depth, int leaf_width,
+                        fff_activation_t act, fff_dtype_t dtype,
+                        const void *node_w, const void *node_b,
+                        const void *leaf_w1, const void *leaf_b1,
+                        const void *leaf_w2, const void *leaf_b2);
+
+/*
+ * FORWARD_I of Algorithm 1 for B tokens, enqueued on `cuda_stream`.
+ *
+ *   x         [B, D]  in
+ *   y         [B, O]  out
+ *   leaf_idx  [B]     out, may be NULL: the region / leaf each token was routed to
+ *
+ * B == 0 is FFF_OK and enqueues nothing.  If B exceeds what fff_reserve was
+ * given, the workspace is grown first (this allocates and synchronises).
+ */
+fff_status_t fff_forward_infer(fff_handle_t h, const void *x, void *y, int32_t *leaf_idx,
+                               int64_t B, void *cuda_stream);
+
+/*
+ * The same computation for buffers in HOST memory (pinned or pageable):
+ * copies x to the device, runs fff_forward_infer, copies y (and leaf_idx when
+ * not NULL) back, and returns after `cuda_stream` has completed.
+ */
+fff_status_t fff_forward_infer_host(fff_handle_t h, const void *x_host, void *y_host,
+                                    int32_t *leaf_idx_host, int64_t B, void *cuda_stream);
+
+/* Free everything the handle owns.  Synchronises the device first; no work of
+ * this handle may be enqueued afterwards. */
+fff_status_t fff_destroy(fff_handle_t h);
+
+/* Size the workspace for batches of up to max_B tokens so that later forwards
+ * allocate nothing.  Allocates and synchronises. */
+fff_status_t fff_reserve(fff_handle_t h, int64_t max_B);
+
+/* Pin the handle to one kernel family (FFF_PATH_*).  FFF_ERR_UNSUPPORTED if
+ * the shapes of this handle cannot run on it. */
+fff_status_t fff_set_path(fff_handle_t h, fff_path_t path);
+
+/*
+ * Stage entry points.  fff_forward_infer computes what these three compute
+ * when called in this order.
+ */
+
+/* Tree descent (Algorithm 1, FORWARD_I, non-leaf branch; paragraph on
+ * inference complexity: d steps, one node network each).
+ *   x [B, D] in;  leaf_idx [B] out. */
+fff_status_t fff_tree_descent(fff_handle_t h, const void *x, int32_t *leaf_idx,
+                              int64_t B, void *cuda_stream);
+
+/* Leaf bucketing: the stable counting sort of token ids by leaf.  Not a step
+ * of the paper (its implementation gathers weights per token); it groups the
+ * tokens so that each leaf's weights are fetched once per batch.
+ *   leaf_idx [B] in, values in [0, 2^depth); ids outside that range are
+ *            ignored and leave their perm entries unwritten
+ *   offsets  [2^depth + 1] out: offsets[j] = #tokens with leaf < j
+ *   perm     [B] out: perm[offsets[j] + r] = r-th smallest token id routed to leaf j
+ * Uses the handle's workspace. */
+fff_status_t fff_leaf_bucketing(fff_handle_t h, const int32_t *leaf_idx, int32_t *offsets,
+                                int32_t *perm, int64_t B, void *cuda_stream);
+
+/* Grouped leaf evaluation with un-permuting write-back (Algorithm 1,
+ * FORWARD_I, leaf branch: return N_{d,j}(x)):
+ * for every i, with t = perm[i] and j = leaf_idx[t]:
+ *   y[t, :] = W2_j act(W1_j x[t, :] + b1_j) + b2_j.
+ *   x [B, D], leaf_idx [B], offsets [2^depth + 1], perm [B] in;  y [B, O] out. */
+fff_status_t fff_grouped_leaf_ff(fff_handle_t h, const void *x, const int32_t *leaf_idx,
+                                 const int32_t *offsets, const int32_t *perm, void *y,
+                                 int64_t B, void *cuda_stream);
+
+/* Copy the bucketing of the handle's most recent forward into caller buffers
+ * (device): perm [B], offsets [2^depth + 1].  Enqueued on `cuda_stream`. */
+fff_status_t fff_debug_get_bucketing(fff_handle_t h, int32_t *perm, int32_t *offsets,
+                                     void *cuda_stream);
+
+/* Synchronise the device and report the device-side status word of the handle:
+ * FFF_OK, or FFF_ERR_DEVICE_TIMEOUT if a bounded wait in a kernel expired since
+ * the last call (the word is cleared). */
+fff_status_t fff_get_last_status(fff_handle_t h);
+
+/* Number of kernels the most recent forward / stage call of this handle enqueued
+ * (-1 for a bad handle). */
+int fff_last_launch_count(fff_handle_t h);
+
+/* Static, never NULL. */
+const char *fff_status_string(fff_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FFF_H */

@@ -1,0 +1,75 @@
+// Shared device helpers for the FFF inference kernels (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace fff {
+
+constexpr unsigned kFullMask = 0xffffffffu;
+
+enum : int { kActRelu = 0, kActGelu = 1 };
+
+// Values written to the per-handle device status word by kernels.
+enum : int { kDevOk = 0, kDevTimeout = 1 };
+
+template <typename T> struct Elem;
+
+template <> struct Elem<float> {
+    static constexpr int kVec = 4;   // elements per 16-byte load
+    __device__ __forceinline__ static float to_float(float v) { return v; }
+    __device__ __forceinline__ static float from_float(float v) { return v; }
+    __device__ __forceinline__ static void load_vec(const float* p, float (&out)[4]) {
+        const float4 v = __ldg(reinterpret_cast<const float4*>(p));
+        out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
+    }
+};
+
+template <> struct Elem<__nv_bfloat16> {
+    static constexpr int kVec = 8;
+    __device__ __forceinline__ static float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+    __device__ __forceinline__ static __nv_bfloat16 from_float(float v) { return __float2bfloat16_rn(v); }
+    __device__ __forceinline__ static void load_vec(const __nv_bfloat16* p, float (&out)[8]) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(p));
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            out[2 * i] = __uint_as_float(w[i] << 16);              // low half = even element
+            out[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);  // high half = odd element
+        }
+    }
+};
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFullMask, v, o);
+    return v;
+}
+
+__device__ __forceinline__ float activate(int act, float v) {
+    if (act == kActRelu) return fmaxf(v, 0.0f);
+    return 0.5f * v * (1.0f + erff(v * 0.70710678118654752440f));
+}
+
+// <a, b> over n elements, evaluated by one warp; every lane returns the sum.
+// `vec` says both rows start on 16-byte boundaries and n is a multiple of kVec.
+template <typename T>
+__device__ __forceinline__ float warp_dot(const T* __restrict__ a, const T* __restrict__ b, int n, bool vec, int lane) {
+    constexpr int V = Elem<T>::kVec;
+    float acc = 0.0f;
+    if (vec) {
+        for (int k = lane * V; k < n; k += 32 * V) {
+            float fa[V], fb[V];
+            Elem<T>::load_vec(a + k, fa);
+            Elem<T>::load_vec(b + k, fb);
+#pragma unroll
+            for (int i = 0; i < V; ++i) acc = fmaf(fa[i], fb[i], acc);
+        }
+    } else {
+        for (int k = lane; k < n; k += 32) acc = fmaf(Elem<T>::to_float(a[k]), Elem<T>::to_float(b[k]), acc);
+    }
+    return warp_sum(acc);
+}
+
+}  // namespace fff
