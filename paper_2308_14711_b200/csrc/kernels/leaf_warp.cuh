@@ -1,0 +1,94 @@
+// Grouped leaf evaluation on CUDA cores with un-permuting write-back.
+//
+// Algorithm 1, FORWARD_I, leaf branch: the token returns N_{d,j}(x), the
+// <D, l, O> feedforward network of its leaf:  y = W2_j act(W1_j x + b1_j) + b2_j.
+//
+// One warp evaluates one token.  Warps walk the tokens in bucket order
+// (perm), so the warps of a CTA mostly work on the same leaf and share its
+// weights through L1/L2.  The row of y is written straight to the token's
+// original position, which is the un-permute step.
+//
+// General path: any D, l, O, both element types, float32 accumulation.  It is
+// the path for float32 layers, for very thin leaves and for buckets of a few
+// tokens, where the work is a gather of weights rather than a contraction.
+#pragma once
+
+#include "common.cuh"
+
+namespace fff {
+
+constexpr int kLeafWarps = 8;
+constexpr int kLeafHiddenUnroll = 4;
+
+// Dynamic shared memory: kLeafWarps * l floats (hidden activations per warp).
+template <typename T>
+__global__ void __launch_bounds__(kLeafWarps * 32)
+k_leaf_warp(const T* __restrict__ x, const int32_t* __restrict__ leaf_idx, const int32_t* __restrict__ perm,
+            const T* __restrict__ w1, const T* __restrict__ b1, const T* __restrict__ w2, const T* __restrict__ b2,
+            T* __restrict__ y, int D, int O, int l, int act, int64_t B, bool vec)
+{
+    extern __shared__ float s_h[];
+    constexpr int V = Elem<T>::kVec;
+    constexpr int U = kLeafHiddenUnroll;
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    float* h = s_h + (size_t)wib * l;
+    const int64_t warp0 = (int64_t)blockIdx.x * kLeafWarps + wib;
+    const int64_t nwarps = (int64_t)gridDim.x * kLeafWarps;
+
+    for (int64_t i = warp0; i < B; i += nwarps) {
+        const int64_t t = perm ? perm[i] : i;
+        const int64_t j = leaf_idx[t];
+        const T* xt = x + t * D;
+        const T* w1j = w1 + j * (int64_t)l * D;
+        const T* b1j = b1 + j * (int64_t)l;
+
+        // hidden layer: U neurons at a time share the loads of x
+        for (int i0 = 0; i0 < l; i0 += U) {
+            float acc[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) acc[u] = 0.0f;
+            if (vec) {
+                for (int k = lane * V; k < D; k += 32 * V) {
+                    float fx[V];
+                    Elem<T>::load_vec(xt + k, fx);
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        if (i0 + u < l) {
+                            float fw[V];
+                            Elem<T>::load_vec(w1j + (int64_t)(i0 + u) * D + k, fw);
+#pragma unroll
+                            for (int e = 0; e < V; ++e) acc[u] = fmaf(fw[e], fx[e], acc[u]);
+                        }
+                    }
+                }
+            } else {
+                for (int k = lane; k < D; k += 32) {
+                    const float fx = Elem<T>::to_float(xt[k]);
+#pragma unroll
+                    for (int u = 0; u < U; ++u)
+                        if (i0 + u < l) acc[u] = fmaf(Elem<T>::to_float(w1j[(int64_t)(i0 + u) * D + k]), fx, acc[u]);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const float s = warp_sum(acc[u]);
+                if (lane == 0 && i0 + u < l) h[i0 + u] = activate(act, s + Elem<T>::to_float(b1j[i0 + u]));
+            }
+        }
+        __syncwarp();
+
+        // output layer: one output neuron per lane
+        const T* w2j = w2 + j * (int64_t)O * l;
+        const T* b2j = b2 + j * (int64_t)O;
+        T* yt = y + t * O;
+        for (int o = lane; o < O; o += 32) {
+            const T* row = w2j + (int64_t)o * l;
+            float acc = Elem<T>::to_float(b2j[o]);
+            for (int q = 0; q < l; ++q) acc = fmaf(Elem<T>::to_float(row[q]), h[q], acc);
+            yt[o] = Elem<T>::from_float(acc);
+        }
+        __syncwarp();
+    }
+}
+
+}  // namespace fff
