@@ -1,0 +1,382 @@
+// C ABI of the FFF inference library: handle management, argument checks,
+// stage planning and kernel launches.  Declarations and the contract of every
+// entry point are in include/fff.h.
+#include "../../include/fff.h"
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdint>
+#include <cstdio>
+#include <cstdlib>
+#include <mutex>
+#include <new>
+#include <set>
+
+#include "kernels/bucket.cuh"
+#include "kernels/common.cuh"
+#include "kernels/descent_warp.cuh"
+#include "kernels/leaf_warp.cuh"
+
+namespace {
+
+constexpr uint64_t kMagic = 0x4646465f42323030ull;   // "FFF_B200"
+
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) switched = (cudaSetDevice(dev) == cudaSuccess);
+    }
+    ~DeviceGuard() { if (switched) cudaSetDevice(prev); }
+};
+
+}  // namespace
+
+struct fff_handle_s {
+    uint64_t magic = kMagic;
+    int device = 0;
+    int sm_count = 148;
+    int D = 0, O = 0, depth = 0, l = 0;
+    int act = 0, dtype = 0;
+    size_t esize = 4;
+    int64_t n_nodes = 0, n_leaves = 1;
+    bool vec_ok = false;          // rows of x / W start on 16-byte boundaries and D % kVec == 0
+
+    // library-owned copies of the parameters, caller layout
+    void *node_w = nullptr, *node_b = nullptr, *w1 = nullptr, *b1 = nullptr, *w2 = nullptr, *b2 = nullptr;
+
+    // workspace
+    int64_t cap_B = 0;
+    int32_t *ws_leaf = nullptr, *ws_perm = nullptr, *ws_offsets = nullptr;
+    int *ws_hist[2] = {nullptr, nullptr};
+    int hist_cur = 0;
+    int *d_status = nullptr;
+
+    // staging for the host-buffer entry point
+    int64_t cap_host_B = 0;
+    void *st_x = nullptr, *st_y = nullptr;
+    int32_t *st_leaf = nullptr;
+
+    int path = FFF_PATH_AUTO;
+    int launches = 0;
+    int64_t last_B = -1;
+};
+
+namespace {
+
+std::mutex g_mu;
+std::set<fff_handle_s*> g_live;
+
+bool live(fff_handle_t h) {
+    if (!h) return false;
+    std::lock_guard<std::mutex> lk(g_mu);
+    return g_live.count(h) != 0 && h->magic == kMagic;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+fff_status_t dmalloc(void** p, size_t bytes) {
+    *p = nullptr;
+    if (bytes == 0) bytes = 16;
+    return cudaMalloc(p, bytes) == cudaSuccess ? FFF_OK : (cudaGetLastError(), FFF_ERR_ALLOC);
+}
+
+void dfree(void* p) { if (p) cudaFree(p); }
+
+fff_status_t clone(void** dst, const void* src, size_t bytes) {
+    fff_status_t s = dmalloc(dst, bytes);
+    if (s != FFF_OK) return s;
+    cudaError_t e = src ? cudaMemcpy(*dst, src, bytes, cudaMemcpyDeviceToDevice) : cudaMemset(*dst, 0, bytes ? bytes : 16);
+    return e == cudaSuccess ? FFF_OK : (cudaGetLastError(), FFF_ERR_CUDA);
+}
+
+void release(fff_handle_s* h) {
+    dfree(h->node_w); dfree(h->node_b); dfree(h->w1); dfree(h->b1); dfree(h->w2); dfree(h->b2);
+    dfree(h->ws_leaf); dfree(h->ws_perm); dfree(h->ws_offsets); dfree(h->ws_hist[0]); dfree(h->ws_hist[1]);
+    dfree(h->d_status); dfree(h->st_x); dfree(h->st_y); dfree(h->st_leaf);
+    h->magic = 0;
+    delete h;
+}
+
+fff_status_t grow_workspace(fff_handle_s* h, int64_t B) {
+    if (B <= h->cap_B) return FFF_OK;
+    if (cudaDeviceSynchronize() != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
+    dfree(h->ws_leaf); dfree(h->ws_perm);
+    h->ws_leaf = h->ws_perm = nullptr;
+    h->cap_B = 0;
+    fff_status_t s;
+    if ((s = dmalloc((void**)&h->ws_leaf, sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
+    if ((s = dmalloc((void**)&h->ws_perm, sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
+    h->cap_B = B;
+    return FFF_OK;
+}
+
+fff_status_t launch_status() {
+    return cudaGetLastError() == cudaSuccess ? FFF_OK : FFF_ERR_CUDA;
+}
+
+// ---- stage launchers -------------------------------------------------------
+
+template <typename T>
+fff_status_t run_descent(fff_handle_s* h, const void* x, int32_t* leaf_idx, int* hist, int64_t B, cudaStream_t st) {
+    const int64_t blocks = std::min<int64_t>((B + fff::kDescentWarps - 1) / fff::kDescentWarps, (int64_t)h->sm_count * 8);
+    fff::k_descent_warp<T><<<(unsigned)blocks, fff::kDescentWarps * 32, 0, st>>>(
+        (const T*)x, (const T*)h->node_w, (const T*)h->node_b, h->D, 0, h->depth, nullptr, leaf_idx, hist, B,
+        h->vec_ok && aligned16(x));
+    ++h->launches;
+    return launch_status();
+}
+
+fff_status_t run_histogram(fff_handle_s* h, const int32_t* keys, int64_t B, cudaStream_t st) {
+    const int64_t blocks = std::min<int64_t>((B + 255) / 256, (int64_t)h->sm_count * 4);
+    fff::k_histogram<<<(unsigned)blocks, 256, 0, st>>>(keys, h->ws_hist[h->hist_cur], B, (int)h->n_leaves);
+    ++h->launches;
+    return launch_status();
+}
+
+// Consumes the current histogram buffer and flips to the other (already zero) one.
+fff_status_t run_bucket(fff_handle_s* h, const int32_t* keys, int32_t* offsets, int32_t* perm, int64_t B, cudaStream_t st) {
+    const int nbins = (int)h->n_leaves;
+    int ctas = std::min(nbins, 32);
+    int per = (nbins + ctas - 1) / ctas;
+    if (per > fff::kBucketMaxBinsPerCta) {
+        per = fff::kBucketMaxBinsPerCta;
+        ctas = (nbins + per - 1) / per;
+    }
+    const size_t smem = sizeof(int) * (size_t)fff::kBucketWarps * per;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        cudaFuncSetAttribute(fff::k_bucket, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)(sizeof(int) * fff::kBucketWarps * fff::kBucketMaxBinsPerCta));
+    });
+    fff::k_bucket<<<ctas, fff::kBucketThreads, smem, st>>>(keys, h->ws_hist[h->hist_cur], h->ws_hist[h->hist_cur ^ 1],
+                                                         offsets, perm, (int)B, nbins, per);
+    h->hist_cur ^= 1;
+    ++h->launches;
+    return launch_status();
+}
+
+template <typename T>
+fff_status_t run_leaf(fff_handle_s* h, const void* x, const int32_t* leaf_idx, const int32_t* perm, void* y,
+                      int64_t B, cudaStream_t st) {
+    const int64_t blocks = std::min<int64_t>((B + fff::kLeafWarps - 1) / fff::kLeafWarps, (int64_t)h->sm_count * 8);
+    const size_t smem = sizeof(float) * (size_t)fff::kLeafWarps * h->l;
+    fff::k_leaf_warp<T><<<(unsigned)blocks, fff::kLeafWarps * 32, smem, st>>>(
+        (const T*)x, leaf_idx, perm, (const T*)h->w1, (const T*)h->b1, (const T*)h->w2, (const T*)h->b2, (T*)y,
+        h->D, h->O, h->l, h->act, B, h->vec_ok && aligned16(x));
+    ++h->launches;
+    return launch_status();
+}
+
+#define FFF_DISPATCH(h, fn, ...) \
+    ((h)->dtype == FFF_DTYPE_F32 ? fn<float>(__VA_ARGS__) : fn<__nv_bfloat16>(__VA_ARGS__))
+
+fff_status_t check_forward_args(fff_handle_t h, int64_t B) {
+    if (!live(h)) return FFF_ERR_BAD_HANDLE;
+    if (B < 0) return FFF_ERR_INVALID_ARG;
+    if (B > INT32_MAX) return FFF_ERR_UNSUPPORTED;
+    return FFF_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* fff_status_string(fff_status_t s) {
+    switch (s) {
+        case FFF_OK: return "ok";
+        case FFF_ERR_INVALID_ARG: return "invalid argument";
+        case FFF_ERR_UNSUPPORTED: return "unsupported configuration";
+        case FFF_ERR_ALLOC: return "allocation failed";
+        case FFF_ERR_CUDA: return "CUDA runtime error";
+        case FFF_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+        case FFF_ERR_BAD_HANDLE: return "bad handle";
+    }
+    return "unknown status";
+}
+
+fff_status_t fff_create(fff_handle_t* out, int D, int O, int depth, int leaf_width, fff_activation_t act,
+                        fff_dtype_t dtype, const void* node_w, const void* node_b, const void* leaf_w1,
+                        const void* leaf_b1, const void* leaf_w2, const void* leaf_b2) {
+    if (!out) return FFF_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (D < 1 || O < 1 || leaf_width < 1 || depth < 0) return FFF_ERR_INVALID_ARG;
+    if (act != FFF_ACT_RELU && act != FFF_ACT_GELU) return FFF_ERR_INVALID_ARG;
+    if (dtype != FFF_DTYPE_F32 && dtype != FFF_DTYPE_BF16) return FFF_ERR_INVALID_ARG;
+    if (depth > FFF_MAX_DEPTH) return FFF_ERR_UNSUPPORTED;
+    if (!leaf_w1 || !leaf_w2 || (depth > 0 && !node_w)) return FFF_ERR_INVALID_ARG;
+    for (const void* p : {node_w, node_b, leaf_w1, leaf_b1, leaf_w2, leaf_b2})
+        if (p && !aligned16(p)) return FFF_ERR_INVALID_ARG;
+
+    fff_handle_s* h = new (std::nothrow) fff_handle_s();
+    if (!h) return FFF_ERR_ALLOC;
+    if (cudaGetDevice(&h->device) != cudaSuccess) { delete h; return cudaGetLastError(), FFF_ERR_CUDA; }
+    cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device);
+    h->D = D; h->O = O; h->depth = depth; h->l = leaf_width; h->act = act; h->dtype = dtype;
+    h->esize = dtype == FFF_DTYPE_F32 ? 4 : 2;
+    h->n_nodes = ((int64_t)1 << depth) - 1;
+    h->n_leaves = (int64_t)1 << depth;
+    h->vec_ok = (D % (int)(16 / h->esize)) == 0;
+
+    const size_t e = h->esize, nn = (size_t)h->n_nodes, nl = (size_t)h->n_leaves;
+    fff_status_t s = FFF_OK;
+    if (s == FFF_OK) s = clone(&h->node_w, node_w, nn * D * e);
+    if (s == FFF_OK) s = clone(&h->node_b, node_b, nn * e);
+    if (s == FFF_OK) s = clone(&h->w1, leaf_w1, nl * leaf_width * D * e);
+    if (s == FFF_OK) s = clone(&h->b1, leaf_b1, nl * leaf_width * e);
+    if (s == FFF_OK) s = clone(&h->w2, leaf_w2, nl * O * leaf_width * e);
+    if (s == FFF_OK) s = clone(&h->b2, leaf_b2, nl * O * e);
+    if (s == FFF_OK) s = clone((void**)&h->ws_offsets, nullptr, sizeof(int32_t) * (nl + 1));
+    if (s == FFF_OK) s = clone((void**)&h->ws_hist[0], nullptr, sizeof(int) * nl);
+    if (s == FFF_OK) s = clone((void**)&h->ws_hist[1], nullptr, sizeof(int) * nl);
+    if (s == FFF_OK) s = clone((void**)&h->d_status, nullptr, sizeof(int));
+    if (s == FFF_OK && cudaDeviceSynchronize() != cudaSuccess) s = (cudaGetLastError(), FFF_ERR_CUDA);
+    if (s != FFF_OK) { release(h); return s; }
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        g_live.insert(h);
+    }
+    *out = h;
+    return FFF_OK;
+}
+
+fff_status_t fff_destroy(fff_handle_t h) {
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        if (!h || g_live.erase(h) == 0) return FFF_ERR_BAD_HANDLE;
+    }
+    DeviceGuard g(h->device);
+    cudaDeviceSynchronize();
+    release(h);
+    return cudaGetLastError() == cudaSuccess ? FFF_OK : FFF_ERR_CUDA;
+}
+
+fff_status_t fff_reserve(fff_handle_t h, int64_t max_B) {
+    fff_status_t s = check_forward_args(h, max_B);
+    if (s != FFF_OK) return s;
+    DeviceGuard g(h->device);
+    return grow_workspace(h, max_B);
+}
+
+fff_status_t fff_set_path(fff_handle_t h, fff_path_t path) {
+    if (!live(h)) return FFF_ERR_BAD_HANDLE;
+    if (path != FFF_PATH_AUTO && path != FFF_PATH_WARP && path != FFF_PATH_TENSOR) return FFF_ERR_INVALID_ARG;
+    if (path == FFF_PATH_TENSOR) return FFF_ERR_UNSUPPORTED;
+    h->path = path;
+    return FFF_OK;
+}
+
+fff_status_t fff_tree_descent(fff_handle_t h, const void* x, int32_t* leaf_idx, int64_t B, void* cuda_stream) {
+    fff_status_t s = check_forward_args(h, B);
+    if (s != FFF_OK) return s;
+    if (B == 0) { h->launches = 0; return FFF_OK; }
+    if (!x || !leaf_idx || !aligned16(x)) return FFF_ERR_INVALID_ARG;
+    DeviceGuard g(h->device);
+    h->launches = 0;
+    return FFF_DISPATCH(h, run_descent, h, x, leaf_idx, nullptr, B, (cudaStream_t)cuda_stream);
+}
+
+fff_status_t fff_leaf_bucketing(fff_handle_t h, const int32_t* leaf_idx, int32_t* offsets, int32_t* perm, int64_t B,
+                                void* cuda_stream) {
+    fff_status_t s = check_forward_args(h, B);
+    if (s != FFF_OK) return s;
+    if (!offsets || (B > 0 && (!leaf_idx || !perm))) return FFF_ERR_INVALID_ARG;
+    DeviceGuard g(h->device);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    h->launches = 0;
+    if (B > 0 && (s = run_histogram(h, leaf_idx, B, st)) != FFF_OK) return s;
+    return run_bucket(h, leaf_idx, offsets, perm, B, st);
+}
+
+fff_status_t fff_grouped_leaf_ff(fff_handle_t h, const void* x, const int32_t* leaf_idx, const int32_t* offsets,
+                                 const int32_t* perm, void* y, int64_t B, void* cuda_stream) {
+    fff_status_t s = check_forward_args(h, B);
+    if (s != FFF_OK) return s;
+    if (B == 0) { h->launches = 0; return FFF_OK; }
+    if (!x || !y || !leaf_idx || !offsets || !perm || !aligned16(x) || !aligned16(y)) return FFF_ERR_INVALID_ARG;
+    DeviceGuard g(h->device);
+    h->launches = 0;
+    return FFF_DISPATCH(h, run_leaf, h, x, leaf_idx, perm, y, B, (cudaStream_t)cuda_stream);
+}
+
+fff_status_t fff_forward_infer(fff_handle_t h, const void* x, void* y, int32_t* leaf_idx, int64_t B, void* cuda_stream) {
+    fff_status_t s = check_forward_args(h, B);
+    if (s != FFF_OK) return s;
+    if (B == 0) { h->launches = 0; h->last_B = 0; return FFF_OK; }
+    if (!x || !y || !aligned16(x) || !aligned16(y)) return FFF_ERR_INVALID_ARG;
+    DeviceGuard g(h->device);
+    if ((s = grow_workspace(h, B)) != FFF_OK) return s;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    int32_t* leaf = leaf_idx ? leaf_idx : h->ws_leaf;
+    h->launches = 0;
+    h->last_B = B;
+    if ((s = FFF_DISPATCH(h, run_descent, h, x, leaf, h->ws_hist[h->hist_cur], B, st)) != FFF_OK) return s;
+    if ((s = run_bucket(h, leaf, h->ws_offsets, h->ws_perm, B, st)) != FFF_OK) return s;
+    return FFF_DISPATCH(h, run_leaf, h, x, leaf, h->ws_perm, y, B, st);
+}
+
+fff_status_t fff_forward_infer_host(fff_handle_t h, const void* x_host, void* y_host, int32_t* leaf_idx_host,
+                                    int64_t B, void* cuda_stream) {
+    fff_status_t s = check_forward_args(h, B);
+    if (s != FFF_OK) return s;
+    if (B == 0) { h->launches = 0; h->last_B = 0; return FFF_OK; }
+    if (!x_host || !y_host) return FFF_ERR_INVALID_ARG;
+    DeviceGuard g(h->device);
+    if (B > h->cap_host_B) {
+        if (cudaDeviceSynchronize() != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
+        dfree(h->st_x); dfree(h->st_y); dfree(h->st_leaf);
+        h->st_x = h->st_y = nullptr; h->st_leaf = nullptr; h->cap_host_B = 0;
+        if ((s = dmalloc(&h->st_x, (size_t)B * h->D * h->esize)) != FFF_OK) return s;
+        if ((s = dmalloc(&h->st_y, (size_t)B * h->O * h->esize)) != FFF_OK) return s;
+        if ((s = dmalloc((void**)&h->st_leaf, (size_t)B * sizeof(int32_t))) != FFF_OK) return s;
+        h->cap_host_B = B;
+    }
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (cudaMemcpyAsync(h->st_x, x_host, (size_t)B * h->D * h->esize, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return cudaGetLastError(), FFF_ERR_CUDA;
+    if ((s = fff_forward_infer(h, h->st_x, h->st_y, h->st_leaf, B, cuda_stream)) != FFF_OK) return s;
+    if (cudaMemcpyAsync(y_host, h->st_y, (size_t)B * h->O * h->esize, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return cudaGetLastError(), FFF_ERR_CUDA;
+    if (leaf_idx_host &&
+        cudaMemcpyAsync(leaf_idx_host, h->st_leaf, (size_t)B * sizeof(int32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return cudaGetLastError(), FFF_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
+    return FFF_OK;
+}
+
+fff_status_t fff_debug_get_bucketing(fff_handle_t h, int32_t* perm, int32_t* offsets, void* cuda_stream) {
+    if (!live(h)) return FFF_ERR_BAD_HANDLE;
+    if (!offsets || h->last_B < 0 || (h->last_B > 0 && !perm)) return FFF_ERR_INVALID_ARG;
+    DeviceGuard g(h->device);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (h->last_B > 0 &&
+        cudaMemcpyAsync(perm, h->ws_perm, sizeof(int32_t) * (size_t)h->last_B, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        return cudaGetLastError(), FFF_ERR_CUDA;
+    if (h->last_B > 0) {
+        if (cudaMemcpyAsync(offsets, h->ws_offsets, sizeof(int32_t) * (size_t)(h->n_leaves + 1), cudaMemcpyDeviceToDevice,
+                            st) != cudaSuccess)
+            return cudaGetLastError(), FFF_ERR_CUDA;
+    } else if (cudaMemsetAsync(offsets, 0, sizeof(int32_t) * (size_t)(h->n_leaves + 1), st) != cudaSuccess) {
+        return cudaGetLastError(), FFF_ERR_CUDA;
+    }
+    return FFF_OK;
+}
+
+fff_status_t fff_get_last_status(fff_handle_t h) {
+    if (!live(h)) return FFF_ERR_BAD_HANDLE;
+    DeviceGuard g(h->device);
+    if (cudaDeviceSynchronize() != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
+    int word = 0;
+    if (cudaMemcpy(&word, h->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
+    if (word != fff::kDevOk) {
+        cudaMemset(h->d_status, 0, sizeof(int));
+        return FFF_ERR_DEVICE_TIMEOUT;
+    }
+    return FFF_OK;
+}
+
+int fff_last_launch_count(fff_handle_t h) { return live(h) ? h->launches : -1; }
+
+}  // extern "C"
