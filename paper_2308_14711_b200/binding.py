@@ -1,0 +1,254 @@
+"""ctypes binding of libfff.so: the same calls as include/fff.h, arguments marshalled only.
+
+Every computation happens in the CUDA library.  If the library has not been
+built (python -m paper_2308_14711_b200.build) loading fails with an error;
+there is no fallback of any kind.
+
+The module-level fff_* functions take raw device addresses (ints); `FFFLayer`
+is a convenience wrapper that takes torch CUDA tensors, checks their dtype,
+shape and contiguity, and passes their data_ptr().
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libfff.so")
+
+FFF_OK = 0
+STATUS_NAMES = {0: "FFF_OK", 1: "FFF_ERR_INVALID_ARG", 2: "FFF_ERR_UNSUPPORTED", 3: "FFF_ERR_ALLOC",
+                4: "FFF_ERR_CUDA", 5: "FFF_ERR_DEVICE_TIMEOUT", 6: "FFF_ERR_BAD_HANDLE"}
+ACTIVATIONS = {"relu": 0, "gelu": 1}
+DTYPES = {"f32": 0, "bf16": 1}
+PATHS = {"auto": 0, "warp": 1, "tensor": 2}
+
+# every symbol include/fff.h declares
+EXPORTS = ["fff_create", "fff_forward_infer", "fff_forward_infer_host", "fff_destroy", "fff_reserve",
+           "fff_set_path", "fff_tree_descent", "fff_leaf_bucketing", "fff_grouped_leaf_ff",
+           "fff_debug_get_bucketing", "fff_get_last_status", "fff_last_launch_count", "fff_status_string"]
+
+
+class FFFError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)} ({status_string(status)})")
+
+
+_lib = None
+
+
+def lib():
+    """Load libfff.so (once). Raises if it is missing: the CUDA library is the only implementation."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} not found: build it with `python -m paper_2308_14711_b200.build` "
+                          "(needs nvcc); there is no CPU fallback")
+    L = C.CDLL(LIB_PATH)
+    vp, i64, ci = C.c_void_p, C.c_int64, C.c_int
+    L.fff_create.argtypes = [C.POINTER(vp), ci, ci, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp]
+    L.fff_forward_infer.argtypes = [vp, vp, vp, vp, i64, vp]
+    L.fff_forward_infer_host.argtypes = [vp, vp, vp, vp, i64, vp]
+    L.fff_destroy.argtypes = [vp]
+    L.fff_reserve.argtypes = [vp, i64]
+    L.fff_set_path.argtypes = [vp, ci]
+    L.fff_tree_descent.argtypes = [vp, vp, vp, i64, vp]
+    L.fff_leaf_bucketing.argtypes = [vp, vp, vp, vp, i64, vp]
+    L.fff_grouped_leaf_ff.argtypes = [vp, vp, vp, vp, vp, vp, i64, vp]
+    L.fff_debug_get_bucketing.argtypes = [vp, vp, vp, vp]
+    L.fff_get_last_status.argtypes = [vp]
+    L.fff_last_launch_count.argtypes = [vp]
+    for name in EXPORTS:
+        getattr(L, name).restype = ci
+    L.fff_status_string.argtypes = [ci]
+    L.fff_status_string.restype = C.c_char_p
+    _lib = L
+    return L
+
+
+def status_string(status: int) -> str:
+    return lib().fff_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != FFF_OK:
+        raise FFFError(status, where)
+
+
+# ---- raw calls: device addresses as ints, 0 / None for NULL ------------------------------------
+
+def fff_create(D, O, depth, leaf_width, act, dtype, node_w, node_b, leaf_w1, leaf_b1, leaf_w2, leaf_b2) -> int:
+    h = C.c_void_p()
+    _check(lib().fff_create(C.byref(h), D, O, depth, leaf_width, act, dtype,
+                            node_w, node_b, leaf_w1, leaf_b1, leaf_w2, leaf_b2), "fff_create")
+    return h.value
+
+
+def fff_forward_infer(h, x, y, leaf_idx, B, stream=None) -> None:
+    _check(lib().fff_forward_infer(h, x, y, leaf_idx, B, stream), "fff_forward_infer")
+
+
+def fff_forward_infer_host(h, x_host, y_host, leaf_idx_host, B, stream=None) -> None:
+    _check(lib().fff_forward_infer_host(h, x_host, y_host, leaf_idx_host, B, stream), "fff_forward_infer_host")
+
+
+def fff_destroy(h) -> None:
+    _check(lib().fff_destroy(h), "fff_destroy")
+
+
+def fff_reserve(h, max_B) -> None:
+    _check(lib().fff_reserve(h, max_B), "fff_reserve")
+
+
+def fff_set_path(h, path) -> None:
+    _check(lib().fff_set_path(h, path), "fff_set_path")
+
+
+def fff_tree_descent(h, x, leaf_idx, B, stream=None) -> None:
+    _check(lib().fff_tree_descent(h, x, leaf_idx, B, stream), "fff_tree_descent")
+
+
+def fff_leaf_bucketing(h, leaf_idx, offsets, perm, B, stream=None) -> None:
+    _check(lib().fff_leaf_bucketing(h, leaf_idx, offsets, perm, B, stream), "fff_leaf_bucketing")
+
+
+def fff_grouped_leaf_ff(h, x, leaf_idx, offsets, perm, y, B, stream=None) -> None:
+    _check(lib().fff_grouped_leaf_ff(h, x, leaf_idx, offsets, perm, y, B, stream), "fff_grouped_leaf_ff")
+
+
+def fff_debug_get_bucketing(h, perm, offsets, stream=None) -> None:
+    _check(lib().fff_debug_get_bucketing(h, perm, offsets, stream), "fff_debug_get_bucketing")
+
+
+def fff_get_last_status(h) -> int:
+    return lib().fff_get_last_status(h)
+
+
+def fff_last_launch_count(h) -> int:
+    return lib().fff_last_launch_count(h)
+
+
+# ---- tensor-level convenience ------------------------------------------------------------------
+
+def _torch():
+    import torch
+    return torch
+
+
+def _ptr(t, dtype, shape, name):
+    if t is None:
+        return None
+    if not t.is_cuda or t.dtype != dtype or not t.is_contiguous() or tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name}: expected contiguous CUDA {dtype} tensor of shape {tuple(shape)}, "
+                         f"got {t.dtype} {tuple(t.shape)} on {t.device}")
+    return t.data_ptr()
+
+
+class FFFLayer:
+    """One FFF layer on the current CUDA device; tensors in, tensors out, all work in libfff.so."""
+
+    def __init__(self, D: int, O: int, depth: int, leaf_width: int, activation: str, dtype: str,
+                 node_w, node_b, w1, b1, w2, b2, path: str = "auto"):
+        torch = _torch()
+        self._h = None
+        self.D, self.O, self.depth, self.l = D, O, depth, leaf_width
+        self.n_leaves = 1 << depth
+        self.tdtype = torch.float32 if dtype == "f32" else torch.bfloat16
+        nn, nl = self.n_leaves - 1, self.n_leaves
+        td = self.tdtype
+        self._h = fff_create(D, O, depth, leaf_width, ACTIVATIONS[activation], DTYPES[dtype],
+                             _ptr(node_w, td, (nn, D), "node_w"), _ptr(node_b, td, (nn,), "node_b"),
+                             _ptr(w1, td, (nl, leaf_width, D), "w1"), _ptr(b1, td, (nl, leaf_width), "b1"),
+                             _ptr(w2, td, (nl, O, leaf_width), "w2"), _ptr(b2, td, (nl, O), "b2"))
+        if path != "auto":
+            self.set_path(path)
+
+    @property
+    def handle(self) -> int:
+        return self._h
+
+    def close(self) -> None:
+        if getattr(self, "_h", None):
+            h, self._h = self._h, None
+            fff_destroy(h)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _stream(self, stream):
+        s = stream if stream is not None else _torch().cuda.current_stream()
+        return s.cuda_stream
+
+    def reserve(self, max_B: int) -> None:
+        fff_reserve(self._h, max_B)
+
+    def set_path(self, path: str) -> None:
+        fff_set_path(self._h, PATHS[path])
+
+    def forward_infer(self, x, y=None, leaf_idx=None, want_leaf_idx: bool = True, stream=None):
+        torch = _torch()
+        B = x.shape[0]
+        if y is None:
+            y = torch.empty((B, self.O), dtype=self.tdtype, device=x.device)
+        if leaf_idx is None and want_leaf_idx:
+            leaf_idx = torch.empty((B,), dtype=torch.int32, device=x.device)
+        fff_forward_infer(self._h, _ptr(x, self.tdtype, (B, self.D), "x"), _ptr(y, self.tdtype, (B, self.O), "y"),
+                          _ptr(leaf_idx, torch.int32, (B,), "leaf_idx"), B, self._stream(stream))
+        return y, leaf_idx
+
+    def forward_infer_host(self, x_host, y_host, leaf_idx_host=None, stream=None) -> None:
+        """x_host / y_host / leaf_idx_host: contiguous CPU tensors (pinned for full copy speed)."""
+        B = x_host.shape[0]
+        assert not x_host.is_cuda and not y_host.is_cuda and x_host.is_contiguous() and y_host.is_contiguous()
+        assert x_host.dtype == self.tdtype and y_host.dtype == self.tdtype
+        assert tuple(x_host.shape) == (B, self.D) and tuple(y_host.shape) == (B, self.O)
+        fff_forward_infer_host(self._h, x_host.data_ptr(), y_host.data_ptr(),
+                               None if leaf_idx_host is None else leaf_idx_host.data_ptr(), B, self._stream(stream))
+
+    def tree_descent(self, x, leaf_idx=None, stream=None):
+        torch = _torch()
+        B = x.shape[0]
+        if leaf_idx is None:
+            leaf_idx = torch.empty((B,), dtype=torch.int32, device=x.device)
+        fff_tree_descent(self._h, _ptr(x, self.tdtype, (B, self.D), "x"), _ptr(leaf_idx, torch.int32, (B,), "leaf_idx"),
+                         B, self._stream(stream))
+        return leaf_idx
+
+    def leaf_bucketing(self, leaf_idx, stream=None):
+        torch = _torch()
+        B = leaf_idx.shape[0]
+        offsets = torch.empty((self.n_leaves + 1,), dtype=torch.int32, device=leaf_idx.device)
+        perm = torch.empty((B,), dtype=torch.int32, device=leaf_idx.device)
+        fff_leaf_bucketing(self._h, _ptr(leaf_idx, torch.int32, (B,), "leaf_idx"), offsets.data_ptr(), perm.data_ptr(),
+                           B, self._stream(stream))
+        return offsets, perm
+
+    def grouped_leaf_ff(self, x, leaf_idx, offsets, perm, y=None, stream=None):
+        torch = _torch()
+        B = x.shape[0]
+        if y is None:
+            y = torch.empty((B, self.O), dtype=self.tdtype, device=x.device)
+        fff_grouped_leaf_ff(self._h, _ptr(x, self.tdtype, (B, self.D), "x"),
+                            _ptr(leaf_idx, torch.int32, (B,), "leaf_idx"),
+                            _ptr(offsets, torch.int32, (self.n_leaves + 1,), "offsets"),
+                            _ptr(perm, torch.int32, (B,), "perm"), _ptr(y, self.tdtype, (B, self.O), "y"),
+                            B, self._stream(stream))
+        return y
+
+    def last_bucketing(self, B: int, stream=None):
+        torch = _torch()
+        perm = torch.empty((B,), dtype=torch.int32, device="cuda")
+        offsets = torch.empty((self.n_leaves + 1,), dtype=torch.int32, device="cuda")
+        fff_debug_get_bucketing(self._h, perm.data_ptr(), offsets.data_ptr(), self._stream(stream))
+        return offsets, perm
+
+    def last_status(self) -> int:
+        return fff_get_last_status(self._h)
+
+    def last_launch_count(self) -> int:
+        return fff_last_launch_count(self._h)
