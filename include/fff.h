@@ -173,6 +173,21 @@ fff_status_t fff_get_last_status(fff_handle_t h);
  * (-1 for a bad handle). */
 int fff_last_launch_count(fff_handle_t h);
 
+/*
+ * Per-launch timing of forwards, for benchmarks.  After fff_profile_begin the
+ * next max_steps calls of fff_forward_infer record a CUDA event on their stream
+ * before the first and after every kernel they launch (at most 16 per forward).
+ * fff_profile_end synchronises the device, writes the mean duration in
+ * milliseconds of each launch position into mean_ms[0 .. fff_profile_launches)
+ * and the number of recorded forwards into *steps, and stops recording.
+ * fff_profile_launch_name(h, i) names the kernel at position i ("" if out of
+ * range); the string is static.
+ */
+fff_status_t fff_profile_begin(fff_handle_t h, int max_steps);
+fff_status_t fff_profile_end(fff_handle_t h, double *mean_ms, int *steps);
+int fff_profile_launches(fff_handle_t h);
+const char *fff_profile_launch_name(fff_handle_t h, int i);
+
 /* Static, never NULL. */
 const char *fff_status_string(fff_status_t s);
 

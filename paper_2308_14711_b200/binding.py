@@ -26,7 +26,8 @@ PATHS = {"auto": 0, "warp": 1, "tensor": 2}
 # every symbol include/fff.h declares
 EXPORTS = ["fff_create", "fff_forward_infer", "fff_forward_infer_host", "fff_destroy", "fff_reserve",
            "fff_set_path", "fff_tree_descent", "fff_leaf_bucketing", "fff_grouped_leaf_ff",
-           "fff_debug_get_bucketing", "fff_get_last_status", "fff_last_launch_count", "fff_status_string"]
+           "fff_debug_get_bucketing", "fff_get_last_status", "fff_last_launch_count", "fff_status_string",
+           "fff_profile_begin", "fff_profile_end", "fff_profile_launches", "fff_profile_launch_name"]
 
 
 class FFFError(RuntimeError):
@@ -60,8 +61,13 @@ def lib():
     L.fff_debug_get_bucketing.argtypes = [vp, vp, vp, vp]
     L.fff_get_last_status.argtypes = [vp]
     L.fff_last_launch_count.argtypes = [vp]
+    L.fff_profile_begin.argtypes = [vp, ci]
+    L.fff_profile_end.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(ci)]
+    L.fff_profile_launches.argtypes = [vp]
+    L.fff_profile_launch_name.argtypes = [vp, ci]
     for name in EXPORTS:
         getattr(L, name).restype = ci
+    L.fff_profile_launch_name.restype = C.c_char_p
     L.fff_status_string.argtypes = [ci]
     L.fff_status_string.restype = C.c_char_p
     _lib = L
@@ -128,6 +134,19 @@ def fff_get_last_status(h) -> int:
 
 def fff_last_launch_count(h) -> int:
     return lib().fff_last_launch_count(h)
+
+
+def fff_profile_begin(h, max_steps) -> None:
+    _check(lib().fff_profile_begin(h, max_steps), "fff_profile_begin")
+
+
+def fff_profile_end(h):
+    """Returns (list of (kernel name, mean ms) per launch position, number of recorded forwards)."""
+    ms = (C.c_double * 16)()
+    steps = C.c_int(0)
+    _check(lib().fff_profile_end(h, ms, C.byref(steps)), "fff_profile_end")
+    n = lib().fff_profile_launches(h)
+    return [(lib().fff_profile_launch_name(h, i).decode(), ms[i]) for i in range(n)], steps.value
 
 
 # ---- tensor-level convenience ------------------------------------------------------------------
@@ -246,6 +265,12 @@ class FFFLayer:
         offsets = torch.empty((self.n_leaves + 1,), dtype=torch.int32, device="cuda")
         fff_debug_get_bucketing(self._h, perm.data_ptr(), offsets.data_ptr(), self._stream(stream))
         return offsets, perm
+
+    def profile_begin(self, max_steps: int) -> None:
+        fff_profile_begin(self._h, max_steps)
+
+    def profile_end(self):
+        return fff_profile_end(self._h)
 
     def last_status(self) -> int:
         return fff_get_last_status(self._h)

@@ -13,6 +13,7 @@
 #include <mutex>
 #include <new>
 #include <set>
+#include <vector>
 
 #include "kernels/bucket.cuh"
 #include "kernels/common.cuh"
@@ -62,6 +63,14 @@ struct fff_handle_s {
     int path = FFF_PATH_AUTO;
     int launches = 0;
     int64_t last_B = -1;
+
+    // optional per-launch timing of forwards (fff_profile_*)
+    static constexpr int kMaxProfLaunches = 16;
+    int prof_max_steps = 0, prof_steps = 0;
+    bool prof_active = false;                     // this forward is being recorded
+    int prof_nlaunch = 0;                         // launches per forward of the recorded steps
+    const char* prof_names[kMaxProfLaunches] = {};
+    std::vector<cudaEvent_t> prof_events;         // [prof_max_steps][kMaxProfLaunches + 1]
 };
 
 namespace {
@@ -92,10 +101,18 @@ fff_status_t clone(void** dst, const void* src, size_t bytes) {
     return e == cudaSuccess ? FFF_OK : (cudaGetLastError(), FFF_ERR_CUDA);
 }
 
+void prof_free(fff_handle_s* h) {
+    for (cudaEvent_t e : h->prof_events) cudaEventDestroy(e);
+    h->prof_events.clear();
+    h->prof_max_steps = h->prof_steps = h->prof_nlaunch = 0;
+    h->prof_active = false;
+}
+
 void release(fff_handle_s* h) {
     dfree(h->node_w); dfree(h->node_b); dfree(h->w1); dfree(h->b1); dfree(h->w2); dfree(h->b2);
     dfree(h->ws_leaf); dfree(h->ws_perm); dfree(h->ws_offsets); dfree(h->ws_hist[0]); dfree(h->ws_hist[1]);
     dfree(h->d_status); dfree(h->st_x); dfree(h->st_y); dfree(h->st_leaf);
+    prof_free(h);
     h->magic = 0;
     delete h;
 }
@@ -113,9 +130,16 @@ fff_status_t grow_workspace(fff_handle_s* h, int64_t B) {
     return FFF_OK;
 }
 
-fff_status_t launch_status() {
+// Called after every kernel launch: counts it, records its profiling event, reports launch errors.
+fff_status_t launched(fff_handle_s* h, cudaStream_t st, const char* name) {
+    const int i = h->launches++;
+    if (h->prof_active && i < fff_handle_s::kMaxProfLaunches) {
+        h->prof_names[i] = name;
+        cudaEventRecord(h->prof_events[(size_t)h->prof_steps * (fff_handle_s::kMaxProfLaunches + 1) + i + 1], st);
+    }
     return cudaGetLastError() == cudaSuccess ? FFF_OK : FFF_ERR_CUDA;
 }
+
 
 // ---- stage launchers -------------------------------------------------------
 
@@ -125,15 +149,13 @@ fff_status_t run_descent(fff_handle_s* h, const void* x, int32_t* leaf_idx, int*
     fff::k_descent_warp<T><<<(unsigned)blocks, fff::kDescentWarps * 32, 0, st>>>(
         (const T*)x, (const T*)h->node_w, (const T*)h->node_b, h->D, 0, h->depth, nullptr, leaf_idx, hist, B,
         h->vec_ok && aligned16(x));
-    ++h->launches;
-    return launch_status();
+    return launched(h, st, "tree_descent_warp");
 }
 
 fff_status_t run_histogram(fff_handle_s* h, const int32_t* keys, int64_t B, cudaStream_t st) {
     const int64_t blocks = std::min<int64_t>((B + 255) / 256, (int64_t)h->sm_count * 4);
     fff::k_histogram<<<(unsigned)blocks, 256, 0, st>>>(keys, h->ws_hist[h->hist_cur], B, (int)h->n_leaves);
-    ++h->launches;
-    return launch_status();
+    return launched(h, st, "leaf_histogram");
 }
 
 // Consumes the current histogram buffer and flips to the other (already zero) one.
@@ -154,8 +176,7 @@ fff_status_t run_bucket(fff_handle_s* h, const int32_t* keys, int32_t* offsets, 
     fff::k_bucket<<<ctas, fff::kBucketThreads, smem, st>>>(keys, h->ws_hist[h->hist_cur], h->ws_hist[h->hist_cur ^ 1],
                                                          offsets, perm, (int)B, nbins, per);
     h->hist_cur ^= 1;
-    ++h->launches;
-    return launch_status();
+    return launched(h, st, "leaf_bucketing");
 }
 
 template <typename T>
@@ -166,8 +187,7 @@ fff_status_t run_leaf(fff_handle_s* h, const void* x, const int32_t* leaf_idx, c
     fff::k_leaf_warp<T><<<(unsigned)blocks, fff::kLeafWarps * 32, smem, st>>>(
         (const T*)x, leaf_idx, perm, (const T*)h->w1, (const T*)h->b1, (const T*)h->w2, (const T*)h->b2, (T*)y,
         h->D, h->O, h->l, h->act, B, h->vec_ok && aligned16(x));
-    ++h->launches;
-    return launch_status();
+    return launched(h, st, "grouped_leaf_ff_warp");
 }
 
 #define FFF_DISPATCH(h, fn, ...) \
@@ -312,9 +332,20 @@ fff_status_t fff_forward_infer(fff_handle_t h, const void* x, void* y, int32_t* 
     int32_t* leaf = leaf_idx ? leaf_idx : h->ws_leaf;
     h->launches = 0;
     h->last_B = B;
-    if ((s = FFF_DISPATCH(h, run_descent, h, x, leaf, h->ws_hist[h->hist_cur], B, st)) != FFF_OK) return s;
-    if ((s = run_bucket(h, leaf, h->ws_offsets, h->ws_perm, B, st)) != FFF_OK) return s;
-    return FFF_DISPATCH(h, run_leaf, h, x, leaf, h->ws_perm, y, B, st);
+    h->prof_active = h->prof_steps < h->prof_max_steps;
+    if (h->prof_active)
+        cudaEventRecord(h->prof_events[(size_t)h->prof_steps * (fff_handle_s::kMaxProfLaunches + 1)], st);
+    s = FFF_DISPATCH(h, run_descent, h, x, leaf, h->ws_hist[h->hist_cur], B, st);
+    if (s == FFF_OK) s = run_bucket(h, leaf, h->ws_offsets, h->ws_perm, B, st);
+    if (s == FFF_OK) s = FFF_DISPATCH(h, run_leaf, h, x, leaf, h->ws_perm, y, B, st);
+    if (h->prof_active) {
+        h->prof_active = false;
+        if (s == FFF_OK && (h->prof_steps == 0 || h->prof_nlaunch == h->launches)) {
+            h->prof_nlaunch = std::min(h->launches, (int)fff_handle_s::kMaxProfLaunches);
+            ++h->prof_steps;
+        }
+    }
+    return s;
 }
 
 fff_status_t fff_forward_infer_host(fff_handle_t h, const void* x_host, void* y_host, int32_t* leaf_idx_host,
@@ -378,5 +409,51 @@ fff_status_t fff_get_last_status(fff_handle_t h) {
 }
 
 int fff_last_launch_count(fff_handle_t h) { return live(h) ? h->launches : -1; }
+
+fff_status_t fff_profile_begin(fff_handle_t h, int max_steps) {
+    if (!live(h)) return FFF_ERR_BAD_HANDLE;
+    if (max_steps < 0 || max_steps > (1 << 20)) return FFF_ERR_INVALID_ARG;
+    DeviceGuard g(h->device);
+    if (cudaDeviceSynchronize() != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
+    prof_free(h);
+    const size_t n = (size_t)max_steps * (fff_handle_s::kMaxProfLaunches + 1);
+    h->prof_events.reserve(n);
+    for (size_t i = 0; i < n; ++i) {
+        cudaEvent_t e;
+        if (cudaEventCreate(&e) != cudaSuccess) { prof_free(h); return cudaGetLastError(), FFF_ERR_ALLOC; }
+        h->prof_events.push_back(e);
+    }
+    h->prof_max_steps = max_steps;
+    return FFF_OK;
+}
+
+int fff_profile_launches(fff_handle_t h) { return live(h) ? h->prof_nlaunch : -1; }
+
+const char* fff_profile_launch_name(fff_handle_t h, int i) {
+    if (!live(h) || i < 0 || i >= h->prof_nlaunch || !h->prof_names[i]) return "";
+    return h->prof_names[i];
+}
+
+fff_status_t fff_profile_end(fff_handle_t h, double* mean_ms, int* steps) {
+    if (!live(h)) return FFF_ERR_BAD_HANDLE;
+    if (!mean_ms || !steps) return FFF_ERR_INVALID_ARG;
+    DeviceGuard g(h->device);
+    if (cudaDeviceSynchronize() != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
+    *steps = h->prof_steps;
+    const int stride = fff_handle_s::kMaxProfLaunches + 1;
+    for (int i = 0; i < h->prof_nlaunch; ++i) {
+        double sum = 0.0;
+        for (int s = 0; s < h->prof_steps; ++s) {
+            float ms = 0.0f;
+            if (cudaEventElapsedTime(&ms, h->prof_events[(size_t)s * stride + i], h->prof_events[(size_t)s * stride + i + 1]) !=
+                cudaSuccess)
+                return cudaGetLastError(), FFF_ERR_CUDA;
+            sum += ms;
+        }
+        mean_ms[i] = h->prof_steps ? sum / h->prof_steps : 0.0;
+    }
+    h->prof_max_steps = 0;      // stop recording; names and counts stay readable until the next begin
+    return FFF_OK;
+}
 
 }  // extern "C"

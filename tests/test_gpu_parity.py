@@ -1,0 +1,174 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the float64 CPU oracle.
+
+Integer results (leaf indices, bucket offsets, bucket permutation) must be bit-exact.
+Outputs must satisfy  |err| <= 1e-5 (1 + |ref|)  for float32 layers and
+|err| <= 2e-2 (1 + |ref|)  with relative L2 error <= 1e-2  for bf16 layers.
+Inputs are margin-enforced (no routing logit within 1e-2 of zero), so the routing decision
+cannot depend on summation order.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import fff_oracle as orc
+from paper_2308_14711_b200 import workloads as wl
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+PATHS = ["auto", "warp"]
+
+
+def small_cfgs():
+    C = wl.FFFConfig
+    return [
+        # ragged D (not a multiple of the vector width), tiny O, float32
+        C("f32_ragged", 50, 3, 3, 5, "relu", "f32", 333, "normal", node_bias_std=0.3),
+        C("f32_mnistlike", 784, 10, 3, 32, "relu", "f32", 517, "normal"),
+        C("f32_gelu_d0", 64, 16, 0, 8, "gelu", "f32", 100, "normal"),
+        C("f32_d1", 32, 32, 1, 4, "gelu", "f32", 65, "normal", node_bias_std=0.5),
+        # bf16: several tiles and a ragged tail, l below / at / above the MMA granule
+        C("bf16_l12", 768, 768, 4, 12, "gelu", "bf16", 1500, "layernorm"),
+        C("bf16_l32", 256, 128, 6, 32, "gelu", "bf16", 3001, "normal"),
+        C("bf16_l1_deep", 128, 64, 10, 1, "gelu", "bf16", 700, "normal"),
+        C("bf16_skew", 128, 256, 7, 16, "relu", "bf16", 4099, "clusters"),
+        C("bf16_ragged", 100, 36, 3, 7, "gelu", "bf16", 257, "normal", node_bias_std=0.2),
+        C("bf16_d0", 128, 128, 0, 48, "gelu", "bf16", 300, "normal"),
+        C("bf16_one_token", 64, 64, 5, 16, "gelu", "bf16", 1, "normal"),
+        C("bf16_l40", 512, 520, 2, 40, "relu", "bf16", 999, "normal"),
+    ]
+
+
+@pytest.fixture(scope="module", params=small_cfgs(), ids=lambda c: c.name)
+def small_case(request):
+    case = util.make_case(request.param, seed=1)
+    y_ref, leaf_ref = orc.forward_i(case.net, case.x, threads=util.ORACLE_THREADS)
+    return case, y_ref, leaf_ref
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_forward_matches_oracle_elementwise(small_case, path):
+    case, y_ref, leaf_ref = small_case
+    cfg = case.cfg
+    layer = util.make_layer(case, path)
+    x = util.to_device(case.x, cfg.dtype)
+    y, leaf = layer.forward_infer(x)
+    torch.cuda.synchronize()
+    assert layer.last_launch_count() > 0
+    np.testing.assert_array_equal(leaf.cpu().numpy(), leaf_ref)
+    off_ref, perm_ref = orc.bucket(leaf_ref, cfg.n_leaves)
+    off, perm = layer.last_bucketing(cfg.B)
+    np.testing.assert_array_equal(off.cpu().numpy(), off_ref)
+    np.testing.assert_array_equal(perm.cpu().numpy(), perm_ref)
+    util.check_outputs(y, y_ref, cfg.dtype)
+    assert layer.last_status() == 0
+    # leaf_idx is optional
+    y2, none = layer.forward_infer(x, want_leaf_idx=False)
+    assert none is None
+    assert torch.equal(y2, y)
+    layer.close()
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_stage_entry_points_match_oracle(small_case, path):
+    case, y_ref, leaf_ref = small_case
+    cfg = case.cfg
+    layer = util.make_layer(case, path)
+    x = util.to_device(case.x, cfg.dtype)
+    leaf = layer.tree_descent(x)
+    np.testing.assert_array_equal(leaf.cpu().numpy(), leaf_ref)
+    off, perm = layer.leaf_bucketing(leaf)
+    off_ref, perm_ref = orc.bucket(leaf_ref, cfg.n_leaves)
+    np.testing.assert_array_equal(off.cpu().numpy(), off_ref)
+    np.testing.assert_array_equal(perm.cpu().numpy(), perm_ref)
+    y = layer.grouped_leaf_ff(x, leaf, off, perm)
+    util.check_outputs(y, y_ref, cfg.dtype)
+    layer.close()
+
+
+def test_runs_are_bit_reproducible(small_case):
+    case, _, _ = small_case
+    layer = util.make_layer(case)
+    x = util.to_device(case.x, case.cfg.dtype)
+    y1, l1 = layer.forward_infer(x)
+    y2, l2 = layer.forward_infer(x)
+    assert torch.equal(y1, y2) and torch.equal(l1, l2)
+    layer.close()
+
+
+@pytest.mark.parametrize("B,depth,kind", [(0, 3, "uniform"), (1, 0, "uniform"), (31, 2, "uniform"), (4097, 5, "uniform"),
+                                          (70001, 11, "uniform"), (50000, 11, "one_bin"), (50000, 11, "zipf"),
+                                          (20000, 15, "uniform"), (3000, 15, "each_own"), (100000, 3, "uniform"),
+                                          (9999, 16, "zipf")])
+def test_bucketing_is_the_stable_counting_sort(B, depth, kind):
+    nl = 1 << depth
+    rng = np.random.default_rng(B + depth)
+    if kind == "uniform":
+        keys = rng.integers(0, nl, size=B)
+    elif kind == "one_bin":
+        keys = np.full(B, nl - 3)
+    elif kind == "each_own":
+        keys = rng.permutation(nl)[:B]
+    else:
+        keys = np.minimum(rng.zipf(1.3, size=B) - 1, nl - 1)
+    keys = keys.astype(np.int32)
+    cfg = wl.FFFConfig("b", 8, 8, depth, 1, "relu", "f32", max(B, 1))
+    w = wl.make_weights(cfg, 0)
+    case = util.Case(cfg, w, None, None, 0)
+    layer = util.make_layer(case)
+    dkeys = torch.from_numpy(keys).cuda()
+    for _ in range(2):      # twice: the histogram buffers alternate between calls
+        off, perm = layer.leaf_bucketing(dkeys)
+        off_ref, perm_ref = orc.bucket(keys, nl)
+        np.testing.assert_array_equal(off.cpu().numpy(), off_ref)
+        np.testing.assert_array_equal(perm.cpu().numpy(), perm_ref)
+    layer.close()
+
+
+def test_host_buffer_entry_point(small_case):
+    case, y_ref, leaf_ref = small_case
+    cfg = case.cfg
+    layer = util.make_layer(case)
+    td = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
+    xh = torch.from_numpy(case.x).to(td).pin_memory()
+    yh = torch.empty((cfg.B, cfg.O), dtype=td).pin_memory()
+    lh = torch.empty((cfg.B,), dtype=torch.int32).pin_memory()
+    layer.forward_infer_host(xh, yh, lh)
+    np.testing.assert_array_equal(lh.numpy(), leaf_ref)
+    util.check_outputs(yh, y_ref, cfg.dtype)
+    layer.close()
+
+
+def test_gpu_argument_errors_are_reported_not_faulted():
+    from paper_2308_14711_b200 import binding
+    cfg = wl.FFFConfig("e", 16, 8, 2, 4, "relu", "f32", 8)
+    case = util.Case(cfg, wl.make_weights(cfg, 0), None, None, 0)
+    layer = util.make_layer(case)
+    x = torch.zeros((8, 16), device="cuda")
+    y = torch.zeros((8, 8), device="cuda")
+    L = binding.lib()
+    h = layer.handle
+    assert L.fff_forward_infer(h, None, y.data_ptr(), None, 8, None) == 1
+    assert L.fff_forward_infer(h, x.data_ptr(), None, None, 8, None) == 1
+    assert L.fff_forward_infer(h, x.data_ptr() + 4, y.data_ptr(), None, 7, None) == 1     # misaligned
+    assert L.fff_forward_infer(h, x.data_ptr(), y.data_ptr(), None, -1, None) == 1
+    assert L.fff_forward_infer(h, x.data_ptr(), y.data_ptr(), None, 0, None) == 0         # empty batch
+    assert L.fff_set_path(h, 9) == 1
+    layer.close()
+    assert L.fff_forward_infer(h, x.data_ptr(), y.data_ptr(), None, 8, None) == 6         # destroyed
+    torch.cuda.synchronize()
+
+
+def test_nan_inputs_stay_in_range():
+    cfg = wl.FFFConfig("n", 64, 32, 4, 8, "gelu", "bf16", 64)
+    case = util.make_case(cfg, 0)
+    layer = util.make_layer(case)
+    x = util.to_device(case.x, "bf16")
+    x[::3] = float("nan")
+    y, leaf = layer.forward_infer(x)
+    torch.cuda.synchronize()
+    lf = leaf.cpu().numpy()
+    assert ((lf >= 0) & (lf < 16)).all()
+    assert torch.isnan(y[::3].float()).all()
+    assert torch.isfinite(y[1::3].float()).all()
+    layer.close()
