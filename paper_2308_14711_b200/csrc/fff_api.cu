@@ -168,11 +168,6 @@ fff_status_t run_bucket(fff_handle_s* h, const int32_t* keys, int32_t* offsets, 
         ctas = (nbins + per - 1) / per;
     }
     const size_t smem = sizeof(int) * (size_t)fff::kBucketWarps * per;
-    static std::once_flag once;
-    std::call_once(once, [] {
-        cudaFuncSetAttribute(fff::k_bucket, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)(sizeof(int) * fff::kBucketWarps * fff::kBucketMaxBinsPerCta));
-    });
     fff::k_bucket<<<ctas, fff::kBucketThreads, smem, st>>>(keys, h->ws_hist[h->hist_cur], h->ws_hist[h->hist_cur ^ 1],
                                                          offsets, perm, (int)B, nbins, per);
     h->hist_cur ^= 1;
@@ -234,6 +229,8 @@ fff_status_t fff_create(fff_handle_t* out, int D, int O, int depth, int leaf_wid
     if (!h) return FFF_ERR_ALLOC;
     if (cudaGetDevice(&h->device) != cudaSuccess) { delete h; return cudaGetLastError(), FFF_ERR_CUDA; }
     cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device);
+    cudaFuncSetAttribute(fff::k_bucket, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         (int)(sizeof(int) * fff::kBucketWarps * fff::kBucketMaxBinsPerCta));
     h->D = D; h->O = O; h->depth = depth; h->l = leaf_width; h->act = act; h->dtype = dtype;
     h->esize = dtype == FFF_DTYPE_F32 ? 4 : 2;
     h->n_nodes = ((int64_t)1 << depth) - 1;
