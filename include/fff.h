@@ -49,7 +49,8 @@ typedef enum {
     FFF_ERR_ALLOC = 3,           /* device or host allocation failed */
     FFF_ERR_CUDA = 4,            /* a CUDA runtime call failed */
     FFF_ERR_DEVICE_TIMEOUT = 5,  /* a bounded device-side wait ran out (read by fff_get_last_status) */
-    FFF_ERR_BAD_HANDLE = 6       /* NULL, destroyed or corrupted handle */
+    FFF_ERR_BAD_HANDLE = 6,      /* NULL, destroyed or corrupted handle */
+    FFF_ERR_TOO_LARGE = 7        /* request exceeds the fixed capacity of fff_leaf_bucketing_static */
 } fff_status_t;
 
 typedef enum {
@@ -149,6 +150,42 @@ fff_status_t fff_tree_descent(fff_handle_t h, const void *x, int32_t *leaf_idx,
  * Uses the handle's workspace. */
 fff_status_t fff_leaf_bucketing(fff_handle_t h, const int32_t *leaf_idx, int32_t *offsets,
                                 int32_t *perm, int64_t B, void *cuda_stream);
+
+/*
+ * Leaf bucketing without any allocation.  (The paper has no counterpart of
+ * this call; it exists for the callers described below.)
+ *
+ * Some callers must not allocate device memory at the point where they need
+ * the bucketing: code running between the begin and end of a memory-pool
+ * accounting window, plugins of a host application that owns all device
+ * memory and forbids cudaMalloc, or latency-critical loops in which an
+ * allocation (which may synchronise the device) is unacceptable.  Such callers
+ * cannot create an fff handle, whose workspace is allocated.  This entry point
+ * computes exactly what fff_leaf_bucketing computes -- same kernels, same
+ * result bit for bit -- but takes no handle and keeps its scratch (the
+ * per-leaf token counts) in a fixed array compiled into the library:
+ * 2 * FFF_STATIC_MAX_BINS int32 counters = 512 KiB, resident on every GPU
+ * that loads the library, for the life of the process.
+ *
+ *   leaf_idx [B] in, values in [0, 2^depth); ids outside are ignored
+ *   offsets  [2^depth + 1] out,  perm [B] out      (as for fff_leaf_bucketing)
+ *   depth    0 <= depth <= FFF_STATIC_MAX_DEPTH;  B <= 2^31 - 1
+ *
+ * Larger requests return FFF_ERR_TOO_LARGE and launch nothing.  The call uses
+ * the current device; all pointers are device pointers on it.  It calls no
+ * cudaMalloc / cudaFree and no allocating library routine.
+ *
+ * The first call on each device looks up the device address of the array
+ * (and sets a kernel attribute); make that first call before starting any
+ * stream capture.  The array is shared by every call in the process and
+ * keeps the previous call's counts, so each call first clears the part it
+ * uses, on `cuda_stream`.  Two calls whose work overlaps on the GPU (different
+ * streams, or different host threads) race on the array: serialise them.
+ */
+#define FFF_STATIC_MAX_DEPTH 16
+#define FFF_STATIC_MAX_BINS (1 << FFF_STATIC_MAX_DEPTH)
+fff_status_t fff_leaf_bucketing_static(const int32_t *leaf_idx, int32_t *offsets, int32_t *perm,
+                                       int64_t B, int depth, void *cuda_stream);
 
 /* Grouped leaf evaluation with un-permuting write-back (Algorithm 1,
  * FORWARD_I, leaf branch: return N_{d,j}(x)):

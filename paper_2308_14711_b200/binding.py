@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(HERE, "libfff.so")
 
 FFF_OK = 0
 STATUS_NAMES = {0: "FFF_OK", 1: "FFF_ERR_INVALID_ARG", 2: "FFF_ERR_UNSUPPORTED", 3: "FFF_ERR_ALLOC",
-                4: "FFF_ERR_CUDA", 5: "FFF_ERR_DEVICE_TIMEOUT", 6: "FFF_ERR_BAD_HANDLE"}
+                4: "FFF_ERR_CUDA", 5: "FFF_ERR_DEVICE_TIMEOUT", 6: "FFF_ERR_BAD_HANDLE", 7: "FFF_ERR_TOO_LARGE"}
 ACTIVATIONS = {"relu": 0, "gelu": 1}
 DTYPES = {"f32": 0, "bf16": 1}
 PATHS = {"auto": 0, "warp": 1, "tensor": 2}
@@ -27,7 +27,8 @@ PATHS = {"auto": 0, "warp": 1, "tensor": 2}
 EXPORTS = ["fff_create", "fff_forward_infer", "fff_forward_infer_host", "fff_destroy", "fff_reserve",
            "fff_set_path", "fff_tree_descent", "fff_leaf_bucketing", "fff_grouped_leaf_ff",
            "fff_debug_get_bucketing", "fff_get_last_status", "fff_last_launch_count", "fff_status_string",
-           "fff_profile_begin", "fff_profile_end", "fff_profile_launches", "fff_profile_launch_name"]
+           "fff_profile_begin", "fff_profile_end", "fff_profile_launches", "fff_profile_launch_name",
+           "fff_leaf_bucketing_static"]
 
 
 class FFFError(RuntimeError):
@@ -61,6 +62,7 @@ def lib():
     L.fff_debug_get_bucketing.argtypes = [vp, vp, vp, vp]
     L.fff_get_last_status.argtypes = [vp]
     L.fff_last_launch_count.argtypes = [vp]
+    L.fff_leaf_bucketing_static.argtypes = [vp, vp, vp, i64, ci, vp]
     L.fff_profile_begin.argtypes = [vp, ci]
     L.fff_profile_end.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(ci)]
     L.fff_profile_launches.argtypes = [vp]
@@ -134,6 +136,11 @@ def fff_get_last_status(h) -> int:
 
 def fff_last_launch_count(h) -> int:
     return lib().fff_last_launch_count(h)
+
+
+def fff_leaf_bucketing_static(leaf_idx, offsets, perm, B, depth, stream=None) -> None:
+    """Handle-free, allocation-free bucketing (scratch compiled into the library; depth <= 16)."""
+    _check(lib().fff_leaf_bucketing_static(leaf_idx, offsets, perm, B, depth, stream), "fff_leaf_bucketing_static")
 
 
 def fff_profile_begin(h, max_steps) -> None:

@@ -197,7 +197,73 @@ fff_status_t check_forward_args(fff_handle_t h, int64_t B) {
 
 }  // namespace
 
+// ---- scratch of fff_leaf_bucketing_static ----------------------------------------------------
+// Two histogram buffers of FFF_STATIC_MAX_BINS counters each, resident on every device that loads the
+// library.  In host code this name only stands for the symbol; the device address comes from
+// cudaGetSymbolAddress (static_scratch_for_current_device).
+static __device__ __align__(256) int g_static_bucket_scratch[2 * FFF_STATIC_MAX_BINS];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+int* g_static_ptr[kMaxDevices] = {};
+
+// Device address of the static scratch on the current device; looked up once per device.
+fff_status_t static_scratch_for_current_device(int** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return FFF_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lk(g_static_mu);
+    if (!g_static_ptr[dev]) {
+        int* p = nullptr;
+        if (cudaGetSymbolAddress((void**)&p, g_static_bucket_scratch) != cudaSuccess || !p)
+            return cudaGetLastError(), FFF_ERR_CUDA;
+        if (cudaFuncSetAttribute(fff::k_bucket, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)(sizeof(int) * fff::kBucketWarps * fff::kBucketMaxBinsPerCta)) != cudaSuccess)
+            return cudaGetLastError(), FFF_ERR_CUDA;
+        g_static_ptr[dev] = p;
+    }
+    *out = g_static_ptr[dev];
+    return FFF_OK;
+}
+
+}  // namespace
+
 extern "C" {
+
+fff_status_t fff_leaf_bucketing_static(const int32_t* leaf_idx, int32_t* offsets, int32_t* perm, int64_t B,
+                                       int depth, void* cuda_stream) {
+    if (B < 0 || depth < 0) return FFF_ERR_INVALID_ARG;
+    if (depth > FFF_STATIC_MAX_DEPTH || B > INT32_MAX) return FFF_ERR_TOO_LARGE;
+    if (!offsets || (B > 0 && (!leaf_idx || !perm))) return FFF_ERR_INVALID_ARG;
+    int* scratch = nullptr;
+    fff_status_t s = static_scratch_for_current_device(&scratch);
+    if (s != FFF_OK) return s;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const int nbins = 1 << depth;
+    int* hist = scratch;                          // must start at zero: holds the previous call's counts
+    int* spare = scratch + FFF_STATIC_MAX_BINS;   // only written (zeroed) by the bucketing kernel
+    if (cudaMemsetAsync(hist, 0, sizeof(int) * (size_t)nbins, st) != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
+    if (B > 0) {
+        int sms = 148;
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        const int64_t blocks = std::min<int64_t>((B + 255) / 256, (int64_t)sms * 4);
+        fff::k_histogram<<<(unsigned)blocks, 256, 0, st>>>(leaf_idx, hist, B, nbins);
+        if (cudaGetLastError() != cudaSuccess) return FFF_ERR_CUDA;
+    }
+    int ctas = std::min(nbins, 32);
+    int per = (nbins + ctas - 1) / ctas;
+    if (per > fff::kBucketMaxBinsPerCta) {
+        per = fff::kBucketMaxBinsPerCta;
+        ctas = (nbins + per - 1) / per;
+    }
+    fff::k_bucket<<<ctas, fff::kBucketThreads, sizeof(int) * (size_t)fff::kBucketWarps * per, st>>>(
+        leaf_idx, hist, spare, offsets, perm, (int)B, nbins, per);
+    return cudaGetLastError() == cudaSuccess ? FFF_OK : FFF_ERR_CUDA;
+}
 
 const char* fff_status_string(fff_status_t s) {
     switch (s) {
@@ -208,6 +274,7 @@ const char* fff_status_string(fff_status_t s) {
         case FFF_ERR_CUDA: return "CUDA runtime error";
         case FFF_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
         case FFF_ERR_BAD_HANDLE: return "bad handle";
+        case FFF_ERR_TOO_LARGE: return "size exceeds the capacity of the static scratch";
     }
     return "unknown status";
 }

@@ -31,8 +31,8 @@ def test_header_symbols_are_exported(lib):
 
 
 def test_status_strings(lib):
-    seen = {binding.status_string(s) for s in range(7)}
-    assert len(seen) == 7 and "ok" in seen
+    seen = {binding.status_string(s) for s in range(8)}
+    assert len(seen) == 8 and "ok" in seen
     assert binding.status_string(99) == "unknown status"
 
 
