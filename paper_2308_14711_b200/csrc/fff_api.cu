@@ -18,6 +18,7 @@
 #include "kernels/bucket.cuh"
 #include "kernels/common.cuh"
 #include "kernels/descent_warp.cuh"
+#include "kernels/leaf_mma.cuh"
 #include "kernels/leaf_warp.cuh"
 
 namespace {
@@ -47,6 +48,14 @@ struct fff_handle_s {
 
     // library-owned copies of the parameters, caller layout
     void *node_w = nullptr, *node_b = nullptr, *w1 = nullptr, *b1 = nullptr, *w2 = nullptr, *b2 = nullptr;
+
+    // tensor-core leaf path: padded hidden width (0 = shapes not eligible) and pre-swizzled stage images
+    int LP = 0;
+    __nv_bfloat16* w1img = nullptr;
+    float* b1img = nullptr;
+    unsigned char* w2img = nullptr;
+    fff::Tile* ws_tiles = nullptr;
+    int* ws_ntiles = nullptr;
 
     // workspace
     int64_t cap_B = 0;
@@ -112,20 +121,33 @@ void release(fff_handle_s* h) {
     dfree(h->node_w); dfree(h->node_b); dfree(h->w1); dfree(h->b1); dfree(h->w2); dfree(h->b2);
     dfree(h->ws_leaf); dfree(h->ws_perm); dfree(h->ws_offsets); dfree(h->ws_hist[0]); dfree(h->ws_hist[1]);
     dfree(h->d_status); dfree(h->st_x); dfree(h->st_y); dfree(h->st_leaf);
+    dfree(h->w1img); dfree(h->b1img); dfree(h->w2img); dfree(h->ws_tiles); dfree(h->ws_ntiles);
     prof_free(h);
     h->magic = 0;
     delete h;
 }
 
+// Upper bound of the tile list: every non-empty bin ends in at most one partial tile.
+size_t max_tiles(const fff_handle_s* h, int64_t B) {
+    return (size_t)(B / fff::kTM + std::min<int64_t>(h->n_leaves, B) + 1);
+}
+
+bool use_tensor_leaf(const fff_handle_s* h) {
+    if (h->LP == 0 || h->path == FFF_PATH_WARP) return false;
+    return h->path == FFF_PATH_TENSOR || h->l >= 8;
+}
+
 fff_status_t grow_workspace(fff_handle_s* h, int64_t B) {
     if (B <= h->cap_B) return FFF_OK;
     if (cudaDeviceSynchronize() != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
-    dfree(h->ws_leaf); dfree(h->ws_perm);
+    dfree(h->ws_leaf); dfree(h->ws_perm); dfree(h->ws_tiles);
     h->ws_leaf = h->ws_perm = nullptr;
+    h->ws_tiles = nullptr;
     h->cap_B = 0;
     fff_status_t s;
     if ((s = dmalloc((void**)&h->ws_leaf, sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
     if ((s = dmalloc((void**)&h->ws_perm, sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
+    if ((s = dmalloc((void**)&h->ws_tiles, sizeof(fff::Tile) * max_tiles(h, B))) != FFF_OK) return s;
     h->cap_B = B;
     return FFF_OK;
 }
@@ -159,7 +181,8 @@ fff_status_t run_histogram(fff_handle_s* h, const int32_t* keys, int64_t B, cuda
 }
 
 // Consumes the current histogram buffer and flips to the other (already zero) one.
-fff_status_t run_bucket(fff_handle_s* h, const int32_t* keys, int32_t* offsets, int32_t* perm, int64_t B, cudaStream_t st) {
+fff_status_t run_bucket(fff_handle_s* h, const int32_t* keys, int32_t* offsets, int32_t* perm, int64_t B, cudaStream_t st,
+                        bool want_tiles) {
     const int nbins = (int)h->n_leaves;
     int ctas = std::min(nbins, 32);
     int per = (nbins + ctas - 1) / ctas;
@@ -169,7 +192,8 @@ fff_status_t run_bucket(fff_handle_s* h, const int32_t* keys, int32_t* offsets, 
     }
     const size_t smem = sizeof(int) * (size_t)fff::kBucketWarps * per;
     fff::k_bucket<<<ctas, fff::kBucketThreads, smem, st>>>(keys, h->ws_hist[h->hist_cur], h->ws_hist[h->hist_cur ^ 1],
-                                                         offsets, perm, (int)B, nbins, per);
+                                                         offsets, perm, (int)B, nbins, per, want_tiles ? fff::kTM : 0,
+                                                         h->ws_tiles, h->ws_ntiles);
     h->hist_cur ^= 1;
     return launched(h, st, "leaf_bucketing");
 }
@@ -183,6 +207,49 @@ fff_status_t run_leaf(fff_handle_s* h, const void* x, const int32_t* leaf_idx, c
         (const T*)x, leaf_idx, perm, (const T*)h->w1, (const T*)h->b1, (const T*)h->w2, (const T*)h->b2, (T*)y,
         h->D, h->O, h->l, h->act, B, h->vec_ok && aligned16(x));
     return launched(h, st, "grouped_leaf_ff_warp");
+}
+
+template <int LP>
+fff_status_t launch_leaf_mma(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, cudaStream_t st) {
+    using L = fff::LeafMmaLayout<LP>;
+    const int per_sm = std::max(1, std::min(2, (int)((227 * 1024) / (L::kSmemBytes + 1024))));
+    const int64_t grid = std::min<int64_t>((int64_t)h->sm_count * per_sm, (int64_t)max_tiles(h, B));
+    fff::k_leaf_mma<LP><<<(unsigned)grid, fff::kLeafMmaThreads, L::kSmemBytes, st>>>(
+        (const __nv_bfloat16*)x, perm, h->ws_tiles, h->ws_ntiles, h->w1img, h->b1img, h->w2img, (__nv_bfloat16*)y, h->D,
+        h->O, h->act, h->d_status);
+    return launched(h, st, "grouped_leaf_ff_mma");
+}
+
+fff_status_t run_leaf_mma(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, cudaStream_t st) {
+    switch (h->LP) {
+        case 16: return launch_leaf_mma<16>(h, x, perm, y, B, st);
+        case 32: return launch_leaf_mma<32>(h, x, perm, y, B, st);
+        case 64: return launch_leaf_mma<64>(h, x, perm, y, B, st);
+    }
+    return FFF_ERR_UNSUPPORTED;
+}
+
+// Build the pre-swizzled stage images of the tensor-core leaf kernel (once, at creation).
+template <typename T>
+fff_status_t pack_leaf_images(fff_handle_s* h) {
+    const int LP = h->LP, U2 = (h->O + fff::kNC - 1) / fff::kNC;
+    const size_t nl = (size_t)h->n_leaves;
+    const size_t stage2 = (size_t)fff::kNC * LP * 2 + fff::kNC * 4;
+    fff_status_t s;
+    if ((s = dmalloc((void**)&h->w1img, nl * LP * h->D * 2)) != FFF_OK) return s;
+    if ((s = dmalloc((void**)&h->b1img, nl * LP * 4)) != FFF_OK) return s;
+    if ((s = dmalloc((void**)&h->w2img, nl * U2 * stage2)) != FFF_OK) return s;
+    if ((s = dmalloc((void**)&h->ws_ntiles, sizeof(int))) != FFF_OK) return s;
+    cudaMemset(h->ws_ntiles, 0, sizeof(int));
+    const int blocks = h->sm_count * 8;
+    fff::k_pack_w1<T><<<blocks, 256>>>((const T*)h->w1, h->w1img, (int)nl, h->l, LP, h->D);
+    fff::k_pack_b1<T><<<blocks, 256>>>((const T*)h->b1, h->b1img, (int)nl, h->l, LP);
+    fff::k_pack_w2<T><<<blocks, 256>>>((const T*)h->w2, (const T*)h->b2, h->w2img, (int)nl, h->l, LP, h->O);
+    if (cudaGetLastError() != cudaSuccess) return FFF_ERR_CUDA;
+    cudaFuncSetAttribute(fff::k_leaf_mma<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, fff::LeafMmaLayout<16>::kSmemBytes);
+    cudaFuncSetAttribute(fff::k_leaf_mma<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, fff::LeafMmaLayout<32>::kSmemBytes);
+    cudaFuncSetAttribute(fff::k_leaf_mma<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, fff::LeafMmaLayout<64>::kSmemBytes);
+    return cudaGetLastError() == cudaSuccess ? FFF_OK : FFF_ERR_CUDA;
 }
 
 #define FFF_DISPATCH(h, fn, ...) \
@@ -261,7 +328,7 @@ fff_status_t fff_leaf_bucketing_static(const int32_t* leaf_idx, int32_t* offsets
         ctas = (nbins + per - 1) / per;
     }
     fff::k_bucket<<<ctas, fff::kBucketThreads, sizeof(int) * (size_t)fff::kBucketWarps * per, st>>>(
-        leaf_idx, hist, spare, offsets, perm, (int)B, nbins, per);
+        leaf_idx, hist, spare, offsets, perm, (int)B, nbins, per, 0, nullptr, nullptr);
     return cudaGetLastError() == cudaSuccess ? FFF_OK : FFF_ERR_CUDA;
 }
 
@@ -316,6 +383,10 @@ fff_status_t fff_create(fff_handle_t* out, int D, int O, int depth, int leaf_wid
     if (s == FFF_OK) s = clone((void**)&h->ws_hist[0], nullptr, sizeof(int) * nl);
     if (s == FFF_OK) s = clone((void**)&h->ws_hist[1], nullptr, sizeof(int) * nl);
     if (s == FFF_OK) s = clone((void**)&h->d_status, nullptr, sizeof(int));
+    if (s == FFF_OK && dtype == FFF_DTYPE_BF16 && D % fff::kKS == 0 && O % 8 == 0 && leaf_width <= 64) {
+        h->LP = leaf_width <= 16 ? 16 : (leaf_width <= 32 ? 32 : 64);
+        s = pack_leaf_images<__nv_bfloat16>(h);
+    }
     if (s == FFF_OK && cudaDeviceSynchronize() != cudaSuccess) s = (cudaGetLastError(), FFF_ERR_CUDA);
     if (s != FFF_OK) { release(h); return s; }
     {
@@ -347,7 +418,7 @@ fff_status_t fff_reserve(fff_handle_t h, int64_t max_B) {
 fff_status_t fff_set_path(fff_handle_t h, fff_path_t path) {
     if (!live(h)) return FFF_ERR_BAD_HANDLE;
     if (path != FFF_PATH_AUTO && path != FFF_PATH_WARP && path != FFF_PATH_TENSOR) return FFF_ERR_INVALID_ARG;
-    if (path == FFF_PATH_TENSOR) return FFF_ERR_UNSUPPORTED;
+    if (path == FFF_PATH_TENSOR && h->LP == 0) return FFF_ERR_UNSUPPORTED;
     h->path = path;
     return FFF_OK;
 }
@@ -371,7 +442,7 @@ fff_status_t fff_leaf_bucketing(fff_handle_t h, const int32_t* leaf_idx, int32_t
     cudaStream_t st = (cudaStream_t)cuda_stream;
     h->launches = 0;
     if (B > 0 && (s = run_histogram(h, leaf_idx, B, st)) != FFF_OK) return s;
-    return run_bucket(h, leaf_idx, offsets, perm, B, st);
+    return run_bucket(h, leaf_idx, offsets, perm, B, st, false);
 }
 
 fff_status_t fff_grouped_leaf_ff(fff_handle_t h, const void* x, const int32_t* leaf_idx, const int32_t* offsets,
@@ -382,7 +453,15 @@ fff_status_t fff_grouped_leaf_ff(fff_handle_t h, const void* x, const int32_t* l
     if (!x || !y || !leaf_idx || !offsets || !perm || !aligned16(x) || !aligned16(y)) return FFF_ERR_INVALID_ARG;
     DeviceGuard g(h->device);
     h->launches = 0;
-    return FFF_DISPATCH(h, run_leaf, h, x, leaf_idx, perm, y, B, (cudaStream_t)cuda_stream);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (use_tensor_leaf(h)) {
+        if ((s = grow_workspace(h, B)) != FFF_OK) return s;
+        fff::k_tiles_from_offsets<<<1, fff::kBucketThreads, 0, st>>>(offsets, (int)h->n_leaves, fff::kTM, h->ws_tiles,
+                                                                     h->ws_ntiles);
+        if ((s = launched(h, st, "tiles_from_offsets")) != FFF_OK) return s;
+        return run_leaf_mma(h, x, perm, y, B, st);
+    }
+    return FFF_DISPATCH(h, run_leaf, h, x, leaf_idx, perm, y, B, st);
 }
 
 fff_status_t fff_forward_infer(fff_handle_t h, const void* x, void* y, int32_t* leaf_idx, int64_t B, void* cuda_stream) {
@@ -400,8 +479,10 @@ fff_status_t fff_forward_infer(fff_handle_t h, const void* x, void* y, int32_t* 
     if (h->prof_active)
         cudaEventRecord(h->prof_events[(size_t)h->prof_steps * (fff_handle_s::kMaxProfLaunches + 1)], st);
     s = FFF_DISPATCH(h, run_descent, h, x, leaf, h->ws_hist[h->hist_cur], B, st);
-    if (s == FFF_OK) s = run_bucket(h, leaf, h->ws_offsets, h->ws_perm, B, st);
-    if (s == FFF_OK) s = FFF_DISPATCH(h, run_leaf, h, x, leaf, h->ws_perm, y, B, st);
+    const bool tensor_leaf = use_tensor_leaf(h);
+    if (s == FFF_OK) s = run_bucket(h, leaf, h->ws_offsets, h->ws_perm, B, st, tensor_leaf);
+    if (s == FFF_OK)
+        s = tensor_leaf ? run_leaf_mma(h, x, h->ws_perm, y, B, st) : FFF_DISPATCH(h, run_leaf, h, x, leaf, h->ws_perm, y, B, st);
     if (h->prof_active) {
         h->prof_active = false;
         if (s == FFF_OK && (h->prof_steps == 0 || h->prof_nlaunch == h->launches)) {

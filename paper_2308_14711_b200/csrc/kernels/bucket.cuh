@@ -43,16 +43,57 @@ k_histogram(const int32_t* __restrict__ keys, int* __restrict__ hist, int64_t B,
     }
 }
 
+// Sum over the block; every thread returns the total.  s_warp: kBucketWarps ints of scratch.
+__device__ __forceinline__ int block_sum(int v, int* s_warp)
+{
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFullMask, v, o);
+    __syncthreads();
+    if (lane == 0) s_warp[w] = v;
+    __syncthreads();
+    int t = s_warp[lane];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(kFullMask, t, o);
+    return t;
+}
+
+// Exclusive prefix sum over the block in thread order.  s_warp: kBucketWarps ints of scratch.
+__device__ __forceinline__ int block_exclusive_scan(int v, int* s_warp)
+{
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int u = __shfl_up_sync(kFullMask, incl, o);
+        if (lane >= o) incl += u;
+    }
+    __syncthreads();
+    if (lane == 31) s_warp[w] = incl;
+    __syncthreads();
+    int ws = s_warp[lane];                     // lane i holds the total of warp i
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int u = __shfl_up_sync(kFullMask, ws, o);
+        if (lane >= o) ws += u;
+    }
+    const int before = __shfl_sync(kFullMask, ws, max(w - 1, 0));
+    return (w > 0 ? before : 0) + incl - v;
+}
+
 // hist: complete histogram of keys.  hist_next: a second histogram buffer that
 // is cleared here for the following call (nobody reads it during this kernel).
+// tile_rows > 0 additionally writes the tile list of the grouped kernels: the
+// tiles of bin 0 first, each bin cut into ceil(count / tile_rows) tiles, and
+// their number into *n_tiles.
 // Dynamic shared memory: kBucketWarps * bins_per_cta ints.
 __global__ void __launch_bounds__(kBucketThreads)
 k_bucket(const int32_t* __restrict__ keys, const int* __restrict__ hist, int* __restrict__ hist_next,
-         int32_t* __restrict__ offsets, int32_t* __restrict__ perm, int B, int nbins, int bins_per_cta)
+         int32_t* __restrict__ offsets, int32_t* __restrict__ perm, int B, int nbins, int bins_per_cta,
+         int tile_rows, Tile* __restrict__ tiles, int* __restrict__ n_tiles)
 {
     extern __shared__ int s_cnt[];                 // [kBucketWarps][bins_per_cta]
     __shared__ int s_warp[kBucketWarps];
-    __shared__ int s_base;
 
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     const int lo = blockIdx.x * bins_per_cta;
@@ -62,20 +103,15 @@ k_bucket(const int32_t* __restrict__ keys, const int* __restrict__ hist, int* __
 
     for (int i = tid; i < kBucketWarps * nb; i += kBucketThreads) s_cnt[i] = 0;
 
-    // tokens in bins below this CTA's range
-    int part = 0;
-    for (int i = tid; i < lo; i += kBucketThreads) part += hist[i];
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(kFullMask, part, o);
-    if (lane == 0) s_warp[w] = part;
-    __syncthreads();
-    if (w == 0) {
-        int v = s_warp[lane];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFullMask, v, o);
-        if (lane == 0) s_base = v;
+    // tokens (and tiles) in bins below this CTA's range
+    int part = 0, tpart = 0;
+    for (int i = tid; i < lo; i += kBucketThreads) {
+        const int c = hist[i];
+        part += c;
+        if (tile_rows > 0) tpart += (c + tile_rows - 1) / tile_rows;
     }
-    __syncthreads();
+    const int base = block_sum(part, s_warp);
+    const int tile_base = tile_rows > 0 ? block_sum(tpart, s_warp) : 0;
 
     // token slice of this warp (a multiple of 32 so that steps never straddle slices)
     const int chunk = (((B + kBucketWarps - 1) / kBucketWarps) + 31) & ~31;
@@ -93,30 +129,13 @@ k_bucket(const int32_t* __restrict__ keys, const int* __restrict__ hist, int* __
     }
     __syncthreads();
 
-    // scan: first output position of every bin, then of every (warp, bin)
+    // scan: first output position of every bin, then of every (warp, bin); tile list
     {
         const int b = lo + tid;
-        const int c = (tid < nb && b < hi) ? hist[b] : 0;
-        int incl = c;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int v = __shfl_up_sync(kFullMask, incl, o);
-            if (lane >= o) incl += v;
-        }
-        if (lane == 31) s_warp[w] = incl;
-        __syncthreads();
-        if (w == 0) {
-            int v = s_warp[lane];
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int u = __shfl_up_sync(kFullMask, v, o);
-                if (lane >= o) v += u;
-            }
-            s_warp[lane] = v;                       // inclusive over warps
-        }
-        __syncthreads();
-        const int start = s_base + (w > 0 ? s_warp[w - 1] : 0) + incl - c;
-        if (tid < nb && b < hi) {
+        const bool mine = tid < nb && b < hi;
+        const int c = mine ? hist[b] : 0;
+        const int start = base + block_exclusive_scan(c, s_warp);
+        if (mine) {
             offsets[b] = start;
             if (b == nbins - 1) offsets[nbins] = start + c;
             int run = start;
@@ -126,6 +145,21 @@ k_bucket(const int32_t* __restrict__ keys, const int* __restrict__ hist, int* __
                 run += c2;
             }
             hist_next[b] = 0;
+        }
+        if (tile_rows > 0) {
+            const int nt = (c + tile_rows - 1) / tile_rows;
+            const int t0 = tile_base + block_exclusive_scan(nt, s_warp);
+            if (mine) {
+                for (int i = 0; i < nt; ++i) {
+                    Tile tl;
+                    tl.bin = b;
+                    tl.start = start + i * tile_rows;
+                    tl.rows = min(tile_rows, c - i * tile_rows);
+                    tl.pad = 0;
+                    tiles[t0 + i] = tl;
+                }
+                if (b == nbins - 1) *n_tiles = t0 + nt;
+            }
         }
     }
     __syncthreads();
@@ -146,6 +180,32 @@ k_bucket(const int32_t* __restrict__ keys, const int* __restrict__ hist, int* __
         if (in) perm[pos + __popc(peers & ((1u << lane) - 1u))] = t;
         __syncwarp();
     }
+}
+
+// Tile list from an existing offsets array (one CTA; used when the caller supplies the bucketing).
+__global__ void __launch_bounds__(kBucketThreads)
+k_tiles_from_offsets(const int32_t* __restrict__ offsets, int nbins, int tile_rows, Tile* __restrict__ tiles,
+                     int* __restrict__ n_tiles)
+{
+    __shared__ int s_warp[kBucketWarps];
+    int tile_base = 0;
+    for (int b0 = 0; b0 < nbins; b0 += kBucketThreads) {
+        const int b = b0 + threadIdx.x;
+        const int start = b < nbins ? offsets[b] : 0;
+        const int c = b < nbins ? offsets[b + 1] - start : 0;
+        const int nt = (c + tile_rows - 1) / tile_rows;
+        const int t0 = tile_base + block_exclusive_scan(nt, s_warp);
+        for (int i = 0; i < nt; ++i) {
+            Tile tl;
+            tl.bin = b;
+            tl.start = start + i * tile_rows;
+            tl.rows = min(tile_rows, c - i * tile_rows);
+            tl.pad = 0;
+            tiles[t0 + i] = tl;
+        }
+        tile_base += block_sum(nt, s_warp);
+    }
+    if (threadIdx.x == 0) *n_tiles = tile_base;
 }
 
 }  // namespace fff

@@ -14,6 +14,12 @@ enum : int { kActRelu = 0, kActGelu = 1 };
 // Values written to the per-handle device status word by kernels.
 enum : int { kDevOk = 0, kDevTimeout = 1 };
 
+// A tile of the grouped kernels: up to a fixed number of consecutive perm entries of one bin
+// (a leaf, or a node position during a staged descent).
+struct Tile {
+    int bin, start, rows, pad;
+};
+
 template <typename T> struct Elem;
 
 template <> struct Elem<float> {

@@ -1,0 +1,302 @@
+// Grouped leaf evaluation on tensor cores (bf16, float32 accumulate) with un-permuting write-back.
+//
+// Algorithm 1, FORWARD_I, leaf branch, for the tokens of one bucket at a time:
+//     H = act(X[T_j] W1_j^T + b1_j)        [|T_j|, l]     (GEMM1, K = D)
+//     Y = H W2_j^T + b2_j                  [|T_j|, O]     (GEMM2, K = l)
+// and row i of Y is stored at the original position of token T_j[i].
+//
+// Work unit: a tile = up to kTM consecutive entries of one bucket.  CTAs are persistent and walk the
+// device-built tile list with a static stride.  Inside a CTA one producer warp streams operands into
+// a ring of shared-memory stages with 1-D bulk (TMA) copies that complete on mbarriers; kTM/16
+// consumer warps each own 16 token rows and run both GEMMs with mma.sync.m16n8k16, keeping H in
+// registers between them (the accumulator fragment of GEMM1 is the A fragment of GEMM2).
+//
+// Ring contents, in order, per tile:
+//   D/kKS   GEMM1 stages: kKS columns of the gathered token rows (one bulk copy per row, rows padded
+//           by 16 bytes in shared memory so that ldmatrix is conflict-free) + the matching slice of
+//           W1_j (one bulk copy of a pre-swizzled image);
+//   O/kNC   GEMM2 stages: kNC rows of W2_j (pre-swizzled image) followed by their float32 biases.
+// The images are written once at handle creation (repack kernels below).
+//
+// Requirements: bf16, D % kKS == 0, O % 8 == 0, l <= 64 (padded to kLP in {16, 32, 64} with zero
+// weights: act(0) * 0 contributes nothing).
+#pragma once
+
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace fff {
+
+constexpr int kTM = 64;          // token rows per tile
+constexpr int kKS = 128;         // K columns per GEMM1 stage
+constexpr int kNC = 256;         // output columns per GEMM2 stage
+constexpr int kStages = 3;
+constexpr int kLeafMmaConsumers = kTM / 16;
+constexpr int kLeafMmaThreads = (kLeafMmaConsumers + 1) * 32;
+constexpr int kXRowBytes = kKS * 2 + 16;                    // padded row of a GEMM1 stage
+constexpr int kOutHalf = 128;                               // outputs accumulated at once per warp
+constexpr int kOutRowBytes = kOutHalf * 2 + 16;             // padded row of the store staging buffer
+
+template <int LP> struct LeafMmaLayout {
+    static constexpr int kW1StageBytes = LP * kKS * 2;
+    static constexpr int kStage1Bytes = kTM * kXRowBytes + kW1StageBytes;
+    static constexpr int kW2Bytes = kNC * LP * 2;
+    static constexpr int kStage2Bytes = kW2Bytes + kNC * 4;             // weights + float32 biases
+    static constexpr int kStageBytes = kStage1Bytes > kStage2Bytes ? kStage1Bytes : kStage2Bytes;
+    static constexpr int kStageStride = (kStageBytes + 127) & ~127;
+    static constexpr int kStagingBytes = kLeafMmaConsumers * 16 * kOutRowBytes;
+    static constexpr int kSmemBytes = kStages * kStageStride + kStagingBytes + 128 /* barriers */ + 128 /* align */;
+};
+
+// ---- one-time repacking of the leaf parameters into stage images --------------------------------
+
+// W1 image: [leaf][D/kKS stages][kKS/64 sub-blocks][LP rows][64 columns], 128-byte swizzled.
+template <typename T>
+__global__ void k_pack_w1(const T* __restrict__ w1, __nv_bfloat16* __restrict__ img, int n_leaves, int l, int LP, int D)
+{
+    const int64_t total = (int64_t)n_leaves * LP * D;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int k = (int)(i % D);
+        const int n = (int)((i / D) % LP);
+        const int64_t j = i / ((int64_t)D * LP);
+        const int u = k / kKS, sb = (k % kKS) / 64, kc = k % 64;
+        const uint32_t off = ptx::swz128((uint32_t)((sb * LP + n) * 128 + kc * 2));
+        const int64_t base = (j * (D / kKS) + u) * (int64_t)(LP * kKS);          // elements
+        const float v = n < l ? Elem<T>::to_float(w1[(j * l + n) * (int64_t)D + k]) : 0.0f;
+        img[base + off / 2] = __float2bfloat16_rn(v);
+    }
+}
+
+// W2 image: [leaf][ceil(O/kNC) stages]{ [kNC rows][LP columns] 128-byte swizzled, then kNC float32 biases }.
+template <typename T>
+__global__ void k_pack_w2(const T* __restrict__ w2, const T* __restrict__ b2, unsigned char* __restrict__ img,
+                          int n_leaves, int l, int LP, int O)
+{
+    const int U2 = (O + kNC - 1) / kNC;
+    const int64_t stage_bytes = (int64_t)kNC * LP * 2 + kNC * 4;
+    const int64_t total = (int64_t)n_leaves * U2 * kNC * (LP + 1);       // LP weights + 1 bias per row
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int c = (int)(i % (LP + 1));
+        const int n = (int)((i / (LP + 1)) % kNC);
+        const int64_t ju = i / ((int64_t)(LP + 1) * kNC);                  // leaf * U2 + stage
+        const int64_t j = ju / U2;
+        const int o = (int)(ju % U2) * kNC + n;
+        unsigned char* st = img + ju * stage_bytes;
+        if (c < LP) {
+            const float v = (o < O && c < l) ? Elem<T>::to_float(w2[(j * O + o) * (int64_t)l + c]) : 0.0f;
+            const uint32_t off = ptx::swz128((uint32_t)(n * LP * 2 + c * 2));
+            *reinterpret_cast<__nv_bfloat16*>(st + off) = __float2bfloat16_rn(v);
+        } else {
+            reinterpret_cast<float*>(st + (int64_t)kNC * LP * 2)[n] = o < O ? Elem<T>::to_float(b2[j * O + o]) : 0.0f;
+        }
+    }
+}
+
+// b1 image: [leaf][LP] float32, zero beyond l.
+template <typename T>
+__global__ void k_pack_b1(const T* __restrict__ b1, float* __restrict__ img, int n_leaves, int l, int LP)
+{
+    const int64_t total = (int64_t)n_leaves * LP;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int n = (int)(i % LP);
+        const int64_t j = i / LP;
+        img[i] = n < l ? Elem<T>::to_float(b1[j * l + n]) : 0.0f;
+    }
+}
+
+// ---- the kernel ------------------------------------------------------------------------------------
+
+template <int LP>
+__global__ void __launch_bounds__(kLeafMmaThreads)
+k_leaf_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ perm,
+           const Tile* __restrict__ tiles, const int* __restrict__ n_tiles,
+           const __nv_bfloat16* __restrict__ w1img, const float* __restrict__ b1img,
+           const unsigned char* __restrict__ w2img, __nv_bfloat16* __restrict__ y,
+           int D, int O, int act, int* __restrict__ status)
+{
+    using L = LeafMmaLayout<LP>;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+    unsigned char* stages = smem;
+    unsigned char* staging = smem + kStages * L::kStageStride;
+    uint64_t* full = reinterpret_cast<uint64_t*>(staging + L::kStagingBytes);
+    uint64_t* empty = full + kStages;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int U1 = D / kKS;
+    const int U2 = (O + kNC - 1) / kNC;
+    const int ntiles = *n_tiles;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            ptx::mbar_init(full + s, 1);
+            ptx::mbar_init(empty + s, kLeafMmaConsumers);
+        }
+        ptx::fence_mbar_init();
+    }
+    __syncthreads();
+
+    int stage = 0;
+    uint32_t phase = 0;
+    bool timed_out = false;
+
+    if (warp == kLeafMmaConsumers) {
+        // ------------------------------------------------------------------ producer warp
+        for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+            const Tile tl = tiles[tile];
+            int64_t tok[kTM / 32];
+#pragma unroll
+            for (int q = 0; q < kTM / 32; ++q) {
+                const int r = q * 32 + lane;
+                tok[q] = r < tl.rows ? perm[tl.start + r] : 0;
+            }
+            for (int u = 0; u < U1; ++u) {
+                if (!timed_out && !ptx::mbar_wait(empty + stage, phase ^ 1)) timed_out = true;
+                unsigned char* st = stages + stage * L::kStageStride;
+                if (lane == 0) {
+                    ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)(tl.rows * kKS * 2 + L::kW1StageBytes));
+                    ptx::bulk_g2s(st + kTM * kXRowBytes, w1img + ((int64_t)tl.bin * U1 + u) * (LP * kKS),
+                                  L::kW1StageBytes, full + stage);
+                }
+                __syncwarp();
+#pragma unroll
+                for (int q = 0; q < kTM / 32; ++q) {
+                    const int r = q * 32 + lane;
+                    if (r < tl.rows) ptx::bulk_g2s(st + r * kXRowBytes, x + tok[q] * D + u * kKS, kKS * 2, full + stage);
+                }
+                if (++stage == kStages) { stage = 0; phase ^= 1; }
+            }
+            for (int u = 0; u < U2; ++u) {
+                if (!timed_out && !ptx::mbar_wait(empty + stage, phase ^ 1)) timed_out = true;
+                if (lane == 0) {
+                    ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)L::kStage2Bytes);
+                    ptx::bulk_g2s(stages + stage * L::kStageStride,
+                                  w2img + ((int64_t)tl.bin * U2 + u) * L::kStage2Bytes, L::kStage2Bytes, full + stage);
+                }
+                __syncwarp();
+                if (++stage == kStages) { stage = 0; phase ^= 1; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ consumer warps
+        const int m0 = warp * 16;
+        unsigned char* my_staging = staging + warp * 16 * kOutRowBytes;
+        const int g = lane >> 2, q4 = lane & 3;
+        for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+            const Tile tl = tiles[tile];
+            const bool active = m0 < tl.rows;          // warps without valid rows only keep the ring moving
+
+            // GEMM1: acc1[nt] = X[m0..m0+16) . W1[nt*8 .. nt*8+8)^T
+            float acc1[LP / 8][4];
+#pragma unroll
+            for (int nt = 0; nt < LP / 8; ++nt)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) acc1[nt][c] = 0.0f;
+
+            for (int u = 0; u < U1; ++u) {
+                if (!timed_out && !ptx::mbar_wait(full + stage, phase)) timed_out = true;
+                if (active) {
+                    const uint32_t xs = ptx::smem_addr(stages + stage * L::kStageStride);
+                    const uint32_t ws = xs + kTM * kXRowBytes;
+                    const uint32_t a_base = xs + (m0 + (lane & 15)) * kXRowBytes + (lane >> 4) * 16;
+                    const int bn = (lane & 7) + ((lane >> 4) << 3);
+                    const int bk = ((lane >> 3) & 1) * 8;
+#pragma unroll
+                    for (int ks = 0; ks < kKS / 16; ++ks) {
+                        uint32_t a0, a1, a2, a3;
+                        ptx::ldmatrix_x4(a_base + ks * 32, a0, a1, a2, a3);
+                        const int kcol = ks * 16 + bk;
+                        const int sb = kcol >> 6, kc = kcol & 63;
+#pragma unroll
+                        for (int np = 0; np < LP / 16; ++np) {
+                            const int n = np * 16 + bn;
+                            uint32_t b0, b1, b2, b3;
+                            ptx::ldmatrix_x4(ws + ptx::swz128((uint32_t)((sb * LP + n) * 128 + kc * 2)), b0, b1, b2, b3);
+                            ptx::mma_bf16(acc1[2 * np], a0, a1, a2, a3, b0, b1);
+                            ptx::mma_bf16(acc1[2 * np + 1], a0, a1, a2, a3, b2, b3);
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(empty + stage);
+                if (++stage == kStages) { stage = 0; phase ^= 1; }
+            }
+
+            // bias + activation; H stays in registers as the A operand of GEMM2
+            uint32_t hA[LP / 8][2];
+            {
+                const float* b1p = b1img + (int64_t)tl.bin * LP;
+#pragma unroll
+                for (int nt = 0; nt < LP / 8; ++nt) {
+                    const float2 b = __ldg(reinterpret_cast<const float2*>(b1p + nt * 8 + 2 * q4));
+                    hA[nt][0] = ptx::pack_bf16(activate(act, acc1[nt][0] + b.x), activate(act, acc1[nt][1] + b.y));
+                    hA[nt][1] = ptx::pack_bf16(activate(act, acc1[nt][2] + b.x), activate(act, acc1[nt][3] + b.y));
+                }
+            }
+
+            // GEMM2 + bias + store
+            for (int u = 0; u < U2; ++u) {
+                if (!timed_out && !ptx::mbar_wait(full + stage, phase)) timed_out = true;
+                if (active) {
+                    const unsigned char* st = stages + stage * L::kStageStride;
+                    const uint32_t ws = ptx::smem_addr(st);
+                    const float* bias = reinterpret_cast<const float*>(st + L::kW2Bytes);
+                    const int bn = (lane & 7) + ((lane >> 4) << 3);
+                    const int bk = ((lane >> 3) & 1) * 8;
+#pragma unroll 1
+                    for (int half = 0; half < kNC / kOutHalf; ++half) {
+                        const int o_base = u * kNC + half * kOutHalf;
+                        if (o_base >= O) break;
+                        float acc2[kOutHalf / 8][4];
+#pragma unroll
+                        for (int nt = 0; nt < kOutHalf / 8; ++nt)
+#pragma unroll
+                            for (int c = 0; c < 4; ++c) acc2[nt][c] = 0.0f;
+#pragma unroll
+                        for (int np = 0; np < kOutHalf / 16; ++np) {
+                            const int n = half * kOutHalf + np * 16 + bn;
+#pragma unroll
+                            for (int kk = 0; kk < LP / 16; ++kk) {
+                                uint32_t b0, b1, b2, b3;
+                                ptx::ldmatrix_x4(ws + ptx::swz128((uint32_t)(n * LP * 2 + (kk * 16 + bk) * 2)), b0, b1, b2, b3);
+                                ptx::mma_bf16(acc2[2 * np], hA[2 * kk][0], hA[2 * kk][1], hA[2 * kk + 1][0], hA[2 * kk + 1][1], b0, b1);
+                                ptx::mma_bf16(acc2[2 * np + 1], hA[2 * kk][0], hA[2 * kk][1], hA[2 * kk + 1][0], hA[2 * kk + 1][1], b2, b3);
+                            }
+                        }
+                        // fragments -> padded staging rows (bf16), then whole 16-byte units to y
+#pragma unroll
+                        for (int nt = 0; nt < kOutHalf / 8; ++nt) {
+                            const float2 b = *reinterpret_cast<const float2*>(bias + half * kOutHalf + nt * 8 + 2 * q4);
+                            *reinterpret_cast<uint32_t*>(my_staging + g * kOutRowBytes + nt * 16 + q4 * 4) =
+                                ptx::pack_bf16(acc2[nt][0] + b.x, acc2[nt][1] + b.y);
+                            *reinterpret_cast<uint32_t*>(my_staging + (g + 8) * kOutRowBytes + nt * 16 + q4 * 4) =
+                                ptx::pack_bf16(acc2[nt][2] + b.x, acc2[nt][3] + b.y);
+                        }
+                        __syncwarp();
+#pragma unroll
+                        for (int it = 0; it < 8; ++it) {
+                            const int r = it * 2 + (lane >> 4);
+                            const int unit = lane & 15;
+                            const int o = o_base + unit * 8;
+                            if (m0 + r < tl.rows && o < O) {
+                                const int64_t t = perm[tl.start + m0 + r];
+                                const uint4 v = *reinterpret_cast<const uint4*>(my_staging + r * kOutRowBytes + unit * 16);
+                                __stcs(reinterpret_cast<uint4*>(y + t * O + o), v);
+                            }
+                        }
+                        __syncwarp();
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(empty + stage);
+                if (++stage == kStages) { stage = 0; phase ^= 1; }
+            }
+        }
+    }
+    if (timed_out) {
+        if (lane == 0) atomicExch(status, kDevTimeout);
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);     // let bulk copies still in flight land before exit
+    }
+}
+
+}  // namespace fff

@@ -16,7 +16,18 @@ from tests import util
 
 pytestmark = pytest.mark.gpu
 
-PATHS = ["auto", "warp"]
+PATHS = ["auto", "warp", "tensor"]
+
+
+def layer_on_path(case, path):
+    """Layer pinned to a kernel family; skips when the shapes cannot run on it."""
+    from paper_2308_14711_b200.binding import FFFError
+    try:
+        return util.make_layer(case, path)
+    except FFFError as e:
+        if e.status == 2:
+            pytest.skip(f"{case.cfg.name}: shapes not eligible for the {path} path")
+        raise
 
 
 def small_cfgs():
@@ -50,7 +61,7 @@ def small_case(request):
 def test_forward_matches_oracle_elementwise(small_case, path):
     case, y_ref, leaf_ref = small_case
     cfg = case.cfg
-    layer = util.make_layer(case, path)
+    layer = layer_on_path(case, path)
     x = util.to_device(case.x, cfg.dtype)
     y, leaf = layer.forward_infer(x)
     torch.cuda.synchronize()
@@ -73,7 +84,7 @@ def test_forward_matches_oracle_elementwise(small_case, path):
 def test_stage_entry_points_match_oracle(small_case, path):
     case, y_ref, leaf_ref = small_case
     cfg = case.cfg
-    layer = util.make_layer(case, path)
+    layer = layer_on_path(case, path)
     x = util.to_device(case.x, cfg.dtype)
     leaf = layer.tree_descent(x)
     np.testing.assert_array_equal(leaf.cpu().numpy(), leaf_ref)
