@@ -60,6 +60,8 @@ struct fff_handle_s {
     // workspace
     int64_t cap_B = 0;
     int32_t *ws_leaf = nullptr, *ws_perm = nullptr, *ws_offsets = nullptr;
+    int32_t* ws_rank = nullptr;   // per-token rank scratch of the bucketing kernel (large batches only)
+    int max_bucket_clusters = 8;
     int *ws_hist[2] = {nullptr, nullptr};
     int hist_cur = 0;
     int *d_status = nullptr;
@@ -121,7 +123,7 @@ void release(fff_handle_s* h) {
     dfree(h->node_w); dfree(h->node_b); dfree(h->w1); dfree(h->b1); dfree(h->w2); dfree(h->b2);
     dfree(h->ws_leaf); dfree(h->ws_perm); dfree(h->ws_offsets); dfree(h->ws_hist[0]); dfree(h->ws_hist[1]);
     dfree(h->d_status); dfree(h->st_x); dfree(h->st_y); dfree(h->st_leaf);
-    dfree(h->w1img); dfree(h->b1img); dfree(h->w2img); dfree(h->ws_tiles); dfree(h->ws_ntiles);
+    dfree(h->w1img); dfree(h->b1img); dfree(h->w2img); dfree(h->ws_tiles); dfree(h->ws_ntiles); dfree(h->ws_rank);
     prof_free(h);
     h->magic = 0;
     delete h;
@@ -140,13 +142,14 @@ bool use_tensor_leaf(const fff_handle_s* h) {
 fff_status_t grow_workspace(fff_handle_s* h, int64_t B) {
     if (B <= h->cap_B) return FFF_OK;
     if (cudaDeviceSynchronize() != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
-    dfree(h->ws_leaf); dfree(h->ws_perm); dfree(h->ws_tiles);
-    h->ws_leaf = h->ws_perm = nullptr;
+    dfree(h->ws_leaf); dfree(h->ws_perm); dfree(h->ws_tiles); dfree(h->ws_rank);
+    h->ws_leaf = h->ws_perm = h->ws_rank = nullptr;
     h->ws_tiles = nullptr;
     h->cap_B = 0;
     fff_status_t s;
     if ((s = dmalloc((void**)&h->ws_leaf, sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
     if ((s = dmalloc((void**)&h->ws_perm, sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
+    if ((s = dmalloc((void**)&h->ws_rank, sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
     if ((s = dmalloc((void**)&h->ws_tiles, sizeof(fff::Tile) * max_tiles(h, B))) != FFF_OK) return s;
     h->cap_B = B;
     return FFF_OK;
@@ -184,16 +187,36 @@ fff_status_t run_histogram(fff_handle_s* h, const int32_t* keys, int64_t B, cuda
 fff_status_t run_bucket(fff_handle_s* h, const int32_t* keys, int32_t* offsets, int32_t* perm, int64_t B, cudaStream_t st,
                         bool want_tiles) {
     const int nbins = (int)h->n_leaves;
-    int ctas = std::min(nbins, 32);
-    int per = (nbins + ctas - 1) / ctas;
-    if (per > fff::kBucketMaxBinsPerCta) {
-        per = fff::kBucketMaxBinsPerCta;
-        ctas = (nbins + per - 1) / per;
-    }
-    const size_t smem = sizeof(int) * (size_t)fff::kBucketWarps * per;
-    fff::k_bucket<<<ctas, fff::kBucketThreads, smem, st>>>(keys, h->ws_hist[h->hist_cur], h->ws_hist[h->hist_cur ^ 1],
-                                                         offsets, perm, (int)B, nbins, per, want_tiles ? fff::kTM : 0,
-                                                         h->ws_tiles, h->ws_ntiles);
+    // Every cluster reads all keys, so more clusters do not shorten the kernel; they only shrink the bin
+    // range (and the number of ballots per step).  All clusters should be resident at once.
+    int clusters = std::max(1, std::min(std::min(nbins / 32, 8), h->max_bucket_clusters));
+    int per = (nbins + clusters - 1) / clusters;
+    if (per > fff::kBucketMaxBinsPerCta) per = fff::kBucketMaxBinsPerCta;
+    clusters = (nbins + per - 1) / per;
+    int bin_bits = 0;
+    while ((1 << bin_bits) < per) ++bin_bits;
+    const bool in_regs = B <= (int64_t)fff::kBucketClusterSize * fff::kBucketWarps * 32 * fff::kBucketKeyRegs;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(clusters * fff::kBucketClusterSize));
+    cfg.blockDim = dim3(fff::kBucketThreads);
+    cfg.dynamicSmemBytes = sizeof(int) * (size_t)(fff::kBucketWarps + 1) * per;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = fff::kBucketClusterSize;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const int* hist = h->ws_hist[h->hist_cur];
+    int* hist_next = h->ws_hist[h->hist_cur ^ 1];
+    const int tile_rows = want_tiles ? (int)fff::kTM : 0;
+    cudaError_t e = in_regs
+        ? cudaLaunchKernelEx(&cfg, fff::k_bucket_cluster<true>, keys, hist, hist_next, offsets, perm, (int)B, nbins, per,
+                             tile_rows, h->ws_tiles, h->ws_ntiles, bin_bits, h->ws_rank)
+        : cudaLaunchKernelEx(&cfg, fff::k_bucket_cluster<false>, keys, hist, hist_next, offsets, perm, (int)B, nbins, per,
+                             tile_rows, h->ws_tiles, h->ws_ntiles, bin_bits, h->ws_rank);
+    if (e != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
     h->hist_cur ^= 1;
     return launched(h, st, "leaf_bucketing");
 }
@@ -363,8 +386,27 @@ fff_status_t fff_create(fff_handle_t* out, int D, int O, int depth, int leaf_wid
     if (!h) return FFF_ERR_ALLOC;
     if (cudaGetDevice(&h->device) != cudaSuccess) { delete h; return cudaGetLastError(), FFF_ERR_CUDA; }
     cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device);
-    cudaFuncSetAttribute(fff::k_bucket, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                         (int)(sizeof(int) * fff::kBucketWarps * fff::kBucketMaxBinsPerCta));
+    {
+        const int smem_max = (int)(sizeof(int) * (fff::kBucketWarps + 1) * fff::kBucketMaxBinsPerCta);
+        cudaFuncSetAttribute(fff::k_bucket_cluster<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max);
+        cudaFuncSetAttribute(fff::k_bucket_cluster<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(fff::kBucketClusterSize);
+        cfg.blockDim = dim3(fff::kBucketThreads);
+        cfg.dynamicSmemBytes = 4096;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = fff::kBucketClusterSize;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, fff::k_bucket_cluster<true>, &cfg) == cudaSuccess && n > 0)
+            h->max_bucket_clusters = n;
+        else
+            cudaGetLastError();
+    }
     h->D = D; h->O = O; h->depth = depth; h->l = leaf_width; h->act = act; h->dtype = dtype;
     h->esize = dtype == FFF_DTYPE_F32 ? 4 : 2;
     h->n_nodes = ((int64_t)1 << depth) - 1;
@@ -439,6 +481,7 @@ fff_status_t fff_leaf_bucketing(fff_handle_t h, const int32_t* leaf_idx, int32_t
     if (s != FFF_OK) return s;
     if (!offsets || (B > 0 && (!leaf_idx || !perm))) return FFF_ERR_INVALID_ARG;
     DeviceGuard g(h->device);
+    if ((s = grow_workspace(h, B)) != FFF_OK) return s;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     h->launches = 0;
     if (B > 0 && (s = run_histogram(h, leaf_idx, B, st)) != FFF_OK) return s;

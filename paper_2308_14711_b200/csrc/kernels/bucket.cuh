@@ -18,6 +18,8 @@
 //   pass 2  each warp re-reads its slice in order and writes perm.
 #pragma once
 
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 
 namespace fff {
@@ -180,6 +182,170 @@ k_bucket(const int32_t* __restrict__ keys, const int* __restrict__ hist, int* __
         if (in) perm[pos + __popc(peers & ((1u << lane) - 1u))] = t;
         __syncwarp();
     }
+}
+
+// ---- cluster version ---------------------------------------------------------------------------
+// Same result as k_bucket, shorter critical path: the token ids are split over the 8 CTAs of a
+// thread-block cluster (256 warp slices instead of 32), the cluster as a whole owns one range of
+// bins, and the per-CTA column totals are exchanged through distributed shared memory.  Each warp
+// loads the keys of its slice in blocks of kBucketKeyRegs independent loads before it touches
+// shared memory, so the slice costs a few memory latencies instead of one per 32 tokens.
+// Lanes holding the same value v (only the low nbits bits may differ) among the lanes with `in` set;
+// built from one ballot per bit, which is far cheaper than the match instruction when a whole SM
+// issues it at once.  The result is only meaningful for lanes with `in` set.
+__device__ __forceinline__ unsigned peers_by_ballot(bool in, int v, int nbits)
+{
+    unsigned peers = __ballot_sync(kFullMask, in);
+    for (int bit = 0; bit < nbits; ++bit) {
+        const bool one = (v >> bit) & 1;
+        const unsigned m = __ballot_sync(kFullMask, one);
+        peers &= one ? m : ~m;
+    }
+    return peers;
+}
+
+constexpr int kBucketClusterSize = 8;
+constexpr int kBucketKeyRegs = 8;
+
+// Each warp makes ONE matching pass over its slice: it records, per token, the rank among the
+// earlier tokens of the same bin inside the slice (in registers when the slice fits kBucketKeyRegs
+// steps, else in `rank_tmp`, B ints of global scratch), and the per-(warp, bin) counts.  After the
+// counts have been turned into absolute start positions, a second, trivial pass writes perm.
+// Dynamic shared memory: (kBucketWarps + 1) * bins_per_cluster ints.
+template <bool kInRegs>
+__global__ void __launch_bounds__(kBucketThreads, 1)
+k_bucket_cluster(const int32_t* __restrict__ keys, const int* __restrict__ hist, int* __restrict__ hist_next,
+                 int32_t* __restrict__ offsets, int32_t* __restrict__ perm, int B, int nbins, int bins_per_cluster,
+                 int tile_rows, Tile* __restrict__ tiles, int* __restrict__ n_tiles, int bin_bits,
+                 int32_t* __restrict__ rank_tmp)
+{
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    extern __shared__ int s_dyn[];
+    __shared__ int s_warp[kBucketWarps];
+    __shared__ int s_pub[2];
+
+    const int nb = bins_per_cluster;
+    int* s_cnt = s_dyn;                            // [kBucketWarps][nb]
+    int* s_tot = s_dyn + kBucketWarps * nb;        // [nb] tokens of this CTA's slices per bin (read by peers)
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    const int rank = (int)cluster.block_rank();
+    const int range = blockIdx.x / kBucketClusterSize;
+    const int lo = range * nb;                     // host launches exactly ceil(nbins / nb) clusters
+    const int hi = min(lo + nb, nbins);
+    const unsigned lt_mask = (1u << lane) - 1u;
+
+    for (int i = tid; i < kBucketWarps * nb; i += kBucketThreads) s_cnt[i] = 0;
+
+    int part = 0, tpart = 0;
+    if (rank == 0) {
+        for (int i = tid; i < lo; i += kBucketThreads) {
+            const int c = hist[i];
+            part += c;
+            if (tile_rows > 0) tpart += (c + tile_rows - 1) / tile_rows;
+        }
+    }
+    const int base = block_sum(part, s_warp);                        // meaningful on rank 0 only
+    const int tile_base = tile_rows > 0 ? block_sum(tpart, s_warp) : 0;
+    if (rank == 0 && tid == 0) { s_pub[0] = base; s_pub[1] = tile_base; }
+
+    const int slices = kBucketClusterSize * kBucketWarps;
+    const int chunk = (((B + slices - 1) / slices) + 31) & ~31;
+    const int t0 = min((rank * kBucketWarps + w) * chunk, B), t1 = min(t0 + chunk, B);
+    int* my = s_cnt + w * nb;
+
+    // pass 1: count and rank inside the slice
+    int kreg[kBucketKeyRegs], rreg[kBucketKeyRegs];
+#pragma unroll
+    for (int i = 0; i < kBucketKeyRegs; ++i) { kreg[i] = -1; rreg[i] = 0; }
+    for (int s0 = t0; s0 < t1; s0 += 32 * kBucketKeyRegs) {
+#pragma unroll
+        for (int i = 0; i < kBucketKeyRegs; ++i) {
+            const int t = s0 + i * 32 + lane;
+            kreg[i] = t < t1 ? __ldg(keys + t) : -1;
+        }
+#pragma unroll
+        for (int i = 0; i < kBucketKeyRegs; ++i) {
+            if (s0 + i * 32 >= t1) break;
+            const int k = kreg[i];
+            const bool in = k >= lo && k < hi;
+            const unsigned peers = peers_by_ballot(in, k - lo, bin_bits);
+            const int leader = in ? __ffs(peers) - 1 : lane;
+            int seen = 0;
+            if (in && lane == leader) {
+                seen = my[k - lo];
+                my[k - lo] = seen + __popc(peers);
+            }
+            seen = __shfl_sync(kFullMask, seen, leader) + __popc(peers & lt_mask);
+            if (kInRegs) rreg[i] = seen;
+            else if (in) rank_tmp[s0 + i * 32 + lane] = seen;
+            __syncwarp();
+        }
+    }
+    __syncthreads();
+
+    // per bin: offsets of the warps inside this CTA, and this CTA's total
+    const int b = lo + tid;
+    const bool mine = tid < nb && b < hi;
+    if (mine) {
+        int run = 0;
+        for (int ww = 0; ww < kBucketWarps; ++ww) {
+            const int c2 = s_cnt[ww * nb + tid];
+            s_cnt[ww * nb + tid] = run;
+            run += c2;
+        }
+        s_tot[tid] = run;
+    }
+    const int c = mine ? hist[b] : 0;
+    const int excl = block_exclusive_scan(c, s_warp);
+    cluster.sync();
+
+    // bin starts (rank 0 publishes the base), tokens of lower-ranked CTAs per bin
+    const int* pub0 = reinterpret_cast<const int*>(cluster.map_shared_rank(s_pub, 0));
+    const int start = pub0[0] + excl;
+    const int tile_base0 = pub0[1];
+    if (mine) {
+        int before = 0;
+        for (int r = 0; r < rank; ++r) before += reinterpret_cast<const int*>(cluster.map_shared_rank(s_tot, r))[tid];
+        const int add = start + before;
+        for (int ww = 0; ww < kBucketWarps; ++ww) s_cnt[ww * nb + tid] += add;
+        if (rank == 0) {
+            offsets[b] = start;
+            if (b == nbins - 1) offsets[nbins] = start + c;
+            hist_next[b] = 0;
+        }
+    }
+    if (tile_rows > 0 && rank == 0) {
+        const int nt = (c + tile_rows - 1) / tile_rows;
+        const int tl0 = tile_base0 + block_exclusive_scan(nt, s_warp);
+        if (mine) {
+            for (int i = 0; i < nt; ++i) {
+                Tile tl;
+                tl.bin = b;
+                tl.start = start + i * tile_rows;
+                tl.rows = min(tile_rows, c - i * tile_rows);
+                tl.pad = 0;
+                tiles[tl0 + i] = tl;
+            }
+            if (b == nbins - 1) *n_tiles = tl0 + nt;
+        }
+    }
+    __syncthreads();
+
+    // pass 2: place
+    if (kInRegs) {
+#pragma unroll
+        for (int i = 0; i < kBucketKeyRegs; ++i) {
+            const int k = kreg[i];
+            if (k >= lo && k < hi) perm[my[k - lo] + rreg[i]] = t0 + i * 32 + lane;
+        }
+    } else {
+        for (int t = t0 + lane; t < t1; t += 32) {
+            const int k = __ldg(keys + t);
+            if (k >= lo && k < hi) perm[my[k - lo] + rank_tmp[t]] = t;
+        }
+    }
+    cluster.sync();      // peers may still be reading this CTA's shared memory
 }
 
 // Tile list from an existing offsets array (one CTA; used when the caller supplies the bucketing).
