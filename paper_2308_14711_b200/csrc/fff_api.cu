@@ -17,6 +17,7 @@
 
 #include "kernels/bucket.cuh"
 #include "kernels/common.cuh"
+#include "kernels/descent_mma.cuh"
 #include "kernels/descent_warp.cuh"
 #include "kernels/leaf_mma.cuh"
 #include "kernels/leaf_warp.cuh"
@@ -62,8 +63,18 @@ struct fff_handle_s {
     int32_t *ws_leaf = nullptr, *ws_perm = nullptr, *ws_offsets = nullptr;
     int32_t* ws_rank = nullptr;   // per-token rank scratch of the bucketing kernel (large batches only)
     int max_bucket_clusters = 8;
-    int *ws_hist[2] = {nullptr, nullptr};
-    int hist_cur = 0;
+    int *ws_hist[2] = {nullptr, nullptr};   // histogram buffers, used alternately
+    int hist_cur = 0;                        // buffer the next histogram is accumulated into (all zero)
+    int hist_dirty[2] = {0, 0};              // leading counters of each buffer that still hold old counts
+
+    // staged descent on tensor cores: consecutive groups of levels, each with its weight image
+    struct DenseStage {
+        int L0 = 0, k = 0, NP = 0;
+        __nv_bfloat16* wimg = nullptr;
+        float* bimg = nullptr;
+    };
+    std::vector<DenseStage> stages;
+    int32_t* ws_pos[2] = {nullptr, nullptr};
     int *d_status = nullptr;
 
     // staging for the host-buffer entry point
@@ -123,6 +134,8 @@ void release(fff_handle_s* h) {
     dfree(h->node_w); dfree(h->node_b); dfree(h->w1); dfree(h->b1); dfree(h->w2); dfree(h->b2);
     dfree(h->ws_leaf); dfree(h->ws_perm); dfree(h->ws_offsets); dfree(h->ws_hist[0]); dfree(h->ws_hist[1]);
     dfree(h->d_status); dfree(h->st_x); dfree(h->st_y); dfree(h->st_leaf);
+    for (auto& sg : h->stages) { dfree(sg.wimg); dfree(sg.bimg); }
+    dfree(h->ws_pos[0]); dfree(h->ws_pos[1]);
     dfree(h->w1img); dfree(h->b1img); dfree(h->w2img); dfree(h->ws_tiles); dfree(h->ws_ntiles); dfree(h->ws_rank);
     prof_free(h);
     h->magic = 0;
@@ -142,14 +155,18 @@ bool use_tensor_leaf(const fff_handle_s* h) {
 fff_status_t grow_workspace(fff_handle_s* h, int64_t B) {
     if (B <= h->cap_B) return FFF_OK;
     if (cudaDeviceSynchronize() != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
-    dfree(h->ws_leaf); dfree(h->ws_perm); dfree(h->ws_tiles); dfree(h->ws_rank);
-    h->ws_leaf = h->ws_perm = h->ws_rank = nullptr;
+    dfree(h->ws_leaf); dfree(h->ws_perm); dfree(h->ws_tiles); dfree(h->ws_rank); dfree(h->ws_pos[0]); dfree(h->ws_pos[1]);
+    h->ws_leaf = h->ws_perm = h->ws_rank = h->ws_pos[0] = h->ws_pos[1] = nullptr;
     h->ws_tiles = nullptr;
     h->cap_B = 0;
     fff_status_t s;
     if ((s = dmalloc((void**)&h->ws_leaf, sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
     if ((s = dmalloc((void**)&h->ws_perm, sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
     if ((s = dmalloc((void**)&h->ws_rank, sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
+    if (h->stages.size() > 1) {
+        if ((s = dmalloc((void**)&h->ws_pos[0], sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
+        if ((s = dmalloc((void**)&h->ws_pos[1], sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
+    }
     if ((s = dmalloc((void**)&h->ws_tiles, sizeof(fff::Tile) * max_tiles(h, B))) != FFF_OK) return s;
     h->cap_B = B;
     return FFF_OK;
@@ -168,25 +185,16 @@ fff_status_t launched(fff_handle_s* h, cudaStream_t st, const char* name) {
 
 // ---- stage launchers -------------------------------------------------------
 
-template <typename T>
-fff_status_t run_descent(fff_handle_s* h, const void* x, int32_t* leaf_idx, int* hist, int64_t B, cudaStream_t st) {
-    const int64_t blocks = std::min<int64_t>((B + fff::kDescentWarps - 1) / fff::kDescentWarps, (int64_t)h->sm_count * 8);
-    fff::k_descent_warp<T><<<(unsigned)blocks, fff::kDescentWarps * 32, 0, st>>>(
-        (const T*)x, (const T*)h->node_w, (const T*)h->node_b, h->D, 0, h->depth, nullptr, leaf_idx, hist, B,
-        h->vec_ok && aligned16(x));
-    return launched(h, st, "tree_descent_warp");
-}
-
 fff_status_t run_histogram(fff_handle_s* h, const int32_t* keys, int64_t B, cudaStream_t st) {
     const int64_t blocks = std::min<int64_t>((B + 255) / 256, (int64_t)h->sm_count * 4);
     fff::k_histogram<<<(unsigned)blocks, 256, 0, st>>>(keys, h->ws_hist[h->hist_cur], B, (int)h->n_leaves);
     return launched(h, st, "leaf_histogram");
 }
 
-// Consumes the current histogram buffer and flips to the other (already zero) one.
-fff_status_t run_bucket(fff_handle_s* h, const int32_t* keys, int32_t* offsets, int32_t* perm, int64_t B, cudaStream_t st,
-                        bool want_tiles) {
-    const int nbins = (int)h->n_leaves;
+// Stable bucketing of B keys in [0, nbins).  Consumes the current histogram buffer (which must hold the
+// histogram of `keys`), clears what is stale in the other buffer and makes that one current.
+fff_status_t run_bucket(fff_handle_s* h, const int32_t* keys, int nbins, int32_t* offsets, int32_t* perm, int64_t B,
+                        cudaStream_t st, bool want_tiles, const char* name) {
     // Every cluster reads all keys, so more clusters do not shorten the kernel; they only shrink the bin
     // range (and the number of ballots per step).  All clusters should be resident at once.
     int clusters = std::max(1, std::min(std::min(nbins / 32, 8), h->max_bucket_clusters));
@@ -208,17 +216,125 @@ fff_status_t run_bucket(fff_handle_s* h, const int32_t* keys, int32_t* offsets, 
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const int* hist = h->ws_hist[h->hist_cur];
-    int* hist_next = h->ws_hist[h->hist_cur ^ 1];
+    const int cur = h->hist_cur, other = cur ^ 1;
+    const int* hist = h->ws_hist[cur];
+    int* hist_next = h->ws_hist[other];
     const int tile_rows = want_tiles ? (int)fff::kTM : 0;
+    const int n_clear = h->hist_dirty[other];
     cudaError_t e = in_regs
         ? cudaLaunchKernelEx(&cfg, fff::k_bucket_cluster<true>, keys, hist, hist_next, offsets, perm, (int)B, nbins, per,
-                             tile_rows, h->ws_tiles, h->ws_ntiles, bin_bits, h->ws_rank)
+                             tile_rows, h->ws_tiles, h->ws_ntiles, bin_bits, h->ws_rank, n_clear)
         : cudaLaunchKernelEx(&cfg, fff::k_bucket_cluster<false>, keys, hist, hist_next, offsets, perm, (int)B, nbins, per,
-                             tile_rows, h->ws_tiles, h->ws_ntiles, bin_bits, h->ws_rank);
+                             tile_rows, h->ws_tiles, h->ws_ntiles, bin_bits, h->ws_rank, n_clear);
     if (e != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
-    h->hist_cur ^= 1;
-    return launched(h, st, "leaf_bucketing");
+    h->hist_dirty[cur] = nbins;
+    h->hist_dirty[other] = 0;
+    h->hist_cur = other;
+    return launched(h, st, name);
+}
+
+template <int NP>
+fff_status_t launch_descent_mma(fff_handle_s* h, const fff_handle_s::DenseStage& sg, const void* x, const int32_t* perm,
+                                bool grouped, int32_t* pos_out, int* hist, int64_t B, cudaStream_t st) {
+    using L = fff::DescentMmaLayout<NP>;
+    const int per_sm = std::max(1, std::min(3, (int)((227 * 1024) / (L::kSmemBytes + 1024))));
+    const int64_t bound = grouped ? (int64_t)max_tiles(h, B) : (B + fff::kTM - 1) / fff::kTM;
+    const int64_t grid = std::max<int64_t>(1, std::min<int64_t>((int64_t)h->sm_count * per_sm, bound));
+    fff::k_descent_mma<NP><<<(unsigned)grid, fff::kLeafMmaThreads, L::kSmemBytes, st>>>(
+        (const __nv_bfloat16*)x, grouped ? perm : nullptr, grouped ? h->ws_tiles : nullptr, h->ws_ntiles,
+        (int)((B + fff::kTM - 1) / fff::kTM), sg.wimg, sg.bimg, pos_out, hist, h->D, (int)B, sg.k, h->d_status);
+    return launched(h, st, "tree_descent_mma");
+}
+
+fff_status_t run_descent_mma(fff_handle_s* h, const fff_handle_s::DenseStage& sg, const void* x, const int32_t* perm,
+                             bool grouped, int32_t* pos_out, int* hist, int64_t B, cudaStream_t st) {
+    switch (sg.NP) {
+        case 16: return launch_descent_mma<16>(h, sg, x, perm, grouped, pos_out, hist, B, st);
+        case 32: return launch_descent_mma<32>(h, sg, x, perm, grouped, pos_out, hist, B, st);
+        case 64: return launch_descent_mma<64>(h, sg, x, perm, grouped, pos_out, hist, B, st);
+    }
+    return FFF_ERR_UNSUPPORTED;
+}
+
+template <typename T>
+fff_status_t run_descent_warp(fff_handle_s* h, const void* x, int level0, int levels, const int32_t* pos_in,
+                              int32_t* pos_out, int* hist, int64_t B, cudaStream_t st) {
+    const int64_t blocks = std::min<int64_t>((B + fff::kDescentWarps - 1) / fff::kDescentWarps, (int64_t)h->sm_count * 8);
+    fff::k_descent_warp<T><<<(unsigned)blocks, fff::kDescentWarps * 32, 0, st>>>(
+        (const T*)x, (const T*)h->node_w, (const T*)h->node_b, h->D, level0, levels, pos_in, pos_out, hist, B,
+        h->vec_ok && aligned16(x));
+    return launched(h, st, "tree_descent_warp");
+}
+
+// Number of leading tensor-core stages to run for a batch of B tokens: a stage pays off while the
+// groups it works on (tokens that share the node at the stage's first level) hold enough tokens to
+// reuse the subtree's weights.
+int dense_stage_count(const fff_handle_s* h, int64_t B) {
+    if (h->stages.empty() || h->path == FFF_PATH_WARP) return 0;
+    if (h->path == FFF_PATH_TENSOR) return (int)h->stages.size();
+    int n = 0;
+    for (const auto& sg : h->stages) {
+        if ((B >> sg.L0) < 16) break;
+        ++n;
+    }
+    return n;
+}
+
+// The whole descent: tensor-core stages (with a bucketing by current node between them), then the
+// remaining levels, if any, one warp per token.  leaf_out receives the leaf index; final_hist (nullable)
+// the histogram of leaves.
+fff_status_t run_descent(fff_handle_s* h, const void* x, int32_t* leaf_out, bool want_hist, int64_t B, cudaStream_t st) {
+    fff_status_t s = FFF_OK;
+    const int n_dense = dense_stage_count(h, B);
+    int level = 0;
+    const int32_t* pos = nullptr;
+    for (int i = 0; i < n_dense; ++i) {
+        const auto& sg = h->stages[i];
+        if (i > 0) {
+            s = run_bucket(h, pos, 1 << level, h->ws_offsets, h->ws_perm, B, st, true, "node_bucketing");
+            if (s != FFF_OK) return s;
+        }
+        const bool last = level + sg.k == h->depth;
+        int32_t* out = last ? leaf_out : h->ws_pos[i & 1];
+        const bool hist_needed = last ? want_hist : (i + 1 < n_dense);
+        s = run_descent_mma(h, sg, x, h->ws_perm, i > 0, out, hist_needed ? h->ws_hist[h->hist_cur] : nullptr, B, st);
+        if (s != FFF_OK) return s;
+        level += sg.k;
+        pos = out;
+    }
+    if (level < h->depth || h->depth == 0) {
+        int* hist = want_hist ? h->ws_hist[h->hist_cur] : nullptr;
+        s = h->dtype == FFF_DTYPE_F32
+                ? run_descent_warp<float>(h, x, level, h->depth - level, pos, leaf_out, hist, B, st)
+                : run_descent_warp<__nv_bfloat16>(h, x, level, h->depth - level, pos, leaf_out, hist, B, st);
+    }
+    return s;
+}
+
+template <typename T>
+fff_status_t pack_node_images(fff_handle_s* h) {
+    const int d = h->depth;
+    const int n_st = (d + 5) / 6;
+    int L0 = 0;
+    for (int i = 0; i < n_st; ++i) {
+        fff_handle_s::DenseStage sg;
+        sg.L0 = L0;
+        sg.k = d / n_st + (i < d % n_st ? 1 : 0);
+        sg.NP = std::max(16, 1 << sg.k);
+        const size_t groups = (size_t)1 << L0;
+        fff_status_t s;
+        if ((s = dmalloc((void**)&sg.wimg, groups * sg.NP * h->D * 2)) != FFF_OK) return s;
+        h->stages.push_back(sg);                       // owned by the handle from here on
+        if ((s = dmalloc((void**)&h->stages.back().bimg, groups * sg.NP * 4)) != FFF_OK) return s;
+        fff::k_pack_nodes<T><<<h->sm_count * 8, 256>>>((const T*)h->node_w, (const T*)h->node_b, h->stages.back().wimg,
+                                                      h->stages.back().bimg, sg.L0, sg.k, sg.NP, h->D);
+        if (cudaGetLastError() != cudaSuccess) return FFF_ERR_CUDA;
+        L0 += sg.k;
+    }
+    cudaFuncSetAttribute(fff::k_descent_mma<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, fff::DescentMmaLayout<16>::kSmemBytes);
+    cudaFuncSetAttribute(fff::k_descent_mma<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, fff::DescentMmaLayout<32>::kSmemBytes);
+    cudaFuncSetAttribute(fff::k_descent_mma<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, fff::DescentMmaLayout<64>::kSmemBytes);
+    return cudaGetLastError() == cudaSuccess ? FFF_OK : FFF_ERR_CUDA;
 }
 
 template <typename T>
@@ -262,8 +378,6 @@ fff_status_t pack_leaf_images(fff_handle_s* h) {
     if ((s = dmalloc((void**)&h->w1img, nl * LP * h->D * 2)) != FFF_OK) return s;
     if ((s = dmalloc((void**)&h->b1img, nl * LP * 4)) != FFF_OK) return s;
     if ((s = dmalloc((void**)&h->w2img, nl * U2 * stage2)) != FFF_OK) return s;
-    if ((s = dmalloc((void**)&h->ws_ntiles, sizeof(int))) != FFF_OK) return s;
-    cudaMemset(h->ws_ntiles, 0, sizeof(int));
     const int blocks = h->sm_count * 8;
     fff::k_pack_w1<T><<<blocks, 256>>>((const T*)h->w1, h->w1img, (int)nl, h->l, LP, h->D);
     fff::k_pack_b1<T><<<blocks, 256>>>((const T*)h->b1, h->b1img, (int)nl, h->l, LP);
@@ -425,6 +539,8 @@ fff_status_t fff_create(fff_handle_t* out, int D, int O, int depth, int leaf_wid
     if (s == FFF_OK) s = clone((void**)&h->ws_hist[0], nullptr, sizeof(int) * nl);
     if (s == FFF_OK) s = clone((void**)&h->ws_hist[1], nullptr, sizeof(int) * nl);
     if (s == FFF_OK) s = clone((void**)&h->d_status, nullptr, sizeof(int));
+    if (s == FFF_OK) s = clone((void**)&h->ws_ntiles, nullptr, sizeof(int));
+    if (s == FFF_OK && dtype == FFF_DTYPE_BF16 && D % fff::kKS == 0 && depth > 0) s = pack_node_images<__nv_bfloat16>(h);
     if (s == FFF_OK && dtype == FFF_DTYPE_BF16 && D % fff::kKS == 0 && O % 8 == 0 && leaf_width <= 64) {
         h->LP = leaf_width <= 16 ? 16 : (leaf_width <= 32 ? 32 : 64);
         s = pack_leaf_images<__nv_bfloat16>(h);
@@ -460,7 +576,7 @@ fff_status_t fff_reserve(fff_handle_t h, int64_t max_B) {
 fff_status_t fff_set_path(fff_handle_t h, fff_path_t path) {
     if (!live(h)) return FFF_ERR_BAD_HANDLE;
     if (path != FFF_PATH_AUTO && path != FFF_PATH_WARP && path != FFF_PATH_TENSOR) return FFF_ERR_INVALID_ARG;
-    if (path == FFF_PATH_TENSOR && h->LP == 0) return FFF_ERR_UNSUPPORTED;
+    if (path == FFF_PATH_TENSOR && h->LP == 0 && h->stages.empty()) return FFF_ERR_UNSUPPORTED;
     h->path = path;
     return FFF_OK;
 }
@@ -471,8 +587,9 @@ fff_status_t fff_tree_descent(fff_handle_t h, const void* x, int32_t* leaf_idx, 
     if (B == 0) { h->launches = 0; return FFF_OK; }
     if (!x || !leaf_idx || !aligned16(x)) return FFF_ERR_INVALID_ARG;
     DeviceGuard g(h->device);
+    if ((s = grow_workspace(h, B)) != FFF_OK) return s;
     h->launches = 0;
-    return FFF_DISPATCH(h, run_descent, h, x, leaf_idx, nullptr, B, (cudaStream_t)cuda_stream);
+    return run_descent(h, x, leaf_idx, false, B, (cudaStream_t)cuda_stream);
 }
 
 fff_status_t fff_leaf_bucketing(fff_handle_t h, const int32_t* leaf_idx, int32_t* offsets, int32_t* perm, int64_t B,
@@ -485,7 +602,7 @@ fff_status_t fff_leaf_bucketing(fff_handle_t h, const int32_t* leaf_idx, int32_t
     cudaStream_t st = (cudaStream_t)cuda_stream;
     h->launches = 0;
     if (B > 0 && (s = run_histogram(h, leaf_idx, B, st)) != FFF_OK) return s;
-    return run_bucket(h, leaf_idx, offsets, perm, B, st, false);
+    return run_bucket(h, leaf_idx, (int)h->n_leaves, offsets, perm, B, st, false, "leaf_bucketing");
 }
 
 fff_status_t fff_grouped_leaf_ff(fff_handle_t h, const void* x, const int32_t* leaf_idx, const int32_t* offsets,
@@ -521,9 +638,9 @@ fff_status_t fff_forward_infer(fff_handle_t h, const void* x, void* y, int32_t* 
     h->prof_active = h->prof_steps < h->prof_max_steps;
     if (h->prof_active)
         cudaEventRecord(h->prof_events[(size_t)h->prof_steps * (fff_handle_s::kMaxProfLaunches + 1)], st);
-    s = FFF_DISPATCH(h, run_descent, h, x, leaf, h->ws_hist[h->hist_cur], B, st);
+    s = run_descent(h, x, leaf, true, B, st);
     const bool tensor_leaf = use_tensor_leaf(h);
-    if (s == FFF_OK) s = run_bucket(h, leaf, h->ws_offsets, h->ws_perm, B, st, tensor_leaf);
+    if (s == FFF_OK) s = run_bucket(h, leaf, (int)h->n_leaves, h->ws_offsets, h->ws_perm, B, st, tensor_leaf, "leaf_bucketing");
     if (s == FFF_OK)
         s = tensor_leaf ? run_leaf_mma(h, x, h->ws_perm, y, B, st) : FFF_DISPATCH(h, run_leaf, h, x, leaf, h->ws_perm, y, B, st);
     if (h->prof_active) {

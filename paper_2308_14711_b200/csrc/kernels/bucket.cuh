@@ -83,8 +83,8 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* s_warp)
     return (w > 0 ? before : 0) + incl - v;
 }
 
-// hist: complete histogram of keys.  hist_next: a second histogram buffer that
-// is cleared here for the following call (nobody reads it during this kernel).
+// hist: complete histogram of keys.  hist_next: a second histogram buffer whose
+// first nbins counters are cleared here (nobody reads it during this kernel).
 // tile_rows > 0 additionally writes the tile list of the grouped kernels: the
 // tiles of bin 0 first, each bin cut into ceil(count / tile_rows) tiles, and
 // their number into *n_tiles.
@@ -217,7 +217,7 @@ __global__ void __launch_bounds__(kBucketThreads, 1)
 k_bucket_cluster(const int32_t* __restrict__ keys, const int* __restrict__ hist, int* __restrict__ hist_next,
                  int32_t* __restrict__ offsets, int32_t* __restrict__ perm, int B, int nbins, int bins_per_cluster,
                  int tile_rows, Tile* __restrict__ tiles, int* __restrict__ n_tiles, int bin_bits,
-                 int32_t* __restrict__ rank_tmp)
+                 int32_t* __restrict__ rank_tmp, int n_clear)
 {
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
@@ -236,6 +236,8 @@ k_bucket_cluster(const int32_t* __restrict__ keys, const int* __restrict__ hist,
     const unsigned lt_mask = (1u << lane) - 1u;
 
     for (int i = tid; i < kBucketWarps * nb; i += kBucketThreads) s_cnt[i] = 0;
+    // clear the other histogram buffer (first n_clear counters hold an earlier call's counts)
+    for (int i = blockIdx.x * kBucketThreads + tid; i < n_clear; i += gridDim.x * kBucketThreads) hist_next[i] = 0;
 
     int part = 0, tpart = 0;
     if (rank == 0) {
@@ -312,7 +314,6 @@ k_bucket_cluster(const int32_t* __restrict__ keys, const int* __restrict__ hist,
         if (rank == 0) {
             offsets[b] = start;
             if (b == nbins - 1) offsets[nbins] = start + c;
-            hist_next[b] = 0;
         }
     }
     if (tile_rows > 0 && rank == 0) {

@@ -1,0 +1,211 @@
+// One stage of the tree descent on tensor cores (bf16, float32 accumulate).
+//
+// Algorithm 1, FORWARD_I, non-leaf branch.  The d sequential node decisions of a token are cut into
+// stages of k <= 6 levels.  A stage starts with the tokens grouped by the node they have reached at
+// level L0 (all tokens at the root for the first stage).  For one group, the 2^k - 1 nodes of the
+// depth-k subtree below that node are the same for every token of the group, so their logits are one
+// narrow GEMM,
+//     logits[|group|, NP] = X[group] . Wsub^T,        NP = 16, 32 or 64 >= 2^k - 1,
+// and the k decisions are then read off the logits by walking the subtree: position p <- 2p + 1 +
+// (logit[p] + b[p] >= 0), starting at p = 0 in the subtree's own breadth-first numbering.  This trades
+// (2^k - 1) / k times more multiply-adds, which the tensor cores absorb, for k times fewer passes
+// over x and no per-token fetch of weight rows.
+//
+// The machinery is that of the grouped leaf kernel: persistent CTAs over a tile list (tiles of up to
+// kTM consecutive entries of one group), a producer warp issuing 1-D bulk (TMA) copies of the
+// gathered token rows and of a pre-swizzled weight image into an mbarrier ring (several producer
+// warps, because one warp issues bulk copies too slowly), kTM/16 consumer
+// warps with mma.sync.m16n8k16.  tiles == NULL means "one group, tokens in natural order".
+//
+// Requirements: bf16, D % kKS == 0.
+#pragma once
+
+#include "common.cuh"
+#include "leaf_mma.cuh"
+#include "ptx.cuh"
+
+namespace fff {
+
+template <int NP> struct DescentMmaLayout {
+    static constexpr int kWStageBytes = NP * kKS * 2;
+    static constexpr int kStageBytes = kTM * kXRowBytes + kWStageBytes;
+    static constexpr int kStageStride = (kStageBytes + 127) & ~127;
+    static constexpr int kLogitRow = NP + 1;                                     // floats, padded
+    static constexpr int kStagingBytes = kLeafMmaConsumers * 16 * kLogitRow * 4;
+    static constexpr int kSmemBytes = kStages * kStageStride + ((kStagingBytes + 127) & ~127) + 128 + 128;
+};
+
+// Weight image of one stage: [group][D/kKS][kKS/64][NP rows][64 columns] 128-byte swizzled, rows in the
+// subtree's breadth-first order (row 2^r - 1 + p = node N_{L0+r, g*2^r + p}); unused rows zero.
+// Bias image: [group][NP] float32.
+template <typename T>
+__global__ void k_pack_nodes(const T* __restrict__ node_w, const T* __restrict__ node_b,
+                             __nv_bfloat16* __restrict__ img, float* __restrict__ bimg,
+                             int L0, int k, int NP, int D)
+{
+    const int64_t groups = (int64_t)1 << L0;
+    const int64_t total = groups * NP * D;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int kk = (int)(i % D);
+        const int n = (int)((i / D) % NP);
+        const int64_t g = i / ((int64_t)D * NP);
+        int r = 0;
+        while (((1 << (r + 1)) - 1) <= n) ++r;                 // level of local node n inside the subtree
+        const bool used = r < k;
+        const int64_t p = n - ((1 << r) - 1);
+        const int64_t row = used ? (((int64_t)1 << (L0 + r)) - 1 + g * ((int64_t)1 << r) + p) : 0;
+        const int u = kk / kKS, sb = (kk % kKS) / 64, kc = kk % 64;
+        const uint32_t off = ptx::swz128((uint32_t)((sb * NP + n) * 128 + kc * 2));
+        const int64_t base = (g * (D / kKS) + u) * (int64_t)(NP * kKS);
+        img[base + off / 2] = __float2bfloat16_rn(used ? Elem<T>::to_float(node_w[row * D + kk]) : 0.0f);
+        if (kk == 0) bimg[g * NP + n] = used ? Elem<T>::to_float(node_b[row]) : 0.0f;
+    }
+}
+
+template <int NP>
+__global__ void __launch_bounds__(kLeafMmaThreads)
+k_descent_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ perm,
+              const Tile* __restrict__ tiles, const int* __restrict__ n_tiles_ptr, int n_tiles_static,
+              const __nv_bfloat16* __restrict__ wimg, const float* __restrict__ bimg,
+              int32_t* __restrict__ pos_out, int* __restrict__ hist,
+              int D, int B, int k, int* __restrict__ status)
+{
+    using L = DescentMmaLayout<NP>;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+    unsigned char* stages = smem;
+    float* staging = reinterpret_cast<float*>(smem + kStages * L::kStageStride);
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStages * L::kStageStride + ((L::kStagingBytes + 127) & ~127));
+    uint64_t* empty = full + kStages;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int U1 = D / kKS;
+    const int ntiles = tiles ? *n_tiles_ptr : n_tiles_static;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            ptx::mbar_init(full + s, kProducerWarps);
+            ptx::mbar_init(empty + s, kLeafMmaConsumers);
+        }
+        ptx::fence_mbar_init();
+    }
+    __syncthreads();
+
+    int stage = 0;
+    uint32_t phase = 0;
+    bool timed_out = false;
+
+    auto get_tile = [&](int t) {
+        Tile tl;
+        if (tiles) {
+            tl = tiles[t];
+        } else {
+            tl.bin = 0;
+            tl.start = t * kTM;
+            tl.rows = min(kTM, B - t * kTM);
+            tl.pad = 0;
+        }
+        return tl;
+    };
+
+    if (warp >= kLeafMmaConsumers) {
+        // ------------------------------------------------------------------ producer warps
+        const int pw = warp - kLeafMmaConsumers;
+        const int r = pw * kRowsPerProducer + lane;               // row of the tile this lane copies
+        for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+            const Tile tl = get_tile(tile);
+            const bool has_row = lane < kRowsPerProducer && r < tl.rows;
+            const int my_rows = max(0, min(kRowsPerProducer, tl.rows - pw * kRowsPerProducer));
+            const int64_t tok = has_row ? (perm ? perm[tl.start + r] : tl.start + r) : 0;
+            for (int u = 0; u < U1; ++u) {
+                if (!timed_out && !ptx::mbar_wait(empty + stage, phase ^ 1)) timed_out = true;
+                unsigned char* st = stages + stage * L::kStageStride;
+                if (lane == 0) {
+                    ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)(my_rows * kKS * 2 + (pw == 0 ? L::kWStageBytes : 0)));
+                    if (pw == 0)
+                        ptx::bulk_g2s(st + kTM * kXRowBytes, wimg + ((int64_t)tl.bin * U1 + u) * (NP * kKS), L::kWStageBytes,
+                                      full + stage);
+                }
+                __syncwarp();
+                if (has_row) ptx::bulk_g2s(st + r * kXRowBytes, x + tok * D + u * kKS, kKS * 2, full + stage);
+                if (++stage == kStages) { stage = 0; phase ^= 1; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ consumer warps
+        const int m0 = warp * 16;
+        float* my_logits = staging + warp * 16 * L::kLogitRow;
+        const int g = lane >> 2, q4 = lane & 3;
+        for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+            const Tile tl = get_tile(tile);
+            const bool active = m0 < tl.rows;
+
+            float acc[NP / 8][4];
+#pragma unroll
+            for (int nt = 0; nt < NP / 8; ++nt)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) acc[nt][c] = 0.0f;
+
+            for (int u = 0; u < U1; ++u) {
+                if (!timed_out && !ptx::mbar_wait(full + stage, phase)) timed_out = true;
+                if (active) {
+                    const uint32_t xs = ptx::smem_addr(stages + stage * L::kStageStride);
+                    const uint32_t ws = xs + kTM * kXRowBytes;
+                    const uint32_t a_base = xs + (m0 + (lane & 15)) * kXRowBytes + (lane >> 4) * 16;
+                    const int bn = (lane & 7) + ((lane >> 4) << 3);
+                    const int bk = ((lane >> 3) & 1) * 8;
+#pragma unroll
+                    for (int ks = 0; ks < kKS / 16; ++ks) {
+                        uint32_t a0, a1, a2, a3;
+                        ptx::ldmatrix_x4(a_base + ks * 32, a0, a1, a2, a3);
+                        const int kcol = ks * 16 + bk;
+                        const int sb = kcol >> 6, kc = kcol & 63;
+#pragma unroll
+                        for (int np = 0; np < NP / 16; ++np) {
+                            const int n = np * 16 + bn;
+                            uint32_t b0, b1, b2, b3;
+                            ptx::ldmatrix_x4(ws + ptx::swz128((uint32_t)((sb * NP + n) * 128 + kc * 2)), b0, b1, b2, b3);
+                            ptx::mma_bf16(acc[2 * np], a0, a1, a2, a3, b0, b1);
+                            ptx::mma_bf16(acc[2 * np + 1], a0, a1, a2, a3, b2, b3);
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(empty + stage);
+                if (++stage == kStages) { stage = 0; phase ^= 1; }
+            }
+
+            if (active) {
+                // logits of the 16 rows of this warp -> shared memory, then one lane per row walks the subtree
+#pragma unroll
+                for (int nt = 0; nt < NP / 8; ++nt) {
+                    my_logits[g * L::kLogitRow + nt * 8 + 2 * q4] = acc[nt][0];
+                    my_logits[g * L::kLogitRow + nt * 8 + 2 * q4 + 1] = acc[nt][1];
+                    my_logits[(g + 8) * L::kLogitRow + nt * 8 + 2 * q4] = acc[nt][2];
+                    my_logits[(g + 8) * L::kLogitRow + nt * 8 + 2 * q4 + 1] = acc[nt][3];
+                }
+                __syncwarp();
+                if (lane < 16 && m0 + lane < tl.rows) {
+                    const float* row = my_logits + lane * L::kLogitRow;
+                    const float* bias = bimg + (int64_t)tl.bin * NP;
+                    int p = 0;
+                    for (int r = 0; r < k; ++r) {
+                        const float logit = row[p] + __ldg(bias + p);
+                        p = 2 * p + 1 + (logit >= 0.0f ? 1 : 0);
+                    }
+                    const int pos = (tl.bin << k) + (p - ((1 << k) - 1));
+                    const int64_t t = perm ? perm[tl.start + m0 + lane] : tl.start + m0 + lane;
+                    pos_out[t] = pos;
+                    if (hist) atomicAdd(hist + pos, 1);
+                }
+                __syncwarp();
+            }
+        }
+    }
+    if (timed_out) {
+        if (lane == 0) atomicExch(status, kDevTimeout);
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);     // let bulk copies still in flight land before exit
+    }
+}
+
+}  // namespace fff

@@ -6,8 +6,8 @@
 // and row i of Y is stored at the original position of token T_j[i].
 //
 // Work unit: a tile = up to kTM consecutive entries of one bucket.  CTAs are persistent and walk the
-// device-built tile list with a static stride.  Inside a CTA one producer warp streams operands into
-// a ring of shared-memory stages with 1-D bulk (TMA) copies that complete on mbarriers; kTM/16
+// device-built tile list with a static stride.  Inside a CTA kProducerWarps producer warps stream operands
+// into a ring of shared-memory stages with 1-D bulk (TMA) copies that complete on mbarriers; kTM/16
 // consumer warps each own 16 token rows and run both GEMMs with mma.sync.m16n8k16, keeping H in
 // registers between them (the accumulator fragment of GEMM1 is the A fragment of GEMM2).
 //
@@ -32,7 +32,11 @@ constexpr int kKS = 128;         // K columns per GEMM1 stage
 constexpr int kNC = 256;         // output columns per GEMM2 stage
 constexpr int kStages = 3;
 constexpr int kLeafMmaConsumers = kTM / 16;
-constexpr int kLeafMmaThreads = (kLeafMmaConsumers + 1) * 32;
+// One warp sustains only about one bulk-copy request per 60 cycles whatever its size, so the row
+// copies of a stage are spread over several producer warps.
+constexpr int kProducerWarps = 4;
+constexpr int kRowsPerProducer = kTM / kProducerWarps;
+constexpr int kLeafMmaThreads = (kLeafMmaConsumers + kProducerWarps) * 32;
 constexpr int kXRowBytes = kKS * 2 + 16;                    // padded row of a GEMM1 stage
 constexpr int kOutHalf = 128;                               // outputs accumulated at once per warp
 constexpr int kOutRowBytes = kOutHalf * 2 + 16;             // padded row of the store staging buffer
@@ -129,7 +133,7 @@ k_leaf_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ perm
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
-            ptx::mbar_init(full + s, 1);
+            ptx::mbar_init(full + s, kProducerWarps);
             ptx::mbar_init(empty + s, kLeafMmaConsumers);
         }
         ptx::fence_mbar_init();
@@ -140,38 +144,38 @@ k_leaf_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ perm
     uint32_t phase = 0;
     bool timed_out = false;
 
-    if (warp == kLeafMmaConsumers) {
-        // ------------------------------------------------------------------ producer warp
+    if (warp >= kLeafMmaConsumers) {
+        // ------------------------------------------------------------------ producer warps
+        const int pw = warp - kLeafMmaConsumers;
+        const int r = pw * kRowsPerProducer + lane;               // row of the tile this lane copies
         for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
             const Tile tl = tiles[tile];
-            int64_t tok[kTM / 32];
-#pragma unroll
-            for (int q = 0; q < kTM / 32; ++q) {
-                const int r = q * 32 + lane;
-                tok[q] = r < tl.rows ? perm[tl.start + r] : 0;
-            }
+            const bool has_row = lane < kRowsPerProducer && r < tl.rows;
+            const int my_rows = max(0, min(kRowsPerProducer, tl.rows - pw * kRowsPerProducer));
+            const int64_t tok = has_row ? perm[tl.start + r] : 0;
             for (int u = 0; u < U1; ++u) {
                 if (!timed_out && !ptx::mbar_wait(empty + stage, phase ^ 1)) timed_out = true;
                 unsigned char* st = stages + stage * L::kStageStride;
                 if (lane == 0) {
-                    ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)(tl.rows * kKS * 2 + L::kW1StageBytes));
-                    ptx::bulk_g2s(st + kTM * kXRowBytes, w1img + ((int64_t)tl.bin * U1 + u) * (LP * kKS),
-                                  L::kW1StageBytes, full + stage);
+                    ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)(my_rows * kKS * 2 + (pw == 0 ? L::kW1StageBytes : 0)));
+                    if (pw == 0)
+                        ptx::bulk_g2s(st + kTM * kXRowBytes, w1img + ((int64_t)tl.bin * U1 + u) * (LP * kKS),
+                                      L::kW1StageBytes, full + stage);
                 }
                 __syncwarp();
-#pragma unroll
-                for (int q = 0; q < kTM / 32; ++q) {
-                    const int r = q * 32 + lane;
-                    if (r < tl.rows) ptx::bulk_g2s(st + r * kXRowBytes, x + tok[q] * D + u * kKS, kKS * 2, full + stage);
-                }
+                if (has_row) ptx::bulk_g2s(st + r * kXRowBytes, x + tok * D + u * kKS, kKS * 2, full + stage);
                 if (++stage == kStages) { stage = 0; phase ^= 1; }
             }
             for (int u = 0; u < U2; ++u) {
                 if (!timed_out && !ptx::mbar_wait(empty + stage, phase ^ 1)) timed_out = true;
                 if (lane == 0) {
-                    ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)L::kStage2Bytes);
-                    ptx::bulk_g2s(stages + stage * L::kStageStride,
-                                  w2img + ((int64_t)tl.bin * U2 + u) * L::kStage2Bytes, L::kStage2Bytes, full + stage);
+                    if (pw == 0) {
+                        ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)L::kStage2Bytes);
+                        ptx::bulk_g2s(stages + stage * L::kStageStride,
+                                      w2img + ((int64_t)tl.bin * U2 + u) * L::kStage2Bytes, L::kStage2Bytes, full + stage);
+                    } else {
+                        ptx::mbar_arrive(full + stage);
+                    }
                 }
                 __syncwarp();
                 if (++stage == kStages) { stage = 0; phase ^= 1; }
