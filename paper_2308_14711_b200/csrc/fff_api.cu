@@ -142,9 +142,16 @@ void release(fff_handle_s* h) {
     delete h;
 }
 
+constexpr int kMinTileRows = 32;
+
 // Upper bound of the tile list: every non-empty bin ends in at most one partial tile.
 size_t max_tiles(const fff_handle_s* h, int64_t B) {
-    return (size_t)(B / fff::kTM + std::min<int64_t>(h->n_leaves, B) + 1);
+    return (size_t)(B / kMinTileRows + std::min<int64_t>(h->n_leaves, B) + 1);
+}
+
+// Token rows per tile of the grouped leaf kernel: short tiles when buckets are small.
+int leaf_tile_rows(const fff_handle_s* h, int64_t B) {
+    return B / h->n_leaves <= 40 ? 32 : 64;
 }
 
 bool use_tensor_leaf(const fff_handle_s* h) {
@@ -194,7 +201,7 @@ fff_status_t run_histogram(fff_handle_s* h, const int32_t* keys, int64_t B, cuda
 // Stable bucketing of B keys in [0, nbins).  Consumes the current histogram buffer (which must hold the
 // histogram of `keys`), clears what is stale in the other buffer and makes that one current.
 fff_status_t run_bucket(fff_handle_s* h, const int32_t* keys, int nbins, int32_t* offsets, int32_t* perm, int64_t B,
-                        cudaStream_t st, bool want_tiles, const char* name) {
+                        cudaStream_t st, int tile_rows, const char* name) {
     // Every cluster reads all keys, so more clusters do not shorten the kernel; they only shrink the bin
     // range (and the number of ballots per step).  All clusters should be resident at once.
     int clusters = std::max(1, std::min(std::min(nbins / 32, 8), h->max_bucket_clusters));
@@ -219,7 +226,6 @@ fff_status_t run_bucket(fff_handle_s* h, const int32_t* keys, int nbins, int32_t
     const int cur = h->hist_cur, other = cur ^ 1;
     const int* hist = h->ws_hist[cur];
     int* hist_next = h->ws_hist[other];
-    const int tile_rows = want_tiles ? (int)fff::kTM : 0;
     const int n_clear = h->hist_dirty[other];
     cudaError_t e = in_regs
         ? cudaLaunchKernelEx(&cfg, fff::k_bucket_cluster<true>, keys, hist, hist_next, offsets, perm, (int)B, nbins, per,
@@ -233,25 +239,28 @@ fff_status_t run_bucket(fff_handle_s* h, const int32_t* keys, int nbins, int32_t
     return launched(h, st, name);
 }
 
-template <int NP>
+template <int NP, int S>
 fff_status_t launch_descent_mma(fff_handle_s* h, const fff_handle_s::DenseStage& sg, const void* x, const int32_t* perm,
                                 bool grouped, int32_t* pos_out, int* hist, int64_t B, cudaStream_t st) {
-    using L = fff::DescentMmaLayout<NP>;
+    using L = fff::DescentMmaLayout<NP, S>;
     const int per_sm = std::max(1, std::min(3, (int)((227 * 1024) / (L::kSmemBytes + 1024))));
-    const int64_t bound = grouped ? (int64_t)max_tiles(h, B) : (B + fff::kTM - 1) / fff::kTM;
+    const int64_t bound = grouped ? (int64_t)max_tiles(h, B) : (B + fff::kDTM - 1) / fff::kDTM;
     const int64_t grid = std::max<int64_t>(1, std::min<int64_t>((int64_t)h->sm_count * per_sm, bound));
-    fff::k_descent_mma<NP><<<(unsigned)grid, fff::kLeafMmaThreads, L::kSmemBytes, st>>>(
+    fff::k_descent_mma<NP, S><<<(unsigned)grid, fff::kDescentThreads, L::kSmemBytes, st>>>(
         (const __nv_bfloat16*)x, grouped ? perm : nullptr, grouped ? h->ws_tiles : nullptr, h->ws_ntiles,
-        (int)((B + fff::kTM - 1) / fff::kTM), sg.wimg, sg.bimg, pos_out, hist, h->D, (int)B, sg.k, h->d_status);
+        (int)((B + fff::kDTM - 1) / fff::kDTM), sg.wimg, sg.bimg, pos_out, hist, h->D, (int)B, sg.k, h->d_status);
     return launched(h, st, "tree_descent_mma");
 }
+
+// Ring depths: as many stages as fit with two CTAs per SM (one for the widest stage).
+constexpr int kDescentStages16 = 4, kDescentStages32 = 4, kDescentStages64 = 6;
 
 fff_status_t run_descent_mma(fff_handle_s* h, const fff_handle_s::DenseStage& sg, const void* x, const int32_t* perm,
                              bool grouped, int32_t* pos_out, int* hist, int64_t B, cudaStream_t st) {
     switch (sg.NP) {
-        case 16: return launch_descent_mma<16>(h, sg, x, perm, grouped, pos_out, hist, B, st);
-        case 32: return launch_descent_mma<32>(h, sg, x, perm, grouped, pos_out, hist, B, st);
-        case 64: return launch_descent_mma<64>(h, sg, x, perm, grouped, pos_out, hist, B, st);
+        case 16: return launch_descent_mma<16, kDescentStages16>(h, sg, x, perm, grouped, pos_out, hist, B, st);
+        case 32: return launch_descent_mma<32, kDescentStages32>(h, sg, x, perm, grouped, pos_out, hist, B, st);
+        case 64: return launch_descent_mma<64, kDescentStages64>(h, sg, x, perm, grouped, pos_out, hist, B, st);
     }
     return FFF_ERR_UNSUPPORTED;
 }
@@ -291,7 +300,7 @@ fff_status_t run_descent(fff_handle_s* h, const void* x, int32_t* leaf_out, bool
     for (int i = 0; i < n_dense; ++i) {
         const auto& sg = h->stages[i];
         if (i > 0) {
-            s = run_bucket(h, pos, 1 << level, h->ws_offsets, h->ws_perm, B, st, true, "node_bucketing");
+            s = run_bucket(h, pos, 1 << level, h->ws_offsets, h->ws_perm, B, st, fff::kDTM, "node_bucketing");
             if (s != FFF_OK) return s;
         }
         const bool last = level + sg.k == h->depth;
@@ -331,9 +340,12 @@ fff_status_t pack_node_images(fff_handle_s* h) {
         if (cudaGetLastError() != cudaSuccess) return FFF_ERR_CUDA;
         L0 += sg.k;
     }
-    cudaFuncSetAttribute(fff::k_descent_mma<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, fff::DescentMmaLayout<16>::kSmemBytes);
-    cudaFuncSetAttribute(fff::k_descent_mma<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, fff::DescentMmaLayout<32>::kSmemBytes);
-    cudaFuncSetAttribute(fff::k_descent_mma<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, fff::DescentMmaLayout<64>::kSmemBytes);
+    cudaFuncSetAttribute(fff::k_descent_mma<16, kDescentStages16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         fff::DescentMmaLayout<16, kDescentStages16>::kSmemBytes);
+    cudaFuncSetAttribute(fff::k_descent_mma<32, kDescentStages32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         fff::DescentMmaLayout<32, kDescentStages32>::kSmemBytes);
+    cudaFuncSetAttribute(fff::k_descent_mma<64, kDescentStages64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         fff::DescentMmaLayout<64, kDescentStages64>::kSmemBytes);
     return cudaGetLastError() == cudaSuccess ? FFF_OK : FFF_ERR_CUDA;
 }
 
@@ -348,22 +360,37 @@ fff_status_t run_leaf(fff_handle_s* h, const void* x, const int32_t* leaf_idx, c
     return launched(h, st, "grouped_leaf_ff_warp");
 }
 
-template <int LP>
+template <int LP, int TM, int S>
 fff_status_t launch_leaf_mma(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, cudaStream_t st) {
-    using L = fff::LeafMmaLayout<LP>;
+    using L = fff::LeafMmaLayout<LP, TM, S>;
+    static bool attr_set[64] = {};
+    if (h->device < 64 && !attr_set[h->device]) {
+        cudaFuncSetAttribute(fff::k_leaf_mma<LP, TM, S>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kSmemBytes);
+        attr_set[h->device] = true;
+    }
     const int per_sm = std::max(1, std::min(2, (int)((227 * 1024) / (L::kSmemBytes + 1024))));
     const int64_t grid = std::min<int64_t>((int64_t)h->sm_count * per_sm, (int64_t)max_tiles(h, B));
-    fff::k_leaf_mma<LP><<<(unsigned)grid, fff::kLeafMmaThreads, L::kSmemBytes, st>>>(
+    fff::k_leaf_mma<LP, TM, S><<<(unsigned)grid, L::kThreads, L::kSmemBytes, st>>>(
         (const __nv_bfloat16*)x, perm, h->ws_tiles, h->ws_ntiles, h->w1img, h->b1img, h->w2img, (__nv_bfloat16*)y, h->D,
         h->O, h->act, h->d_status);
     return launched(h, st, "grouped_leaf_ff_mma");
 }
 
-fff_status_t run_leaf_mma(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, cudaStream_t st) {
-    switch (h->LP) {
-        case 16: return launch_leaf_mma<16>(h, x, perm, y, B, st);
-        case 32: return launch_leaf_mma<32>(h, x, perm, y, B, st);
-        case 64: return launch_leaf_mma<64>(h, x, perm, y, B, st);
+// Ring depth per (LP, TM): what fits twice into an SM's shared memory (once for LP = 64).
+fff_status_t run_leaf_mma(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, int tile_rows,
+                          cudaStream_t st) {
+    if (tile_rows == 32) {
+        switch (h->LP) {
+            case 16: return launch_leaf_mma<16, 32, 6>(h, x, perm, y, B, st);
+            case 32: return launch_leaf_mma<32, 32, 5>(h, x, perm, y, B, st);
+            case 64: return launch_leaf_mma<64, 32, 4>(h, x, perm, y, B, st);
+        }
+    } else {
+        switch (h->LP) {
+            case 16: return launch_leaf_mma<16, 64, 4>(h, x, perm, y, B, st);
+            case 32: return launch_leaf_mma<32, 64, 3>(h, x, perm, y, B, st);
+            case 64: return launch_leaf_mma<64, 64, 5>(h, x, perm, y, B, st);
+        }
     }
     return FFF_ERR_UNSUPPORTED;
 }
@@ -383,9 +410,6 @@ fff_status_t pack_leaf_images(fff_handle_s* h) {
     fff::k_pack_b1<T><<<blocks, 256>>>((const T*)h->b1, h->b1img, (int)nl, h->l, LP);
     fff::k_pack_w2<T><<<blocks, 256>>>((const T*)h->w2, (const T*)h->b2, h->w2img, (int)nl, h->l, LP, h->O);
     if (cudaGetLastError() != cudaSuccess) return FFF_ERR_CUDA;
-    cudaFuncSetAttribute(fff::k_leaf_mma<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, fff::LeafMmaLayout<16>::kSmemBytes);
-    cudaFuncSetAttribute(fff::k_leaf_mma<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, fff::LeafMmaLayout<32>::kSmemBytes);
-    cudaFuncSetAttribute(fff::k_leaf_mma<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, fff::LeafMmaLayout<64>::kSmemBytes);
     return cudaGetLastError() == cudaSuccess ? FFF_OK : FFF_ERR_CUDA;
 }
 
@@ -602,7 +626,7 @@ fff_status_t fff_leaf_bucketing(fff_handle_t h, const int32_t* leaf_idx, int32_t
     cudaStream_t st = (cudaStream_t)cuda_stream;
     h->launches = 0;
     if (B > 0 && (s = run_histogram(h, leaf_idx, B, st)) != FFF_OK) return s;
-    return run_bucket(h, leaf_idx, (int)h->n_leaves, offsets, perm, B, st, false, "leaf_bucketing");
+    return run_bucket(h, leaf_idx, (int)h->n_leaves, offsets, perm, B, st, 0, "leaf_bucketing");
 }
 
 fff_status_t fff_grouped_leaf_ff(fff_handle_t h, const void* x, const int32_t* leaf_idx, const int32_t* offsets,
@@ -616,10 +640,11 @@ fff_status_t fff_grouped_leaf_ff(fff_handle_t h, const void* x, const int32_t* l
     cudaStream_t st = (cudaStream_t)cuda_stream;
     if (use_tensor_leaf(h)) {
         if ((s = grow_workspace(h, B)) != FFF_OK) return s;
-        fff::k_tiles_from_offsets<<<1, fff::kBucketThreads, 0, st>>>(offsets, (int)h->n_leaves, fff::kTM, h->ws_tiles,
+        const int tile_rows = leaf_tile_rows(h, B);
+        fff::k_tiles_from_offsets<<<1, fff::kBucketThreads, 0, st>>>(offsets, (int)h->n_leaves, tile_rows, h->ws_tiles,
                                                                      h->ws_ntiles);
         if ((s = launched(h, st, "tiles_from_offsets")) != FFF_OK) return s;
-        return run_leaf_mma(h, x, perm, y, B, st);
+        return run_leaf_mma(h, x, perm, y, B, tile_rows, st);
     }
     return FFF_DISPATCH(h, run_leaf, h, x, leaf_idx, perm, y, B, st);
 }
@@ -640,9 +665,11 @@ fff_status_t fff_forward_infer(fff_handle_t h, const void* x, void* y, int32_t* 
         cudaEventRecord(h->prof_events[(size_t)h->prof_steps * (fff_handle_s::kMaxProfLaunches + 1)], st);
     s = run_descent(h, x, leaf, true, B, st);
     const bool tensor_leaf = use_tensor_leaf(h);
-    if (s == FFF_OK) s = run_bucket(h, leaf, (int)h->n_leaves, h->ws_offsets, h->ws_perm, B, st, tensor_leaf, "leaf_bucketing");
+    const int tile_rows = tensor_leaf ? leaf_tile_rows(h, B) : 0;
+    if (s == FFF_OK) s = run_bucket(h, leaf, (int)h->n_leaves, h->ws_offsets, h->ws_perm, B, st, tile_rows, "leaf_bucketing");
     if (s == FFF_OK)
-        s = tensor_leaf ? run_leaf_mma(h, x, h->ws_perm, y, B, st) : FFF_DISPATCH(h, run_leaf, h, x, leaf, h->ws_perm, y, B, st);
+        s = tensor_leaf ? run_leaf_mma(h, x, h->ws_perm, y, B, tile_rows, st)
+                        : FFF_DISPATCH(h, run_leaf, h, x, leaf, h->ws_perm, y, B, st);
     if (h->prof_active) {
         h->prof_active = false;
         if (s == FFF_OK && (h->prof_steps == 0 || h->prof_nlaunch == h->launches)) {

@@ -12,10 +12,9 @@
 // over x and no per-token fetch of weight rows.
 //
 // The machinery is that of the grouped leaf kernel: persistent CTAs over a tile list (tiles of up to
-// kTM consecutive entries of one group), a producer warp issuing 1-D bulk (TMA) copies of the
-// gathered token rows and of a pre-swizzled weight image into an mbarrier ring (several producer
-// warps, because one warp issues bulk copies too slowly), kTM/16 consumer
-// warps with mma.sync.m16n8k16.  tiles == NULL means "one group, tokens in natural order".
+// 64 consecutive entries of one group), producer warps that copy the gathered token rows with
+// 16-byte cp.async and a pre-swizzled weight image with one bulk (TMA) copy per stage into an
+// mbarrier ring, and 4 consumer warps with mma.sync.m16n8k16.  tiles == NULL means "one group, tokens in natural order".
 //
 // Requirements: bf16, D % kKS == 0.
 #pragma once
@@ -26,13 +25,18 @@
 
 namespace fff {
 
-template <int NP> struct DescentMmaLayout {
+constexpr int kDTM = 64;                                   // token rows per tile of the descent stages
+constexpr int kDescentConsumers = kDTM / 16;
+constexpr int kDescentThreads = (kDescentConsumers + kProducerWarps) * 32;
+
+template <int NP, int S> struct DescentMmaLayout {
     static constexpr int kWStageBytes = NP * kKS * 2;
-    static constexpr int kStageBytes = kTM * kXRowBytes + kWStageBytes;
+    static constexpr int kStageBytes = kDTM * kXRowBytes + kWStageBytes;
     static constexpr int kStageStride = (kStageBytes + 127) & ~127;
     static constexpr int kLogitRow = NP + 1;                                     // floats, padded
-    static constexpr int kStagingBytes = kLeafMmaConsumers * 16 * kLogitRow * 4;
-    static constexpr int kSmemBytes = kStages * kStageStride + ((kStagingBytes + 127) & ~127) + 128 + 128;
+    static constexpr int kStagingBytes = kDescentConsumers * 16 * kLogitRow * 4;
+    static constexpr int kSmemBytes = S * kStageStride + ((kStagingBytes + 127) & ~127) + 128 + 128;
+    static_assert(S <= kMaxStages, "barrier area holds 2 * kMaxStages mbarriers");
 };
 
 // Weight image of one stage: [group][D/kKS][kKS/64][NP rows][64 columns] 128-byte swizzled, rows in the
@@ -62,15 +66,18 @@ __global__ void k_pack_nodes(const T* __restrict__ node_w, const T* __restrict__
     }
 }
 
-template <int NP>
-__global__ void __launch_bounds__(kLeafMmaThreads)
+template <int NP, int S>
+__global__ void __launch_bounds__(kDescentThreads)
 k_descent_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ perm,
               const Tile* __restrict__ tiles, const int* __restrict__ n_tiles_ptr, int n_tiles_static,
               const __nv_bfloat16* __restrict__ wimg, const float* __restrict__ bimg,
               int32_t* __restrict__ pos_out, int* __restrict__ hist,
               int D, int B, int k, int* __restrict__ status)
 {
-    using L = DescentMmaLayout<NP>;
+    using L = DescentMmaLayout<NP, S>;
+    constexpr int kStages = S;
+    constexpr int kTM = kDTM;
+    constexpr int kLeafMmaConsumers = kDescentConsumers;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     unsigned char* stages = smem;
@@ -84,7 +91,7 @@ k_descent_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ p
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
-            ptx::mbar_init(full + s, kProducerWarps);
+            ptx::mbar_init(full + s, kProducerThreads + 1);     // every producer thread + the weight copy
             ptx::mbar_init(empty + s, kLeafMmaConsumers);
         }
         ptx::fence_mbar_init();
@@ -110,24 +117,29 @@ k_descent_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ p
 
     if (warp >= kLeafMmaConsumers) {
         // ------------------------------------------------------------------ producer warps
-        const int pw = warp - kLeafMmaConsumers;
-        const int r = pw * kRowsPerProducer + lane;               // row of the tile this lane copies
+        const int ptid = threadIdx.x - kLeafMmaConsumers * 32;
+        const int prow = ptid >> 4, pchunk = ptid & 15;
         for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
             const Tile tl = get_tile(tile);
-            const bool has_row = lane < kRowsPerProducer && r < tl.rows;
-            const int my_rows = max(0, min(kRowsPerProducer, tl.rows - pw * kRowsPerProducer));
-            const int64_t tok = has_row ? (perm ? perm[tl.start + r] : tl.start + r) : 0;
+            const __nv_bfloat16* src[kTM / kRowsPerPass];
+#pragma unroll
+            for (int i = 0; i < kTM / kRowsPerPass; ++i) {
+                const int r = i * kRowsPerPass + prow;
+                const int64_t tok = r < tl.rows ? (perm ? perm[tl.start + r] : tl.start + r) : -1;
+                src[i] = tok >= 0 ? x + tok * D + pchunk * 8 : nullptr;
+            }
             for (int u = 0; u < U1; ++u) {
                 if (!timed_out && !ptx::mbar_wait(empty + stage, phase ^ 1)) timed_out = true;
                 unsigned char* st = stages + stage * L::kStageStride;
-                if (lane == 0) {
-                    ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)(my_rows * kKS * 2 + (pw == 0 ? L::kWStageBytes : 0)));
-                    if (pw == 0)
-                        ptx::bulk_g2s(st + kTM * kXRowBytes, wimg + ((int64_t)tl.bin * U1 + u) * (NP * kKS), L::kWStageBytes,
-                                      full + stage);
+                if (ptid == 0) {
+                    ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)L::kWStageBytes);
+                    ptx::bulk_g2s(st + kTM * kXRowBytes, wimg + ((int64_t)tl.bin * U1 + u) * (NP * kKS), L::kWStageBytes,
+                                  full + stage);
                 }
-                __syncwarp();
-                if (has_row) ptx::bulk_g2s(st + r * kXRowBytes, x + tok * D + u * kKS, kKS * 2, full + stage);
+#pragma unroll
+                for (int i = 0; i < kTM / kRowsPerPass; ++i)
+                    if (src[i]) ptx::cp_async16(st + (i * kRowsPerPass + prow) * kXRowBytes + pchunk * 16, src[i] + u * kKS);
+                ptx::cp_async_mbar_arrive(full + stage);
                 if (++stage == kStages) { stage = 0; phase ^= 1; }
             }
         }
@@ -139,6 +151,14 @@ k_descent_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ p
         for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
             const Tile tl = get_tile(tile);
             const bool active = m0 < tl.rows;
+
+            // epilogue operands, fetched now so that their latency hides behind the K loop
+            const int my_row = m0 + (lane & 15);
+            const int64_t my_tok = (active && my_row < tl.rows) ? (perm ? perm[tl.start + my_row] : tl.start + my_row) : -1;
+            float2 bias2[NP / 8];
+#pragma unroll
+            for (int nt = 0; nt < NP / 8; ++nt)
+                bias2[nt] = __ldg(reinterpret_cast<const float2*>(bimg + (int64_t)tl.bin * NP + nt * 8 + 2 * q4));
 
             float acc[NP / 8][4];
 #pragma unroll
@@ -179,23 +199,18 @@ k_descent_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ p
                 // logits of the 16 rows of this warp -> shared memory, then one lane per row walks the subtree
 #pragma unroll
                 for (int nt = 0; nt < NP / 8; ++nt) {
-                    my_logits[g * L::kLogitRow + nt * 8 + 2 * q4] = acc[nt][0];
-                    my_logits[g * L::kLogitRow + nt * 8 + 2 * q4 + 1] = acc[nt][1];
-                    my_logits[(g + 8) * L::kLogitRow + nt * 8 + 2 * q4] = acc[nt][2];
-                    my_logits[(g + 8) * L::kLogitRow + nt * 8 + 2 * q4 + 1] = acc[nt][3];
+                    my_logits[g * L::kLogitRow + nt * 8 + 2 * q4] = acc[nt][0] + bias2[nt].x;
+                    my_logits[g * L::kLogitRow + nt * 8 + 2 * q4 + 1] = acc[nt][1] + bias2[nt].y;
+                    my_logits[(g + 8) * L::kLogitRow + nt * 8 + 2 * q4] = acc[nt][2] + bias2[nt].x;
+                    my_logits[(g + 8) * L::kLogitRow + nt * 8 + 2 * q4 + 1] = acc[nt][3] + bias2[nt].y;
                 }
                 __syncwarp();
-                if (lane < 16 && m0 + lane < tl.rows) {
+                if (lane < 16 && my_tok >= 0) {
                     const float* row = my_logits + lane * L::kLogitRow;
-                    const float* bias = bimg + (int64_t)tl.bin * NP;
                     int p = 0;
-                    for (int r = 0; r < k; ++r) {
-                        const float logit = row[p] + __ldg(bias + p);
-                        p = 2 * p + 1 + (logit >= 0.0f ? 1 : 0);
-                    }
+                    for (int r = 0; r < k; ++r) p = 2 * p + 1 + (row[p] >= 0.0f ? 1 : 0);
                     const int pos = (tl.bin << k) + (p - ((1 << k) - 1));
-                    const int64_t t = perm ? perm[tl.start + m0 + lane] : tl.start + m0 + lane;
-                    pos_out[t] = pos;
+                    pos_out[my_tok] = pos;
                     if (hist) atomicAdd(hist + pos, 1);
                 }
                 __syncwarp();

@@ -5,16 +5,16 @@
 //     Y = H W2_j^T + b2_j                  [|T_j|, O]     (GEMM2, K = l)
 // and row i of Y is stored at the original position of token T_j[i].
 //
-// Work unit: a tile = up to kTM consecutive entries of one bucket.  CTAs are persistent and walk the
+// Work unit: a tile = up to TM consecutive entries of one bucket.  CTAs are persistent and walk the
 // device-built tile list with a static stride.  Inside a CTA kProducerWarps producer warps stream operands
-// into a ring of shared-memory stages with 1-D bulk (TMA) copies that complete on mbarriers; kTM/16
+// into a ring of shared-memory stages with 1-D bulk (TMA) copies that complete on mbarriers; TM/16
 // consumer warps each own 16 token rows and run both GEMMs with mma.sync.m16n8k16, keeping H in
 // registers between them (the accumulator fragment of GEMM1 is the A fragment of GEMM2).
 //
 // Ring contents, in order, per tile:
-//   D/kKS   GEMM1 stages: kKS columns of the gathered token rows (one bulk copy per row, rows padded
-//           by 16 bytes in shared memory so that ldmatrix is conflict-free) + the matching slice of
-//           W1_j (one bulk copy of a pre-swizzled image);
+//   D/kKS   GEMM1 stages: kKS columns of the gathered token rows (16-byte cp.async, rows padded by
+//           16 bytes in shared memory so that ldmatrix is conflict-free) + the matching slice of W1_j
+//           (one bulk copy of a pre-swizzled image);
 //   O/kNC   GEMM2 stages: kNC rows of W2_j (pre-swizzled image) followed by their float32 biases.
 // The images are written once at handle creation (repack kernels below).
 //
@@ -27,29 +27,35 @@
 
 namespace fff {
 
-constexpr int kTM = 64;          // token rows per tile
 constexpr int kKS = 128;         // K columns per GEMM1 stage
 constexpr int kNC = 256;         // output columns per GEMM2 stage
-constexpr int kStages = 3;
-constexpr int kLeafMmaConsumers = kTM / 16;
-// One warp sustains only about one bulk-copy request per 60 cycles whatever its size, so the row
-// copies of a stage are spread over several producer warps.
+// A warp needs about 70 cycles per bulk-copy request whatever its size, which is far too slow for
+// one 256-byte request per gathered row.  The token rows are therefore copied with 16-byte cp.async
+// by all threads of the producer warps (16 threads per row piece); bulk copies are kept for the
+// weight images, where one request moves kilobytes.
 constexpr int kProducerWarps = 4;
-constexpr int kRowsPerProducer = kTM / kProducerWarps;
-constexpr int kLeafMmaThreads = (kLeafMmaConsumers + kProducerWarps) * 32;
+constexpr int kProducerThreads = kProducerWarps * 32;
+constexpr int kRowsPerPass = kProducerThreads / 16;       // rows covered by one cp.async of every producer thread
 constexpr int kXRowBytes = kKS * 2 + 16;                    // padded row of a GEMM1 stage
 constexpr int kOutHalf = 128;                               // outputs accumulated at once per warp
 constexpr int kOutRowBytes = kOutHalf * 2 + 16;             // padded row of the store staging buffer
+constexpr int kMaxStages = 8;
 
-template <int LP> struct LeafMmaLayout {
+// LP: padded hidden width.  TM: token rows per tile (32 or 64).  S: ring stages.  Memory latency under
+// load is a few microseconds, so what matters is how many useful bytes the ring keeps in flight per
+// SM: small buckets get short tiles and a deeper ring instead of half-empty 64-row slots.
+template <int LP, int TM, int S> struct LeafMmaLayout {
+    static constexpr int kConsumers = TM / 16;
+    static constexpr int kThreads = (kConsumers + kProducerWarps) * 32;
     static constexpr int kW1StageBytes = LP * kKS * 2;
-    static constexpr int kStage1Bytes = kTM * kXRowBytes + kW1StageBytes;
+    static constexpr int kStage1Bytes = TM * kXRowBytes + kW1StageBytes;
     static constexpr int kW2Bytes = kNC * LP * 2;
     static constexpr int kStage2Bytes = kW2Bytes + kNC * 4;             // weights + float32 biases
     static constexpr int kStageBytes = kStage1Bytes > kStage2Bytes ? kStage1Bytes : kStage2Bytes;
     static constexpr int kStageStride = (kStageBytes + 127) & ~127;
-    static constexpr int kStagingBytes = kLeafMmaConsumers * 16 * kOutRowBytes;
-    static constexpr int kSmemBytes = kStages * kStageStride + kStagingBytes + 128 /* barriers */ + 128 /* align */;
+    static constexpr int kStagingBytes = kConsumers * 16 * kOutRowBytes;
+    static constexpr int kSmemBytes = S * kStageStride + kStagingBytes + 128 /* barriers */ + 128 /* align */;
+    static_assert(S <= kMaxStages, "barrier area holds 2 * kMaxStages mbarriers");
 };
 
 // ---- one-time repacking of the leaf parameters into stage images --------------------------------
@@ -110,15 +116,18 @@ __global__ void k_pack_b1(const T* __restrict__ b1, float* __restrict__ img, int
 
 // ---- the kernel ------------------------------------------------------------------------------------
 
-template <int LP>
-__global__ void __launch_bounds__(kLeafMmaThreads)
+template <int LP, int TM, int S>
+__global__ void __launch_bounds__((TM / 16 + kProducerWarps) * 32)
 k_leaf_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ perm,
            const Tile* __restrict__ tiles, const int* __restrict__ n_tiles,
            const __nv_bfloat16* __restrict__ w1img, const float* __restrict__ b1img,
            const unsigned char* __restrict__ w2img, __nv_bfloat16* __restrict__ y,
            int D, int O, int act, int* __restrict__ status)
 {
-    using L = LeafMmaLayout<LP>;
+    using L = LeafMmaLayout<LP, TM, S>;
+    constexpr int kStages = S;
+    constexpr int kTM = TM;
+    constexpr int kLeafMmaConsumers = L::kConsumers;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     unsigned char* stages = smem;
@@ -133,7 +142,7 @@ k_leaf_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ perm
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
-            ptx::mbar_init(full + s, kProducerWarps);
+            ptx::mbar_init(full + s, kProducerThreads + 1);     // every producer thread + the weight copy
             ptx::mbar_init(empty + s, kLeafMmaConsumers);
         }
         ptx::fence_mbar_init();
@@ -146,38 +155,38 @@ k_leaf_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ perm
 
     if (warp >= kLeafMmaConsumers) {
         // ------------------------------------------------------------------ producer warps
-        const int pw = warp - kLeafMmaConsumers;
-        const int r = pw * kRowsPerProducer + lane;               // row of the tile this lane copies
+        const int ptid = threadIdx.x - kLeafMmaConsumers * 32;
+        const int prow = ptid >> 4, pchunk = ptid & 15;
         for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
             const Tile tl = tiles[tile];
-            const bool has_row = lane < kRowsPerProducer && r < tl.rows;
-            const int my_rows = max(0, min(kRowsPerProducer, tl.rows - pw * kRowsPerProducer));
-            const int64_t tok = has_row ? perm[tl.start + r] : 0;
+            const __nv_bfloat16* src[kTM / kRowsPerPass];
+#pragma unroll
+            for (int i = 0; i < kTM / kRowsPerPass; ++i) {
+                const int r = i * kRowsPerPass + prow;
+                src[i] = r < tl.rows ? x + (int64_t)perm[tl.start + r] * D + pchunk * 8 : nullptr;
+            }
             for (int u = 0; u < U1; ++u) {
                 if (!timed_out && !ptx::mbar_wait(empty + stage, phase ^ 1)) timed_out = true;
                 unsigned char* st = stages + stage * L::kStageStride;
-                if (lane == 0) {
-                    ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)(my_rows * kKS * 2 + (pw == 0 ? L::kW1StageBytes : 0)));
-                    if (pw == 0)
-                        ptx::bulk_g2s(st + kTM * kXRowBytes, w1img + ((int64_t)tl.bin * U1 + u) * (LP * kKS),
-                                      L::kW1StageBytes, full + stage);
+                if (ptid == 0) {
+                    ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)L::kW1StageBytes);
+                    ptx::bulk_g2s(st + kTM * kXRowBytes, w1img + ((int64_t)tl.bin * U1 + u) * (LP * kKS), L::kW1StageBytes,
+                                  full + stage);
                 }
-                __syncwarp();
-                if (has_row) ptx::bulk_g2s(st + r * kXRowBytes, x + tok * D + u * kKS, kKS * 2, full + stage);
+#pragma unroll
+                for (int i = 0; i < kTM / kRowsPerPass; ++i)
+                    if (src[i]) ptx::cp_async16(st + (i * kRowsPerPass + prow) * kXRowBytes + pchunk * 16, src[i] + u * kKS);
+                ptx::cp_async_mbar_arrive(full + stage);
                 if (++stage == kStages) { stage = 0; phase ^= 1; }
             }
             for (int u = 0; u < U2; ++u) {
                 if (!timed_out && !ptx::mbar_wait(empty + stage, phase ^ 1)) timed_out = true;
-                if (lane == 0) {
-                    if (pw == 0) {
-                        ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)L::kStage2Bytes);
-                        ptx::bulk_g2s(stages + stage * L::kStageStride,
-                                      w2img + ((int64_t)tl.bin * U2 + u) * L::kStage2Bytes, L::kStage2Bytes, full + stage);
-                    } else {
-                        ptx::mbar_arrive(full + stage);
-                    }
+                if (ptid == 0) {
+                    ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)L::kStage2Bytes);
+                    ptx::bulk_g2s(stages + stage * L::kStageStride, w2img + ((int64_t)tl.bin * U2 + u) * L::kStage2Bytes,
+                                  L::kStage2Bytes, full + stage);
                 }
-                __syncwarp();
+                ptx::mbar_arrive(full + stage);
                 if (++stage == kStages) { stage = 0; phase ^= 1; }
             }
         }
@@ -189,6 +198,14 @@ k_leaf_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ perm
         for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
             const Tile tl = tiles[tile];
             const bool active = m0 < tl.rows;          // warps without valid rows only keep the ring moving
+
+            // epilogue operands, fetched now so that their latency hides behind the K loop
+            const int my_row = m0 + (lane & 15);
+            const int64_t my_tok = (active && my_row < tl.rows) ? perm[tl.start + my_row] : -1;
+            float2 b1r[LP / 8];
+#pragma unroll
+            for (int nt = 0; nt < LP / 8; ++nt)
+                b1r[nt] = __ldg(reinterpret_cast<const float2*>(b1img + (int64_t)tl.bin * LP + nt * 8 + 2 * q4));
 
             // GEMM1: acc1[nt] = X[m0..m0+16) . W1[nt*8 .. nt*8+8)^T
             float acc1[LP / 8][4];
@@ -229,10 +246,9 @@ k_leaf_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ perm
             // bias + activation; H stays in registers as the A operand of GEMM2
             uint32_t hA[LP / 8][2];
             {
-                const float* b1p = b1img + (int64_t)tl.bin * LP;
 #pragma unroll
                 for (int nt = 0; nt < LP / 8; ++nt) {
-                    const float2 b = __ldg(reinterpret_cast<const float2*>(b1p + nt * 8 + 2 * q4));
+                    const float2 b = b1r[nt];
                     hA[nt][0] = ptx::pack_bf16(activate(act, acc1[nt][0] + b.x), activate(act, acc1[nt][1] + b.y));
                     hA[nt][1] = ptx::pack_bf16(activate(act, acc1[nt][2] + b.x), activate(act, acc1[nt][3] + b.y));
                 }
@@ -282,8 +298,8 @@ k_leaf_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ perm
                             const int r = it * 2 + (lane >> 4);
                             const int unit = lane & 15;
                             const int o = o_base + unit * 8;
-                            if (m0 + r < tl.rows && o < O) {
-                                const int64_t t = perm[tl.start + m0 + r];
+                            const int64_t t = __shfl_sync(kFullMask, my_tok, r);
+                            if (t >= 0 && o < O) {
                                 const uint4 v = *reinterpret_cast<const uint4*>(my_staging + r * kOutRowBytes + unit * 16);
                                 __stcs(reinterpret_cast<uint4*>(y + t * O + o), v);
                             }
