@@ -56,16 +56,15 @@ struct fff_handle_s {
     float* b1img = nullptr;
     unsigned char* w2img = nullptr;
     fff::Tile* ws_tiles = nullptr;
-    int* ws_ntiles = nullptr;
 
     // workspace
     int64_t cap_B = 0;
     int32_t *ws_leaf = nullptr, *ws_perm = nullptr, *ws_offsets = nullptr;
     int32_t* ws_rank = nullptr;   // per-token rank scratch of the bucketing kernel (large batches only)
     int max_bucket_clusters = 8;
-    int *ws_hist[2] = {nullptr, nullptr};   // histogram buffers, used alternately
-    int hist_cur = 0;                        // buffer the next histogram is accumulated into (all zero)
-    int hist_dirty[2] = {0, 0};              // leading counters of each buffer that still hold old counts
+    int32_t* last_perm = nullptr; // where the most recent forward left its leaf permutation
+    int32_t* ws_perm2 = nullptr;  // second permutation buffer: successive bucketings alternate between the two
+    int32_t* ws_offsets2[2] = {nullptr, nullptr};   // offsets of the intermediate (node) bucketings
 
     // staged descent on tensor cores: consecutive groups of levels, each with its weight image
     struct DenseStage {
@@ -132,11 +131,11 @@ void prof_free(fff_handle_s* h) {
 
 void release(fff_handle_s* h) {
     dfree(h->node_w); dfree(h->node_b); dfree(h->w1); dfree(h->b1); dfree(h->w2); dfree(h->b2);
-    dfree(h->ws_leaf); dfree(h->ws_perm); dfree(h->ws_offsets); dfree(h->ws_hist[0]); dfree(h->ws_hist[1]);
+    dfree(h->ws_leaf); dfree(h->ws_perm); dfree(h->ws_perm2); dfree(h->ws_offsets); dfree(h->ws_offsets2[0]); dfree(h->ws_offsets2[1]);
     dfree(h->d_status); dfree(h->st_x); dfree(h->st_y); dfree(h->st_leaf);
     for (auto& sg : h->stages) { dfree(sg.wimg); dfree(sg.bimg); }
     dfree(h->ws_pos[0]); dfree(h->ws_pos[1]);
-    dfree(h->w1img); dfree(h->b1img); dfree(h->w2img); dfree(h->ws_tiles); dfree(h->ws_ntiles); dfree(h->ws_rank);
+    dfree(h->w1img); dfree(h->b1img); dfree(h->w2img); dfree(h->ws_tiles); dfree(h->ws_rank);
     prof_free(h);
     h->magic = 0;
     delete h;
@@ -144,10 +143,11 @@ void release(fff_handle_s* h) {
 
 constexpr int kMinTileRows = 32;
 
-// Upper bound of the tile list: every non-empty bin ends in at most one partial tile.
-size_t max_tiles(const fff_handle_s* h, int64_t B) {
-    return (size_t)(B / kMinTileRows + std::min<int64_t>(h->n_leaves, B) + 1);
-}
+// Length of a tile list: floor(B / tile_rows) + nbins entries, some of them empty (see k_bucket_cluster).
+int tile_list_len(int64_t B, int tile_rows, int nbins) { return (int)(B / tile_rows) + nbins; }
+
+// Capacity of the tile buffer: the longest list any stage can ask for.
+size_t max_tiles(const fff_handle_s* h, int64_t B) { return (size_t)(B / kMinTileRows + h->n_leaves + 1); }
 
 // Token rows per tile of the grouped leaf kernel: short tiles when buckets are small.
 int leaf_tile_rows(const fff_handle_s* h, int64_t B) {
@@ -162,13 +162,15 @@ bool use_tensor_leaf(const fff_handle_s* h) {
 fff_status_t grow_workspace(fff_handle_s* h, int64_t B) {
     if (B <= h->cap_B) return FFF_OK;
     if (cudaDeviceSynchronize() != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
-    dfree(h->ws_leaf); dfree(h->ws_perm); dfree(h->ws_tiles); dfree(h->ws_rank); dfree(h->ws_pos[0]); dfree(h->ws_pos[1]);
-    h->ws_leaf = h->ws_perm = h->ws_rank = h->ws_pos[0] = h->ws_pos[1] = nullptr;
+    dfree(h->ws_leaf); dfree(h->ws_perm); dfree(h->ws_perm2); dfree(h->ws_tiles); dfree(h->ws_rank); dfree(h->ws_pos[0]);
+    dfree(h->ws_pos[1]);
+    h->ws_leaf = h->ws_perm = h->ws_perm2 = h->ws_rank = h->ws_pos[0] = h->ws_pos[1] = nullptr;
     h->ws_tiles = nullptr;
     h->cap_B = 0;
     fff_status_t s;
     if ((s = dmalloc((void**)&h->ws_leaf, sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
     if ((s = dmalloc((void**)&h->ws_perm, sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
+    if ((s = dmalloc((void**)&h->ws_perm2, sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
     if ((s = dmalloc((void**)&h->ws_rank, sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
     if (h->stages.size() > 1) {
         if ((s = dmalloc((void**)&h->ws_pos[0], sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
@@ -192,29 +194,21 @@ fff_status_t launched(fff_handle_s* h, cudaStream_t st, const char* name) {
 
 // ---- stage launchers -------------------------------------------------------
 
-fff_status_t run_histogram(fff_handle_s* h, const int32_t* keys, int64_t B, cudaStream_t st) {
-    const int64_t blocks = std::min<int64_t>((B + 255) / 256, (int64_t)h->sm_count * 4);
-    fff::k_histogram<<<(unsigned)blocks, 256, 0, st>>>(keys, h->ws_hist[h->hist_cur], B, (int)h->n_leaves);
-    return launched(h, st, "leaf_histogram");
-}
+// What a bucketing refines: nothing (all tokens in natural order), or the previous bucketing.
+struct Coarse {
+    const int32_t* perm = nullptr;      // previous permutation
+    const int32_t* offsets = nullptr;   // its offsets, one segment per coarse bin
+    int bins = 0;                       // number of coarse bins
+};
 
-// Stable bucketing of B keys in [0, nbins).  Consumes the current histogram buffer (which must hold the
-// histogram of `keys`), clears what is stale in the other buffer and makes that one current.
-fff_status_t run_bucket(fff_handle_s* h, const int32_t* keys, int nbins, int32_t* offsets, int32_t* perm, int64_t B,
-                        cudaStream_t st, int tile_rows, const char* name) {
-    // Every cluster reads all keys, so more clusters do not shorten the kernel; they only shrink the bin
-    // range (and the number of ballots per step).  All clusters should be resident at once.
-    int clusters = std::max(1, std::min(std::min(nbins / 32, 8), h->max_bucket_clusters));
-    int per = (nbins + clusters - 1) / clusters;
-    if (per > fff::kBucketMaxBinsPerCta) per = fff::kBucketMaxBinsPerCta;
-    clusters = (nbins + per - 1) / per;
-    int bin_bits = 0;
-    while ((1 << bin_bits) < per) ++bin_bits;
-    const bool in_regs = B <= (int64_t)fff::kBucketClusterSize * fff::kBucketWarps * 32 * fff::kBucketKeyRegs;
+template <int NW>
+cudaError_t launch_bucket(int clusters, size_t smem, cudaStream_t st, const int32_t* keys, const int32_t* perm_in,
+                          const int32_t* seg_offsets, int32_t* offsets, int32_t* perm, int B, int nbins, int nb, int bin_bits,
+                          int tile_rows, fff::Tile* tiles, int n_tiles_total, int32_t* rank_tmp) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(clusters * fff::kBucketClusterSize));
-    cfg.blockDim = dim3(fff::kBucketThreads);
-    cfg.dynamicSmemBytes = sizeof(int) * (size_t)(fff::kBucketWarps + 1) * per;
+    cfg.blockDim = dim3(NW * 32);
+    cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -223,32 +217,54 @@ fff_status_t run_bucket(fff_handle_s* h, const int32_t* keys, int nbins, int32_t
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const int cur = h->hist_cur, other = cur ^ 1;
-    const int* hist = h->ws_hist[cur];
-    int* hist_next = h->ws_hist[other];
-    const int n_clear = h->hist_dirty[other];
-    cudaError_t e = in_regs
-        ? cudaLaunchKernelEx(&cfg, fff::k_bucket_cluster<true>, keys, hist, hist_next, offsets, perm, (int)B, nbins, per,
-                             tile_rows, h->ws_tiles, h->ws_ntiles, bin_bits, h->ws_rank, n_clear)
-        : cudaLaunchKernelEx(&cfg, fff::k_bucket_cluster<false>, keys, hist, hist_next, offsets, perm, (int)B, nbins, per,
-                             tile_rows, h->ws_tiles, h->ws_ntiles, bin_bits, h->ws_rank, n_clear);
+    return cudaLaunchKernelEx(&cfg, fff::k_bucket_cluster<NW>, keys, perm_in, seg_offsets, offsets, perm, B, nbins, nb, bin_bits,
+                              tile_rows, tiles, n_tiles_total, rank_tmp);
+}
+
+// Stable bucketing of B keys in [0, nbins) into (offsets, perm).  If `coarse` describes a bucketing by
+// key >> log2(nbins / coarse.bins), only the inside of each coarse bucket is re-ordered (one cluster per
+// coarse bucket); otherwise clusters split the bin range and each scans all keys.
+// tile_rows > 0 also writes the tile list (tile_list_len(B, tile_rows, nbins) entries) into ws_tiles.
+fff_status_t run_bucket(fff_handle_s* h, const int32_t* keys, int nbins, const Coarse& coarse, int32_t* offsets,
+                        int32_t* perm, int64_t B, cudaStream_t st, int tile_rows, const char* name) {
+    const int n_tiles_total = tile_rows > 0 ? tile_list_len(B, tile_rows, nbins) : 0;
+    cudaError_t e;
+    if (coarse.perm && nbins / coarse.bins <= fff::kBucketMaxBinsPerCta) {
+        const int nb = nbins / coarse.bins;
+        int bin_bits = 0;
+        while ((1 << bin_bits) < nb) ++bin_bits;
+        if (nb <= 256)
+            e = launch_bucket<8>(coarse.bins, sizeof(int) * (size_t)(8 + 1) * nb, st, keys, coarse.perm, coarse.offsets, offsets,
+                                 perm, (int)B, nbins, nb, bin_bits, tile_rows, h->ws_tiles, n_tiles_total, h->ws_rank);
+        else
+            e = launch_bucket<32>(coarse.bins, sizeof(int) * (size_t)(32 + 1) * nb, st, keys, coarse.perm, coarse.offsets,
+                                  offsets, perm, (int)B, nbins, nb, bin_bits, tile_rows, h->ws_tiles, n_tiles_total, h->ws_rank);
+    } else {
+        // Every cluster reads all keys, so more clusters do not shorten the kernel; they only shrink the
+        // bin range (and the number of ballots per step).
+        int clusters = std::max(1, std::min(std::min(nbins / 32, 8), h->max_bucket_clusters));
+        int nb = (nbins + clusters - 1) / clusters;
+        if (nb > fff::kBucketMaxBinsPerCta) nb = fff::kBucketMaxBinsPerCta;
+        clusters = (nbins + nb - 1) / nb;
+        int bin_bits = 0;
+        while ((1 << bin_bits) < nb) ++bin_bits;
+        e = launch_bucket<32>(clusters, sizeof(int) * (size_t)(32 + 1) * nb, st, keys, nullptr, nullptr, offsets, perm, (int)B,
+                              nbins, nb, bin_bits, tile_rows, h->ws_tiles, n_tiles_total, h->ws_rank);
+    }
     if (e != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
-    h->hist_dirty[cur] = nbins;
-    h->hist_dirty[other] = 0;
-    h->hist_cur = other;
     return launched(h, st, name);
 }
 
 template <int NP, int S>
 fff_status_t launch_descent_mma(fff_handle_s* h, const fff_handle_s::DenseStage& sg, const void* x, const int32_t* perm,
-                                bool grouped, int32_t* pos_out, int* hist, int64_t B, cudaStream_t st) {
+                                bool grouped, int32_t* pos_out, int64_t B, cudaStream_t st) {
     using L = fff::DescentMmaLayout<NP, S>;
     const int per_sm = std::max(1, std::min(3, (int)((227 * 1024) / (L::kSmemBytes + 1024))));
-    const int64_t bound = grouped ? (int64_t)max_tiles(h, B) : (B + fff::kDTM - 1) / fff::kDTM;
-    const int64_t grid = std::max<int64_t>(1, std::min<int64_t>((int64_t)h->sm_count * per_sm, bound));
+    const int n_tiles = grouped ? tile_list_len(B, fff::kDTM, 1 << sg.L0) : (int)((B + fff::kDTM - 1) / fff::kDTM);
+    const int64_t grid = std::max<int64_t>(1, std::min<int64_t>((int64_t)h->sm_count * per_sm, n_tiles));
     fff::k_descent_mma<NP, S><<<(unsigned)grid, fff::kDescentThreads, L::kSmemBytes, st>>>(
-        (const __nv_bfloat16*)x, grouped ? perm : nullptr, grouped ? h->ws_tiles : nullptr, h->ws_ntiles,
-        (int)((B + fff::kDTM - 1) / fff::kDTM), sg.wimg, sg.bimg, pos_out, hist, h->D, (int)B, sg.k, h->d_status);
+        (const __nv_bfloat16*)x, grouped ? perm : nullptr, grouped ? h->ws_tiles : nullptr, n_tiles, sg.wimg, sg.bimg, pos_out,
+        h->D, (int)B, sg.k, h->d_status);
     return launched(h, st, "tree_descent_mma");
 }
 
@@ -256,21 +272,21 @@ fff_status_t launch_descent_mma(fff_handle_s* h, const fff_handle_s::DenseStage&
 constexpr int kDescentStages16 = 4, kDescentStages32 = 4, kDescentStages64 = 6;
 
 fff_status_t run_descent_mma(fff_handle_s* h, const fff_handle_s::DenseStage& sg, const void* x, const int32_t* perm,
-                             bool grouped, int32_t* pos_out, int* hist, int64_t B, cudaStream_t st) {
+                             bool grouped, int32_t* pos_out, int64_t B, cudaStream_t st) {
     switch (sg.NP) {
-        case 16: return launch_descent_mma<16, kDescentStages16>(h, sg, x, perm, grouped, pos_out, hist, B, st);
-        case 32: return launch_descent_mma<32, kDescentStages32>(h, sg, x, perm, grouped, pos_out, hist, B, st);
-        case 64: return launch_descent_mma<64, kDescentStages64>(h, sg, x, perm, grouped, pos_out, hist, B, st);
+        case 16: return launch_descent_mma<16, kDescentStages16>(h, sg, x, perm, grouped, pos_out, B, st);
+        case 32: return launch_descent_mma<32, kDescentStages32>(h, sg, x, perm, grouped, pos_out, B, st);
+        case 64: return launch_descent_mma<64, kDescentStages64>(h, sg, x, perm, grouped, pos_out, B, st);
     }
     return FFF_ERR_UNSUPPORTED;
 }
 
 template <typename T>
 fff_status_t run_descent_warp(fff_handle_s* h, const void* x, int level0, int levels, const int32_t* pos_in,
-                              int32_t* pos_out, int* hist, int64_t B, cudaStream_t st) {
+                              int32_t* pos_out, int64_t B, cudaStream_t st) {
     const int64_t blocks = std::min<int64_t>((B + fff::kDescentWarps - 1) / fff::kDescentWarps, (int64_t)h->sm_count * 8);
     fff::k_descent_warp<T><<<(unsigned)blocks, fff::kDescentWarps * 32, 0, st>>>(
-        (const T*)x, (const T*)h->node_w, (const T*)h->node_b, h->D, level0, levels, pos_in, pos_out, hist, B,
+        (const T*)x, (const T*)h->node_w, (const T*)h->node_b, h->D, level0, levels, pos_in, pos_out, B,
         h->vec_ok && aligned16(x));
     return launched(h, st, "tree_descent_warp");
 }
@@ -290,33 +306,38 @@ int dense_stage_count(const fff_handle_s* h, int64_t B) {
 }
 
 // The whole descent: tensor-core stages (with a bucketing by current node between them), then the
-// remaining levels, if any, one warp per token.  leaf_out receives the leaf index; final_hist (nullable)
-// the histogram of leaves.
-fff_status_t run_descent(fff_handle_s* h, const void* x, int32_t* leaf_out, bool want_hist, int64_t B, cudaStream_t st) {
+// remaining levels, if any, one warp per token.  leaf_out receives the leaf index.  *coarse describes
+// the last node bucketing made on the way (the leaf bucketing can refine it instead of starting over).
+fff_status_t run_descent(fff_handle_s* h, const void* x, int32_t* leaf_out, Coarse* coarse, int64_t B, cudaStream_t st) {
     fff_status_t s = FFF_OK;
     const int n_dense = dense_stage_count(h, B);
     int level = 0;
     const int32_t* pos = nullptr;
+    Coarse prev;
     for (int i = 0; i < n_dense; ++i) {
         const auto& sg = h->stages[i];
         if (i > 0) {
-            s = run_bucket(h, pos, 1 << level, h->ws_offsets, h->ws_perm, B, st, fff::kDTM, "node_bucketing");
+            // bucket by the node reached so far; buffers alternate so that the previous level stays readable
+            int32_t* perm_out = (i & 1) ? h->ws_perm2 : h->ws_perm;
+            int32_t* off_out = h->ws_offsets2[i & 1];
+            s = run_bucket(h, pos, 1 << level, prev, off_out, perm_out, B, st, fff::kDTM, "node_bucketing");
             if (s != FFF_OK) return s;
+            prev.perm = perm_out;
+            prev.offsets = off_out;
+            prev.bins = 1 << level;
         }
         const bool last = level + sg.k == h->depth;
         int32_t* out = last ? leaf_out : h->ws_pos[i & 1];
-        const bool hist_needed = last ? want_hist : (i + 1 < n_dense);
-        s = run_descent_mma(h, sg, x, h->ws_perm, i > 0, out, hist_needed ? h->ws_hist[h->hist_cur] : nullptr, B, st);
+        s = run_descent_mma(h, sg, x, prev.perm, i > 0, out, B, st);
         if (s != FFF_OK) return s;
         level += sg.k;
         pos = out;
     }
     if (level < h->depth || h->depth == 0) {
-        int* hist = want_hist ? h->ws_hist[h->hist_cur] : nullptr;
-        s = h->dtype == FFF_DTYPE_F32
-                ? run_descent_warp<float>(h, x, level, h->depth - level, pos, leaf_out, hist, B, st)
-                : run_descent_warp<__nv_bfloat16>(h, x, level, h->depth - level, pos, leaf_out, hist, B, st);
+        s = h->dtype == FFF_DTYPE_F32 ? run_descent_warp<float>(h, x, level, h->depth - level, pos, leaf_out, B, st)
+                                      : run_descent_warp<__nv_bfloat16>(h, x, level, h->depth - level, pos, leaf_out, B, st);
     }
+    if (coarse) *coarse = prev;
     return s;
 }
 
@@ -362,6 +383,7 @@ fff_status_t run_leaf(fff_handle_s* h, const void* x, const int32_t* leaf_idx, c
 
 template <int LP, int TM, int S>
 fff_status_t launch_leaf_mma(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, cudaStream_t st) {
+    const int n_tiles = tile_list_len(B, TM, (int)h->n_leaves);
     using L = fff::LeafMmaLayout<LP, TM, S>;
     static bool attr_set[64] = {};
     if (h->device < 64 && !attr_set[h->device]) {
@@ -369,9 +391,9 @@ fff_status_t launch_leaf_mma(fff_handle_s* h, const void* x, const int32_t* perm
         attr_set[h->device] = true;
     }
     const int per_sm = std::max(1, std::min(2, (int)((227 * 1024) / (L::kSmemBytes + 1024))));
-    const int64_t grid = std::min<int64_t>((int64_t)h->sm_count * per_sm, (int64_t)max_tiles(h, B));
+    const int64_t grid = std::min<int64_t>((int64_t)h->sm_count * per_sm, n_tiles);
     fff::k_leaf_mma<LP, TM, S><<<(unsigned)grid, L::kThreads, L::kSmemBytes, st>>>(
-        (const __nv_bfloat16*)x, perm, h->ws_tiles, h->ws_ntiles, h->w1img, h->b1img, h->w2img, (__nv_bfloat16*)y, h->D,
+        (const __nv_bfloat16*)x, perm, h->ws_tiles, n_tiles, h->w1img, h->b1img, h->w2img, (__nv_bfloat16*)y, h->D,
         h->O, h->act, h->d_status);
     return launched(h, st, "grouped_leaf_ff_mma");
 }
@@ -526,8 +548,7 @@ fff_status_t fff_create(fff_handle_t* out, int D, int O, int depth, int leaf_wid
     cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device);
     {
         const int smem_max = (int)(sizeof(int) * (fff::kBucketWarps + 1) * fff::kBucketMaxBinsPerCta);
-        cudaFuncSetAttribute(fff::k_bucket_cluster<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max);
-        cudaFuncSetAttribute(fff::k_bucket_cluster<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max);
+        cudaFuncSetAttribute(fff::k_bucket_cluster<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max);
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(fff::kBucketClusterSize);
         cfg.blockDim = dim3(fff::kBucketThreads);
@@ -540,7 +561,7 @@ fff_status_t fff_create(fff_handle_t* out, int D, int O, int depth, int leaf_wid
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, fff::k_bucket_cluster<true>, &cfg) == cudaSuccess && n > 0)
+        if (cudaOccupancyMaxActiveClusters(&n, fff::k_bucket_cluster<32>, &cfg) == cudaSuccess && n > 0)
             h->max_bucket_clusters = n;
         else
             cudaGetLastError();
@@ -560,10 +581,9 @@ fff_status_t fff_create(fff_handle_t* out, int D, int O, int depth, int leaf_wid
     if (s == FFF_OK) s = clone(&h->w2, leaf_w2, nl * O * leaf_width * e);
     if (s == FFF_OK) s = clone(&h->b2, leaf_b2, nl * O * e);
     if (s == FFF_OK) s = clone((void**)&h->ws_offsets, nullptr, sizeof(int32_t) * (nl + 1));
-    if (s == FFF_OK) s = clone((void**)&h->ws_hist[0], nullptr, sizeof(int) * nl);
-    if (s == FFF_OK) s = clone((void**)&h->ws_hist[1], nullptr, sizeof(int) * nl);
+    if (s == FFF_OK) s = clone((void**)&h->ws_offsets2[0], nullptr, sizeof(int32_t) * (nl + 1));
+    if (s == FFF_OK) s = clone((void**)&h->ws_offsets2[1], nullptr, sizeof(int32_t) * (nl + 1));
     if (s == FFF_OK) s = clone((void**)&h->d_status, nullptr, sizeof(int));
-    if (s == FFF_OK) s = clone((void**)&h->ws_ntiles, nullptr, sizeof(int));
     if (s == FFF_OK && dtype == FFF_DTYPE_BF16 && D % fff::kKS == 0 && depth > 0) s = pack_node_images<__nv_bfloat16>(h);
     if (s == FFF_OK && dtype == FFF_DTYPE_BF16 && D % fff::kKS == 0 && O % 8 == 0 && leaf_width <= 64) {
         h->LP = leaf_width <= 16 ? 16 : (leaf_width <= 32 ? 32 : 64);
@@ -613,7 +633,7 @@ fff_status_t fff_tree_descent(fff_handle_t h, const void* x, int32_t* leaf_idx, 
     DeviceGuard g(h->device);
     if ((s = grow_workspace(h, B)) != FFF_OK) return s;
     h->launches = 0;
-    return run_descent(h, x, leaf_idx, false, B, (cudaStream_t)cuda_stream);
+    return run_descent(h, x, leaf_idx, nullptr, B, (cudaStream_t)cuda_stream);
 }
 
 fff_status_t fff_leaf_bucketing(fff_handle_t h, const int32_t* leaf_idx, int32_t* offsets, int32_t* perm, int64_t B,
@@ -625,8 +645,7 @@ fff_status_t fff_leaf_bucketing(fff_handle_t h, const int32_t* leaf_idx, int32_t
     if ((s = grow_workspace(h, B)) != FFF_OK) return s;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     h->launches = 0;
-    if (B > 0 && (s = run_histogram(h, leaf_idx, B, st)) != FFF_OK) return s;
-    return run_bucket(h, leaf_idx, (int)h->n_leaves, offsets, perm, B, st, 0, "leaf_bucketing");
+    return run_bucket(h, leaf_idx, (int)h->n_leaves, Coarse(), offsets, perm, B, st, 0, "leaf_bucketing");
 }
 
 fff_status_t fff_grouped_leaf_ff(fff_handle_t h, const void* x, const int32_t* leaf_idx, const int32_t* offsets,
@@ -642,7 +661,7 @@ fff_status_t fff_grouped_leaf_ff(fff_handle_t h, const void* x, const int32_t* l
         if ((s = grow_workspace(h, B)) != FFF_OK) return s;
         const int tile_rows = leaf_tile_rows(h, B);
         fff::k_tiles_from_offsets<<<1, fff::kBucketThreads, 0, st>>>(offsets, (int)h->n_leaves, tile_rows, h->ws_tiles,
-                                                                     h->ws_ntiles);
+                                                                     tile_list_len(B, tile_rows, (int)h->n_leaves));
         if ((s = launched(h, st, "tiles_from_offsets")) != FFF_OK) return s;
         return run_leaf_mma(h, x, perm, y, B, tile_rows, st);
     }
@@ -663,13 +682,17 @@ fff_status_t fff_forward_infer(fff_handle_t h, const void* x, void* y, int32_t* 
     h->prof_active = h->prof_steps < h->prof_max_steps;
     if (h->prof_active)
         cudaEventRecord(h->prof_events[(size_t)h->prof_steps * (fff_handle_s::kMaxProfLaunches + 1)], st);
-    s = run_descent(h, x, leaf, true, B, st);
+    Coarse coarse;
+    s = run_descent(h, x, leaf, &coarse, B, st);
     const bool tensor_leaf = use_tensor_leaf(h);
     const int tile_rows = tensor_leaf ? leaf_tile_rows(h, B) : 0;
-    if (s == FFF_OK) s = run_bucket(h, leaf, (int)h->n_leaves, h->ws_offsets, h->ws_perm, B, st, tile_rows, "leaf_bucketing");
+    // the final permutation goes to whichever buffer the last node bucketing did not use
+    h->last_perm = coarse.perm == h->ws_perm ? h->ws_perm2 : h->ws_perm;
     if (s == FFF_OK)
-        s = tensor_leaf ? run_leaf_mma(h, x, h->ws_perm, y, B, tile_rows, st)
-                        : FFF_DISPATCH(h, run_leaf, h, x, leaf, h->ws_perm, y, B, st);
+        s = run_bucket(h, leaf, (int)h->n_leaves, coarse, h->ws_offsets, h->last_perm, B, st, tile_rows, "leaf_bucketing");
+    if (s == FFF_OK)
+        s = tensor_leaf ? run_leaf_mma(h, x, h->last_perm, y, B, tile_rows, st)
+                        : FFF_DISPATCH(h, run_leaf, h, x, leaf, h->last_perm, y, B, st);
     if (h->prof_active) {
         h->prof_active = false;
         if (s == FFF_OK && (h->prof_steps == 0 || h->prof_nlaunch == h->launches)) {
@@ -715,7 +738,7 @@ fff_status_t fff_debug_get_bucketing(fff_handle_t h, int32_t* perm, int32_t* off
     DeviceGuard g(h->device);
     cudaStream_t st = (cudaStream_t)cuda_stream;
     if (h->last_B > 0 &&
-        cudaMemcpyAsync(perm, h->ws_perm, sizeof(int32_t) * (size_t)h->last_B, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        cudaMemcpyAsync(perm, h->last_perm, sizeof(int32_t) * (size_t)h->last_B, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
         return cudaGetLastError(), FFF_ERR_CUDA;
     if (h->last_B > 0) {
         if (cudaMemcpyAsync(offsets, h->ws_offsets, sizeof(int32_t) * (size_t)(h->n_leaves + 1), cudaMemcpyDeviceToDevice,

@@ -185,11 +185,29 @@ k_bucket(const int32_t* __restrict__ keys, const int* __restrict__ hist, int* __
 }
 
 // ---- cluster version ---------------------------------------------------------------------------
-// Same result as k_bucket, shorter critical path: the token ids are split over the 8 CTAs of a
-// thread-block cluster (256 warp slices instead of 32), the cluster as a whole owns one range of
-// bins, and the per-CTA column totals are exchanged through distributed shared memory.  Each warp
-// loads the keys of its slice in blocks of kBucketKeyRegs independent loads before it touches
-// shared memory, so the slice costs a few memory latencies instead of one per 32 tokens.
+// Self-contained stable bucketing: no histogram input, no atomics.
+//
+// A thread-block cluster of 8 CTAs owns one contiguous range of bins and one list of candidate
+// tokens; it counts, scans and places on its own:
+//   * global mode (seg_offsets == NULL): the candidates are all B tokens in natural order; cluster c
+//     owns bins [c*nb, (c+1)*nb) and ignores tokens whose key falls outside (it still counts the
+//     tokens with smaller keys, which gives the first output position of its range);
+//   * segmented mode: the tokens were already bucketed by a coarser key (perm_in, seg_offsets) and
+//     refining that order only moves tokens inside their old bucket.  Cluster c handles the tokens
+//     perm_in[seg_offsets[c] .. seg_offsets[c+1]), whose keys all lie in [c*nb, (c+1)*nb), and writes
+//     exactly that range of perm_out.  Work is spread over all old buckets at once.
+// The candidate list is split into 8 * NW contiguous slices, one per warp of the cluster.  Each warp
+// makes one matching pass over its slice (keys in registers when the slice has at most
+// 32 * kBucketKeyRegs tokens, else the per-token rank goes through `rank_tmp`), per-CTA totals are
+// exchanged through distributed shared memory, and a second trivial pass writes perm_out.
+//
+// Tile list (tile_rows > 0): cluster c writes the tiles of its bins starting at entry
+// floor(first_position / tile_rows) + c*nb -- an upper bound of the number of tiles before it -- and
+// pads its region up to the next cluster's start with empty tiles (rows = 0), so that the list has a
+// size known on the host, n_tiles_total = floor(B / tile_rows) + nbins, and needs no global scan.
+constexpr int kBucketClusterSize = 8;
+constexpr int kBucketKeyRegs = 8;
+
 // Lanes holding the same value v (only the low nbits bits may differ) among the lanes with `in` set;
 // built from one ballot per bit, which is far cheaper than the match instruction when a whole SM
 // issues it at once.  The result is only meaningful for lanes with `in` set.
@@ -204,73 +222,98 @@ __device__ __forceinline__ unsigned peers_by_ballot(bool in, int v, int nbits)
     return peers;
 }
 
-constexpr int kBucketClusterSize = 8;
-constexpr int kBucketKeyRegs = 8;
+template <int NW> __device__ __forceinline__ int block_sum_nw(int v, int* s_warp)
+{
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFullMask, v, o);
+    __syncthreads();
+    if (lane == 0) s_warp[w] = v;
+    __syncthreads();
+    int t = lane < NW ? s_warp[lane] : 0;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(kFullMask, t, o);
+    return t;
+}
 
-// Each warp makes ONE matching pass over its slice: it records, per token, the rank among the
-// earlier tokens of the same bin inside the slice (in registers when the slice fits kBucketKeyRegs
-// steps, else in `rank_tmp`, B ints of global scratch), and the per-(warp, bin) counts.  After the
-// counts have been turned into absolute start positions, a second, trivial pass writes perm.
-// Dynamic shared memory: (kBucketWarps + 1) * bins_per_cluster ints.
-template <bool kInRegs>
-__global__ void __launch_bounds__(kBucketThreads, 1)
-k_bucket_cluster(const int32_t* __restrict__ keys, const int* __restrict__ hist, int* __restrict__ hist_next,
-                 int32_t* __restrict__ offsets, int32_t* __restrict__ perm, int B, int nbins, int bins_per_cluster,
-                 int tile_rows, Tile* __restrict__ tiles, int* __restrict__ n_tiles, int bin_bits,
-                 int32_t* __restrict__ rank_tmp, int n_clear)
+// Exclusive prefix sum over the block in thread order; *total receives the block total.
+template <int NW> __device__ __forceinline__ int block_exclusive_scan_nw(int v, int* s_warp, int* total)
+{
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int u = __shfl_up_sync(kFullMask, incl, o);
+        if (lane >= o) incl += u;
+    }
+    __syncthreads();
+    if (lane == 31) s_warp[w] = incl;
+    __syncthreads();
+    int ws = lane < NW ? s_warp[lane] : 0;        // lane i holds the total of warp i
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int u = __shfl_up_sync(kFullMask, ws, o);
+        if (lane >= o) ws += u;
+    }
+    *total = __shfl_sync(kFullMask, ws, NW - 1);
+    const int before = __shfl_sync(kFullMask, ws, max(w - 1, 0));
+    return (w > 0 ? before : 0) + incl - v;
+}
+
+// Dynamic shared memory: (NW + 1) * nb ints.  Requires nb <= NW * 32.
+template <int NW>
+__global__ void __launch_bounds__(NW * 32, NW == 32 ? 1 : 4)
+k_bucket_cluster(const int32_t* __restrict__ keys, const int32_t* __restrict__ perm_in,
+                 const int32_t* __restrict__ seg_offsets, int32_t* __restrict__ offsets_out,
+                 int32_t* __restrict__ perm_out, int B, int nbins, int nb, int bin_bits, int tile_rows,
+                 Tile* __restrict__ tiles, int n_tiles_total, int32_t* __restrict__ rank_tmp)
 {
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
+    constexpr int kThreads = NW * 32;
     extern __shared__ int s_dyn[];
-    __shared__ int s_warp[kBucketWarps];
-    __shared__ int s_pub[2];
+    __shared__ int s_warp[32];
+    __shared__ int s_below;                          // tokens of this CTA's slices with a key below the range
 
-    const int nb = bins_per_cluster;
-    int* s_cnt = s_dyn;                            // [kBucketWarps][nb]
-    int* s_tot = s_dyn + kBucketWarps * nb;        // [nb] tokens of this CTA's slices per bin (read by peers)
+    int* s_cnt = s_dyn;                              // [NW][nb]
+    int* s_tot = s_dyn + NW * nb;                    // [nb] tokens of this CTA's slices per bin (read by peers)
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     const int rank = (int)cluster.block_rank();
-    const int range = blockIdx.x / kBucketClusterSize;
-    const int lo = range * nb;                     // host launches exactly ceil(nbins / nb) clusters
-    const int hi = min(lo + nb, nbins);
+    const int c = blockIdx.x / kBucketClusterSize;
+    const int n_clusters = gridDim.x / kBucketClusterSize;
+    const int lo = c * nb, hi = min(lo + nb, nbins);
+    const int seg_lo = seg_offsets ? seg_offsets[c] : 0;
+    const int seg_hi = seg_offsets ? seg_offsets[c + 1] : B;
     const unsigned lt_mask = (1u << lane) - 1u;
 
-    for (int i = tid; i < kBucketWarps * nb; i += kBucketThreads) s_cnt[i] = 0;
-    // clear the other histogram buffer (first n_clear counters hold an earlier call's counts)
-    for (int i = blockIdx.x * kBucketThreads + tid; i < n_clear; i += gridDim.x * kBucketThreads) hist_next[i] = 0;
+    for (int i = tid; i < NW * nb; i += kThreads) s_cnt[i] = 0;
+    __syncthreads();
 
-    int part = 0, tpart = 0;
-    if (rank == 0) {
-        for (int i = tid; i < lo; i += kBucketThreads) {
-            const int c = hist[i];
-            part += c;
-            if (tile_rows > 0) tpart += (c + tile_rows - 1) / tile_rows;
-        }
-    }
-    const int base = block_sum(part, s_warp);                        // meaningful on rank 0 only
-    const int tile_base = tile_rows > 0 ? block_sum(tpart, s_warp) : 0;
-    if (rank == 0 && tid == 0) { s_pub[0] = base; s_pub[1] = tile_base; }
-
-    const int slices = kBucketClusterSize * kBucketWarps;
-    const int chunk = (((B + slices - 1) / slices) + 31) & ~31;
-    const int t0 = min((rank * kBucketWarps + w) * chunk, B), t1 = min(t0 + chunk, B);
+    const int slices = kBucketClusterSize * NW;
+    const int chunk = ((((seg_hi - seg_lo) + slices - 1) / slices) + 31) & ~31;
+    const int t0 = min(seg_lo + (rank * NW + w) * chunk, seg_hi), t1 = min(t0 + chunk, seg_hi);
+    const bool in_regs = chunk <= 32 * kBucketKeyRegs;       // uniform over the cluster
     int* my = s_cnt + w * nb;
 
     // pass 1: count and rank inside the slice
-    int kreg[kBucketKeyRegs], rreg[kBucketKeyRegs];
+    int kreg[kBucketKeyRegs], rreg[kBucketKeyRegs], treg[kBucketKeyRegs];
 #pragma unroll
-    for (int i = 0; i < kBucketKeyRegs; ++i) { kreg[i] = -1; rreg[i] = 0; }
+    for (int i = 0; i < kBucketKeyRegs; ++i) { kreg[i] = -1; rreg[i] = 0; treg[i] = 0; }
+    int below = 0;
     for (int s0 = t0; s0 < t1; s0 += 32 * kBucketKeyRegs) {
 #pragma unroll
         for (int i = 0; i < kBucketKeyRegs; ++i) {
-            const int t = s0 + i * 32 + lane;
-            kreg[i] = t < t1 ? __ldg(keys + t) : -1;
+            const int idx = s0 + i * 32 + lane;
+            treg[i] = idx < t1 ? (perm_in ? __ldg(perm_in + idx) : idx) : -1;
         }
+#pragma unroll
+        for (int i = 0; i < kBucketKeyRegs; ++i) kreg[i] = treg[i] >= 0 ? __ldg(keys + treg[i]) : -1;
 #pragma unroll
         for (int i = 0; i < kBucketKeyRegs; ++i) {
             if (s0 + i * 32 >= t1) break;
             const int k = kreg[i];
             const bool in = k >= lo && k < hi;
+            below += (k >= 0 && k < lo) ? 1 : 0;
             const unsigned peers = peers_by_ballot(in, k - lo, bin_bits);
             const int leader = in ? __ffs(peers) - 1 : lane;
             int seen = 0;
@@ -279,11 +322,12 @@ k_bucket_cluster(const int32_t* __restrict__ keys, const int* __restrict__ hist,
                 my[k - lo] = seen + __popc(peers);
             }
             seen = __shfl_sync(kFullMask, seen, leader) + __popc(peers & lt_mask);
-            if (kInRegs) rreg[i] = seen;
+            if (in_regs) rreg[i] = seen;
             else if (in) rank_tmp[s0 + i * 32 + lane] = seen;
             __syncwarp();
         }
     }
+    const int below_cta = seg_offsets ? 0 : block_sum_nw<NW>(below, s_warp);
     __syncthreads();
 
     // per bin: offsets of the warps inside this CTA, and this CTA's total
@@ -291,68 +335,86 @@ k_bucket_cluster(const int32_t* __restrict__ keys, const int* __restrict__ hist,
     const bool mine = tid < nb && b < hi;
     if (mine) {
         int run = 0;
-        for (int ww = 0; ww < kBucketWarps; ++ww) {
+        for (int ww = 0; ww < NW; ++ww) {
             const int c2 = s_cnt[ww * nb + tid];
             s_cnt[ww * nb + tid] = run;
             run += c2;
         }
         s_tot[tid] = run;
     }
-    const int c = mine ? hist[b] : 0;
-    const int excl = block_exclusive_scan(c, s_warp);
+    if (tid == 0) s_below = below_cta;
     cluster.sync();
 
-    // bin starts (rank 0 publishes the base), tokens of lower-ranked CTAs per bin
-    const int* pub0 = reinterpret_cast<const int*>(cluster.map_shared_rank(s_pub, 0));
-    const int start = pub0[0] + excl;
-    const int tile_base0 = pub0[1];
+    // totals over the cluster, tokens of lower-ranked CTAs, first position of every bin
+    int total = 0, before = 0;
     if (mine) {
-        int before = 0;
-        for (int r = 0; r < rank; ++r) before += reinterpret_cast<const int*>(cluster.map_shared_rank(s_tot, r))[tid];
+#pragma unroll
+        for (int r = 0; r < kBucketClusterSize; ++r) {
+            const int v = reinterpret_cast<const int*>(cluster.map_shared_rank(s_tot, r))[tid];
+            total += v;
+            if (r < rank) before += v;
+        }
+    }
+    int first = seg_lo;                              // first output position of the cluster's range
+    if (!seg_offsets) {
+        first = 0;
+#pragma unroll
+        for (int r = 0; r < kBucketClusterSize; ++r) first += *reinterpret_cast<const int*>(cluster.map_shared_rank(&s_below, r));
+    }
+    int cluster_total = 0;
+    const int start = first + block_exclusive_scan_nw<NW>(total, s_warp, &cluster_total);
+    if (mine) {
         const int add = start + before;
-        for (int ww = 0; ww < kBucketWarps; ++ww) s_cnt[ww * nb + tid] += add;
+        for (int ww = 0; ww < NW; ++ww) s_cnt[ww * nb + tid] += add;
         if (rank == 0) {
-            offsets[b] = start;
-            if (b == nbins - 1) offsets[nbins] = start + c;
+            offsets_out[b] = start;
+            if (b == nbins - 1) offsets_out[nbins] = start + total;
         }
     }
     if (tile_rows > 0 && rank == 0) {
-        const int nt = (c + tile_rows - 1) / tile_rows;
-        const int tl0 = tile_base0 + block_exclusive_scan(nt, s_warp);
+        const int nt = (total + tile_rows - 1) / tile_rows;
+        int n_mine = 0;
+        const int region = first / tile_rows + lo;
+        const int tl0 = region + block_exclusive_scan_nw<NW>(nt, s_warp, &n_mine);
         if (mine) {
             for (int i = 0; i < nt; ++i) {
                 Tile tl;
                 tl.bin = b;
                 tl.start = start + i * tile_rows;
-                tl.rows = min(tile_rows, c - i * tile_rows);
+                tl.rows = min(tile_rows, total - i * tile_rows);
                 tl.pad = 0;
                 tiles[tl0 + i] = tl;
             }
-            if (b == nbins - 1) *n_tiles = tl0 + nt;
         }
+        const int region_end = c == n_clusters - 1 ? n_tiles_total : (first + cluster_total) / tile_rows + hi;
+        Tile empty;
+        empty.bin = 0; empty.start = 0; empty.rows = 0; empty.pad = 0;
+        for (int i = region + n_mine + tid; i < region_end; i += kThreads) tiles[i] = empty;
     }
     __syncthreads();
 
     // pass 2: place
-    if (kInRegs) {
+    if (in_regs) {
 #pragma unroll
         for (int i = 0; i < kBucketKeyRegs; ++i) {
             const int k = kreg[i];
-            if (k >= lo && k < hi) perm[my[k - lo] + rreg[i]] = t0 + i * 32 + lane;
+            if (k >= lo && k < hi) perm_out[my[k - lo] + rreg[i]] = treg[i];
         }
     } else {
-        for (int t = t0 + lane; t < t1; t += 32) {
+        for (int idx = t0 + lane; idx < t1; idx += 32) {
+            const int t = perm_in ? __ldg(perm_in + idx) : idx;
             const int k = __ldg(keys + t);
-            if (k >= lo && k < hi) perm[my[k - lo] + rank_tmp[t]] = t;
+            if (k >= lo && k < hi) perm_out[my[k - lo] + rank_tmp[idx]] = t;
         }
     }
     cluster.sync();      // peers may still be reading this CTA's shared memory
 }
 
-// Tile list from an existing offsets array (one CTA; used when the caller supplies the bucketing).
+// Tile list from an existing offsets array (one CTA; used when the caller supplies the bucketing),
+// padded with empty tiles up to n_tiles_total = floor(B / tile_rows) + nbins.
 __global__ void __launch_bounds__(kBucketThreads)
 k_tiles_from_offsets(const int32_t* __restrict__ offsets, int nbins, int tile_rows, Tile* __restrict__ tiles,
-                     int* __restrict__ n_tiles)
+                     int n_tiles_total)
 {
     __shared__ int s_warp[kBucketWarps];
     int tile_base = 0;
@@ -372,7 +434,9 @@ k_tiles_from_offsets(const int32_t* __restrict__ offsets, int nbins, int tile_ro
         }
         tile_base += block_sum(nt, s_warp);
     }
-    if (threadIdx.x == 0) *n_tiles = tile_base;
+    Tile empty;
+    empty.bin = 0; empty.start = 0; empty.rows = 0; empty.pad = 0;
+    for (int i = tile_base + threadIdx.x; i < n_tiles_total; i += kBucketThreads) tiles[i] = empty;
 }
 
 }  // namespace fff

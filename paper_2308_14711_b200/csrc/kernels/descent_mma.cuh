@@ -69,9 +69,9 @@ __global__ void k_pack_nodes(const T* __restrict__ node_w, const T* __restrict__
 template <int NP, int S>
 __global__ void __launch_bounds__(kDescentThreads)
 k_descent_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ perm,
-              const Tile* __restrict__ tiles, const int* __restrict__ n_tiles_ptr, int n_tiles_static,
+              const Tile* __restrict__ tiles, int n_tiles_total,
               const __nv_bfloat16* __restrict__ wimg, const float* __restrict__ bimg,
-              int32_t* __restrict__ pos_out, int* __restrict__ hist,
+              int32_t* __restrict__ pos_out,
               int D, int B, int k, int* __restrict__ status)
 {
     using L = DescentMmaLayout<NP, S>;
@@ -87,7 +87,7 @@ k_descent_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ p
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int U1 = D / kKS;
-    const int ntiles = tiles ? *n_tiles_ptr : n_tiles_static;
+    const int ntiles = n_tiles_total;      // a device-built list may contain empty tiles (rows = 0)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -121,6 +121,7 @@ k_descent_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ p
         const int prow = ptid >> 4, pchunk = ptid & 15;
         for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
             const Tile tl = get_tile(tile);
+            if (tl.rows == 0) continue;
             const __nv_bfloat16* src[kTM / kRowsPerPass];
 #pragma unroll
             for (int i = 0; i < kTM / kRowsPerPass; ++i) {
@@ -150,6 +151,7 @@ k_descent_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ p
         const int g = lane >> 2, q4 = lane & 3;
         for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
             const Tile tl = get_tile(tile);
+            if (tl.rows == 0) continue;
             const bool active = m0 < tl.rows;
 
             // epilogue operands, fetched now so that their latency hides behind the K loop
@@ -211,7 +213,6 @@ k_descent_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ p
                     for (int r = 0; r < k; ++r) p = 2 * p + 1 + (row[p] >= 0.0f ? 1 : 0);
                     const int pos = (tl.bin << k) + (p - ((1 << k) - 1));
                     pos_out[my_tok] = pos;
-                    if (hist) atomicAdd(hist + pos, 1);
                 }
                 __syncwarp();
             }

@@ -19,12 +19,12 @@ constexpr int kDescentWarps = 8;
 
 // level0 / pos_in: the walk starts at node N_{level0, pos_in[t]} (pos_in NULL = position 0)
 // and continues for `levels` levels; pos_out[t] receives the position reached at level
-// level0 + levels.  hist (nullable) counts tokens per final position.
+// level0 + levels.
 template <typename T>
 __global__ void __launch_bounds__(kDescentWarps * 32)
 k_descent_warp(const T* __restrict__ x, const T* __restrict__ node_w, const T* __restrict__ node_b,
                int D, int level0, int levels, const int32_t* __restrict__ pos_in,
-               int32_t* __restrict__ pos_out, int* __restrict__ hist, int64_t B, bool vec)
+               int32_t* __restrict__ pos_out, int64_t B, bool vec)
 {
     const int lane = threadIdx.x & 31;
     const int64_t warp0 = (int64_t)blockIdx.x * kDescentWarps + (threadIdx.x >> 5);
@@ -37,10 +37,7 @@ k_descent_warp(const T* __restrict__ x, const T* __restrict__ node_w, const T* _
             const float logit = warp_dot<T>(node_w + row * D, xt, D, vec, lane) + Elem<T>::to_float(node_b[row]);
             n = 2 * n + (logit >= 0.0f ? 1 : 0);
         }
-        if (lane == 0) {
-            pos_out[t] = (int32_t)n;
-            if (hist) atomicAdd(hist + n, 1);
-        }
+        if (lane == 0) pos_out[t] = (int32_t)n;
     }
 }
 

@@ -119,7 +119,7 @@ __global__ void k_pack_b1(const T* __restrict__ b1, float* __restrict__ img, int
 template <int LP, int TM, int S>
 __global__ void __launch_bounds__((TM / 16 + kProducerWarps) * 32)
 k_leaf_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ perm,
-           const Tile* __restrict__ tiles, const int* __restrict__ n_tiles,
+           const Tile* __restrict__ tiles, int n_tiles_total,
            const __nv_bfloat16* __restrict__ w1img, const float* __restrict__ b1img,
            const unsigned char* __restrict__ w2img, __nv_bfloat16* __restrict__ y,
            int D, int O, int act, int* __restrict__ status)
@@ -138,7 +138,7 @@ k_leaf_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ perm
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int U1 = D / kKS;
     const int U2 = (O + kNC - 1) / kNC;
-    const int ntiles = *n_tiles;
+    const int ntiles = n_tiles_total;      // the list may contain empty tiles (rows = 0)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -159,6 +159,7 @@ k_leaf_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ perm
         const int prow = ptid >> 4, pchunk = ptid & 15;
         for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
             const Tile tl = tiles[tile];
+            if (tl.rows == 0) continue;
             const __nv_bfloat16* src[kTM / kRowsPerPass];
 #pragma unroll
             for (int i = 0; i < kTM / kRowsPerPass; ++i) {
@@ -197,6 +198,7 @@ k_leaf_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ perm
         const int g = lane >> 2, q4 = lane & 3;
         for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
             const Tile tl = tiles[tile];
+            if (tl.rows == 0) continue;
             const bool active = m0 < tl.rows;          // warps without valid rows only keep the ring moving
 
             // epilogue operands, fetched now so that their latency hides behind the K loop
