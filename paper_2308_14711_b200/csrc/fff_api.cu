@@ -411,7 +411,7 @@ fff_status_t run_leaf_mma(fff_handle_s* h, const void* x, const int32_t* perm, v
         switch (h->LP) {
             case 16: return launch_leaf_mma<16, 64, 4>(h, x, perm, y, B, st);
             case 32: return launch_leaf_mma<32, 64, 3>(h, x, perm, y, B, st);
-            case 64: return launch_leaf_mma<64, 64, 5>(h, x, perm, y, B, st);
+            case 64: return launch_leaf_mma<64, 64, 4>(h, x, perm, y, B, st);
         }
     }
     return FFF_ERR_UNSUPPORTED;

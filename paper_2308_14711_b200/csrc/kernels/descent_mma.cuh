@@ -130,7 +130,7 @@ k_descent_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ p
                 src[i] = tok >= 0 ? x + tok * D + pchunk * 8 : nullptr;
             }
             for (int u = 0; u < U1; ++u) {
-                if (!timed_out && !ptx::mbar_wait(empty + stage, phase ^ 1)) timed_out = true;
+                if (!timed_out && !ptx::mbar_wait_relaxed(empty + stage, phase ^ 1)) timed_out = true;
                 unsigned char* st = stages + stage * L::kStageStride;
                 if (ptid == 0) {
                     ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)L::kWStageBytes);

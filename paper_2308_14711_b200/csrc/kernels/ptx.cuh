@@ -53,6 +53,19 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     return true;
 }
 
+// The same for waits that are not latency-critical (producers waiting for a free slot): sleeps
+// between polls so that the polling warp leaves the issue slots of its scheduler to the warps that
+// do the arithmetic.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        __nanosleep(200);
+        if (clock64() - t0 > kWaitCycles) return false;
+    }
+    return true;
+}
+
 // Global -> shared bulk copy of `bytes` (multiple of 16, both addresses 16-byte aligned),
 // completion counted in bytes on `bar`.
 __device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {
