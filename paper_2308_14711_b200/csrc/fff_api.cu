@@ -82,6 +82,7 @@ struct fff_handle_s {
     int32_t *st_leaf = nullptr;
 
     int path = FFF_PATH_AUTO;
+    bool pdl = true;              // launch every kernel of a forward but the first as a programmatic dependent
     int launches = 0;
     int64_t last_B = -1;
 
@@ -120,6 +121,38 @@ fff_status_t clone(void** dst, const void* src, size_t bytes) {
     if (s != FFF_OK) return s;
     cudaError_t e = src ? cudaMemcpy(*dst, src, bytes, cudaMemcpyDeviceToDevice) : cudaMemset(*dst, 0, bytes ? bytes : 16);
     return e == cudaSuccess ? FFF_OK : (cudaGetLastError(), FFF_ERR_CUDA);
+}
+
+// Launch a kernel of the forward chain.  Every launch after the first of a call carries the
+// programmatic-stream-serialization attribute: the kernel may be scheduled while its predecessor is
+// still draining, runs its prologue, and waits in griddepcontrol.wait (cudaGridDependencySynchronize)
+// until the predecessor has completed and flushed its results.  Every kernel launched through here
+// calls that wait before its first global read.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chain(fff_handle_s* h, void (*kern)(KArgs...), unsigned grid, unsigned block, size_t smem, cudaStream_t st,
+                         int cluster, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    if (cluster > 1) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = (unsigned)cluster;
+        attr[n].val.clusterDim.y = 1;
+        attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    if (h->pdl && h->launches > 0 && !h->prof_active) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = (unsigned)n;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
 }
 
 void prof_free(fff_handle_s* h) {
@@ -202,23 +235,12 @@ struct Coarse {
 };
 
 template <int NW>
-cudaError_t launch_bucket(int clusters, size_t smem, cudaStream_t st, const int32_t* keys, const int32_t* perm_in,
-                          const int32_t* seg_offsets, int32_t* offsets, int32_t* perm, int B, int nbins, int nb, int bin_bits,
-                          int tile_rows, fff::Tile* tiles, int n_tiles_total, int32_t* rank_tmp) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(clusters * fff::kBucketClusterSize));
-    cfg.blockDim = dim3(NW * 32);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = fff::kBucketClusterSize;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, fff::k_bucket_cluster<NW>, keys, perm_in, seg_offsets, offsets, perm, B, nbins, nb, bin_bits,
-                              tile_rows, tiles, n_tiles_total, rank_tmp);
+cudaError_t launch_bucket(fff_handle_s* h, int clusters, size_t smem, cudaStream_t st, const int32_t* keys,
+                          const int32_t* perm_in, const int32_t* seg_offsets, int32_t* offsets, int32_t* perm, int B, int nbins,
+                          int nb, int bin_bits, int tile_rows, fff::Tile* tiles, int n_tiles_total, int32_t* rank_tmp) {
+    return launch_chain(h, fff::k_bucket_cluster<NW>, (unsigned)(clusters * fff::kBucketClusterSize), NW * 32, smem, st,
+                        fff::kBucketClusterSize, keys, perm_in, seg_offsets, offsets, perm, B, nbins, nb, bin_bits, tile_rows,
+                        tiles, n_tiles_total, rank_tmp);
 }
 
 // Stable bucketing of B keys in [0, nbins) into (offsets, perm).  If `coarse` describes a bucketing by
@@ -234,10 +256,10 @@ fff_status_t run_bucket(fff_handle_s* h, const int32_t* keys, int nbins, const C
         int bin_bits = 0;
         while ((1 << bin_bits) < nb) ++bin_bits;
         if (nb <= 256)
-            e = launch_bucket<8>(coarse.bins, sizeof(int) * (size_t)(8 + 1) * nb, st, keys, coarse.perm, coarse.offsets, offsets,
+            e = launch_bucket<8>(h, coarse.bins, sizeof(int) * (size_t)(8 + 1) * nb, st, keys, coarse.perm, coarse.offsets, offsets,
                                  perm, (int)B, nbins, nb, bin_bits, tile_rows, h->ws_tiles, n_tiles_total, h->ws_rank);
         else
-            e = launch_bucket<32>(coarse.bins, sizeof(int) * (size_t)(32 + 1) * nb, st, keys, coarse.perm, coarse.offsets,
+            e = launch_bucket<32>(h, coarse.bins, sizeof(int) * (size_t)(32 + 1) * nb, st, keys, coarse.perm, coarse.offsets,
                                   offsets, perm, (int)B, nbins, nb, bin_bits, tile_rows, h->ws_tiles, n_tiles_total, h->ws_rank);
     } else {
         // Every cluster reads all keys, so more clusters do not shorten the kernel; they only shrink the
@@ -248,7 +270,7 @@ fff_status_t run_bucket(fff_handle_s* h, const int32_t* keys, int nbins, const C
         clusters = (nbins + nb - 1) / nb;
         int bin_bits = 0;
         while ((1 << bin_bits) < nb) ++bin_bits;
-        e = launch_bucket<32>(clusters, sizeof(int) * (size_t)(32 + 1) * nb, st, keys, nullptr, nullptr, offsets, perm, (int)B,
+        e = launch_bucket<32>(h, clusters, sizeof(int) * (size_t)(32 + 1) * nb, st, keys, nullptr, nullptr, offsets, perm, (int)B,
                               nbins, nb, bin_bits, tile_rows, h->ws_tiles, n_tiles_total, h->ws_rank);
     }
     if (e != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
@@ -262,9 +284,10 @@ fff_status_t launch_descent_mma(fff_handle_s* h, const fff_handle_s::DenseStage&
     const int per_sm = std::max(1, std::min(3, (int)((227 * 1024) / (L::kSmemBytes + 1024))));
     const int n_tiles = grouped ? tile_list_len(B, fff::kDTM, 1 << sg.L0) : (int)((B + fff::kDTM - 1) / fff::kDTM);
     const int64_t grid = std::max<int64_t>(1, std::min<int64_t>((int64_t)h->sm_count * per_sm, n_tiles));
-    fff::k_descent_mma<NP, S><<<(unsigned)grid, fff::kDescentThreads, L::kSmemBytes, st>>>(
-        (const __nv_bfloat16*)x, grouped ? perm : nullptr, grouped ? h->ws_tiles : nullptr, n_tiles, sg.wimg, sg.bimg, pos_out,
-        h->D, (int)B, sg.k, h->d_status);
+    if (launch_chain(h, fff::k_descent_mma<NP, S>, (unsigned)grid, fff::kDescentThreads, L::kSmemBytes, st, 1,
+                     (const __nv_bfloat16*)x, grouped ? perm : nullptr, grouped ? h->ws_tiles : nullptr, n_tiles, sg.wimg,
+                     sg.bimg, pos_out, h->D, (int)B, sg.k, h->d_status) != cudaSuccess)
+        return cudaGetLastError(), FFF_ERR_CUDA;
     return launched(h, st, "tree_descent_mma");
 }
 
@@ -285,9 +308,10 @@ template <typename T>
 fff_status_t run_descent_warp(fff_handle_s* h, const void* x, int level0, int levels, const int32_t* pos_in,
                               int32_t* pos_out, int64_t B, cudaStream_t st) {
     const int64_t blocks = std::min<int64_t>((B + fff::kDescentWarps - 1) / fff::kDescentWarps, (int64_t)h->sm_count * 8);
-    fff::k_descent_warp<T><<<(unsigned)blocks, fff::kDescentWarps * 32, 0, st>>>(
-        (const T*)x, (const T*)h->node_w, (const T*)h->node_b, h->D, level0, levels, pos_in, pos_out, B,
-        h->vec_ok && aligned16(x));
+    if (launch_chain(h, fff::k_descent_warp<T>, (unsigned)blocks, fff::kDescentWarps * 32, 0, st, 1, (const T*)x,
+                     (const T*)h->node_w, (const T*)h->node_b, h->D, level0, levels, pos_in, pos_out, B,
+                     h->vec_ok && aligned16(x)) != cudaSuccess)
+        return cudaGetLastError(), FFF_ERR_CUDA;
     return launched(h, st, "tree_descent_warp");
 }
 
@@ -375,9 +399,10 @@ fff_status_t run_leaf(fff_handle_s* h, const void* x, const int32_t* leaf_idx, c
                       int64_t B, cudaStream_t st) {
     const int64_t blocks = std::min<int64_t>((B + fff::kLeafWarps - 1) / fff::kLeafWarps, (int64_t)h->sm_count * 8);
     const size_t smem = sizeof(float) * (size_t)fff::kLeafWarps * h->l;
-    fff::k_leaf_warp<T><<<(unsigned)blocks, fff::kLeafWarps * 32, smem, st>>>(
-        (const T*)x, leaf_idx, perm, (const T*)h->w1, (const T*)h->b1, (const T*)h->w2, (const T*)h->b2, (T*)y,
-        h->D, h->O, h->l, h->act, B, h->vec_ok && aligned16(x));
+    if (launch_chain(h, fff::k_leaf_warp<T>, (unsigned)blocks, fff::kLeafWarps * 32, smem, st, 1, (const T*)x, leaf_idx, perm,
+                     (const T*)h->w1, (const T*)h->b1, (const T*)h->w2, (const T*)h->b2, (T*)y, h->D, h->O, h->l, h->act, B,
+                     h->vec_ok && aligned16(x)) != cudaSuccess)
+        return cudaGetLastError(), FFF_ERR_CUDA;
     return launched(h, st, "grouped_leaf_ff_warp");
 }
 
@@ -392,9 +417,10 @@ fff_status_t launch_leaf_mma(fff_handle_s* h, const void* x, const int32_t* perm
     }
     const int per_sm = std::max(1, std::min(2, (int)((227 * 1024) / (L::kSmemBytes + 1024))));
     const int64_t grid = std::min<int64_t>((int64_t)h->sm_count * per_sm, n_tiles);
-    fff::k_leaf_mma<LP, TM, S><<<(unsigned)grid, L::kThreads, L::kSmemBytes, st>>>(
-        (const __nv_bfloat16*)x, perm, h->ws_tiles, n_tiles, h->w1img, h->b1img, h->w2img, (__nv_bfloat16*)y, h->D,
-        h->O, h->act, h->d_status);
+    if (launch_chain(h, fff::k_leaf_mma<LP, TM, S>, (unsigned)grid, L::kThreads, L::kSmemBytes, st, 1,
+                     (const __nv_bfloat16*)x, perm, h->ws_tiles, n_tiles, h->w1img, h->b1img, h->w2img, (__nv_bfloat16*)y, h->D,
+                     h->O, h->act, h->d_status) != cudaSuccess)
+        return cudaGetLastError(), FFF_ERR_CUDA;
     return launched(h, st, "grouped_leaf_ff_mma");
 }
 

@@ -282,6 +282,8 @@ k_bucket_cluster(const int32_t* __restrict__ keys, const int32_t* __restrict__ p
     const int c = blockIdx.x / kBucketClusterSize;
     const int n_clusters = gridDim.x / kBucketClusterSize;
     const int lo = c * nb, hi = min(lo + nb, nbins);
+    pdl_trigger();
+    pdl_wait();
     const int seg_lo = seg_offsets ? seg_offsets[c] : 0;
     const int seg_hi = seg_offsets ? seg_offsets[c + 1] : B;
     const unsigned lt_mask = (1u << lane) - 1u;

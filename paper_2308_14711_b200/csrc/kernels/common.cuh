@@ -20,6 +20,13 @@ struct Tile {
     int bin, start, rows, pad;
 };
 
+// Programmatic dependent launch.  pdl_trigger: the next kernel in the stream may be scheduled from now
+// on.  pdl_wait: block until the previous kernel in the stream has completed and its writes are
+// visible; must precede the first read of anything that kernel produced.  Both are no-ops for a
+// kernel that was launched the ordinary way.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 template <typename T> struct Elem;
 
 template <> struct Elem<float> {

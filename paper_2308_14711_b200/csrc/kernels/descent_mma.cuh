@@ -14,7 +14,8 @@
 // The machinery is that of the grouped leaf kernel: persistent CTAs over a tile list (tiles of up to
 // 64 consecutive entries of one group), producer warps that copy the gathered token rows with
 // 16-byte cp.async and a pre-swizzled weight image with one bulk (TMA) copy per stage into an
-// mbarrier ring, and 4 consumer warps with mma.sync.m16n8k16.  tiles == NULL means "one group, tokens in natural order".
+// mbarrier ring, and 8 consumer warps with mma.sync.m16n8k16 (two per 16-row m-tile, taking alternate
+// k-steps).  tiles == NULL means "one group, tokens in natural order".
 //
 // Requirements: bf16, D % kKS == 0.
 #pragma once
@@ -26,7 +27,11 @@
 namespace fff {
 
 constexpr int kDTM = 64;                                   // token rows per tile of the descent stages
-constexpr int kDescentConsumers = kDTM / 16;
+constexpr int kDescentMTiles = kDTM / 16;
+// Two warps share each 16-row m-tile and take alternate k-steps (a single warp would crawl along one
+// chain of dependent mma); the pair adds its partial logits up through shared memory.
+constexpr int kDescentKSplit = 2;
+constexpr int kDescentConsumers = kDescentMTiles * kDescentKSplit;
 constexpr int kDescentThreads = (kDescentConsumers + kProducerWarps) * 32;
 
 template <int NP, int S> struct DescentMmaLayout {
@@ -34,7 +39,9 @@ template <int NP, int S> struct DescentMmaLayout {
     static constexpr int kStageBytes = kDTM * kXRowBytes + kWStageBytes;
     static constexpr int kStageStride = (kStageBytes + 127) & ~127;
     static constexpr int kLogitRow = NP + 1;                                     // floats, padded
-    static constexpr int kStagingBytes = kDescentConsumers * 16 * kLogitRow * 4;
+    // one scratch area per warp pair: partial accumulators (fragment order), then the 16 logit rows
+    static constexpr int kPairScratch = (16 * kLogitRow * 4 > NP * 64 ? 16 * kLogitRow * 4 : NP * 64);
+    static constexpr int kStagingBytes = kDescentMTiles * kPairScratch;
     static constexpr int kSmemBytes = S * kStageStride + ((kStagingBytes + 127) & ~127) + 128 + 128;
     static_assert(S <= kMaxStages, "barrier area holds 2 * kMaxStages mbarriers");
 };
@@ -67,7 +74,7 @@ __global__ void k_pack_nodes(const T* __restrict__ node_w, const T* __restrict__
 }
 
 template <int NP, int S>
-__global__ void __launch_bounds__(kDescentThreads)
+__global__ void __launch_bounds__(kDescentThreads, NP <= 32 ? 2 : 1)
 k_descent_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ perm,
               const Tile* __restrict__ tiles, int n_tiles_total,
               const __nv_bfloat16* __restrict__ wimg, const float* __restrict__ bimg,
@@ -81,7 +88,7 @@ k_descent_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ p
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     unsigned char* stages = smem;
-    float* staging = reinterpret_cast<float*>(smem + kStages * L::kStageStride);
+    unsigned char* staging = smem + kStages * L::kStageStride;
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStages * L::kStageStride + ((L::kStagingBytes + 127) & ~127));
     uint64_t* empty = full + kStages;
 
@@ -96,7 +103,9 @@ k_descent_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ p
         }
         ptx::fence_mbar_init();
     }
+    pdl_trigger();
     __syncthreads();
+    pdl_wait();
 
     int stage = 0;
     uint32_t phase = 0;
@@ -146,9 +155,12 @@ k_descent_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ p
         }
     } else {
         // ------------------------------------------------------------------ consumer warps
-        const int m0 = warp * 16;
-        float* my_logits = staging + warp * 16 * L::kLogitRow;
+        const int mi = warp % kDescentMTiles, ni = warp / kDescentMTiles;
+        const int m0 = mi * 16;
+        float* pair = reinterpret_cast<float*>(staging + mi * L::kPairScratch);
         const int g = lane >> 2, q4 = lane & 3;
+        const int bn = (lane & 7) + ((lane >> 4) << 3);
+        const int bk = ((lane >> 3) & 1) * 8;
         for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
             const Tile tl = get_tile(tile);
             if (tl.rows == 0) continue;
@@ -156,11 +168,13 @@ k_descent_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ p
 
             // epilogue operands, fetched now so that their latency hides behind the K loop
             const int my_row = m0 + (lane & 15);
-            const int64_t my_tok = (active && my_row < tl.rows) ? (perm ? perm[tl.start + my_row] : tl.start + my_row) : -1;
+            const int64_t my_tok =
+                (ni == 0 && active && my_row < tl.rows) ? (perm ? perm[tl.start + my_row] : tl.start + my_row) : -1;
             float2 bias2[NP / 8];
 #pragma unroll
             for (int nt = 0; nt < NP / 8; ++nt)
-                bias2[nt] = __ldg(reinterpret_cast<const float2*>(bimg + (int64_t)tl.bin * NP + nt * 8 + 2 * q4));
+                bias2[nt] = ni == 0 ? __ldg(reinterpret_cast<const float2*>(bimg + (int64_t)tl.bin * NP + nt * 8 + 2 * q4))
+                                    : make_float2(0.0f, 0.0f);
 
             float acc[NP / 8][4];
 #pragma unroll
@@ -174,10 +188,9 @@ k_descent_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ p
                     const uint32_t xs = ptx::smem_addr(stages + stage * L::kStageStride);
                     const uint32_t ws = xs + kTM * kXRowBytes;
                     const uint32_t a_base = xs + (m0 + (lane & 15)) * kXRowBytes + (lane >> 4) * 16;
-                    const int bn = (lane & 7) + ((lane >> 4) << 3);
-                    const int bk = ((lane >> 3) & 1) * 8;
 #pragma unroll
-                    for (int ks = 0; ks < kKS / 16; ++ks) {
+                    for (int kq = 0; kq < (kKS / 16) / kDescentKSplit; ++kq) {
+                        const int ks = kq * kDescentKSplit + ni;
                         uint32_t a0, a1, a2, a3;
                         ptx::ldmatrix_x4(a_base + ks * 32, a0, a1, a2, a3);
                         const int kcol = ks * 16 + bk;
@@ -197,25 +210,40 @@ k_descent_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ p
                 if (++stage == kStages) { stage = 0; phase ^= 1; }
             }
 
-            if (active) {
-                // logits of the 16 rows of this warp -> shared memory, then one lane per row walks the subtree
+            // the second warp of the pair hands over its partial sums; the first adds them, lays the 16
+            // logit rows out in shared memory, and one lane per row walks the subtree
+            if (ni == 1) {
 #pragma unroll
-                for (int nt = 0; nt < NP / 8; ++nt) {
-                    my_logits[g * L::kLogitRow + nt * 8 + 2 * q4] = acc[nt][0] + bias2[nt].x;
-                    my_logits[g * L::kLogitRow + nt * 8 + 2 * q4 + 1] = acc[nt][1] + bias2[nt].y;
-                    my_logits[(g + 8) * L::kLogitRow + nt * 8 + 2 * q4] = acc[nt][2] + bias2[nt].x;
-                    my_logits[(g + 8) * L::kLogitRow + nt * 8 + 2 * q4 + 1] = acc[nt][3] + bias2[nt].y;
-                }
-                __syncwarp();
-                if (lane < 16 && my_tok >= 0) {
-                    const float* row = my_logits + lane * L::kLogitRow;
-                    int p = 0;
-                    for (int r = 0; r < k; ++r) p = 2 * p + 1 + (row[p] >= 0.0f ? 1 : 0);
-                    const int pos = (tl.bin << k) + (p - ((1 << k) - 1));
-                    pos_out[my_tok] = pos;
-                }
-                __syncwarp();
+                for (int nt = 0; nt < NP / 8; ++nt)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) pair[(nt * 4 + c) * 32 + lane] = acc[nt][c];
             }
+            asm volatile("bar.sync %0, %1;" ::"r"(1 + mi), "r"(kDescentKSplit * 32) : "memory");
+            if (ni == 0) {
+#pragma unroll
+                for (int nt = 0; nt < NP / 8; ++nt)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) acc[nt][c] += pair[(nt * 4 + c) * 32 + lane];
+                __syncwarp();       // every lane has read its partials before the area is reused for the rows
+                if (active) {
+#pragma unroll
+                    for (int nt = 0; nt < NP / 8; ++nt) {
+                        pair[g * L::kLogitRow + nt * 8 + 2 * q4] = acc[nt][0] + bias2[nt].x;
+                        pair[g * L::kLogitRow + nt * 8 + 2 * q4 + 1] = acc[nt][1] + bias2[nt].y;
+                        pair[(g + 8) * L::kLogitRow + nt * 8 + 2 * q4] = acc[nt][2] + bias2[nt].x;
+                        pair[(g + 8) * L::kLogitRow + nt * 8 + 2 * q4 + 1] = acc[nt][3] + bias2[nt].y;
+                    }
+                    __syncwarp();
+                    if (lane < 16 && my_tok >= 0) {
+                        const float* row = pair + lane * L::kLogitRow;
+                        int p = 0;
+                        for (int r = 0; r < k; ++r) p = 2 * p + 1 + (row[p] >= 0.0f ? 1 : 0);
+                        pos_out[my_tok] = (tl.bin << k) + (p - ((1 << k) - 1));
+                    }
+                    __syncwarp();
+                }
+            }
+            asm volatile("bar.sync %0, %1;" ::"r"(1 + mi), "r"(kDescentKSplit * 32) : "memory");
         }
     }
     if (timed_out) {

@@ -26,6 +26,8 @@ k_descent_warp(const T* __restrict__ x, const T* __restrict__ node_w, const T* _
                int D, int level0, int levels, const int32_t* __restrict__ pos_in,
                int32_t* __restrict__ pos_out, int64_t B, bool vec)
 {
+    pdl_trigger();
+    pdl_wait();
     const int lane = threadIdx.x & 31;
     const int64_t warp0 = (int64_t)blockIdx.x * kDescentWarps + (threadIdx.x >> 5);
     const int64_t nwarps = (int64_t)gridDim.x * kDescentWarps;

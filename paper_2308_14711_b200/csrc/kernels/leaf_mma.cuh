@@ -157,7 +157,9 @@ k_leaf_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ perm
         }
         ptx::fence_mbar_init();
     }
+    pdl_trigger();
     __syncthreads();
+    pdl_wait();
 
     int stage = 0;
     uint32_t phase = 0;

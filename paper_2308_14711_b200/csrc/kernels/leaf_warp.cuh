@@ -28,6 +28,8 @@ k_leaf_warp(const T* __restrict__ x, const int32_t* __restrict__ leaf_idx, const
             T* __restrict__ y, int D, int O, int l, int act, int64_t B, bool vec)
 {
     extern __shared__ float s_h[];
+    pdl_trigger();
+    pdl_wait();
     constexpr int V = Elem<T>::kVec;
     constexpr int U = kLeafHiddenUnroll;
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
