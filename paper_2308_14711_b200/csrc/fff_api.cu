@@ -63,6 +63,8 @@ struct fff_handle_s {
     int32_t* ws_rank = nullptr;   // per-token rank scratch of the bucketing kernel (large batches only)
     int max_bucket_clusters = 8;
     int32_t* last_perm = nullptr; // where the most recent forward left its leaf permutation
+    int* ws_matrix = nullptr;     // per-CTA bin totals of the grid-wide bucketing kernel
+    int coop_ctas = 0;            // CTAs of that kernel that are resident at once (0 = cooperative launch unavailable)
     int32_t* ws_perm2 = nullptr;  // second permutation buffer: successive bucketings alternate between the two
     int32_t* ws_offsets2[2] = {nullptr, nullptr};   // offsets of the intermediate (node) bucketings
 
@@ -168,7 +170,7 @@ void release(fff_handle_s* h) {
     dfree(h->d_status); dfree(h->st_x); dfree(h->st_y); dfree(h->st_leaf);
     for (auto& sg : h->stages) { dfree(sg.wimg); dfree(sg.bimg); }
     dfree(h->ws_pos[0]); dfree(h->ws_pos[1]);
-    dfree(h->w1img); dfree(h->b1img); dfree(h->w2img); dfree(h->ws_tiles); dfree(h->ws_rank);
+    dfree(h->w1img); dfree(h->b1img); dfree(h->w2img); dfree(h->ws_tiles); dfree(h->ws_rank); dfree(h->ws_matrix);
     prof_free(h);
     h->magic = 0;
     delete h;
@@ -261,6 +263,19 @@ fff_status_t run_bucket(fff_handle_s* h, const int32_t* keys, int nbins, const C
         else
             e = launch_bucket<32>(h, coarse.bins, sizeof(int) * (size_t)(32 + 1) * nb, st, keys, coarse.perm, coarse.offsets,
                                   offsets, perm, (int)B, nbins, nb, bin_bits, tile_rows, h->ws_tiles, n_tiles_total, h->ws_rank);
+    } else if (h->coop_ctas > 0 && nbins <= fff::kBucketMaxBinsPerCta && B >= 4096) {
+        // few bins, no previous bucketing: one token slice per SM and one grid-wide barrier
+        const int ctas = (int)std::min<int64_t>(h->coop_ctas, (B + 255) / 256);
+        int bin_bits = 0;
+        while ((1 << bin_bits) < nbins) ++bin_bits;
+        int Bi = (int)B, tr = tile_rows, nbi = nbins, ntt = n_tiles_total;
+        const int32_t* k = keys;
+        fff::Tile* tiles = h->ws_tiles;
+        int32_t* rank = h->ws_rank;
+        int* matrix = h->ws_matrix;
+        void* args[] = {&k, &offsets, &perm, &Bi, &nbi, &bin_bits, &tr, &tiles, &ntt, &rank, &matrix};
+        e = cudaLaunchCooperativeKernel((const void*)fff::k_bucket_coop, dim3((unsigned)ctas), dim3(fff::kCoopThreads), args,
+                                        sizeof(int) * (size_t)(fff::kCoopWarps + 2) * nbins, st);
     } else {
         // Every cluster reads all keys, so more clusters do not shorten the kernel; they only shrink the
         // bin range (and the number of ballots per step).
@@ -610,6 +625,21 @@ fff_status_t fff_create(fff_handle_t* out, int D, int O, int depth, int leaf_wid
     if (s == FFF_OK) s = clone((void**)&h->ws_offsets2[0], nullptr, sizeof(int32_t) * (nl + 1));
     if (s == FFF_OK) s = clone((void**)&h->ws_offsets2[1], nullptr, sizeof(int32_t) * (nl + 1));
     if (s == FFF_OK) s = clone((void**)&h->d_status, nullptr, sizeof(int));
+    {
+        int coop = 0, per_sm = 0;
+        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, h->device);
+        const int smem_max = (int)(sizeof(int) * (fff::kCoopWarps + 2) * fff::kBucketMaxBinsPerCta);
+        cudaFuncSetAttribute(fff::k_bucket_coop, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max);
+        if (coop && cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fff::k_bucket_coop, fff::kCoopThreads, smem_max) ==
+                        cudaSuccess &&
+            per_sm > 0) {
+            h->coop_ctas = h->sm_count;          // one CTA per SM is always resident
+            if (s == FFF_OK)
+                s = clone((void**)&h->ws_matrix, nullptr, sizeof(int) * (size_t)h->coop_ctas * fff::kBucketMaxBinsPerCta);
+        } else {
+            cudaGetLastError();
+        }
+    }
     if (s == FFF_OK && dtype == FFF_DTYPE_BF16 && D % fff::kKS == 0 && depth > 0) s = pack_node_images<__nv_bfloat16>(h);
     if (s == FFF_OK && dtype == FFF_DTYPE_BF16 && D % fff::kKS == 0 && O % 8 == 0 && leaf_width <= 64) {
         h->LP = leaf_width <= 16 ? 16 : (leaf_width <= 32 ? 32 : 64);

@@ -412,6 +412,174 @@ k_bucket_cluster(const int32_t* __restrict__ keys, const int32_t* __restrict__ p
     cluster.sync();      // peers may still be reading this CTA's shared memory
 }
 
+// ---- grid-wide version for few bins ----------------------------------------------------------------
+// Global bucketing (all B tokens in natural order) of at most kBucketMaxBinsPerCta bins with the work
+// spread over the whole GPU: CTA c of G takes the c-th contiguous slice of the tokens, counts per
+// (warp, bin), publishes its per-bin totals as row c of a G x nbins matrix in global memory, and after
+// one grid-wide barrier (cooperative launch; all CTAs are resident) adds up the rows of the CTAs before
+// it.  Same result as k_bucket_cluster, which needs one cluster (8 SMs) to scan every token.
+// The tile list is written dense and padded with empty tiles up to n_tiles_total.
+constexpr int kCoopWarps = 8;
+constexpr int kCoopThreads = kCoopWarps * 32;
+
+// Dynamic shared memory: (kCoopWarps + 2) * nbins ints.
+__global__ void __launch_bounds__(kCoopThreads)
+k_bucket_coop(const int32_t* __restrict__ keys, int32_t* __restrict__ offsets_out, int32_t* __restrict__ perm_out, int B,
+              int nbins, int bin_bits, int tile_rows, Tile* __restrict__ tiles, int n_tiles_total,
+              int32_t* __restrict__ rank_tmp, int* __restrict__ matrix)
+{
+    namespace cg = cooperative_groups;
+    extern __shared__ int s_dyn[];
+    __shared__ int s_warp[32];
+    int* s_cnt = s_dyn;                              // [kCoopWarps][nbins]
+    int* s_start = s_dyn + kCoopWarps * nbins;       // [nbins] first position of the bin
+    int* s_total = s_start + nbins;                  // [nbins] tokens in the bin
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    const int G = gridDim.x, c = blockIdx.x;
+    const unsigned lt_mask = (1u << lane) - 1u;
+
+    pdl_trigger();
+    for (int i = tid; i < (kCoopWarps + 2) * nbins; i += kCoopThreads) s_cnt[i] = 0;     // counts, starts and totals
+    __syncthreads();
+    pdl_wait();
+
+    const int slices = G * kCoopWarps;
+    const int chunk = (((B + slices - 1) / slices) + 31) & ~31;
+    const int t0 = min((c * kCoopWarps + w) * chunk, B), t1 = min(t0 + chunk, B);
+    const bool in_regs = chunk <= 32 * kBucketKeyRegs;
+    int* my = s_cnt + w * nbins;
+
+    // pass 1: count and rank inside the slice
+    int kreg[kBucketKeyRegs], rreg[kBucketKeyRegs];
+#pragma unroll
+    for (int i = 0; i < kBucketKeyRegs; ++i) { kreg[i] = -1; rreg[i] = 0; }
+    for (int s0 = t0; s0 < t1; s0 += 32 * kBucketKeyRegs) {
+#pragma unroll
+        for (int i = 0; i < kBucketKeyRegs; ++i) {
+            const int t = s0 + i * 32 + lane;
+            kreg[i] = t < t1 ? __ldg(keys + t) : -1;
+        }
+#pragma unroll
+        for (int i = 0; i < kBucketKeyRegs; ++i) {
+            if (s0 + i * 32 >= t1) break;
+            const int k = kreg[i];
+            const bool in = k >= 0 && k < nbins;
+            const unsigned peers = peers_by_ballot(in, k, bin_bits);
+            const int leader = in ? __ffs(peers) - 1 : lane;
+            int seen = 0;
+            if (in && lane == leader) {
+                seen = my[k];
+                my[k] = seen + __popc(peers);
+            }
+            seen = __shfl_sync(kFullMask, seen, leader) + __popc(peers & lt_mask);
+            if (in_regs) rreg[i] = seen;
+            else if (in) rank_tmp[s0 + i * 32 + lane] = seen;
+            __syncwarp();
+        }
+    }
+    __syncthreads();
+
+    // per bin: offsets of the warps inside this CTA; the CTA total goes to row c of the matrix
+    for (int b = tid; b < nbins; b += kCoopThreads) {
+        int run = 0;
+        for (int ww = 0; ww < kCoopWarps; ++ww) {
+            const int c2 = s_cnt[ww * nbins + b];
+            s_cnt[ww * nbins + b] = run;
+            run += c2;
+        }
+        matrix[c * nbins + b] = run;
+    }
+    __threadfence();
+    cg::this_grid().sync();
+
+    // tokens of the CTAs before this one, and bin totals: column sums of the matrix.  P threads share a
+    // bin (P = threads / nbins when that is > 1) and every thread keeps 8 independent loads in flight.
+    {
+        const int P = nbins < kCoopThreads ? kCoopThreads / nbins : 1;
+        for (int b = tid % (nbins < kCoopThreads ? nbins : kCoopThreads); b < nbins; b += kCoopThreads) {
+            const int part = nbins < kCoopThreads ? tid / nbins : 0;
+            int before = 0, total = 0;
+            for (int r0 = part; r0 < G; r0 += 8 * P) {
+                int v[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int r = r0 + j * P;
+                    v[j] = r < G ? __ldcg(matrix + r * nbins + b) : 0;
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    total += v[j];
+                    if (r0 + j * P < c) before += v[j];
+                }
+            }
+            if (P > 1) {
+                // add up the P partial sums of the bin: the threads of one bin are nbins apart
+                atomicAdd(&s_total[b], total);
+                atomicAdd(&s_start[b], before);
+            } else {
+                s_total[b] = total;
+                s_start[b] = before;      // completed below with the first position of the bin
+            }
+        }
+    }
+    __syncthreads();
+    // exclusive scan of the totals over the bins (chunks of kCoopThreads bins, running carry)
+    int carry = 0;
+    for (int b0 = 0; b0 < nbins; b0 += kCoopThreads) {
+        const int b = b0 + tid;
+        const int v = b < nbins ? s_total[b] : 0;
+        int chunk_total = 0;
+        const int ex = carry + block_exclusive_scan_nw<kCoopWarps>(v, s_warp, &chunk_total);
+        if (b < nbins) {
+            const int add = ex + s_start[b];
+            for (int ww = 0; ww < kCoopWarps; ++ww) s_cnt[ww * nbins + b] += add;
+            s_start[b] = ex;
+            if (c == 0) {
+                offsets_out[b] = ex;
+                if (b == nbins - 1) offsets_out[nbins] = ex + v;
+            }
+        }
+        carry += chunk_total;
+    }
+    __syncthreads();
+    if (tile_rows > 0 && c == 0) {
+        int tile_base = 0;
+        for (int b0 = 0; b0 < nbins; b0 += kCoopThreads) {
+            const int b = b0 + tid;
+            const int total = b < nbins ? s_total[b] : 0;
+            const int nt = (total + tile_rows - 1) / tile_rows;
+            int n_chunk = 0;
+            const int tl0 = tile_base + block_exclusive_scan_nw<kCoopWarps>(nt, s_warp, &n_chunk);
+            for (int i = 0; i < nt; ++i) {
+                Tile tl;
+                tl.bin = b;
+                tl.start = s_start[b] + i * tile_rows;
+                tl.rows = min(tile_rows, total - i * tile_rows);
+                tl.pad = 0;
+                tiles[tl0 + i] = tl;
+            }
+            tile_base += n_chunk;
+        }
+        Tile empty;
+        empty.bin = 0; empty.start = 0; empty.rows = 0; empty.pad = 0;
+        for (int i = tile_base + tid; i < n_tiles_total; i += kCoopThreads) tiles[i] = empty;
+    }
+
+    // pass 2: place
+    if (in_regs) {
+#pragma unroll
+        for (int i = 0; i < kBucketKeyRegs; ++i) {
+            const int k = kreg[i];
+            if (k >= 0 && k < nbins) perm_out[my[k] + rreg[i]] = t0 + i * 32 + lane;
+        }
+    } else {
+        for (int t = t0 + lane; t < t1; t += 32) {
+            const int k = __ldg(keys + t);
+            if (k >= 0 && k < nbins) perm_out[my[k] + rank_tmp[t]] = t;
+        }
+    }
+}
+
 // Tile list from an existing offsets array (one CTA; used when the caller supplies the bucketing),
 // padded with empty tiles up to n_tiles_total = floor(B / tile_rows) + nbins.
 __global__ void __launch_bounds__(kBucketThreads)
