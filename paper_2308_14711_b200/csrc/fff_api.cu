@@ -292,29 +292,39 @@ fff_status_t run_bucket(fff_handle_s* h, const int32_t* keys, int nbins, const C
     return launched(h, st, name);
 }
 
-template <int NP, int S>
+constexpr int kSmemBudget = 227 * 1024 - 1024;      // usable shared memory of an SM, less the per-CTA reservation
+
+template <int NP>
 fff_status_t launch_descent_mma(fff_handle_s* h, const fff_handle_s::DenseStage& sg, const void* x, const int32_t* perm,
                                 bool grouped, int32_t* pos_out, int64_t B, cudaStream_t st) {
-    using L = fff::DescentMmaLayout<NP, S>;
-    const int per_sm = std::max(1, std::min(3, (int)((227 * 1024) / (L::kSmemBytes + 1024))));
+    using L = fff::DescentMmaLayout<NP>;
+    // A single-group stage keeps its weight image resident if at least 3 ring stages still fit.
+    const int res_bytes = NP * h->D * 2;
+    const bool resident = !grouped && L::smem_bytes(3, res_bytes) <= kSmemBudget;
+    // two CTAs per SM when that leaves at least 3 stages each, else one CTA with as many as fit
+    auto stages_for = [&](int budget) {
+        const int per = resident ? L::kXStageBytes : L::kStageStride;
+        return std::min((int)fff::kMaxStages, (budget - L::kFixedBytes - (resident ? res_bytes : 0)) / per);
+    };
+    int per_sm = 2, stages = stages_for(kSmemBudget / 2 - 1024);
+    if (stages < 3) { per_sm = 1; stages = stages_for(kSmemBudget); }
+    if (stages < 2) return FFF_ERR_UNSUPPORTED;
+    const int smem = L::smem_bytes(stages, resident ? res_bytes : 0);
     const int n_tiles = grouped ? tile_list_len(B, fff::kDTM, 1 << sg.L0) : (int)((B + fff::kDTM - 1) / fff::kDTM);
     const int64_t grid = std::max<int64_t>(1, std::min<int64_t>((int64_t)h->sm_count * per_sm, n_tiles));
-    if (launch_chain(h, fff::k_descent_mma<NP, S>, (unsigned)grid, fff::kDescentThreads, L::kSmemBytes, st, 1,
+    if (launch_chain(h, fff::k_descent_mma<NP>, (unsigned)grid, fff::kDescentThreads, (size_t)smem, st, 1,
                      (const __nv_bfloat16*)x, grouped ? perm : nullptr, grouped ? h->ws_tiles : nullptr, n_tiles, sg.wimg,
-                     sg.bimg, pos_out, h->D, (int)B, sg.k, h->d_status) != cudaSuccess)
+                     sg.bimg, pos_out, h->D, (int)B, sg.k, stages, resident ? 1 : 0, h->d_status) != cudaSuccess)
         return cudaGetLastError(), FFF_ERR_CUDA;
     return launched(h, st, "tree_descent_mma");
 }
 
-// Ring depths: as many stages as fit with two CTAs per SM (one for the widest stage).
-constexpr int kDescentStages16 = 4, kDescentStages32 = 4, kDescentStages64 = 6;
-
 fff_status_t run_descent_mma(fff_handle_s* h, const fff_handle_s::DenseStage& sg, const void* x, const int32_t* perm,
                              bool grouped, int32_t* pos_out, int64_t B, cudaStream_t st) {
     switch (sg.NP) {
-        case 16: return launch_descent_mma<16, kDescentStages16>(h, sg, x, perm, grouped, pos_out, B, st);
-        case 32: return launch_descent_mma<32, kDescentStages32>(h, sg, x, perm, grouped, pos_out, B, st);
-        case 64: return launch_descent_mma<64, kDescentStages64>(h, sg, x, perm, grouped, pos_out, B, st);
+        case 16: return launch_descent_mma<16>(h, sg, x, perm, grouped, pos_out, B, st);
+        case 32: return launch_descent_mma<32>(h, sg, x, perm, grouped, pos_out, B, st);
+        case 64: return launch_descent_mma<64>(h, sg, x, perm, grouped, pos_out, B, st);
     }
     return FFF_ERR_UNSUPPORTED;
 }
@@ -400,12 +410,9 @@ fff_status_t pack_node_images(fff_handle_s* h) {
         if (cudaGetLastError() != cudaSuccess) return FFF_ERR_CUDA;
         L0 += sg.k;
     }
-    cudaFuncSetAttribute(fff::k_descent_mma<16, kDescentStages16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                         fff::DescentMmaLayout<16, kDescentStages16>::kSmemBytes);
-    cudaFuncSetAttribute(fff::k_descent_mma<32, kDescentStages32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                         fff::DescentMmaLayout<32, kDescentStages32>::kSmemBytes);
-    cudaFuncSetAttribute(fff::k_descent_mma<64, kDescentStages64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                         fff::DescentMmaLayout<64, kDescentStages64>::kSmemBytes);
+    cudaFuncSetAttribute(fff::k_descent_mma<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+    cudaFuncSetAttribute(fff::k_descent_mma<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+    cudaFuncSetAttribute(fff::k_descent_mma<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
     return cudaGetLastError() == cudaSuccess ? FFF_OK : FFF_ERR_CUDA;
 }
 

@@ -34,16 +34,22 @@ constexpr int kDescentKSplit = 2;
 constexpr int kDescentConsumers = kDescentMTiles * kDescentKSplit;
 constexpr int kDescentThreads = (kDescentConsumers + kProducerWarps) * 32;
 
-template <int NP, int S> struct DescentMmaLayout {
+// The ring depth and the stage stride are run-time values: a stage holds the token rows and, unless the
+// whole weight image of the (single) group is kept resident in shared memory, the matching weight slice.
+template <int NP> struct DescentMmaLayout {
     static constexpr int kWStageBytes = NP * kKS * 2;
-    static constexpr int kStageBytes = kDTM * kXRowBytes + kWStageBytes;
+    static constexpr int kXStageBytes = kDTM * kXRowBytes;
+    static constexpr int kStageBytes = kXStageBytes + kWStageBytes;
     static constexpr int kStageStride = (kStageBytes + 127) & ~127;
     static constexpr int kLogitRow = NP + 1;                                     // floats, padded
     // one scratch area per warp pair: partial accumulators (fragment order), then the 16 logit rows
     static constexpr int kPairScratch = (16 * kLogitRow * 4 > NP * 64 ? 16 * kLogitRow * 4 : NP * 64);
     static constexpr int kStagingBytes = kDescentMTiles * kPairScratch;
-    static constexpr int kSmemBytes = S * kStageStride + ((kStagingBytes + 127) & ~127) + 128 + 128;
-    static_assert(S <= kMaxStages, "barrier area holds 2 * kMaxStages mbarriers");
+    static constexpr int kFixedBytes = ((kStagingBytes + 127) & ~127) + 256 /* barriers */ + 128 /* align */;
+    // shared memory of a launch with `stages` ring stages; resident_bytes = NP * D * 2 or 0
+    static constexpr int smem_bytes(int stages, int resident_bytes) {
+        return stages * (resident_bytes ? kXStageBytes : kStageStride) + kFixedBytes + resident_bytes;
+    }
 };
 
 // Weight image of one stage: [group][D/kKS][kKS/64][NP rows][64 columns] 128-byte swizzled, rows in the
@@ -73,24 +79,28 @@ __global__ void k_pack_nodes(const T* __restrict__ node_w, const T* __restrict__
     }
 }
 
-template <int NP, int S>
+// resident != 0 (single-group stage only, tiles == NULL): the whole weight image of the group is copied
+// into shared memory once per CTA and the ring carries token rows only.
+template <int NP>
 __global__ void __launch_bounds__(kDescentThreads, NP <= 32 ? 2 : 1)
 k_descent_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ perm,
               const Tile* __restrict__ tiles, int n_tiles_total,
               const __nv_bfloat16* __restrict__ wimg, const float* __restrict__ bimg,
               int32_t* __restrict__ pos_out,
-              int D, int B, int k, int* __restrict__ status)
+              int D, int B, int k, int kStages, int resident, int* __restrict__ status)
 {
-    using L = DescentMmaLayout<NP, S>;
-    constexpr int kStages = S;
+    using L = DescentMmaLayout<NP>;
     constexpr int kTM = kDTM;
     constexpr int kLeafMmaConsumers = kDescentConsumers;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+    const int stage_stride = resident ? L::kXStageBytes : L::kStageStride;
     unsigned char* stages = smem;
-    unsigned char* staging = smem + kStages * L::kStageStride;
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStages * L::kStageStride + ((L::kStagingBytes + 127) & ~127));
-    uint64_t* empty = full + kStages;
+    unsigned char* staging = smem + kStages * stage_stride;
+    uint64_t* full = reinterpret_cast<uint64_t*>(staging + ((L::kStagingBytes + 127) & ~127));
+    uint64_t* empty = full + kMaxStages;
+    uint64_t* wbar = empty + kMaxStages;                               // completion of the resident weight copy
+    unsigned char* wres = reinterpret_cast<unsigned char*>(full) + 256;  // resident weight image
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int U1 = D / kKS;
@@ -101,11 +111,17 @@ k_descent_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ p
             ptx::mbar_init(full + s, kProducerThreads + 1);     // every producer thread + the weight copy
             ptx::mbar_init(empty + s, kLeafMmaConsumers);
         }
+        ptx::mbar_init(wbar, 1);
         ptx::fence_mbar_init();
     }
     pdl_trigger();
     __syncthreads();
     pdl_wait();
+    if (resident && threadIdx.x == 0) {
+        ptx::mbar_arrive_expect_tx(wbar, (uint32_t)(NP * D * 2));
+        for (int u = 0; u < D / kKS; ++u)
+            ptx::bulk_g2s(wres + u * L::kWStageBytes, wimg + (int64_t)u * (NP * kKS), L::kWStageBytes, wbar);
+    }
 
     int stage = 0;
     uint32_t phase = 0;
@@ -140,11 +156,15 @@ k_descent_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ p
             }
             for (int u = 0; u < U1; ++u) {
                 if (!timed_out && !ptx::mbar_wait_relaxed(empty + stage, phase ^ 1)) timed_out = true;
-                unsigned char* st = stages + stage * L::kStageStride;
+                unsigned char* st = stages + stage * stage_stride;
                 if (ptid == 0) {
-                    ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)L::kWStageBytes);
-                    ptx::bulk_g2s(st + kTM * kXRowBytes, wimg + ((int64_t)tl.bin * U1 + u) * (NP * kKS), L::kWStageBytes,
-                                  full + stage);
+                    if (resident) {
+                        ptx::mbar_arrive(full + stage);
+                    } else {
+                        ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)L::kWStageBytes);
+                        ptx::bulk_g2s(st + kTM * kXRowBytes, wimg + ((int64_t)tl.bin * U1 + u) * (NP * kKS), L::kWStageBytes,
+                                      full + stage);
+                    }
                 }
 #pragma unroll
                 for (int i = 0; i < kTM / kRowsPerPass; ++i)
@@ -161,6 +181,7 @@ k_descent_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ p
         const int g = lane >> 2, q4 = lane & 3;
         const int bn = (lane & 7) + ((lane >> 4) << 3);
         const int bk = ((lane >> 3) & 1) * 8;
+        if (resident && !ptx::mbar_wait(wbar, 0)) timed_out = true;
         for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
             const Tile tl = get_tile(tile);
             if (tl.rows == 0) continue;
@@ -185,8 +206,8 @@ k_descent_mma(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ p
             for (int u = 0; u < U1; ++u) {
                 if (!timed_out && !ptx::mbar_wait(full + stage, phase)) timed_out = true;
                 if (active) {
-                    const uint32_t xs = ptx::smem_addr(stages + stage * L::kStageStride);
-                    const uint32_t ws = xs + kTM * kXRowBytes;
+                    const uint32_t xs = ptx::smem_addr(stages + stage * stage_stride);
+                    const uint32_t ws = resident ? ptx::smem_addr(wres + u * L::kWStageBytes) : xs + kTM * kXRowBytes;
                     const uint32_t a_base = xs + (m0 + (lane & 15)) * kXRowBytes + (lane >> 4) * 16;
 #pragma unroll
                     for (int kq = 0; kq < (kKS / 16) / kDescentKSplit; ++kq) {
