@@ -34,7 +34,7 @@ if ROOT not in sys.path:
 
 import numpy as np  # noqa: E402
 
-from paper_2308_14711_b200 import workloads as wl  # noqa: E402
+from paper_2308_14711_b200 import replicas, workloads as wl  # noqa: E402
 
 DEFAULT_CONFIG = "vit_d8_l12_bf16"
 FALLBACK_HBM_GBS = 6650.0
@@ -235,11 +235,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         torch.cuda.synchronize()
 
     def max_over_ranks(v: float) -> float:
-        if dist is None:
-            return v
-        t = torch.tensor([v], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return replicas.max_over_ranks(v, dist, "cuda")
 
     peaks = measured_peaks()
     cfg = wl.CONFIGS[args.config]
@@ -260,7 +256,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     ms_prof, _, prof, _, _ = time_device(layer, xs, ys, ls, args.steps, 3, profile=True)
     status = layer.last_status()
     ms_per_step = ms / args.steps
-    value = world * B * args.steps / (ms * 1e-3)
+    value = replicas.whole_job_throughput(B, args.steps, world, ms)
 
     leaves_touched = int(torch.unique(ls[0]).numel())
     kernels, prof_steps = prof
@@ -377,9 +373,13 @@ def cpu_baseline(cfg, w_host, x_host, budget_s: float = 20.0) -> dict:
     t = time.perf_counter()
     orc.forward_i(net, x_host[:n], threads=cores)
     dt = time.perf_counter() - t
+    n1 = max(64, n // max(cores, 1))
+    t = time.perf_counter()
+    orc.forward_i(net, x_host[:n1], threads=1)
+    dt1 = time.perf_counter() - t
     return {"value": n / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"first {n} of {cfg.B} tokens of {cfg.name}, one pass, float64 C oracle, {cores} threads",
-            "seconds": round(dt, 3)}
+            "seconds": round(dt, 3), "single_thread_value": n1 / dt1, "single_thread_sample_tokens": n1}
 
 
 def run_reference(args, rank: int, world: int):
