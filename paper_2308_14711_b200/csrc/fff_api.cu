@@ -186,6 +186,12 @@ size_t max_tiles(const fff_handle_s* h, int64_t B) { return (size_t)(B / kMinTil
 
 // Token rows per tile of the grouped leaf kernel: short tiles when buckets are small.
 int leaf_tile_rows(const fff_handle_s* h, int64_t B) {
+    static const int forced = [] {
+        const char* e = std::getenv("FFF_LEAF_TILE_ROWS");      // tuning aid: 32 or 64
+        const int v = e ? std::atoi(e) : 0;
+        return (v == 32 || v == 64) ? v : 0;
+    }();
+    if (forced) return forced;
     return B / h->n_leaves <= 40 ? 32 : 64;
 }
 
@@ -398,7 +404,10 @@ fff_status_t pack_node_images(fff_handle_s* h) {
     for (int i = 0; i < n_st; ++i) {
         fff_handle_s::DenseStage sg;
         sg.L0 = L0;
-        sg.k = d / n_st + (i < d % n_st ? 1 : 0);
+        {
+            static const bool small_first = std::getenv("FFF_SMALL_STAGE_FIRST") != nullptr;      // tuning aid
+            sg.k = d / n_st + ((small_first ? i >= n_st - d % n_st : i < d % n_st) ? 1 : 0);
+        }
         sg.NP = std::max(16, 1 << sg.k);
         const size_t groups = (size_t)1 << L0;
         fff_status_t s;
