@@ -63,6 +63,7 @@ struct fff_handle_s {
     int32_t* ws_rank = nullptr;   // per-token rank scratch of the bucketing kernel (large batches only)
     int max_bucket_clusters = 8;
     int32_t* last_perm = nullptr; // where the most recent forward left its leaf permutation
+    bool bucketing_pending = false;   // the last forward skipped the leaf bucketing; ws_leaf holds its leaf indices
     int* ws_matrix = nullptr;     // per-CTA bin totals of the grid-wide bucketing kernel
     int coop_ctas = 0;            // CTAs of that kernel that are resident at once (0 = cooperative launch unavailable)
     int32_t* ws_perm2 = nullptr;  // second permutation buffer: successive bucketings alternate between the two
@@ -259,7 +260,9 @@ fff_status_t run_bucket(fff_handle_s* h, const int32_t* keys, int nbins, const C
                         int32_t* perm, int64_t B, cudaStream_t st, int tile_rows, const char* name) {
     const int n_tiles_total = tile_rows > 0 ? tile_list_len(B, tile_rows, nbins) : 0;
     cudaError_t e;
-    if (coarse.perm && nbins / coarse.bins <= fff::kBucketMaxBinsPerCta) {
+    // Refining pays while the coarse buckets are few and large; thousands of tiny buckets would mean
+    // thousands of tiny clusters, and scanning all keys from a few clusters is cheaper then.
+    if (coarse.perm && nbins / coarse.bins <= fff::kBucketMaxBinsPerCta && coarse.bins <= 256) {
         const int nb = nbins / coarse.bins;
         int bin_bits = 0;
         while ((1 << bin_bits) < nb) ++bin_bits;
@@ -754,17 +757,30 @@ fff_status_t fff_forward_infer(fff_handle_t h, const void* x, void* y, int32_t* 
     h->prof_active = h->prof_steps < h->prof_max_steps;
     if (h->prof_active)
         cudaEventRecord(h->prof_events[(size_t)h->prof_steps * (fff_handle_s::kMaxProfLaunches + 1)], st);
+    const bool tensor_leaf = use_tensor_leaf(h);
+    // With fewer than about 4 tokens per leaf the warp leaf kernel gains nothing from bucket order (no
+    // weights to share), so the bucketing is left out of the forward and made on demand
+    // (fff_debug_get_bucketing) from the leaf indices, which then also live in the workspace.
+    const bool lazy_bucketing = !tensor_leaf && B < 4 * h->n_leaves;
+    if (lazy_bucketing) leaf = h->ws_leaf;
     Coarse coarse;
     s = run_descent(h, x, leaf, &coarse, B, st);
-    const bool tensor_leaf = use_tensor_leaf(h);
     const int tile_rows = tensor_leaf ? leaf_tile_rows(h, B) : 0;
     // the final permutation goes to whichever buffer the last node bucketing did not use
     h->last_perm = coarse.perm == h->ws_perm ? h->ws_perm2 : h->ws_perm;
-    if (s == FFF_OK)
-        s = run_bucket(h, leaf, (int)h->n_leaves, coarse, h->ws_offsets, h->last_perm, B, st, tile_rows, "leaf_bucketing");
-    if (s == FFF_OK)
-        s = tensor_leaf ? run_leaf_mma(h, x, h->last_perm, y, B, tile_rows, st)
-                        : FFF_DISPATCH(h, run_leaf, h, x, leaf, h->last_perm, y, B, st);
+    h->bucketing_pending = lazy_bucketing;
+    if (lazy_bucketing) {
+        if (s == FFF_OK && leaf_idx &&
+            cudaMemcpyAsync(leaf_idx, leaf, sizeof(int32_t) * (size_t)B, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+            s = (cudaGetLastError(), FFF_ERR_CUDA);
+        if (s == FFF_OK) s = FFF_DISPATCH(h, run_leaf, h, x, leaf, nullptr, y, B, st);
+    } else {
+        if (s == FFF_OK)
+            s = run_bucket(h, leaf, (int)h->n_leaves, coarse, h->ws_offsets, h->last_perm, B, st, tile_rows, "leaf_bucketing");
+        if (s == FFF_OK)
+            s = tensor_leaf ? run_leaf_mma(h, x, h->last_perm, y, B, tile_rows, st)
+                            : FFF_DISPATCH(h, run_leaf, h, x, leaf, h->last_perm, y, B, st);
+    }
     if (h->prof_active) {
         h->prof_active = false;
         if (s == FFF_OK && (h->prof_steps == 0 || h->prof_nlaunch == h->launches)) {
@@ -809,6 +825,15 @@ fff_status_t fff_debug_get_bucketing(fff_handle_t h, int32_t* perm, int32_t* off
     if (!offsets || h->last_B < 0 || (h->last_B > 0 && !perm)) return FFF_ERR_INVALID_ARG;
     DeviceGuard g(h->device);
     cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (h->last_B > 0 && h->bucketing_pending) {
+        const int saved = h->launches;
+        h->launches = 0;           // an ordinary launch: nothing of this call precedes it in the stream
+        const fff_status_t bs = run_bucket(h, h->ws_leaf, (int)h->n_leaves, Coarse(), h->ws_offsets, h->last_perm, h->last_B, st,
+                                           0, "leaf_bucketing");
+        h->launches = saved;
+        if (bs != FFF_OK) return bs;
+        h->bucketing_pending = false;
+    }
     if (h->last_B > 0 &&
         cudaMemcpyAsync(perm, h->last_perm, sizeof(int32_t) * (size_t)h->last_B, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
         return cudaGetLastError(), FFF_ERR_CUDA;

@@ -79,15 +79,31 @@ k_leaf_warp(const T* __restrict__ x, const int32_t* __restrict__ leaf_idx, const
         }
         __syncwarp();
 
-        // output layer: one output neuron per lane
+        // output layer.  Thin leaves (l = 1, rows of W2 are single elements): 8 / 4 consecutive outputs per
+        // lane with 16-byte loads of W2, b2 and a 16-byte store of y.  Otherwise one output neuron per lane,
+        // four rows in flight.
         const T* w2j = w2 + j * (int64_t)O * l;
         const T* b2j = b2 + j * (int64_t)O;
         T* yt = y + t * O;
-        for (int o = lane; o < O; o += 32) {
-            const T* row = w2j + (int64_t)o * l;
-            float acc = Elem<T>::to_float(b2j[o]);
-            for (int q = 0; q < l; ++q) acc = fmaf(Elem<T>::to_float(row[q]), h[q], acc);
-            yt[o] = Elem<T>::from_float(acc);
+        if (l == 1 && vec && (O % V) == 0) {
+            const float h0 = h[0];
+            for (int o = lane * V; o < O; o += 32 * V) {
+                float fw[V], fb[V];
+                Elem<T>::load_vec(w2j + o, fw);
+                Elem<T>::load_vec(b2j + o, fb);
+                alignas(16) T out[V];
+#pragma unroll
+                for (int e = 0; e < V; ++e) out[e] = Elem<T>::from_float(fmaf(fw[e], h0, fb[e]));
+                *reinterpret_cast<uint4*>(yt + o) = *reinterpret_cast<const uint4*>(out);
+            }
+        } else {
+#pragma unroll 4
+            for (int o = lane; o < O; o += 32) {
+                const T* row = w2j + (int64_t)o * l;
+                float acc = Elem<T>::to_float(b2j[o]);
+                for (int q = 0; q < l; ++q) acc = fmaf(Elem<T>::to_float(row[q]), h[q], acc);
+                yt[o] = Elem<T>::from_float(acc);
+            }
         }
         __syncwarp();
     }
