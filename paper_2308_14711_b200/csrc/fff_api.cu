@@ -18,6 +18,7 @@
 #include "kernels/bucket.cuh"
 #include "kernels/common.cuh"
 #include "kernels/descent_mma.cuh"
+#include "kernels/descent_umma.cuh"
 #include "kernels/descent_warp.cuh"
 #include "kernels/leaf_mma.cuh"
 #include "kernels/leaf_warp.cuh"
@@ -72,10 +73,13 @@ struct fff_handle_s {
     // staged descent on tensor cores: consecutive groups of levels, each with its weight image
     struct DenseStage {
         int L0 = 0, k = 0, NP = 0;
+        bool umma = false;            // first stage on the tcgen05 kernel (up to 8 levels)
         __nv_bfloat16* wimg = nullptr;
         float* bimg = nullptr;
     };
     std::vector<DenseStage> stages;
+    // the same with a first stage of up to 8 levels on the tcgen05 kernel (empty = not available)
+    std::vector<DenseStage> ustages;
     int32_t* ws_pos[2] = {nullptr, nullptr};
     int *d_status = nullptr;
 
@@ -170,6 +174,7 @@ void release(fff_handle_s* h) {
     dfree(h->ws_leaf); dfree(h->ws_perm); dfree(h->ws_perm2); dfree(h->ws_offsets); dfree(h->ws_offsets2[0]); dfree(h->ws_offsets2[1]);
     dfree(h->d_status); dfree(h->st_x); dfree(h->st_y); dfree(h->st_leaf);
     for (auto& sg : h->stages) { dfree(sg.wimg); dfree(sg.bimg); }
+    for (auto& sg : h->ustages) { dfree(sg.wimg); dfree(sg.bimg); }
     dfree(h->ws_pos[0]); dfree(h->ws_pos[1]);
     dfree(h->w1img); dfree(h->b1img); dfree(h->w2img); dfree(h->ws_tiles); dfree(h->ws_rank); dfree(h->ws_matrix);
     prof_free(h);
@@ -214,7 +219,7 @@ fff_status_t grow_workspace(fff_handle_s* h, int64_t B) {
     if ((s = dmalloc((void**)&h->ws_perm, sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
     if ((s = dmalloc((void**)&h->ws_perm2, sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
     if ((s = dmalloc((void**)&h->ws_rank, sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
-    if (h->stages.size() > 1) {
+    if (h->stages.size() > 1 || h->ustages.size() > 1) {
         if ((s = dmalloc((void**)&h->ws_pos[0], sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
         if ((s = dmalloc((void**)&h->ws_pos[1], sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
     }
@@ -338,6 +343,67 @@ fff_status_t run_descent_mma(fff_handle_s* h, const fff_handle_s::DenseStage& sg
     return FFF_ERR_UNSUPPORTED;
 }
 
+// cuTensorMapEncodeTiled, looked up once through the runtime (the library does not link the driver).
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static const EncodeTiledFn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess) {
+            cudaGetLastError();
+            p = nullptr;
+        }
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// Tensor map of the bf16 token matrix x[B, D] for boxes of box_rows x 64 columns, 128-byte swizzled;
+// rows past B read as zeros.
+bool make_x_tensor_map(CUtensorMap* tm, const void* x, int64_t B, int D, int box_rows) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return false;
+    const cuuint64_t gdim[2] = {(cuuint64_t)D, (cuuint64_t)B};
+    const cuuint64_t gstride[1] = {(cuuint64_t)D * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)fff::kUKB, (cuuint32_t)box_rows};
+    const cuuint32_t estride[2] = {1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(x), gdim, gstride, box, estride,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int NP>
+fff_status_t launch_descent_umma(fff_handle_s* h, const fff_handle_s::DenseStage& sg, const void* x, int32_t* pos_out,
+                                 int64_t B, cudaStream_t st) {
+    using L = fff::DescentUmmaLayout<NP>;
+    const int stages = std::min((int)fff::kUmmaMaxStages, (kSmemBudget - L::smem_bytes(0)) / L::kStageBytes);
+    if (stages < 2) return FFF_ERR_UNSUPPORTED;
+    CUtensorMap tm;
+    if (!make_x_tensor_map(&tm, x, B, h->D, fff::kUM)) return FFF_ERR_CUDA;
+    const int64_t n_tiles = (B + fff::kUM - 1) / fff::kUM;
+    const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(h->sm_count, n_tiles));
+    if (launch_chain(h, fff::k_descent_umma<NP>, (unsigned)grid, fff::kUmmaThreads, (size_t)L::smem_bytes(stages), st, 1, tm,
+                     (const __nv_bfloat16*)sg.wimg, (const float*)sg.bimg, pos_out, h->D, (int)B, sg.k, stages,
+                     h->d_status) != cudaSuccess)
+        return cudaGetLastError(), FFF_ERR_CUDA;
+    return launched(h, st, "tree_descent_umma");
+}
+
+fff_status_t run_descent_umma(fff_handle_s* h, const fff_handle_s::DenseStage& sg, const void* x, int32_t* pos_out, int64_t B,
+                              cudaStream_t st) {
+    switch (sg.NP) {
+        case 32: return launch_descent_umma<32>(h, sg, x, pos_out, B, st);
+        case 64: return launch_descent_umma<64>(h, sg, x, pos_out, B, st);
+        case 128: return launch_descent_umma<128>(h, sg, x, pos_out, B, st);
+        case 256: return launch_descent_umma<256>(h, sg, x, pos_out, B, st);
+    }
+    return FFF_ERR_UNSUPPORTED;
+}
+
 template <typename T>
 fff_status_t run_descent_warp(fff_handle_s* h, const void* x, int level0, int levels, const int32_t* pos_in,
                               int32_t* pos_out, int64_t B, cudaStream_t st) {
@@ -352,11 +418,16 @@ fff_status_t run_descent_warp(fff_handle_s* h, const void* x, int level0, int le
 // Number of leading tensor-core stages to run for a batch of B tokens: a stage pays off while the
 // groups it works on (tokens that share the node at the stage's first level) hold enough tokens to
 // reuse the subtree's weights.
+const std::vector<fff_handle_s::DenseStage>& stage_plan(const fff_handle_s* h) {
+    return h->ustages.empty() ? h->stages : h->ustages;
+}
+
 int dense_stage_count(const fff_handle_s* h, int64_t B) {
-    if (h->stages.empty() || h->path == FFF_PATH_WARP) return 0;
-    if (h->path == FFF_PATH_TENSOR) return (int)h->stages.size();
+    const auto& plan = stage_plan(h);
+    if (plan.empty() || h->path == FFF_PATH_WARP) return 0;
+    if (h->path == FFF_PATH_TENSOR) return (int)plan.size();
     int n = 0;
-    for (const auto& sg : h->stages) {
+    for (const auto& sg : plan) {
         if ((B >> sg.L0) < 16) break;
         ++n;
     }
@@ -372,8 +443,9 @@ fff_status_t run_descent(fff_handle_s* h, const void* x, int32_t* leaf_out, Coar
     int level = 0;
     const int32_t* pos = nullptr;
     Coarse prev;
+    const auto& plan = stage_plan(h);
     for (int i = 0; i < n_dense; ++i) {
-        const auto& sg = h->stages[i];
+        const auto& sg = plan[i];
         if (i > 0) {
             // bucket by the node reached so far; buffers alternate so that the previous level stays readable
             int32_t* perm_out = (i & 1) ? h->ws_perm2 : h->ws_perm;
@@ -386,7 +458,7 @@ fff_status_t run_descent(fff_handle_s* h, const void* x, int32_t* leaf_out, Coar
         }
         const bool last = level + sg.k == h->depth;
         int32_t* out = last ? leaf_out : h->ws_pos[i & 1];
-        s = run_descent_mma(h, sg, x, prev.perm, i > 0, out, B, st);
+        s = sg.umma ? run_descent_umma(h, sg, x, out, B, st) : run_descent_mma(h, sg, x, prev.perm, i > 0, out, B, st);
         if (s != FFF_OK) return s;
         level += sg.k;
         pos = out;
@@ -399,28 +471,74 @@ fff_status_t run_descent(fff_handle_s* h, const void* x, int32_t* leaf_out, Coar
     return s;
 }
 
+// Packs the weight image of one stage (levels L0 .. L0 + k - 1) and appends it to `plan`.
+template <typename T>
+fff_status_t pack_stage(fff_handle_s* h, std::vector<fff_handle_s::DenseStage>& plan, int L0, int k, int NP, bool umma) {
+    fff_handle_s::DenseStage sg;
+    sg.L0 = L0;
+    sg.k = k;
+    sg.NP = NP;
+    sg.umma = umma;
+    const size_t groups = (size_t)1 << L0;
+    fff_status_t s;
+    if ((s = dmalloc((void**)&sg.wimg, groups * sg.NP * h->D * 2)) != FFF_OK) return s;
+    plan.push_back(sg);                            // owned by the handle from here on
+    if ((s = dmalloc((void**)&plan.back().bimg, groups * sg.NP * 4)) != FFF_OK) return s;
+    fff::k_pack_nodes<T><<<h->sm_count * 8, 256>>>((const T*)h->node_w, (const T*)h->node_b, plan.back().wimg, plan.back().bimg,
+                                                  sg.L0, sg.k, sg.NP, h->D);
+    return cudaGetLastError() == cudaSuccess ? FFF_OK : FFF_ERR_CUDA;
+}
+
+// Levels per stage when `levels` levels are cut into stages of at most 6, larger stages first.
+std::vector<int> cut_levels(int levels) {
+    std::vector<int> ks;
+    const int n_st = (levels + 5) / 6;
+    static const bool small_first = std::getenv("FFF_SMALL_STAGE_FIRST") != nullptr;      // tuning aid
+    for (int i = 0; i < n_st; ++i)
+        ks.push_back(levels / n_st + ((small_first ? i >= n_st - levels % n_st : i < levels % n_st) ? 1 : 0));
+    return ks;
+}
+
 template <typename T>
 fff_status_t pack_node_images(fff_handle_s* h) {
     const int d = h->depth;
-    const int n_st = (d + 5) / 6;
+    fff_status_t s;
+    // plan for the mma.sync kernels alone: stages of at most 6 levels
     int L0 = 0;
-    for (int i = 0; i < n_st; ++i) {
-        fff_handle_s::DenseStage sg;
-        sg.L0 = L0;
-        {
-            static const bool small_first = std::getenv("FFF_SMALL_STAGE_FIRST") != nullptr;      // tuning aid
-            sg.k = d / n_st + ((small_first ? i >= n_st - d % n_st : i < d % n_st) ? 1 : 0);
+    for (int k : cut_levels(d)) {
+        if ((s = pack_stage<T>(h, h->stages, L0, k, std::max(16, 1 << k), false)) != FFF_OK) return s;
+        L0 += k;
+    }
+    // plan with a first stage of up to 8 levels on the tcgen05 kernel, the rest as above
+    if (encode_tiled_fn() && h->D % fff::kUKB == 0 && std::getenv("FFF_NO_UMMA") == nullptr) {
+        std::vector<int> ks;
+        if (const char* e = std::getenv("FFF_STAGE_PLAN")) {       // tuning aid: "8,3" = 8 levels, then 3
+            int sum = 0;
+            for (const char* p = e; *p;) {
+                const int v = std::atoi(p);
+                ks.push_back(v);
+                sum += v;
+                while (*p && *p != ',') ++p;
+                if (*p == ',') ++p;
+            }
+            bool ok = sum == d && !ks.empty() && ks[0] >= 1 && ks[0] <= 8;
+            for (size_t i = 1; i < ks.size(); ++i) ok = ok && ks[i] >= 1 && ks[i] <= 6;
+            if (!ok) ks.clear();
         }
-        sg.NP = std::max(16, 1 << sg.k);
-        const size_t groups = (size_t)1 << L0;
-        fff_status_t s;
-        if ((s = dmalloc((void**)&sg.wimg, groups * sg.NP * h->D * 2)) != FFF_OK) return s;
-        h->stages.push_back(sg);                       // owned by the handle from here on
-        if ((s = dmalloc((void**)&h->stages.back().bimg, groups * sg.NP * 4)) != FFF_OK) return s;
-        fff::k_pack_nodes<T><<<h->sm_count * 8, 256>>>((const T*)h->node_w, (const T*)h->node_b, h->stages.back().wimg,
-                                                      h->stages.back().bimg, sg.L0, sg.k, sg.NP, h->D);
-        if (cudaGetLastError() != cudaSuccess) return FFF_ERR_CUDA;
-        L0 += sg.k;
+        if (ks.empty()) {
+            ks.push_back(std::min(d, 8));
+            for (int k : cut_levels(d - ks[0])) ks.push_back(k);
+        }
+        L0 = 0;
+        for (size_t i = 0; i < ks.size(); ++i) {
+            const int np = i == 0 ? std::max(32, 1 << ks[i]) : std::max(16, 1 << ks[i]);
+            if ((s = pack_stage<T>(h, h->ustages, L0, ks[i], np, i == 0)) != FFF_OK) return s;
+            L0 += ks[i];
+        }
+        cudaFuncSetAttribute(fff::k_descent_umma<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+        cudaFuncSetAttribute(fff::k_descent_umma<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+        cudaFuncSetAttribute(fff::k_descent_umma<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+        cudaFuncSetAttribute(fff::k_descent_umma<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
     }
     cudaFuncSetAttribute(fff::k_descent_mma<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
     cudaFuncSetAttribute(fff::k_descent_mma<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);

@@ -1,0 +1,184 @@
+// First stage of the tree descent on the fifth-generation tensor cores (tcgen05, bf16 -> float32).
+//
+// Algorithm 1, FORWARD_I, non-leaf branch.  At the root every token faces the same subtree, so the
+// logits of all 2^k - 1 nodes of its first k <= 8 levels are one dense GEMM
+//     logits[B, NP] = X . Wsub^T,        NP = 32, 64, 128 or 256 >= 2^k - 1,
+// and the k decisions of a token are read off its row of logits: p <- 2p + 1 + (logit[p] + b[p] >= 0),
+// starting at p = 0 in the subtree's breadth-first numbering.  A logit of exactly zero (either sign)
+// goes right, NaN goes left, as in the scalar walk.
+//
+// One persistent CTA per SM works on tiles of 128 consecutive tokens:
+//   warp 4   producer: per K-block of 64 columns, one tiled tensor-map load of the 128 x 64 token
+//            tile (128-byte swizzled by the copy engine) and one bulk copy of the matching NP x 64
+//            slice of the pre-swizzled weight image into a ring of shared-memory stages;
+//   warp 5   MMA issuer: four tcgen05.mma (M = 128, N = NP, K = 16) per stage into one of two
+//            accumulators in tensor memory; tcgen05.commit frees the stage and, after the last
+//            K-block, publishes the accumulator;
+//   warps 0-3  epilogue: each thread owns one token (= one tensor-memory lane), reads its NP logits
+//            with tcgen05.ld, turns them into NP decision bits, frees the accumulator and walks the
+//            subtree on the bits.
+// The tensor pipe, the copy engine and the epilogue overlap across tiles through the two accumulators.
+//
+// Every wait is bounded (see ptx.cuh); tensor memory is released on every exit path.
+//
+// Requirements: bf16, D % 64 == 0, x 16-byte aligned.
+#pragma once
+
+#include <cuda.h>      // CUtensorMap
+
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace fff {
+
+constexpr int kUM = 128;                 // token rows per tile = rows of one tcgen05.mma
+constexpr int kUKB = 64;                 // columns per K-block: 128 bytes, one swizzle line
+constexpr int kUmmaEpilogueWarps = 4;
+constexpr int kUmmaThreads = (kUmmaEpilogueWarps + 2) * 32;
+constexpr int kUmmaMaxStages = 8;
+
+template <int NP> struct DescentUmmaLayout {
+    static_assert(NP == 32 || NP == 64 || NP == 128 || NP == 256, "accumulator width");
+    static constexpr int kXStageBytes = kUM * kUKB * 2;
+    static constexpr int kWStageBytes = NP * kUKB * 2;
+    static constexpr int kStageBytes = kXStageBytes + kWStageBytes;          // a multiple of 1024
+    static constexpr int kBarrierBytes = 256;                                // 2 * kUmmaMaxStages + 4 mbarriers, tmem slot
+    static constexpr int kTmemCols = 2 * NP;                                 // two accumulators
+    static constexpr int smem_bytes(int stages) { return 1024 + stages * kStageBytes + kBarrierBytes + NP * 4; }
+};
+
+// wimg: [D / 64][NP rows][64 columns] 128-byte swizzled (the single-group image of k_pack_nodes),
+// bimg: [NP] float32.  pos_out[t] = position reached at level k.
+template <int NP>
+__global__ void __launch_bounds__(kUmmaThreads, 1)
+k_descent_umma(const __grid_constant__ CUtensorMap tmap_x, const __nv_bfloat16* __restrict__ wimg,
+               const float* __restrict__ bimg, int32_t* __restrict__ pos_out, int D, int B, int k, int kStages,
+               int* __restrict__ status)
+{
+    using L = DescentUmmaLayout<NP>;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* full = reinterpret_cast<uint64_t*>(ring + kStages * L::kStageBytes);
+    uint64_t* empty = full + kUmmaMaxStages;
+    uint64_t* acc_full = empty + kUmmaMaxStages;
+    uint64_t* acc_empty = acc_full + 2;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    float* bias = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(full) + L::kBarrierBytes);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_tiles = (B + kUM - 1) / kUM;
+    const int KB = D / kUKB;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            ptx::mbar_init(full + s, 1);
+            ptx::mbar_init(empty + s, 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            ptx::mbar_init(acc_full + a, 1);
+            ptx::mbar_init(acc_empty + a, kUmmaEpilogueWarps * 32);
+        }
+        ptx::fence_mbar_init();
+        ptx::prefetch_tensormap(&tmap_x);
+    }
+    if (warp == 5) {
+        ptx::tmem_alloc(tmem_slot, L::kTmemCols);
+        ptx::tmem_relinquish_alloc_permit();
+    }
+    for (int i = threadIdx.x; i < NP; i += kUmmaThreads) bias[i] = bimg[i];    // a parameter image, not a predecessor's output
+    ptx::tc_fence_before_sync();
+    pdl_trigger();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    pdl_wait();
+    const uint32_t tmem_base = *tmem_slot;
+
+    bool timed_out = false;
+    if (warp == 4) {
+        // ------------------------------------------------------------------ producer
+        int stage = 0;
+        uint32_t phase = 0;
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+            for (int kb = 0; kb < KB; ++kb) {
+                if (!timed_out && !ptx::mbar_wait_relaxed(empty + stage, phase ^ 1)) timed_out = true;
+                if (lane == 0) {
+                    unsigned char* st = ring + stage * L::kStageBytes;
+                    ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)L::kStageBytes);
+                    ptx::tma_load_2d(st, &tmap_x, kb * kUKB, tile * kUM, full + stage);
+                    ptx::bulk_g2s(st + L::kXStageBytes, wimg + (int64_t)kb * (NP * kUKB), L::kWStageBytes, full + stage);
+                }
+                __syncwarp();
+                if (++stage == kStages) { stage = 0; phase ^= 1; }
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------------------------ MMA issuer
+        constexpr uint32_t idesc = ptx::umma_idesc_bf16(kUM, NP);
+        int stage = 0;
+        uint32_t phase = 0;
+        int it = 0;
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
+            const int a = it & 1;
+            if (!timed_out && !ptx::mbar_wait(acc_empty + a, ((it >> 1) & 1) ^ 1)) timed_out = true;
+            ptx::tc_fence_after_sync();
+            for (int kb = 0; kb < KB; ++kb) {
+                if (!timed_out && !ptx::mbar_wait(full + stage, phase)) timed_out = true;
+                ptx::tc_fence_after_sync();
+                if (lane == 0) {
+                    const uint32_t xs = ptx::smem_addr(ring + stage * L::kStageBytes);
+                    const uint64_t ad = ptx::umma_desc_k128(xs), bd = ptx::umma_desc_k128(xs + L::kXStageBytes);
+#pragma unroll
+                    for (int j = 0; j < kUKB / 16; ++j)
+                        ptx::umma_bf16(tmem_base + a * NP, ad + 2 * j, bd + 2 * j, idesc, (kb | j) != 0 ? 1u : 0u);
+                    ptx::umma_commit(empty + stage);
+                    if (kb == KB - 1) ptx::umma_commit(acc_full + a);
+                }
+                __syncwarp();
+                if (++stage == kStages) { stage = 0; phase ^= 1; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue: one token per thread
+        int it = 0;
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
+            const int a = it & 1;
+            if (!timed_out && !ptx::mbar_wait(acc_full + a, (it >> 1) & 1)) timed_out = true;
+            ptx::tc_fence_after_sync();
+            uint32_t bits[NP / 32];
+#pragma unroll
+            for (int c = 0; c < NP / 32; ++c) {
+                uint32_t v[32];
+                ptx::tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + a * NP + c * 32, v);
+                ptx::tmem_ld_wait();
+                uint32_t m = 0;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) m |= (__uint_as_float(v[j]) + bias[c * 32 + j] >= 0.0f ? 1u : 0u) << j;
+                bits[c] = m;
+            }
+            ptx::tc_fence_before_sync();
+            ptx::mbar_arrive(acc_empty + a);
+
+            int p = 0;
+            for (int r = 0; r < k; ++r) {
+                uint32_t w = bits[0];
+#pragma unroll
+                for (int c = 1; c < NP / 32; ++c) w = (p >> 5) == c ? bits[c] : w;
+                p = 2 * p + 1 + (int)((w >> (p & 31)) & 1u);
+            }
+            const int tok = tile * kUM + warp * 32 + lane;
+            if (tok < B) pos_out[tok] = p - ((1 << k) - 1);
+        }
+    }
+    if (timed_out) {
+        if (lane == 0) atomicExch(status, kDevTimeout);
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);     // let copies and MMAs still in flight finish before exit
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 5) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, L::kTmemCols);
+    }
+}
+
+}  // namespace fff
