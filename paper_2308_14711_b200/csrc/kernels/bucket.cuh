@@ -492,12 +492,47 @@ k_bucket_coop(const int32_t* __restrict__ keys, int32_t* __restrict__ offsets_ou
     __threadfence();
     cg::this_grid().sync();
 
-    // tokens of the CTAs before this one, and bin totals: column sums of the matrix.  P threads share a
-    // bin (P = threads / nbins when that is > 1) and every thread keeps 8 independent loads in flight.
-    {
+    // tokens of the CTAs before this one, and bin totals: column sums of the matrix.  Four bins go in
+    // one 16-byte load when nbins % 4 == 0; P threads share a column (P = threads / columns when that is
+    // > 1) and every thread keeps kInFlight independent loads in flight.
+    if ((nbins & 3) == 0) {
+        constexpr int kInFlight = 10;
+        const int V = nbins >> 2;
+        const int cols = V < kCoopThreads ? V : kCoopThreads;
+        const int P = V < kCoopThreads ? kCoopThreads / V : 1;
+        const int part = V < kCoopThreads ? tid / V : 0;
+        const int4* m4 = reinterpret_cast<const int4*>(matrix);
+        for (int vb = tid % cols; vb < V && part < P; vb += kCoopThreads) {
+            int4 before = make_int4(0, 0, 0, 0), total = make_int4(0, 0, 0, 0);
+            for (int r0 = part; r0 < G; r0 += kInFlight * P) {
+                int4 v[kInFlight];
+#pragma unroll
+                for (int j = 0; j < kInFlight; ++j) {
+                    const int r = r0 + j * P;
+                    v[j] = r < G ? __ldcg(m4 + r * V + vb) : make_int4(0, 0, 0, 0);
+                }
+#pragma unroll
+                for (int j = 0; j < kInFlight; ++j) {
+                    total.x += v[j].x; total.y += v[j].y; total.z += v[j].z; total.w += v[j].w;
+                    if (r0 + j * P < c) { before.x += v[j].x; before.y += v[j].y; before.z += v[j].z; before.w += v[j].w; }
+                }
+            }
+            const int b = 4 * vb;
+            if (P > 1) {
+                atomicAdd(&s_total[b], total.x); atomicAdd(&s_total[b + 1], total.y);
+                atomicAdd(&s_total[b + 2], total.z); atomicAdd(&s_total[b + 3], total.w);
+                atomicAdd(&s_start[b], before.x); atomicAdd(&s_start[b + 1], before.y);
+                atomicAdd(&s_start[b + 2], before.z); atomicAdd(&s_start[b + 3], before.w);
+            } else {
+                s_total[b] = total.x; s_total[b + 1] = total.y; s_total[b + 2] = total.z; s_total[b + 3] = total.w;
+                s_start[b] = before.x; s_start[b + 1] = before.y; s_start[b + 2] = before.z; s_start[b + 3] = before.w;
+            }
+        }
+    } else {
         const int P = nbins < kCoopThreads ? kCoopThreads / nbins : 1;
         for (int b = tid % (nbins < kCoopThreads ? nbins : kCoopThreads); b < nbins; b += kCoopThreads) {
             const int part = nbins < kCoopThreads ? tid / nbins : 0;
+            if (part >= P) break;
             int before = 0, total = 0;
             for (int r0 = part; r0 < G; r0 += 8 * P) {
                 int v[8];
@@ -513,7 +548,6 @@ k_bucket_coop(const int32_t* __restrict__ keys, int32_t* __restrict__ offsets_ou
                 }
             }
             if (P > 1) {
-                // add up the P partial sums of the bin: the threads of one bin are nbins apart
                 atomicAdd(&s_total[b], total);
                 atomicAdd(&s_start[b], before);
             } else {
