@@ -21,6 +21,7 @@
 #include "kernels/descent_umma.cuh"
 #include "kernels/descent_warp.cuh"
 #include "kernels/leaf_mma.cuh"
+#include "kernels/leaf_umma.cuh"
 #include "kernels/leaf_warp.cuh"
 
 namespace {
@@ -56,6 +57,8 @@ struct fff_handle_s {
     __nv_bfloat16* w1img = nullptr;
     float* b1img = nullptr;
     unsigned char* w2img = nullptr;
+    __nv_bfloat16* w2uimg = nullptr;   // W2 pieces of the tcgen05 leaf kernel (nullptr = kernel not available)
+    int* ws_sched = nullptr;           // its tile counter and finished-CTA counter (zero between launches)
     fff::Tile* ws_tiles = nullptr;
 
     // workspace
@@ -176,7 +179,7 @@ void release(fff_handle_s* h) {
     for (auto& sg : h->stages) { dfree(sg.wimg); dfree(sg.bimg); }
     for (auto& sg : h->ustages) { dfree(sg.wimg); dfree(sg.bimg); }
     dfree(h->ws_pos[0]); dfree(h->ws_pos[1]);
-    dfree(h->w1img); dfree(h->b1img); dfree(h->w2img); dfree(h->ws_tiles); dfree(h->ws_rank); dfree(h->ws_matrix);
+    dfree(h->w1img); dfree(h->b1img); dfree(h->w2img); dfree(h->w2uimg); dfree(h->ws_sched); dfree(h->ws_tiles); dfree(h->ws_rank); dfree(h->ws_matrix);
     prof_free(h);
     h->magic = 0;
     delete h;
@@ -197,6 +200,7 @@ int leaf_tile_rows(const fff_handle_s* h, int64_t B) {
         const int v = e ? std::atoi(e) : 0;
         return (v == 32 || v == 64) ? v : 0;
     }();
+    if (h->w2uimg) return fff::kLUM;              // the tcgen05 kernel works on 128-row tiles
     if (forced) return forced;
     return B / h->n_leaves <= 40 ? 32 : 64;
 }
@@ -576,9 +580,39 @@ fff_status_t launch_leaf_mma(fff_handle_s* h, const void* x, const int32_t* perm
     return launched(h, st, "grouped_leaf_ff_mma");
 }
 
+template <int LP>
+fff_status_t launch_leaf_umma(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, cudaStream_t st) {
+    using L = fff::LeafUmmaLayout<LP>;
+    const int n_tiles = tile_list_len(B, fff::kLUM, (int)h->n_leaves);
+    const int stages = std::min((int)fff::kLUMaxStages, (kSmemBudget - L::smem_bytes(0, h->O)) / L::kStageBytes);
+    if (stages < 2) return FFF_ERR_UNSUPPORTED;
+    static bool attr_set[64] = {};
+    if (h->device < 64 && !attr_set[h->device]) {
+        cudaFuncSetAttribute(fff::k_leaf_umma<LP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+        attr_set[h->device] = true;
+    }
+    CUtensorMap tm;
+    if (!make_x_tensor_map(&tm, x, B, h->D, 1)) return FFF_ERR_CUDA;       // one-row boxes: rows are gathered four at a time
+    const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(h->sm_count, n_tiles));
+    const int wide = (reinterpret_cast<uintptr_t>(y) & 31u) == 0 ? 1 : 0;
+    if (launch_chain(h, fff::k_leaf_umma<LP>, (unsigned)grid, fff::kLUThreads, (size_t)L::smem_bytes(stages, h->O), st, 1, tm, perm,
+                     (const fff::Tile*)h->ws_tiles, n_tiles, (const __nv_bfloat16*)h->w1img, (const float*)h->b1img,
+                     (const __nv_bfloat16*)h->w2uimg, (const __nv_bfloat16*)h->b2, (__nv_bfloat16*)y, h->D, h->O, h->act, stages,
+                     wide, h->ws_sched, h->d_status) != cudaSuccess)
+        return cudaGetLastError(), FFF_ERR_CUDA;
+    return launched(h, st, "grouped_leaf_ff_umma");
+}
+
 // Ring depth per (LP, TM): what fits twice into an SM's shared memory (once for LP = 64).
 fff_status_t run_leaf_mma(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, int tile_rows,
                           cudaStream_t st) {
+    if (tile_rows == fff::kLUM && h->w2uimg) {
+        switch (h->LP) {
+            case 16: return launch_leaf_umma<16>(h, x, perm, y, B, st);
+            case 32: return launch_leaf_umma<32>(h, x, perm, y, B, st);
+            case 64: return launch_leaf_umma<64>(h, x, perm, y, B, st);
+        }
+    }
     if (tile_rows == 32) {
         switch (h->LP) {
             case 16: return launch_leaf_mma<16, 32, 6>(h, x, perm, y, B, st);
@@ -610,6 +644,14 @@ fff_status_t pack_leaf_images(fff_handle_s* h) {
     fff::k_pack_b1<T><<<blocks, 256>>>((const T*)h->b1, h->b1img, (int)nl, h->l, LP);
     fff::k_pack_w2<T><<<blocks, 256>>>((const T*)h->w2, (const T*)h->b2, h->w2img, (int)nl, h->l, LP, h->O);
     if (cudaGetLastError() != cudaSuccess) return FFF_ERR_CUDA;
+    // the tcgen05 kernel: W2 in pieces of 128 output features, and its scheduler words
+    if (encode_tiled_fn() && h->O % 16 == 0 && h->D % fff::kLUKB == 0 && std::getenv("FFF_NO_UMMA_LEAF") == nullptr) {
+        const size_t P = (size_t)(h->O + fff::kLUPiece - 1) / fff::kLUPiece;
+        if ((s = dmalloc((void**)&h->w2uimg, nl * P * fff::kLUPiece * LP * 2)) != FFF_OK) return s;
+        if ((s = clone((void**)&h->ws_sched, nullptr, 2 * sizeof(int))) != FFF_OK) return s;
+        fff::k_pack_w2_umma<T><<<blocks, 256>>>((const T*)h->w2, h->w2uimg, (int)nl, h->l, LP, h->O);
+        if (cudaGetLastError() != cudaSuccess) return FFF_ERR_CUDA;
+    }
     return cudaGetLastError() == cudaSuccess ? FFF_OK : FFF_ERR_CUDA;
 }
 

@@ -126,6 +126,27 @@ __device__ __forceinline__ void tma_load_2d(void* dst_smem, const void* tmap, in
         : "memory");
 }
 
+// The same for four separate rows r0..r3 of a tensor map whose box is one row high: the four row
+// pieces land in consecutive rows of the shared-memory tile (4 x box width bytes in all).
+__device__ __forceinline__ void tma_gather4(void* dst_smem, const void* tmap, int c0, int r0, int r1, int r2, int r3,
+                                            uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3, %4, %5, %6}], [%7];" ::"r"(smem_addr(dst_smem)),
+        "l"(tmap), "r"(c0), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(smem_addr(bar))
+        : "memory");
+}
+
+// Makes shared-memory writes of this thread visible to the asynchronous proxy (tensor cores, TMA).
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// 32-byte global store (address 32-byte aligned).
+__device__ __forceinline__ void st_global_v8(void* p, const uint32_t* v) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]),
+                 "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+                 : "memory");
+}
+
 __device__ __forceinline__ void prefetch_tensormap(const void* tmap) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
 }
@@ -147,17 +168,20 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
 __device__ __forceinline__ void tc_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// Shared-memory matrix descriptor of a K-major operand tile whose rows are 128 bytes (64 bf16) long
-// and 128-byte swizzled, 8-row groups 1024 bytes apart; the tile starts on a 1024-byte boundary.
-// Adding 2 to the descriptor moves the start 32 bytes (one K = 16 step) along the row.
-__device__ __forceinline__ uint64_t umma_desc_k128(uint32_t saddr) {
+// Shared-memory matrix descriptor of a K-major operand tile with densely packed rows of row_bytes =
+// 32, 64 or 128 bytes (16, 32 or 64 bf16), swizzled in the mode of that width, 8-row groups
+// 8 * row_bytes apart; the tile starts on a 1024-byte boundary.  Adding 2 to the descriptor moves the
+// start 32 bytes (one K = 16 step) along the row.
+__device__ __forceinline__ uint64_t umma_desc_rows(uint32_t saddr, int row_bytes) {
+    const uint64_t mode = row_bytes == 128 ? 2 : row_bytes == 64 ? 4 : 6;     // 128-, 64-, 32-byte swizzle
     uint64_t d = (uint64_t)((saddr & 0x3FFFFu) >> 4);      // start address / 16
-    d |= (uint64_t)1 << 16;                                // leading-dimension offset (unused by this layout)
-    d |= (uint64_t)(1024 >> 4) << 32;                      // stride between 8-row groups / 16
+    d |= (uint64_t)1 << 16;                                // leading-dimension offset (unused by these layouts)
+    d |= (uint64_t)((8 * row_bytes) >> 4) << 32;           // stride between 8-row groups / 16
     d |= (uint64_t)1 << 46;                                // descriptor version of this architecture
-    d |= (uint64_t)2 << 61;                                // 128-byte swizzle
+    d |= mode << 61;
     return d;
 }
+__device__ __forceinline__ uint64_t umma_desc_k128(uint32_t saddr) { return umma_desc_rows(saddr, 128); }
 
 // Instruction descriptor: bf16 x bf16 -> float32, both operands K-major, M rows, N columns.
 __host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N) {
