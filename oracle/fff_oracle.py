@@ -7,6 +7,7 @@ loops in fff_oracle.c; nothing here is shared with the CUDA path.
 from __future__ import annotations
 
 import ctypes as C
+import threading
 from concurrent.futures import ThreadPoolExecutor
 from typing import Dict, Optional, Tuple
 
@@ -22,32 +23,41 @@ _ip = C.POINTER(C.c_int32)
 _lp = C.POINTER(C.c_long)
 
 
+_lib_lock = threading.Lock()
+
+
 def lib():
     global _lib
     if _lib is None:
-        L = C.CDLL(_build.build())
-        L.fff_oracle_descend.argtypes = [C.c_int, C.c_int, _dp, _dp, _dp, C.c_long, C.c_long, _ip, _dp, _lp]
-        L.fff_oracle_descend.restype = None
-        L.fff_oracle_forward_i.argtypes = [C.c_int] * 5 + [_dp] * 7 + [C.c_long, C.c_long, _dp, _ip, _lp, _lp]
-        L.fff_oracle_forward_i.restype = None
-        L.fff_oracle_forward_t.argtypes = [C.c_int] * 5 + [_dp] * 7 + [C.c_long, _dp]
-        L.fff_oracle_forward_t.restype = None
-        L.fff_oracle_forward_all_leaves_masked.argtypes = [C.c_int] * 5 + [_dp] * 5 + [C.c_long, _ip, _dp]
-        L.fff_oracle_forward_all_leaves_masked.restype = None
-        L.fff_oracle_brute_force_leaf.argtypes = [C.c_int, C.c_int, _dp, _dp, _dp, _ip]
-        L.fff_oracle_brute_force_leaf.restype = C.c_int
-        L.fff_oracle_bucket.argtypes = [_ip, C.c_long, C.c_long, _ip, _ip]
-        L.fff_oracle_bucket.restype = None
-        for name in ("training_size", "inference_size"):
-            f = getattr(L, "fff_oracle_" + name)
-            f.argtypes = [C.c_int] * 3
-            f.restype = C.c_long
-        L.fff_oracle_training_width.argtypes = [C.c_int, C.c_int]
-        L.fff_oracle_training_width.restype = C.c_long
-        L.fff_oracle_inference_width.argtypes = [C.c_int]
-        L.fff_oracle_inference_width.restype = C.c_long
-        _lib = L
+        with _lib_lock:
+            if _lib is None:
+                _lib = _load()
     return _lib
+
+
+def _load():
+    L = C.CDLL(_build.build())
+    L.fff_oracle_descend.argtypes = [C.c_int, C.c_int, _dp, _dp, _dp, C.c_long, C.c_long, _ip, _dp, _lp]
+    L.fff_oracle_descend.restype = None
+    L.fff_oracle_forward_i.argtypes = [C.c_int] * 5 + [_dp] * 7 + [C.c_long, C.c_long, _dp, _ip, _lp, _lp]
+    L.fff_oracle_forward_i.restype = None
+    L.fff_oracle_forward_t.argtypes = [C.c_int] * 5 + [_dp] * 7 + [C.c_long, _dp]
+    L.fff_oracle_forward_t.restype = None
+    L.fff_oracle_forward_all_leaves_masked.argtypes = [C.c_int] * 5 + [_dp] * 5 + [C.c_long, _ip, _dp]
+    L.fff_oracle_forward_all_leaves_masked.restype = None
+    L.fff_oracle_brute_force_leaf.argtypes = [C.c_int, C.c_int, _dp, _dp, _dp, _ip]
+    L.fff_oracle_brute_force_leaf.restype = C.c_int
+    L.fff_oracle_bucket.argtypes = [_ip, C.c_long, C.c_long, _ip, _ip]
+    L.fff_oracle_bucket.restype = None
+    for name in ("training_size", "inference_size"):
+        f = getattr(L, "fff_oracle_" + name)
+        f.argtypes = [C.c_int] * 3
+        f.restype = C.c_long
+    L.fff_oracle_training_width.argtypes = [C.c_int, C.c_int]
+    L.fff_oracle_training_width.restype = C.c_long
+    L.fff_oracle_inference_width.argtypes = [C.c_int]
+    L.fff_oracle_inference_width.restype = C.c_long
+    return L
 
 
 def _d(a) -> np.ndarray:

@@ -57,7 +57,7 @@ struct fff_handle_s {
     __nv_bfloat16* w1img = nullptr;
     float* b1img = nullptr;
     unsigned char* w2img = nullptr;
-    __nv_bfloat16* w2uimg = nullptr;   // W2 pieces of the tcgen05 leaf kernel (nullptr = kernel not available)
+    unsigned char* w2uimg = nullptr;   // W2 pieces (+ biases) of the tcgen05 leaf kernel (nullptr = kernel not available)
     int* ws_sched = nullptr;           // its tile counter and finished-CTA counter (zero between launches)
     fff::Tile* ws_tiles = nullptr;
 
@@ -584,7 +584,7 @@ template <int LP>
 fff_status_t launch_leaf_umma(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, cudaStream_t st) {
     using L = fff::LeafUmmaLayout<LP>;
     const int n_tiles = tile_list_len(B, fff::kLUM, (int)h->n_leaves);
-    const int stages = std::min((int)fff::kLUMaxStages, (kSmemBudget - L::smem_bytes(0, h->O)) / L::kStageBytes);
+    const int stages = std::min((int)fff::kLUMaxStages, (kSmemBudget - L::smem_bytes(0)) / L::kStageBytes);
     if (stages < 2) return FFF_ERR_UNSUPPORTED;
     static bool attr_set[64] = {};
     if (h->device < 64 && !attr_set[h->device]) {
@@ -595,10 +595,10 @@ fff_status_t launch_leaf_umma(fff_handle_s* h, const void* x, const int32_t* per
     if (!make_x_tensor_map(&tm, x, B, h->D, 1)) return FFF_ERR_CUDA;       // one-row boxes: rows are gathered four at a time
     const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(h->sm_count, n_tiles));
     const int wide = (reinterpret_cast<uintptr_t>(y) & 31u) == 0 ? 1 : 0;
-    if (launch_chain(h, fff::k_leaf_umma<LP>, (unsigned)grid, fff::kLUThreads, (size_t)L::smem_bytes(stages, h->O), st, 1, tm, perm,
+    if (launch_chain(h, fff::k_leaf_umma<LP>, (unsigned)grid, fff::kLUThreads, (size_t)L::smem_bytes(stages), st, 1, tm, perm,
                      (const fff::Tile*)h->ws_tiles, n_tiles, (const __nv_bfloat16*)h->w1img, (const float*)h->b1img,
-                     (const __nv_bfloat16*)h->w2uimg, (const __nv_bfloat16*)h->b2, (__nv_bfloat16*)y, h->D, h->O, h->act, stages,
-                     wide, h->ws_sched, h->d_status) != cudaSuccess)
+                     (const unsigned char*)h->w2uimg, (__nv_bfloat16*)y, h->D, h->O, h->act, stages, wide, h->ws_sched,
+                     h->d_status) != cudaSuccess)
         return cudaGetLastError(), FFF_ERR_CUDA;
     return launched(h, st, "grouped_leaf_ff_umma");
 }
@@ -647,9 +647,9 @@ fff_status_t pack_leaf_images(fff_handle_s* h) {
     // the tcgen05 kernel: W2 in pieces of 128 output features, and its scheduler words
     if (encode_tiled_fn() && h->O % 16 == 0 && h->D % fff::kLUKB == 0 && std::getenv("FFF_NO_UMMA_LEAF") == nullptr) {
         const size_t P = (size_t)(h->O + fff::kLUPiece - 1) / fff::kLUPiece;
-        if ((s = dmalloc((void**)&h->w2uimg, nl * P * fff::kLUPiece * LP * 2)) != FFF_OK) return s;
+        if ((s = dmalloc((void**)&h->w2uimg, nl * P * ((size_t)fff::kLUPiece * LP * 2 + fff::kLUPiece * 4))) != FFF_OK) return s;
         if ((s = clone((void**)&h->ws_sched, nullptr, 2 * sizeof(int))) != FFF_OK) return s;
-        fff::k_pack_w2_umma<T><<<blocks, 256>>>((const T*)h->w2, h->w2uimg, (int)nl, h->l, LP, h->O);
+        fff::k_pack_w2_umma<T><<<blocks, 256>>>((const T*)h->w2, (const T*)h->b2, h->w2uimg, (int)nl, h->l, LP, h->O);
         if (cudaGetLastError() != cudaSuccess) return FFF_ERR_CUDA;
     }
     return cudaGetLastError() == cudaSuccess ? FFF_OK : FFF_ERR_CUDA;

@@ -8,17 +8,21 @@
 //
 // Work unit: a tile = up to 128 consecutive entries of one bucket = the 128 rows of one tcgen05.mma.
 // One persistent CTA per SM takes tiles from a device-wide counter, in list order.  Warp roles:
-//   warps 0-3   epilogue, one token row (= one tensor-memory lane) per thread: H = act(acc1 + b1) to
+//   warps 0-7   epilogue.  A thread owns one token row (= one tensor-memory lane; warps w and w + 4
+//               share the lanes of quarter w % 4) and one half of the columns: H = act(acc1 + b1) to
 //               shared memory as the A operand of GEMM2; then, per piece of 128 output columns,
-//               acc2 + b2 -> bf16 -> 32-byte stores straight to the token's row of y;
-//   warp 4      tile scheduler: claims list entries with an atomic counter, skips empty ones and
+//               acc2 + b2 -> bf16 -> 32-byte stores straight to the token's row of y.  One warp per
+//               scheduler issues too slowly for this, hence two;
+//   warp 8      tile scheduler: claims list entries with an atomic counter, skips empty ones and
 //               publishes the tiles a few ahead through a small shared-memory queue;
-//   warp 5      GEMM1 issuer: per K-block of 64 columns four tcgen05.mma (M = 128, N = LP, K = 16);
-//   warp 6      GEMM2: bulk copies of the W2 pieces into their own small ring and, per piece,
-//               LP/16 tcgen05.mma (M = 128, N = 128) into one of two accumulators;
-//   warps 7-10  gather of the token rows: per K-block one tile::gather4 tensor-map load per 4 rows
-//               (4 x 128 bytes, 128-byte swizzled by the copy engine), 32 rows per warp; the first of
-//               them also starts the bulk copy of the matching W1 K-block.
+//   warp 9      GEMM1 issuer: per K-block of 64 columns four tcgen05.mma (M = 128, N = LP, K = 16);
+//   warp 10     GEMM2: bulk copies of the W2 pieces (each followed by its 128 float32 biases) into
+//               their own ring and, per piece, LP/16 tcgen05.mma (M = 128, N = 128) into one of two
+//               accumulators;
+//   warps 11-14 gather of the token rows: per K-block one tile::gather4 tensor-map load per 4 rows
+//               (4 x 128 bytes, 128-byte swizzled by the copy engine), the 4-row groups dealt
+//               round-robin to the four warps; the first of them also starts the bulk copy of the
+//               matching W1 K-block.
 // GEMM1 of the next tile runs while the epilogue of the current one drains, and the row gathers never
 // stop in between: loads and stores overlap across tiles.
 //
@@ -40,8 +44,11 @@ namespace fff {
 constexpr int kLUM = 128;                  // token rows per tile
 constexpr int kLUKB = 64;                  // columns per K-block of GEMM1
 constexpr int kLUPiece = 128;              // output columns per GEMM2 piece
-constexpr int kLUGatherWarps = kLUM / 32;
-constexpr int kLUWarps = 4 + 3 + kLUGatherWarps;
+constexpr int kLUEpiWarps = 8;
+constexpr int kLUGatherWarps = 4;
+constexpr int kLUSchedWarp = kLUEpiWarps, kLUGemm1Warp = kLUEpiWarps + 1, kLUGemm2Warp = kLUEpiWarps + 2;
+constexpr int kLUFirstGatherWarp = kLUEpiWarps + 3;
+constexpr int kLUWarps = kLUEpiWarps + 3 + kLUGatherWarps;
 constexpr int kLUThreads = kLUWarps * 32;
 constexpr int kLUMaxStages = 8;
 constexpr int kLUMaxW2Slots = 8;
@@ -56,15 +63,15 @@ template <int LP> struct LeafUmmaLayout {
     static constexpr int kXStageBytes = kLUM * kLUKB * 2;
     static constexpr int kW1StageBytes = LP * kLUKB * 2;
     static constexpr int kStageBytes = kXStageBytes + kW1StageBytes;         // a multiple of 1024
-    static constexpr int kW2PieceBytes = kLUPiece * kRowBytes;               // a multiple of 1024
+    static constexpr int kW2Bytes = kLUPiece * kRowBytes;                    // weights of a piece
+    static constexpr int kW2PieceBytes = kW2Bytes + kLUPiece * 4;            // + float32 biases
+    static constexpr int kW2SlotStride = (kW2PieceBytes + 1023) & ~1023;
     static constexpr int kHBytes = kLUM * kRowBytes;
     // W2 ring: a whole tile's pieces (O <= 1024) when they are small, so that no copy waits for an MMA just issued
     static constexpr int kW2Slots = LP <= 32 ? 8 : 4;
     static constexpr int kBarrierBytes = 512;
-    // plus the float32 biases of the tile's leaf: LP of b1, O (rounded up to 128) of b2
-    static constexpr int smem_bytes(int stages, int O) {
-        return 1024 + stages * kStageBytes + kW2Slots * kW2PieceBytes + kHBytes + kBarrierBytes +
-               (LP + ((O + 127) & ~127)) * 4;
+    static constexpr int smem_bytes(int stages) {
+        return 1024 + stages * kStageBytes + kW2Slots * kW2SlotStride + kHBytes + kBarrierBytes;
     }
 };
 
@@ -75,40 +82,46 @@ __host__ __device__ __forceinline__ uint32_t swz_rows(uint32_t off, int row_byte
     return off ^ (((off >> 7) & (uint32_t)(row_bytes / 16 - 1)) << 4);
 }
 
-// W2 image for GEMM2: [leaf][ceil(O/128) pieces][128 rows (output features)][LP columns], swizzled per piece.
+// W2 image for GEMM2: [leaf][ceil(O/128) pieces]{ [128 rows (output features)][LP columns] swizzled,
+// then the 128 float32 biases of those features }.
 template <typename T>
-__global__ void k_pack_w2_umma(const T* __restrict__ w2, __nv_bfloat16* __restrict__ img, int n_leaves, int l, int LP, int O)
+__global__ void k_pack_w2_umma(const T* __restrict__ w2, const T* __restrict__ b2, unsigned char* __restrict__ img,
+                               int n_leaves, int l, int LP, int O)
 {
     const int P = (O + kLUPiece - 1) / kLUPiece;
-    const int64_t total = (int64_t)n_leaves * P * kLUPiece * LP;
+    const int64_t piece_bytes = (int64_t)kLUPiece * LP * 2 + kLUPiece * 4;
+    const int64_t total = (int64_t)n_leaves * P * kLUPiece * (LP + 1);      // LP weights + 1 bias per row
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-        const int c = (int)(i % LP);
-        const int n = (int)((i / LP) % kLUPiece);
-        const int64_t jp = i / ((int64_t)LP * kLUPiece);                   // leaf * P + piece
+        const int c = (int)(i % (LP + 1));
+        const int n = (int)((i / (LP + 1)) % kLUPiece);
+        const int64_t jp = i / ((int64_t)(LP + 1) * kLUPiece);             // leaf * P + piece
         const int64_t j = jp / P;
         const int o = (int)(jp % P) * kLUPiece + n;
-        const float v = (o < O && c < l) ? Elem<T>::to_float(w2[(j * O + o) * (int64_t)l + c]) : 0.0f;
-        const uint32_t off = swz_rows((uint32_t)(n * LP * 2 + c * 2), LP * 2);
-        img[jp * (int64_t)(kLUPiece * LP) + off / 2] = __float2bfloat16_rn(v);
+        unsigned char* piece = img + jp * piece_bytes;
+        if (c < LP) {
+            const float v = (o < O && c < l) ? Elem<T>::to_float(w2[(j * O + o) * (int64_t)l + c]) : 0.0f;
+            *reinterpret_cast<__nv_bfloat16*>(piece + swz_rows((uint32_t)(n * LP * 2 + c * 2), LP * 2)) = __float2bfloat16_rn(v);
+        } else {
+            reinterpret_cast<float*>(piece + (int64_t)kLUPiece * LP * 2)[n] = o < O ? Elem<T>::to_float(b2[j * O + o]) : 0.0f;
+        }
     }
 }
 
-// sched: two ints, both zero before the first launch and again after every launch: [0] tiles handed
-// out so far, [1] CTAs that have finished.
+// sched: two ints, both zero before the first launch and again after every launch: [0] list entries
+// handed out so far, [1] CTAs that have finished.
 template <int LP>
 __global__ void __launch_bounds__(kLUThreads, 1)
 k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restrict__ perm,
             const Tile* __restrict__ tiles, int n_tiles_total,
             const __nv_bfloat16* __restrict__ w1img, const float* __restrict__ b1img,
-            const __nv_bfloat16* __restrict__ w2img, const __nv_bfloat16* __restrict__ b2,
-            __nv_bfloat16* __restrict__ y, int D, int O, int act, int kStages, int wide_stores,
-            int* __restrict__ sched, int* __restrict__ status)
+            const unsigned char* __restrict__ w2img, __nv_bfloat16* __restrict__ y,
+            int D, int O, int act, int kStages, int wide_stores, int* __restrict__ sched, int* __restrict__ status)
 {
     using L = LeafUmmaLayout<LP>;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     unsigned char* w2ring = ring + kStages * L::kStageBytes;
-    unsigned char* hbuf = w2ring + L::kW2Slots * L::kW2PieceBytes;
+    unsigned char* hbuf = w2ring + L::kW2Slots * L::kW2SlotStride;
     uint64_t* full = reinterpret_cast<uint64_t*>(hbuf + L::kHBytes);
     uint64_t* empty = full + kLUMaxStages;
     uint64_t* w2_full = empty + kLUMaxStages;
@@ -122,8 +135,6 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
     uint64_t* y_empty = y_full + 2;         // [2]
     Tile* queue = reinterpret_cast<Tile*>(y_empty + 2);                      // [kLUQueue]
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(queue + kLUQueue);
-    float* s_b1 = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(full) + L::kBarrierBytes);     // [LP]
-    float* s_b2 = s_b1 + LP;                                                                                // [O]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int KB = D / kLUKB;
@@ -136,23 +147,23 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
         }
         for (int s = 0; s < L::kW2Slots; ++s) {
             ptx::mbar_init(w2_full + s, 1);
-            ptx::mbar_init(w2_empty + s, 1);
+            ptx::mbar_init(w2_empty + s, 1 + kLUEpiWarps);      // the MMAs that read the weights + every reader of the biases
         }
         for (int s = 0; s < kLUQueue; ++s) {
             ptx::mbar_init(q_full + s, 1);
             ptx::mbar_init(q_empty + s, kLUConsumerWarps);
         }
         ptx::mbar_init(acc1_full, 1);
-        ptx::mbar_init(acc1_empty, 128);
-        ptx::mbar_init(h_full, 128);
+        ptx::mbar_init(acc1_empty, kLUEpiWarps * 32);
+        ptx::mbar_init(h_full, kLUEpiWarps * 32);
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(y_full + b, 1);
-            ptx::mbar_init(y_empty + b, 128);
+            ptx::mbar_init(y_empty + b, kLUEpiWarps * 32);
         }
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(&tmap_x);
     }
-    if (warp == 5) {
+    if (warp == kLUGemm1Warp) {
         ptx::tmem_alloc(tmem_slot, kLUTmemCols);
         ptx::tmem_relinquish_alloc_permit();
     }
@@ -164,7 +175,7 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
     const uint32_t tmem_base = *tmem_slot;
 
     bool timed_out = false;
-    const int max_iters = 2 * n_tiles_total + kLUQueue + 1;     // no role loops longer than this, whatever it reads
+    const int max_iters = n_tiles_total + kLUQueue + 1;     // no role loops longer than this, whatever it reads
 
     // Consumers take the tiles in the order the scheduler published them; rows < 0 ends the sequence.
     int q_slot = 0;
@@ -178,13 +189,12 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
         return tl;
     };
 
-    if (warp == 4) {
+    if (warp == kLUSchedWarp) {
         // ------------------------------------------------------------------ scheduler
         int fetched = 0;
-        bool done = false;
         Tile last;
         last.bin = 0; last.start = 0; last.rows = -1; last.pad = 0;
-        while (!done) {
+        for (;;) {
             int idx = 0;
             if (lane == 0) idx = atomicAdd(sched, 1);
             idx = __shfl_sync(kFullMask, idx, 0);
@@ -209,19 +219,20 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
             __syncwarp();
             if (++q_slot == kLUQueue) { q_slot = 0; q_phase ^= 1; }
         }
-    } else if (warp >= 7) {
+    } else if (warp >= kLUFirstGatherWarp) {
         // ------------------------------------------------------------------ row gathers
-        const int gw = warp - 7;
+        const int gw = warp - kLUFirstGatherWarp;
         int stage = 0;
         uint32_t phase = 0;
         for (int it = 0; it < max_iters; ++it) {
             const Tile tl = next_tile();
             if (tl.rows <= 0) break;
-            const int rows_here = min(max(tl.rows - gw * 32, 0), 32);
-            const int groups = (rows_here + 3) >> 2;                   // gather4 requests of this warp per K-block
+            // 4-row group g = lane * kLUGatherWarps + gw of the tile belongs to this lane
+            const int total_groups = (tl.rows + 3) >> 2;
+            const int groups = max((total_groups - gw + kLUGatherWarps - 1) / kLUGatherWarps, 0);     // of this warp
+            const int first = (lane * kLUGatherWarps + gw) * 4;
             int r[4] = {0, 0, 0, 0};
             if (lane < groups) {
-                const int first = gw * 32 + lane * 4;
 #pragma unroll
                 for (int i = 0; i < 4; ++i) r[i] = perm[tl.start + min(first + i, tl.rows - 1)];
             }
@@ -237,12 +248,12 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                 }
                 __syncwarp();
                 if (lane < groups)
-                    ptx::tma_gather4(ring + stage * L::kStageBytes + (gw * 32 + lane * 4) * 128, &tmap_x, kb * kLUKB, r[0], r[1],
-                                     r[2], r[3], full + stage);
+                    ptx::tma_gather4(ring + stage * L::kStageBytes + first * 128, &tmap_x, kb * kLUKB, r[0], r[1], r[2], r[3],
+                                     full + stage);
                 if (++stage == kStages) { stage = 0; phase ^= 1; }
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == kLUGemm1Warp) {
         // ------------------------------------------------------------------ GEMM1 issuer
         constexpr uint32_t idesc = ptx::umma_idesc_bf16(kLUM, LP);
         int stage = 0;
@@ -268,7 +279,7 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                 if (++stage == kStages) { stage = 0; phase ^= 1; }
             }
         }
-    } else if (warp == 6) {
+    } else if (warp == kLUGemm2Warp) {
         // ------------------------------------------------------------------ W2 copies + GEMM2 issuer
         int ld_slot = 0, mm_slot = 0;
         uint32_t ld_phase = 0, mm_phase = 0;
@@ -277,13 +288,13 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
         for (int it = 0; it < max_iters; ++it) {
             const Tile tl = next_tile();
             if (tl.rows <= 0) break;
-            const __nv_bfloat16* w2j = w2img + (int64_t)tl.bin * P * (kLUPiece * LP);
+            const unsigned char* w2j = w2img + (int64_t)tl.bin * P * L::kW2PieceBytes;
             int loaded = 0;
             auto load_piece = [&]() {
                 if (!timed_out && !ptx::mbar_wait(w2_empty + ld_slot, ld_phase ^ 1)) timed_out = true;
                 if (lane == 0) {
                     ptx::mbar_arrive_expect_tx(w2_full + ld_slot, (uint32_t)L::kW2PieceBytes);
-                    ptx::bulk_g2s(w2ring + ld_slot * L::kW2PieceBytes, w2j + (int64_t)loaded * (kLUPiece * LP), L::kW2PieceBytes,
+                    ptx::bulk_g2s(w2ring + ld_slot * L::kW2SlotStride, w2j + (int64_t)loaded * L::kW2PieceBytes, L::kW2PieceBytes,
                                   w2_full + ld_slot);
                 }
                 __syncwarp();
@@ -294,7 +305,6 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
             if (!timed_out && !ptx::mbar_wait(h_full, it & 1)) timed_out = true;
             ptx::tc_fence_after_sync();
             for (int p = 0; p < P; ++p, ++pc) {
-                if (loaded < P) load_piece();
                 const int b = pc & 1;
                 if (!timed_out && !ptx::mbar_wait(w2_full + mm_slot, mm_phase)) timed_out = true;
                 if (!timed_out && !ptx::mbar_wait(y_empty + b, ((pc >> 1) & 1) ^ 1)) timed_out = true;
@@ -303,7 +313,7 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                     const int n = min(kLUPiece, O - p * kLUPiece);
                     const uint32_t idesc = ptx::umma_idesc_bf16(kLUM, n);
                     const uint64_t ad = ptx::umma_desc_rows(hs, L::kRowBytes);
-                    const uint64_t bd = ptx::umma_desc_rows(ptx::smem_addr(w2ring + mm_slot * L::kW2PieceBytes), L::kRowBytes);
+                    const uint64_t bd = ptx::umma_desc_rows(ptx::smem_addr(w2ring + mm_slot * L::kW2SlotStride), L::kRowBytes);
 #pragma unroll
                     for (int kk = 0; kk < LP / 16; ++kk)
                         ptx::umma_bf16(tmem_base + kLUAcc2Col + b * kLUPiece, ad + 2 * kk, bd + 2 * kk, idesc, kk != 0 ? 1u : 0u);
@@ -312,77 +322,76 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                 }
                 __syncwarp();
                 if (++mm_slot == L::kW2Slots) { mm_slot = 0; mm_phase ^= 1; }
+                if (loaded < P) load_piece();                    // only when a tile has more pieces than ring slots
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue: one token row per thread
-        const int row = warp * 32 + lane;
-        const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+        // ------------------------------------------------------------------ epilogue: one token row and one column half per thread
+        const int quarter = warp & 3, half = warp >> 2;
+        const int row = quarter * 32 + lane;
+        const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        constexpr int HC = LP / 2;                               // H columns of this thread
         int pc = 0;
+        int w2_slot = 0;
+        uint32_t w2_phase = 0;
         for (int it = 0; it < max_iters; ++it) {
             const Tile tl = next_tile();
             if (tl.rows <= 0) break;
             const int64_t tok = row < tl.rows ? perm[tl.start + row] : -1;
-            // biases of this tile's leaf as float32 in shared memory (the four warps share them)
-            asm volatile("bar.sync 1, 128;" ::: "memory");       // everyone is done with the previous tile's biases
-            if (row < LP) s_b1[row] = __ldg(b1img + (int64_t)tl.bin * LP + row);
-            for (int i = row; i < O / 8; i += 128) {
-                const uint4 bb = __ldg(reinterpret_cast<const uint4*>(b2 + (int64_t)tl.bin * O) + i);
-                const uint32_t bw[4] = {bb.x, bb.y, bb.z, bb.w};
+            float b1r[HC];
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    s_b2[8 * i + 2 * e] = __uint_as_float(bw[e] << 16);
-                    s_b2[8 * i + 2 * e + 1] = __uint_as_float(bw[e] & 0xFFFF0000u);
-                }
+            for (int j = 0; j < HC; j += 4) {
+                const float4 t = __ldg(reinterpret_cast<const float4*>(b1img + (int64_t)tl.bin * LP + half * HC + j));
+                b1r[j] = t.x; b1r[j + 1] = t.y; b1r[j + 2] = t.z; b1r[j + 3] = t.w;
             }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
 
-            // H = act(acc1 + b1) -> bf16 -> this thread's row of the A operand of GEMM2
+            // H = act(acc1 + b1) -> bf16 -> this thread's part of its row of the A operand of GEMM2
             if (!timed_out && !ptx::mbar_wait(acc1_full, it & 1)) timed_out = true;
             ptx::tc_fence_after_sync();
             {
-                uint32_t hp[LP / 2];
-#pragma unroll
-                for (int c0 = 0; c0 < LP; c0 += 32) {
-                    uint32_t v[32];
-                    ptx::tmem_ld32(lane_base + c0, v);        // columns past LP of the last load are not used
-                    ptx::tmem_ld_wait();
-#pragma unroll
-                    for (int j = 0; j < 32 && c0 + j < LP; j += 2) {
-                        hp[(c0 + j) / 2] = ptx::pack_bf16(activate(act, __uint_as_float(v[j]) + s_b1[c0 + j]),
-                                                          activate(act, __uint_as_float(v[j + 1]) + s_b1[c0 + j + 1]));
-                    }
-                }
+                uint32_t v[32];
+                ptx::tmem_ld32(lane_base + half * HC, v);      // columns past HC are not used
+                ptx::tmem_ld_wait();
                 ptx::tc_fence_before_sync();
                 ptx::mbar_arrive(acc1_empty);
+                uint32_t hp[HC / 2];
 #pragma unroll
-                for (int c = 0; c < LP / 8; ++c)
-                    *reinterpret_cast<uint4*>(hbuf + swz_rows((uint32_t)(row * L::kRowBytes + c * 16), L::kRowBytes)) =
+                for (int j = 0; j < HC; j += 2)
+                    hp[j / 2] = ptx::pack_bf16(activate(act, __uint_as_float(v[j]) + b1r[j]),
+                                               activate(act, __uint_as_float(v[j + 1]) + b1r[j + 1]));
+#pragma unroll
+                for (int c = 0; c < HC / 8; ++c)
+                    *reinterpret_cast<uint4*>(hbuf + swz_rows((uint32_t)(row * L::kRowBytes + (half * HC / 8 + c) * 16), L::kRowBytes)) =
                         make_uint4(hp[4 * c], hp[4 * c + 1], hp[4 * c + 2], hp[4 * c + 3]);
                 ptx::fence_proxy_async();
                 ptx::mbar_arrive(h_full);
             }
 
-            // Y pieces
+            // Y pieces: this thread's 64 of the 128 columns
             __nv_bfloat16* yrow = y + (tok >= 0 ? tok : 0) * O;
             for (int p = 0; p < P; ++p, ++pc) {
                 const int b = pc & 1;
                 if (!timed_out && !ptx::mbar_wait(y_full + b, (pc >> 1) & 1)) timed_out = true;
+                if (!timed_out && !ptx::mbar_wait(w2_full + w2_slot, w2_phase)) timed_out = true;     // biases: landed long ago
                 ptx::tc_fence_after_sync();
+                const float* bias = reinterpret_cast<const float*>(w2ring + w2_slot * L::kW2SlotStride + L::kW2Bytes);
                 const int ncols = min(kLUPiece, O - p * kLUPiece);
-#pragma unroll 1
-                for (int c0 = 0; c0 < ncols; c0 += 32) {
+#pragma unroll
+                for (int cc = 0; cc < 2; ++cc) {
+                    const int c0 = half * 64 + cc * 32;
                     uint32_t v[32];
                     ptx::tmem_ld32(lane_base + kLUAcc2Col + b * kLUPiece + c0, v);
                     ptx::tmem_ld_wait();
                     const int o0 = p * kLUPiece + c0;
-                    const int nv = min(32, ncols - c0);              // 16 or 32
+                    const int nv = min(32, ncols - c0);              // <= 0, 16 or 32
                     uint32_t out[16];
 #pragma unroll
-                    for (int e = 0; e < 16; ++e)
-                        out[e] = ptx::pack_bf16(__uint_as_float(v[2 * e]) + s_b2[o0 + 2 * e],
-                                                __uint_as_float(v[2 * e + 1]) + s_b2[o0 + 2 * e + 1]);
-                    if (tok >= 0) {
+                    for (int e = 0; e < 8; ++e) {
+                        const float4 bb = *reinterpret_cast<const float4*>(bias + c0 + 4 * e);
+                        out[2 * e] = ptx::pack_bf16(__uint_as_float(v[4 * e]) + bb.x, __uint_as_float(v[4 * e + 1]) + bb.y);
+                        out[2 * e + 1] = ptx::pack_bf16(__uint_as_float(v[4 * e + 2]) + bb.z, __uint_as_float(v[4 * e + 3]) + bb.w);
+                    }
+                    if (tok >= 0 && nv > 0) {
                         if (wide_stores && nv == 32) {
                             ptx::st_global_v8(yrow + o0, out);
                             ptx::st_global_v8(yrow + o0 + 16, out + 8);
@@ -397,6 +406,9 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                 }
                 ptx::tc_fence_before_sync();
                 ptx::mbar_arrive(y_empty + b);
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(w2_empty + w2_slot);
+                if (++w2_slot == L::kW2Slots) { w2_slot = 0; w2_phase ^= 1; }
             }
         }
     }
@@ -406,7 +418,7 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == kLUGemm1Warp) {
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, kLUTmemCols);
     }
