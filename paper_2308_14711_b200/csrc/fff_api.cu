@@ -155,7 +155,9 @@ cudaError_t launch_chain(fff_handle_s* h, void (*kern)(KArgs...), unsigned grid,
         attr[n].val.clusterDim.z = 1;
         ++n;
     }
-    if (h->pdl && h->launches > 0 && !h->prof_active) {
+    // (also the first kernel of a call: it may then start its prologue while the last kernel of the
+    // previous call on this stream drains; with any other predecessor the attribute changes nothing)
+    if (h->pdl && !h->prof_active) {
         attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[n].val.programmaticStreamSerializationAllowed = 1;
         ++n;
@@ -200,7 +202,10 @@ int leaf_tile_rows(const fff_handle_s* h, int64_t B) {
         const int v = e ? std::atoi(e) : 0;
         return (v == 32 || v == 64) ? v : 0;
     }();
-    if (h->w2uimg) return fff::kLUM;              // the tcgen05 kernel works on 128-row tiles
+    // The tcgen05 kernel works on 128-row tiles and wins when buckets fill them reasonably well; with thin
+    // buckets (measured at 32 tokens per leaf) the mma.sync kernel on 32-row tiles is ahead.
+    static const bool force_umma = std::getenv("FFF_FORCE_UMMA_LEAF") != nullptr;      // tuning aid
+    if (h->w2uimg && (force_umma || B >= 48 * h->n_leaves)) return fff::kLUM;
     if (forced) return forced;
     return B / h->n_leaves <= 40 ? 32 : 64;
 }
@@ -529,10 +534,9 @@ fff_status_t pack_node_images(fff_handle_s* h) {
             for (size_t i = 1; i < ks.size(); ++i) ok = ok && ks[i] >= 1 && ks[i] <= 6;
             if (!ok) ks.clear();
         }
-        if (ks.empty()) {
-            ks.push_back(std::min(d, 8));
-            for (int k : cut_levels(d - ks[0])) ks.push_back(k);
-        }
+        // Up to 8 levels in one stage when that is the whole tree (no node bucketing at all); deeper
+        // trees measured best with the usual cut into stages of at most 6 levels.
+        if (ks.empty()) ks = d <= 8 ? std::vector<int>{d} : cut_levels(d);
         L0 = 0;
         for (size_t i = 0; i < ks.size(); ++i) {
             const int np = i == 0 ? std::max(32, 1 << ks[i]) : std::max(16, 1 << ks[i]);

@@ -11,8 +11,9 @@
 //   warps 0-7   epilogue.  A thread owns one token row (= one tensor-memory lane; warps w and w + 4
 //               share the lanes of quarter w % 4) and one half of the columns: H = act(acc1 + b1) to
 //               shared memory as the A operand of GEMM2; then, per piece of 128 output columns,
-//               acc2 + b2 -> bf16 -> 32-byte stores straight to the token's row of y.  One warp per
-//               scheduler issues too slowly for this, hence two;
+//               acc2 + b2 -> bf16 -> 32-byte stores straight to the token's row of y.  Two warps per
+//               quarter measured faster than one and than four; quarters without valid rows (short
+//               tiles) only keep the barriers moving;
 //   warp 8      tile scheduler: claims list entries with an atomic counter, skips empty ones and
 //               publishes the tiles a few ahead through a small shared-memory queue;
 //   warp 9      GEMM1 issuer: per K-block of 64 columns four tcgen05.mma (M = 128, N = LP, K = 16);
@@ -45,6 +46,7 @@ constexpr int kLUM = 128;                  // token rows per tile
 constexpr int kLUKB = 64;                  // columns per K-block of GEMM1
 constexpr int kLUPiece = 128;              // output columns per GEMM2 piece
 constexpr int kLUEpiWarps = 8;
+constexpr int kLUColParts = kLUEpiWarps / 4;       // epilogue warps per lane quarter = column parts per piece
 constexpr int kLUGatherWarps = 4;
 constexpr int kLUSchedWarp = kLUEpiWarps, kLUGemm1Warp = kLUEpiWarps + 1, kLUGemm2Warp = kLUEpiWarps + 2;
 constexpr int kLUFirstGatherWarp = kLUEpiWarps + 3;
@@ -326,22 +328,24 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue: one token row and one column half per thread
-        const int quarter = warp & 3, half = warp >> 2;
+        // ------------------------------------------------------------------ epilogue: one token row and one column part per thread
+        const int quarter = warp & 3, part = warp >> 2;
         const int row = quarter * 32 + lane;
         const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
-        constexpr int HC = LP / 2;                               // H columns of this thread
+        constexpr int HC = LP / kLUColParts;                     // H columns of this thread (4, 8 or 16)
+        constexpr int YC = kLUPiece / kLUColParts;               // y columns of this thread per piece
         int pc = 0;
         int w2_slot = 0;
         uint32_t w2_phase = 0;
         for (int it = 0; it < max_iters; ++it) {
             const Tile tl = next_tile();
             if (tl.rows <= 0) break;
+            const bool active = quarter * 32 < tl.rows;          // this warp's lanes hold valid rows
             const int64_t tok = row < tl.rows ? perm[tl.start + row] : -1;
             float b1r[HC];
 #pragma unroll
             for (int j = 0; j < HC; j += 4) {
-                const float4 t = __ldg(reinterpret_cast<const float4*>(b1img + (int64_t)tl.bin * LP + half * HC + j));
+                const float4 t = __ldg(reinterpret_cast<const float4*>(b1img + (int64_t)tl.bin * LP + part * HC + j));
                 b1r[j] = t.x; b1r[j + 1] = t.y; b1r[j + 2] = t.z; b1r[j + 3] = t.w;
             }
 
@@ -349,25 +353,34 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
             if (!timed_out && !ptx::mbar_wait(acc1_full, it & 1)) timed_out = true;
             ptx::tc_fence_after_sync();
             {
-                uint32_t v[32];
-                ptx::tmem_ld32(lane_base + half * HC, v);      // columns past HC are not used
-                ptx::tmem_ld_wait();
+                uint32_t hp[HC / 2];
+                if (active) {
+                    uint32_t v[32];
+                    ptx::tmem_ld32(lane_base + part * HC, v);      // columns past HC are not used
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < HC; j += 2)
+                        hp[j / 2] = ptx::pack_bf16(activate(act, __uint_as_float(v[j]) + b1r[j]),
+                                                   activate(act, __uint_as_float(v[j + 1]) + b1r[j + 1]));
+                }
                 ptx::tc_fence_before_sync();
                 ptx::mbar_arrive(acc1_empty);
-                uint32_t hp[HC / 2];
+                if (active) {
+                    if constexpr (HC == 4) {
+                        unsigned char* dst = hbuf + swz_rows((uint32_t)(row * L::kRowBytes + (part >> 1) * 16), L::kRowBytes) + (part & 1) * 8;
+                        *reinterpret_cast<uint2*>(dst) = make_uint2(hp[0], hp[1]);
+                    } else {
 #pragma unroll
-                for (int j = 0; j < HC; j += 2)
-                    hp[j / 2] = ptx::pack_bf16(activate(act, __uint_as_float(v[j]) + b1r[j]),
-                                               activate(act, __uint_as_float(v[j + 1]) + b1r[j + 1]));
-#pragma unroll
-                for (int c = 0; c < HC / 8; ++c)
-                    *reinterpret_cast<uint4*>(hbuf + swz_rows((uint32_t)(row * L::kRowBytes + (half * HC / 8 + c) * 16), L::kRowBytes)) =
-                        make_uint4(hp[4 * c], hp[4 * c + 1], hp[4 * c + 2], hp[4 * c + 3]);
-                ptx::fence_proxy_async();
+                        for (int c = 0; c < HC / 8; ++c)
+                            *reinterpret_cast<uint4*>(hbuf + swz_rows((uint32_t)(row * L::kRowBytes + (part * HC / 8 + c) * 16), L::kRowBytes)) =
+                                make_uint4(hp[4 * c], hp[4 * c + 1], hp[4 * c + 2], hp[4 * c + 3]);
+                    }
+                    ptx::fence_proxy_async();
+                }
                 ptx::mbar_arrive(h_full);
             }
 
-            // Y pieces: this thread's 64 of the 128 columns
+            // Y pieces: this thread's share of the 128 columns
             __nv_bfloat16* yrow = y + (tok >= 0 ? tok : 0) * O;
             for (int p = 0; p < P; ++p, ++pc) {
                 const int b = pc & 1;
@@ -377,30 +390,32 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                 const float* bias = reinterpret_cast<const float*>(w2ring + w2_slot * L::kW2SlotStride + L::kW2Bytes);
                 const int ncols = min(kLUPiece, O - p * kLUPiece);
 #pragma unroll
-                for (int cc = 0; cc < 2; ++cc) {
-                    const int c0 = half * 64 + cc * 32;
-                    uint32_t v[32];
-                    ptx::tmem_ld32(lane_base + kLUAcc2Col + b * kLUPiece + c0, v);
-                    ptx::tmem_ld_wait();
-                    const int o0 = p * kLUPiece + c0;
+                for (int cc = 0; cc < YC / 32; ++cc) {
+                    const int c0 = part * YC + cc * 32;
                     const int nv = min(32, ncols - c0);              // <= 0, 16 or 32
-                    uint32_t out[16];
+                    if (active && nv > 0) {
+                        uint32_t v[32];
+                        ptx::tmem_ld32(lane_base + kLUAcc2Col + b * kLUPiece + c0, v);
+                        ptx::tmem_ld_wait();
+                        const int o0 = p * kLUPiece + c0;
+                        uint32_t out[16];
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        const float4 bb = *reinterpret_cast<const float4*>(bias + c0 + 4 * e);
-                        out[2 * e] = ptx::pack_bf16(__uint_as_float(v[4 * e]) + bb.x, __uint_as_float(v[4 * e + 1]) + bb.y);
-                        out[2 * e + 1] = ptx::pack_bf16(__uint_as_float(v[4 * e + 2]) + bb.z, __uint_as_float(v[4 * e + 3]) + bb.w);
-                    }
-                    if (tok >= 0 && nv > 0) {
-                        if (wide_stores && nv == 32) {
-                            ptx::st_global_v8(yrow + o0, out);
-                            ptx::st_global_v8(yrow + o0 + 16, out + 8);
-                        } else {
+                        for (int e = 0; e < 8; ++e) {
+                            const float4 bb = *reinterpret_cast<const float4*>(bias + c0 + 4 * e);
+                            out[2 * e] = ptx::pack_bf16(__uint_as_float(v[4 * e]) + bb.x, __uint_as_float(v[4 * e + 1]) + bb.y);
+                            out[2 * e + 1] = ptx::pack_bf16(__uint_as_float(v[4 * e + 2]) + bb.z, __uint_as_float(v[4 * e + 3]) + bb.w);
+                        }
+                        if (tok >= 0) {
+                            if (wide_stores && nv == 32) {
+                                ptx::st_global_v8(yrow + o0, out);
+                                ptx::st_global_v8(yrow + o0 + 16, out + 8);
+                            } else {
 #pragma unroll
-                            for (int q = 0; q < 4; ++q)
-                                if (q * 8 < nv)
-                                    *reinterpret_cast<uint4*>(yrow + o0 + q * 8) =
-                                        make_uint4(out[4 * q], out[4 * q + 1], out[4 * q + 2], out[4 * q + 3]);
+                                for (int q = 0; q < 4; ++q)
+                                    if (q * 8 < nv)
+                                        *reinterpret_cast<uint4*>(yrow + o0 + q * 8) =
+                                            make_uint4(out[4 * q], out[4 * q + 1], out[4 * q + 2], out[4 * q + 3]);
+                            }
                         }
                     }
                 }
