@@ -202,10 +202,10 @@ int leaf_tile_rows(const fff_handle_s* h, int64_t B) {
         const int v = e ? std::atoi(e) : 0;
         return (v == 32 || v == 64) ? v : 0;
     }();
-    // The tcgen05 kernel works on 128-row tiles and wins when buckets fill them reasonably well; with thin
-    // buckets (measured at 32 tokens per leaf) the mma.sync kernel on 32-row tiles is ahead.
-    static const bool force_umma = std::getenv("FFF_FORCE_UMMA_LEAF") != nullptr;      // tuning aid
-    if (h->w2uimg && (force_umma || B >= 48 * h->n_leaves)) return fff::kLUM;
+    // The tcgen05 kernel works on 128-row tiles.  Measured against the mma.sync kernel it is far ahead when
+    // some buckets are large (skewed routing), about level with uniformly thin buckets of 32 tokens, and is
+    // left out only when buckets are thinner still (every tile costs its epilogue a fixed few microseconds).
+    if (h->w2uimg && B >= 16 * h->n_leaves) return fff::kLUM;
     if (forced) return forced;
     return B / h->n_leaves <= 40 ? 32 : 64;
 }
@@ -599,9 +599,10 @@ fff_status_t launch_leaf_umma(fff_handle_s* h, const void* x, const int32_t* per
     if (!make_x_tensor_map(&tm, x, B, h->D, 1)) return FFF_ERR_CUDA;       // one-row boxes: rows are gathered four at a time
     const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(h->sm_count, n_tiles));
     const int wide = (reinterpret_cast<uintptr_t>(y) & 31u) == 0 ? 1 : 0;
+    const int passes = 1;      // two passes (full tiles first) measured slightly slower
     if (launch_chain(h, fff::k_leaf_umma<LP>, (unsigned)grid, fff::kLUThreads, (size_t)L::smem_bytes(stages), st, 1, tm, perm,
                      (const fff::Tile*)h->ws_tiles, n_tiles, (const __nv_bfloat16*)h->w1img, (const float*)h->b1img,
-                     (const unsigned char*)h->w2uimg, (__nv_bfloat16*)y, h->D, h->O, h->act, stages, wide, h->ws_sched,
+                     (const unsigned char*)h->w2uimg, (__nv_bfloat16*)y, h->D, h->O, h->act, stages, wide, passes, h->ws_sched,
                      h->d_status) != cudaSuccess)
         return cudaGetLastError(), FFF_ERR_CUDA;
     return launched(h, st, "grouped_leaf_ff_umma");

@@ -65,6 +65,21 @@ __device__ __forceinline__ float activate(int act, float v) {
     return 0.5f * v * (1.0f + erff(v * 0.70710678118654752440f));
 }
 
+// The same for kernels whose result is rounded to bf16 right away: erf by the rational-times-exponential
+// formula 7.1.26 of Abramowitz & Stegun (absolute error below 1.5e-7, far inside half a bf16 ulp of the
+// GELU value), one exponential and one division instead of the long polynomial of erff.
+__device__ __forceinline__ float activate_bf16(int act, float v) {
+    if (act == kActRelu) return fmaxf(v, 0.0f);
+    const float z = fabsf(v) * 0.70710678118654752440f;
+    const float t = __fdividef(1.0f, fmaf(0.3275911f, z, 1.0f));
+    float poly = fmaf(1.061405429f, t, -1.453152027f);
+    poly = fmaf(poly, t, 1.421413741f);
+    poly = fmaf(poly, t, -0.284496736f);
+    poly = fmaf(poly, t, 0.254829592f);
+    const float e = 1.0f - poly * t * __expf(-z * z);          // erf(|v| / sqrt 2)
+    return 0.5f * v * (1.0f + copysignf(e, v));
+}
+
 // <a, b> over n elements, evaluated by one warp; every lane returns the sum.
 // `vec` says both rows start on 16-byte boundaries and n is a multiple of kVec.
 template <typename T>

@@ -12,10 +12,12 @@
 //               share the lanes of quarter w % 4) and one half of the columns: H = act(acc1 + b1) to
 //               shared memory as the A operand of GEMM2; then, per piece of 128 output columns,
 //               acc2 + b2 -> bf16 -> 32-byte stores straight to the token's row of y.  Two warps per
-//               quarter measured faster than one and than four; quarters without valid rows (short
-//               tiles) only keep the barriers moving;
+//               quarter measured faster than one, three (with 96-column pieces) and four; quarters
+//               without valid rows (short tiles) only keep the barriers moving;
 //   warp 8      tile scheduler: claims list entries with an atomic counter, skips empty ones and
-//               publishes the tiles a few ahead through a small shared-memory queue;
+//               publishes them through a small shared-memory queue.  A tile is claimed only when the
+//               gathers have started on the one before it: claiming further ahead would hand a CTA
+//               work long before it can do it and leave other SMs idle at the end;
 //   warp 9      GEMM1 issuer: per K-block of 64 columns four tcgen05.mma (M = 128, N = LP, K = 16);
 //   warp 10     GEMM2: bulk copies of the W2 pieces (each followed by its 128 float32 biases) into
 //               their own ring and, per piece, LP/16 tcgen05.mma (M = 128, N = 128) into one of two
@@ -32,7 +34,7 @@
 //
 // Every wait is bounded (see ptx.cuh); tensor memory is released on every exit path.
 //
-// Requirements: bf16, D % 64 == 0, O % 16 == 0, l <= 64 (padded to LP in {16, 32, 64}), x 16-byte aligned.
+// Requirements: bf16, D % 128 == 0, O % 16 == 0, l <= 64 (padded to LP in {16, 32, 64}), x 16-byte aligned.
 #pragma once
 
 #include <cuda.h>      // CUtensorMap
@@ -45,15 +47,18 @@ namespace fff {
 constexpr int kLUM = 128;                  // token rows per tile
 constexpr int kLUKB = 64;                  // columns per K-block of GEMM1
 constexpr int kLUPiece = 128;              // output columns per GEMM2 piece
+constexpr int kLUAccStride = 128;          // tensor-memory columns between the two GEMM2 accumulators
 constexpr int kLUEpiWarps = 8;
 constexpr int kLUColParts = kLUEpiWarps / 4;       // epilogue warps per lane quarter = column parts per piece
+constexpr int kLUHParts = 2;                       // of which this many compute H
+static_assert(kLUPiece % (32 * kLUColParts) == 0, "whole 32-column tensor-memory loads per piece and thread");
 constexpr int kLUGatherWarps = 4;
 constexpr int kLUSchedWarp = kLUEpiWarps, kLUGemm1Warp = kLUEpiWarps + 1, kLUGemm2Warp = kLUEpiWarps + 2;
 constexpr int kLUFirstGatherWarp = kLUEpiWarps + 3;
 constexpr int kLUWarps = kLUEpiWarps + 3 + kLUGatherWarps;
 constexpr int kLUThreads = kLUWarps * 32;
 constexpr int kLUMaxStages = 8;
-constexpr int kLUMaxW2Slots = 8;
+constexpr int kLUMaxW2Slots = 12;
 constexpr int kLUQueue = 4;                // tiles published ahead by the scheduler
 constexpr int kLUConsumerWarps = kLUWarps - 1;     // every warp but the scheduler reads the tile queue
 constexpr int kLUAcc2Col = 64;             // first tensor-memory column of the two GEMM2 accumulators
@@ -62,8 +67,14 @@ constexpr int kLUTmemCols = 512;
 template <int LP> struct LeafUmmaLayout {
     static_assert(LP == 16 || LP == 32 || LP == 64, "padded hidden width");
     static constexpr int kRowBytes = LP * 2;                                 // row of H and of a W2 piece
-    static constexpr int kXStageBytes = kLUM * kLUKB * 2;
-    static constexpr int kW1StageBytes = LP * kLUKB * 2;
+    // A ring stage holds kSub K-blocks of 64 columns (each a 128-byte swizzled operand tile of its own):
+    // every stage costs each role a fixed few hundred cycles of barrier traffic, so two K-blocks share one
+    // where shared memory allows.
+    static constexpr int kSub = LP <= 32 ? 2 : 1;
+    static constexpr int kXSubBytes = kLUM * kLUKB * 2;
+    static constexpr int kW1SubBytes = LP * kLUKB * 2;
+    static constexpr int kXStageBytes = kSub * kXSubBytes;
+    static constexpr int kW1StageBytes = kSub * kW1SubBytes;
     static constexpr int kStageBytes = kXStageBytes + kW1StageBytes;         // a multiple of 1024
     static constexpr int kW2Bytes = kLUPiece * kRowBytes;                    // weights of a piece
     static constexpr int kW2PieceBytes = kW2Bytes + kLUPiece * 4;            // + float32 biases
@@ -71,7 +82,7 @@ template <int LP> struct LeafUmmaLayout {
     static constexpr int kHBytes = kLUM * kRowBytes;
     // W2 ring: a whole tile's pieces (O <= 1024) when they are small, so that no copy waits for an MMA just issued
     static constexpr int kW2Slots = LP <= 32 ? 8 : 4;
-    static constexpr int kBarrierBytes = 512;
+    static constexpr int kBarrierBytes = 640;
     static constexpr int smem_bytes(int stages) {
         return 1024 + stages * kStageBytes + kW2Slots * kW2SlotStride + kHBytes + kBarrierBytes;
     }
@@ -117,7 +128,7 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
             const Tile* __restrict__ tiles, int n_tiles_total,
             const __nv_bfloat16* __restrict__ w1img, const float* __restrict__ b1img,
             const unsigned char* __restrict__ w2img, __nv_bfloat16* __restrict__ y,
-            int D, int O, int act, int kStages, int wide_stores, int* __restrict__ sched, int* __restrict__ status)
+            int D, int O, int act, int kStages, int wide_stores, int passes, int* __restrict__ sched, int* __restrict__ status)
 {
     using L = LeafUmmaLayout<LP>;
     extern __shared__ unsigned char smem_raw[];
@@ -137,9 +148,10 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
     uint64_t* y_empty = y_full + 2;         // [2]
     Tile* queue = reinterpret_cast<Tile*>(y_empty + 2);                      // [kLUQueue]
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(queue + kLUQueue);
+    uint64_t* want = reinterpret_cast<uint64_t*>(tmem_slot + 2);             // the gathers have started another tile
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int KB = D / kLUKB;
+    const int KB = D / (kLUKB * L::kSub);                   // ring stages per tile
     const int P = (O + kLUPiece - 1) / kLUPiece;
 
     if (threadIdx.x == 0) {
@@ -155,6 +167,7 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
             ptx::mbar_init(q_full + s, 1);
             ptx::mbar_init(q_empty + s, kLUConsumerWarps);
         }
+        ptx::mbar_init(want, 1);
         ptx::mbar_init(acc1_full, 1);
         ptx::mbar_init(acc1_empty, kLUEpiWarps * 32);
         ptx::mbar_init(h_full, kLUEpiWarps * 32);
@@ -194,15 +207,22 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
     if (warp == kLUSchedWarp) {
         // ------------------------------------------------------------------ scheduler
         int fetched = 0;
+        int published = 0;
         Tile last;
         last.bin = 0; last.start = 0; last.rows = -1; last.pad = 0;
         for (;;) {
+            // tile n >= 2 is claimed once the gathers have started tile n - 1
+            if (published >= 2 && !timed_out && !ptx::mbar_wait_relaxed(want, (uint32_t)(published - 1) & 1u)) timed_out = true;
             int idx = 0;
             if (lane == 0) idx = atomicAdd(sched, 1);
             idx = __shfl_sync(kFullMask, idx, 0);
-            if (idx >= n_tiles_total || ++fetched > max_iters) break;
-            const Tile c = tiles[idx];
+            if (idx >= passes * n_tiles_total || ++fetched > passes * max_iters) break;
+            // with two passes the full tiles go first and the ragged ones last, so that the work handed out
+            // at the end comes in small pieces
+            const int second = idx >= n_tiles_total ? 1 : 0;
+            const Tile c = tiles[idx - second * n_tiles_total];
             if (c.rows <= 0 || c.rows > kLUM) continue;          // empty list entry
+            if (passes == 2 && (c.rows == kLUM) != (second == 0)) continue;
             if (!timed_out && !ptx::mbar_wait_relaxed(q_empty + q_slot, q_phase ^ 1)) timed_out = true;
             if (lane == 0) {
                 queue[q_slot] = c;
@@ -210,6 +230,7 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
             }
             __syncwarp();
             if (++q_slot == kLUQueue) { q_slot = 0; q_phase ^= 1; }
+            ++published;
         }
         // end of the sequence; after a timeout every slot gets the marker so that stragglers stop too
         for (int s = 0; s < (timed_out ? kLUQueue : 1); ++s) {
@@ -229,6 +250,7 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
         for (int it = 0; it < max_iters; ++it) {
             const Tile tl = next_tile();
             if (tl.rows <= 0) break;
+            if (gw == 0 && lane == 0) ptx::mbar_arrive(want);
             // 4-row group g = lane * kLUGatherWarps + gw of the tile belongs to this lane
             const int total_groups = (tl.rows + 3) >> 2;
             const int groups = max((total_groups - gw + kLUGatherWarps - 1) / kLUGatherWarps, 0);     // of this warp
@@ -241,17 +263,20 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
             for (int kb = 0; kb < KB; ++kb) {
                 if (!timed_out && !ptx::mbar_wait_relaxed(empty + stage, phase ^ 1)) timed_out = true;
                 if (lane == 0) {
-                    const uint32_t bytes = (uint32_t)groups * 512u + (gw == 0 ? (uint32_t)L::kW1StageBytes : 0u);
+                    const uint32_t bytes = (uint32_t)groups * (512u * L::kSub) + (gw == 0 ? (uint32_t)L::kW1StageBytes : 0u);
                     if (bytes > 0) ptx::mbar_arrive_expect_tx(full + stage, bytes);
                     else ptx::mbar_arrive(full + stage);
                     if (gw == 0)
                         ptx::bulk_g2s(ring + stage * L::kStageBytes + L::kXStageBytes,
-                                      w1img + ((int64_t)tl.bin * KB + kb) * (LP * kLUKB), L::kW1StageBytes, full + stage);
+                                      w1img + ((int64_t)tl.bin * KB + kb) * (L::kSub * LP * kLUKB), L::kW1StageBytes, full + stage);
                 }
                 __syncwarp();
-                if (lane < groups)
-                    ptx::tma_gather4(ring + stage * L::kStageBytes + first * 128, &tmap_x, kb * kLUKB, r[0], r[1], r[2], r[3],
-                                     full + stage);
+                if (lane < groups) {
+#pragma unroll
+                    for (int sb = 0; sb < L::kSub; ++sb)
+                        ptx::tma_gather4(ring + stage * L::kStageBytes + sb * L::kXSubBytes + first * 128, &tmap_x,
+                                         (kb * L::kSub + sb) * kLUKB, r[0], r[1], r[2], r[3], full + stage);
+                }
                 if (++stage == kStages) { stage = 0; phase ^= 1; }
             }
         }
@@ -270,10 +295,14 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                 ptx::tc_fence_after_sync();
                 if (lane == 0) {
                     const uint32_t xs = ptx::smem_addr(ring + stage * L::kStageBytes);
-                    const uint64_t ad = ptx::umma_desc_k128(xs), bd = ptx::umma_desc_k128(xs + L::kXStageBytes);
 #pragma unroll
-                    for (int j = 0; j < kLUKB / 16; ++j)
-                        ptx::umma_bf16(tmem_base, ad + 2 * j, bd + 2 * j, idesc, (kb | j) != 0 ? 1u : 0u);
+                    for (int sb = 0; sb < L::kSub; ++sb) {
+                        const uint64_t ad = ptx::umma_desc_k128(xs + sb * L::kXSubBytes);
+                        const uint64_t bd = ptx::umma_desc_k128(xs + L::kXStageBytes + sb * L::kW1SubBytes);
+#pragma unroll
+                        for (int j = 0; j < kLUKB / 16; ++j)
+                            ptx::umma_bf16(tmem_base, ad + 2 * j, bd + 2 * j, idesc, (kb | sb | j) != 0 ? 1u : 0u);
+                    }
                     ptx::umma_commit(empty + stage);
                     if (kb == KB - 1) ptx::umma_commit(acc1_full);
                 }
@@ -318,7 +347,7 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                     const uint64_t bd = ptx::umma_desc_rows(ptx::smem_addr(w2ring + mm_slot * L::kW2SlotStride), L::kRowBytes);
 #pragma unroll
                     for (int kk = 0; kk < LP / 16; ++kk)
-                        ptx::umma_bf16(tmem_base + kLUAcc2Col + b * kLUPiece, ad + 2 * kk, bd + 2 * kk, idesc, kk != 0 ? 1u : 0u);
+                        ptx::umma_bf16(tmem_base + kLUAcc2Col + b * kLUAccStride, ad + 2 * kk, bd + 2 * kk, idesc, kk != 0 ? 1u : 0u);
                     ptx::umma_commit(w2_empty + mm_slot);
                     ptx::umma_commit(y_full + b);
                 }
@@ -332,7 +361,7 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
         const int quarter = warp & 3, part = warp >> 2;
         const int row = quarter * 32 + lane;
         const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
-        constexpr int HC = LP / kLUColParts;                     // H columns of this thread (4, 8 or 16)
+        constexpr int HC = LP / kLUHParts;                       // H columns of a thread that computes H
         constexpr int YC = kLUPiece / kLUColParts;               // y columns of this thread per piece
         int pc = 0;
         int w2_slot = 0;
@@ -341,11 +370,12 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
             const Tile tl = next_tile();
             if (tl.rows <= 0) break;
             const bool active = quarter * 32 < tl.rows;          // this warp's lanes hold valid rows
+            const bool h_active = active && part < kLUHParts;
             const int64_t tok = row < tl.rows ? perm[tl.start + row] : -1;
             float b1r[HC];
 #pragma unroll
             for (int j = 0; j < HC; j += 4) {
-                const float4 t = __ldg(reinterpret_cast<const float4*>(b1img + (int64_t)tl.bin * LP + part * HC + j));
+                const float4 t = __ldg(reinterpret_cast<const float4*>(b1img + (int64_t)tl.bin * LP + (part % kLUHParts) * HC + j));
                 b1r[j] = t.x; b1r[j + 1] = t.y; b1r[j + 2] = t.z; b1r[j + 3] = t.w;
             }
 
@@ -354,27 +384,22 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
             ptx::tc_fence_after_sync();
             {
                 uint32_t hp[HC / 2];
-                if (active) {
+                if (h_active) {
                     uint32_t v[32];
                     ptx::tmem_ld32(lane_base + part * HC, v);      // columns past HC are not used
                     ptx::tmem_ld_wait();
 #pragma unroll
                     for (int j = 0; j < HC; j += 2)
-                        hp[j / 2] = ptx::pack_bf16(activate(act, __uint_as_float(v[j]) + b1r[j]),
-                                                   activate(act, __uint_as_float(v[j + 1]) + b1r[j + 1]));
+                        hp[j / 2] = ptx::pack_bf16(activate_bf16(act, __uint_as_float(v[j]) + b1r[j]),
+                                                   activate_bf16(act, __uint_as_float(v[j + 1]) + b1r[j + 1]));
                 }
                 ptx::tc_fence_before_sync();
                 ptx::mbar_arrive(acc1_empty);
-                if (active) {
-                    if constexpr (HC == 4) {
-                        unsigned char* dst = hbuf + swz_rows((uint32_t)(row * L::kRowBytes + (part >> 1) * 16), L::kRowBytes) + (part & 1) * 8;
-                        *reinterpret_cast<uint2*>(dst) = make_uint2(hp[0], hp[1]);
-                    } else {
+                if (h_active) {
 #pragma unroll
-                        for (int c = 0; c < HC / 8; ++c)
-                            *reinterpret_cast<uint4*>(hbuf + swz_rows((uint32_t)(row * L::kRowBytes + (part * HC / 8 + c) * 16), L::kRowBytes)) =
-                                make_uint4(hp[4 * c], hp[4 * c + 1], hp[4 * c + 2], hp[4 * c + 3]);
-                    }
+                    for (int c = 0; c < HC / 8; ++c)
+                        *reinterpret_cast<uint4*>(hbuf + swz_rows((uint32_t)(row * L::kRowBytes + (part * HC / 8 + c) * 16), L::kRowBytes)) =
+                            make_uint4(hp[4 * c], hp[4 * c + 1], hp[4 * c + 2], hp[4 * c + 3]);
                     ptx::fence_proxy_async();
                 }
                 ptx::mbar_arrive(h_full);
@@ -395,7 +420,7 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                     const int nv = min(32, ncols - c0);              // <= 0, 16 or 32
                     if (active && nv > 0) {
                         uint32_t v[32];
-                        ptx::tmem_ld32(lane_base + kLUAcc2Col + b * kLUPiece + c0, v);
+                        ptx::tmem_ld32(lane_base + kLUAcc2Col + b * kLUAccStride + c0, v);
                         ptx::tmem_ld_wait();
                         const int o0 = p * kLUPiece + c0;
                         uint32_t out[16];
