@@ -195,8 +195,13 @@ int tile_list_len(int64_t B, int tile_rows, int nbins) { return (int)(B / tile_r
 // Capacity of the tile buffer: the longest list any stage can ask for.
 size_t max_tiles(const fff_handle_s* h, int64_t B) { return (size_t)(B / kMinTileRows + h->n_leaves + 1); }
 
-// Token rows per tile of the grouped leaf kernel: short tiles when buckets are small.
-int leaf_tile_rows(const fff_handle_s* h, int64_t B) {
+// Which tensor-core leaf kernel runs, and on tiles of how many token rows.
+struct LeafPlan {
+    int tile_rows = 0;
+    bool umma = false;
+};
+
+LeafPlan leaf_plan(const fff_handle_s* h, int64_t B) {
     static const int forced = [] {
         const char* e = std::getenv("FFF_LEAF_TILE_ROWS");      // tuning aid: 32 or 64
         const int v = e ? std::atoi(e) : 0;
@@ -205,9 +210,16 @@ int leaf_tile_rows(const fff_handle_s* h, int64_t B) {
     // The tcgen05 kernel works on 128-row tiles.  Measured against the mma.sync kernel it is far ahead when
     // some buckets are large (skewed routing), about level with uniformly thin buckets of 32 tokens, and is
     // left out only when buckets are thinner still (every tile costs its epilogue a fixed few microseconds).
-    if (h->w2uimg && B >= 16 * h->n_leaves) return fff::kLUM;
-    if (forced) return forced;
-    return B / h->n_leaves <= 40 ? 32 : 64;
+    if (h->w2uimg && B >= 16 * h->n_leaves) {
+        static const int umma_rows = [] {
+            const char* e = std::getenv("FFF_UMMA_TILE_ROWS");  // tuning aid: a multiple of 4 up to 128
+            const int v = e ? std::atoi(e) : 0;
+            return (v >= 4 && v <= fff::kLUM && v % 4 == 0) ? v : 0;
+        }();
+        return LeafPlan{umma_rows ? umma_rows : fff::kLUM, true};
+    }
+    if (forced) return LeafPlan{forced, false};
+    return LeafPlan{B / h->n_leaves <= 40 ? 32 : 64, false};
 }
 
 bool use_tensor_leaf(const fff_handle_s* h) {
@@ -585,9 +597,10 @@ fff_status_t launch_leaf_mma(fff_handle_s* h, const void* x, const int32_t* perm
 }
 
 template <int LP>
-fff_status_t launch_leaf_umma(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, cudaStream_t st) {
+fff_status_t launch_leaf_umma(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, int tile_rows,
+                              cudaStream_t st) {
     using L = fff::LeafUmmaLayout<LP>;
-    const int n_tiles = tile_list_len(B, fff::kLUM, (int)h->n_leaves);
+    const int n_tiles = tile_list_len(B, tile_rows, (int)h->n_leaves);
     const int stages = std::min((int)fff::kLUMaxStages, (kSmemBudget - L::smem_bytes(0)) / L::kStageBytes);
     if (stages < 2) return FFF_ERR_UNSUPPORTED;
     static bool attr_set[64] = {};
@@ -609,13 +622,14 @@ fff_status_t launch_leaf_umma(fff_handle_s* h, const void* x, const int32_t* per
 }
 
 // Ring depth per (LP, TM): what fits twice into an SM's shared memory (once for LP = 64).
-fff_status_t run_leaf_mma(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, int tile_rows,
+fff_status_t run_leaf_mma(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, const LeafPlan& plan,
                           cudaStream_t st) {
-    if (tile_rows == fff::kLUM && h->w2uimg) {
+    const int tile_rows = plan.tile_rows;
+    if (plan.umma && h->w2uimg) {
         switch (h->LP) {
-            case 16: return launch_leaf_umma<16>(h, x, perm, y, B, st);
-            case 32: return launch_leaf_umma<32>(h, x, perm, y, B, st);
-            case 64: return launch_leaf_umma<64>(h, x, perm, y, B, st);
+            case 16: return launch_leaf_umma<16>(h, x, perm, y, B, tile_rows, st);
+            case 32: return launch_leaf_umma<32>(h, x, perm, y, B, tile_rows, st);
+            case 64: return launch_leaf_umma<64>(h, x, perm, y, B, tile_rows, st);
         }
     }
     if (tile_rows == 32) {
@@ -899,11 +913,12 @@ fff_status_t fff_grouped_leaf_ff(fff_handle_t h, const void* x, const int32_t* l
     cudaStream_t st = (cudaStream_t)cuda_stream;
     if (use_tensor_leaf(h)) {
         if ((s = grow_workspace(h, B)) != FFF_OK) return s;
-        const int tile_rows = leaf_tile_rows(h, B);
+        const LeafPlan plan = leaf_plan(h, B);
+        const int tile_rows = plan.tile_rows;
         fff::k_tiles_from_offsets<<<1, fff::kBucketThreads, 0, st>>>(offsets, (int)h->n_leaves, tile_rows, h->ws_tiles,
                                                                      tile_list_len(B, tile_rows, (int)h->n_leaves));
         if ((s = launched(h, st, "tiles_from_offsets")) != FFF_OK) return s;
-        return run_leaf_mma(h, x, perm, y, B, tile_rows, st);
+        return run_leaf_mma(h, x, perm, y, B, plan, st);
     }
     return FFF_DISPATCH(h, run_leaf, h, x, leaf_idx, perm, y, B, st);
 }
@@ -930,7 +945,8 @@ fff_status_t fff_forward_infer(fff_handle_t h, const void* x, void* y, int32_t* 
     if (lazy_bucketing) leaf = h->ws_leaf;
     Coarse coarse;
     s = run_descent(h, x, leaf, &coarse, B, st);
-    const int tile_rows = tensor_leaf ? leaf_tile_rows(h, B) : 0;
+    const LeafPlan plan = tensor_leaf ? leaf_plan(h, B) : LeafPlan{};
+    const int tile_rows = plan.tile_rows;
     // the final permutation goes to whichever buffer the last node bucketing did not use
     h->last_perm = coarse.perm == h->ws_perm ? h->ws_perm2 : h->ws_perm;
     h->bucketing_pending = lazy_bucketing;
@@ -943,7 +959,7 @@ fff_status_t fff_forward_infer(fff_handle_t h, const void* x, void* y, int32_t* 
         if (s == FFF_OK)
             s = run_bucket(h, leaf, (int)h->n_leaves, coarse, h->ws_offsets, h->last_perm, B, st, tile_rows, "leaf_bucketing");
         if (s == FFF_OK)
-            s = tensor_leaf ? run_leaf_mma(h, x, h->last_perm, y, B, tile_rows, st)
+            s = tensor_leaf ? run_leaf_mma(h, x, h->last_perm, y, B, plan, st)
                             : FFF_DISPATCH(h, run_leaf, h, x, leaf, h->last_perm, y, B, st);
     }
     if (h->prof_active) {
