@@ -47,6 +47,11 @@ def small_cfgs():
         C("bf16_d0", 128, 128, 0, 48, "gelu", "bf16", 300, "normal"),
         C("bf16_one_token", 64, 64, 5, 16, "gelu", "bf16", 1, "normal"),
         C("bf16_l40", 512, 520, 2, 40, "relu", "bf16", 999, "normal"),
+        # O not a multiple of the 128-column output pieces; fewer tokens than one 128-row tile
+        C("bf16_o208", 384, 208, 5, 20, "gelu", "bf16", 2000, "normal"),
+        C("bf16_tiny_batch", 128, 144, 3, 16, "relu", "bf16", 37, "normal", node_bias_std=0.2),
+        # eight levels in one dense stage (255 nodes), small batch
+        C("bf16_d8_small", 256, 64, 8, 8, "gelu", "bf16", 5000, "layernorm"),
     ]
 
 
