@@ -615,7 +615,7 @@ fff_status_t launch_leaf_umma(fff_handle_s* h, const void* x, const int32_t* per
     const int passes = 1;      // two passes (full tiles first) measured slightly slower
     if (launch_chain(h, fff::k_leaf_umma<LP>, (unsigned)grid, fff::kLUThreads, (size_t)L::smem_bytes(stages), st, 1, tm, perm,
                      (const fff::Tile*)h->ws_tiles, n_tiles, (const __nv_bfloat16*)h->w1img, (const float*)h->b1img,
-                     (const unsigned char*)h->w2uimg, (__nv_bfloat16*)y, h->D, h->O, h->act, stages, wide, passes, h->ws_sched,
+                     (const unsigned char*)h->w2uimg, (__nv_bfloat16*)y, h->D, h->O, h->l, h->act, stages, wide, passes, h->ws_sched,
                      h->d_status) != cudaSuccess)
         return cudaGetLastError(), FFF_ERR_CUDA;
     return launched(h, st, "grouped_leaf_ff_umma");

@@ -112,7 +112,10 @@ __global__ void k_pack_w2_umma(const T* __restrict__ w2, const T* __restrict__ b
         const int o = (int)(jp % P) * kLUPiece + n;
         unsigned char* piece = img + jp * piece_bytes;
         if (c < LP) {
-            const float v = (o < O && c < l) ? Elem<T>::to_float(w2[(j * O + o) * (int64_t)l + c]) : 0.0f;
+            // a spare padded column (l < LP) carries the output bias: H gets a constant 1 there, so GEMM2 adds
+            // b2 by itself and the epilogue has no bias to fetch and add (b2 is bf16 already: exact)
+            float v = (o < O && c < l) ? Elem<T>::to_float(w2[(j * O + o) * (int64_t)l + c]) : 0.0f;
+            if (c == l && o < O) v = Elem<T>::to_float(b2[j * O + o]);
             *reinterpret_cast<__nv_bfloat16*>(piece + swz_rows((uint32_t)(n * LP * 2 + c * 2), LP * 2)) = __float2bfloat16_rn(v);
         } else {
             reinterpret_cast<float*>(piece + (int64_t)kLUPiece * LP * 2)[n] = o < O ? Elem<T>::to_float(b2[j * O + o]) : 0.0f;
@@ -128,7 +131,8 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
             const Tile* __restrict__ tiles, int n_tiles_total,
             const __nv_bfloat16* __restrict__ w1img, const float* __restrict__ b1img,
             const unsigned char* __restrict__ w2img, __nv_bfloat16* __restrict__ y,
-            int D, int O, int act, int kStages, int wide_stores, int passes, int* __restrict__ sched, int* __restrict__ status)
+            int D, int O, int l, int act, int kStages, int wide_stores, int passes, int* __restrict__ sched,
+            int* __restrict__ status)
 {
     using L = LeafUmmaLayout<LP>;
     extern __shared__ unsigned char smem_raw[];
@@ -389,9 +393,13 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                     ptx::tmem_ld32(lane_base + part * HC, v);      // columns past HC are not used
                     ptx::tmem_ld_wait();
 #pragma unroll
-                    for (int j = 0; j < HC; j += 2)
-                        hp[j / 2] = ptx::pack_bf16(activate_bf16(act, __uint_as_float(v[j]) + b1r[j]),
-                                                   activate_bf16(act, __uint_as_float(v[j + 1]) + b1r[j + 1]));
+                    for (int j = 0; j < HC; j += 2) {
+                        float h0 = activate_bf16(act, __uint_as_float(v[j]) + b1r[j]);
+                        float h1 = activate_bf16(act, __uint_as_float(v[j + 1]) + b1r[j + 1]);
+                        if (part * HC + j == l) h0 = 1.0f;           // the bias column (only when l < LP)
+                        if (part * HC + j + 1 == l) h1 = 1.0f;
+                        hp[j / 2] = ptx::pack_bf16(h0, h1);
+                    }
                 }
                 ptx::tc_fence_before_sync();
                 ptx::mbar_arrive(acc1_empty);
@@ -424,11 +432,17 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                         ptx::tmem_ld_wait();
                         const int o0 = p * kLUPiece + c0;
                         uint32_t out[16];
+                        if (l < LP) {                                // bias already added by GEMM2
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) {
-                            const float4 bb = *reinterpret_cast<const float4*>(bias + c0 + 4 * e);
-                            out[2 * e] = ptx::pack_bf16(__uint_as_float(v[4 * e]) + bb.x, __uint_as_float(v[4 * e + 1]) + bb.y);
-                            out[2 * e + 1] = ptx::pack_bf16(__uint_as_float(v[4 * e + 2]) + bb.z, __uint_as_float(v[4 * e + 3]) + bb.w);
+                            for (int e = 0; e < 16; ++e)
+                                out[e] = ptx::pack_bf16(__uint_as_float(v[2 * e]), __uint_as_float(v[2 * e + 1]));
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) {
+                                const float4 bb = *reinterpret_cast<const float4*>(bias + c0 + 4 * e);
+                                out[2 * e] = ptx::pack_bf16(__uint_as_float(v[4 * e]) + bb.x, __uint_as_float(v[4 * e + 1]) + bb.y);
+                                out[2 * e + 1] = ptx::pack_bf16(__uint_as_float(v[4 * e + 2]) + bb.z, __uint_as_float(v[4 * e + 3]) + bb.w);
+                            }
                         }
                         if (tok >= 0) {
                             if (wide_stores && nv == 32) {
