@@ -65,6 +65,8 @@ struct fff_handle_s {
     int64_t cap_B = 0;
     int32_t *ws_leaf = nullptr, *ws_perm = nullptr, *ws_offsets = nullptr;
     int32_t* ws_rank = nullptr;   // per-token rank scratch of the bucketing kernel (large batches only)
+    uint8_t* ws_rank8 = nullptr;  // rank of every token inside its 128-token tile, left by the first descent stage
+    uint8_t* ws_counts8 = nullptr;   // and that stage's per-tile counts, [ceil(B/128)][<= 256]
     int max_bucket_clusters = 8;
     int32_t* last_perm = nullptr; // where the most recent forward left its leaf permutation
     bool bucketing_pending = false;   // the last forward skipped the leaf bucketing; ws_leaf holds its leaf indices
@@ -181,7 +183,7 @@ void release(fff_handle_s* h) {
     for (auto& sg : h->stages) { dfree(sg.wimg); dfree(sg.bimg); }
     for (auto& sg : h->ustages) { dfree(sg.wimg); dfree(sg.bimg); }
     dfree(h->ws_pos[0]); dfree(h->ws_pos[1]);
-    dfree(h->w1img); dfree(h->b1img); dfree(h->w2img); dfree(h->w2uimg); dfree(h->ws_sched); dfree(h->ws_tiles); dfree(h->ws_rank); dfree(h->ws_matrix);
+    dfree(h->w1img); dfree(h->b1img); dfree(h->w2img); dfree(h->w2uimg); dfree(h->ws_sched); dfree(h->ws_tiles); dfree(h->ws_rank); dfree(h->ws_rank8); dfree(h->ws_counts8); dfree(h->ws_matrix);
     prof_free(h);
     h->magic = 0;
     delete h;
@@ -231,6 +233,8 @@ fff_status_t grow_workspace(fff_handle_s* h, int64_t B) {
     if (B <= h->cap_B) return FFF_OK;
     if (cudaDeviceSynchronize() != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
     dfree(h->ws_leaf); dfree(h->ws_perm); dfree(h->ws_perm2); dfree(h->ws_tiles); dfree(h->ws_rank); dfree(h->ws_pos[0]);
+    dfree(h->ws_rank8); dfree(h->ws_counts8);
+    h->ws_rank8 = h->ws_counts8 = nullptr;
     dfree(h->ws_pos[1]);
     h->ws_leaf = h->ws_perm = h->ws_perm2 = h->ws_rank = h->ws_pos[0] = h->ws_pos[1] = nullptr;
     h->ws_tiles = nullptr;
@@ -240,6 +244,10 @@ fff_status_t grow_workspace(fff_handle_s* h, int64_t B) {
     if ((s = dmalloc((void**)&h->ws_perm, sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
     if ((s = dmalloc((void**)&h->ws_perm2, sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
     if ((s = dmalloc((void**)&h->ws_rank, sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
+    if (!h->ustages.empty()) {
+        if ((s = dmalloc((void**)&h->ws_rank8, (size_t)B)) != FFF_OK) return s;
+        if ((s = dmalloc((void**)&h->ws_counts8, (size_t)((B + 127) / 128) * 256)) != FFF_OK) return s;
+    }
     if (h->stages.size() > 1 || h->ustages.size() > 1) {
         if ((s = dmalloc((void**)&h->ws_pos[0], sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
         if ((s = dmalloc((void**)&h->ws_pos[1], sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
@@ -267,6 +275,8 @@ struct Coarse {
     const int32_t* perm = nullptr;      // previous permutation
     const int32_t* offsets = nullptr;   // its offsets, one segment per coarse bin
     int bins = 0;                       // number of coarse bins
+    bool ranked = false;                // no previous bucketing, but the keys come with the first descent stage's
+                                        // per-tile ranks and counts (ws_rank8, ws_counts8)
 };
 
 template <int NW>
@@ -286,6 +296,18 @@ fff_status_t run_bucket(fff_handle_s* h, const int32_t* keys, int nbins, const C
                         int32_t* perm, int64_t B, cudaStream_t st, int tile_rows, const char* name) {
     const int n_tiles_total = tile_rows > 0 ? tile_list_len(B, tile_rows, nbins) : 0;
     cudaError_t e;
+    const int64_t n_src = (B + fff::kRankTile - 1) / fff::kRankTile;
+    const int64_t ranked_ctas = std::min<int64_t>(h->sm_count, n_src);
+    if (coarse.ranked && !coarse.perm && nbins >= 16 && nbins <= 256 && B > 0 &&
+        (n_src + ranked_ctas - 1) / ranked_ctas <= fff::kRankedMaxTilesPerCta) {
+        // the descent kernel has done the ranking: sum its per-tile counts and scatter
+        if (launch_chain(h, fff::k_bucket_ranked, (unsigned)ranked_ctas, fff::kRankedThreads,
+                         sizeof(int) * (size_t)(3 + fff::kRankedMaxTilesPerCta) * nbins, st, 1, keys, (const uint8_t*)h->ws_rank8,
+                         (const uint8_t*)h->ws_counts8, offsets, perm, (int)B, nbins, tile_rows, h->ws_tiles,
+                         n_tiles_total) != cudaSuccess)
+            return cudaGetLastError(), FFF_ERR_CUDA;
+        return launched(h, st, name);
+    }
     // Refining pays while the coarse buckets are few and large; thousands of tiny buckets would mean
     // thousands of tiny clusters, and scanning all keys from a few clusters is cheaper then.
     if (coarse.perm && nbins / coarse.bins <= fff::kBucketMaxBinsPerCta && coarse.bins <= 256) {
@@ -407,9 +429,10 @@ fff_status_t launch_descent_umma(fff_handle_s* h, const fff_handle_s::DenseStage
     if (!make_x_tensor_map(&tm, x, B, h->D, fff::kUM)) return FFF_ERR_CUDA;
     const int64_t n_tiles = (B + fff::kUM - 1) / fff::kUM;
     const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(h->sm_count, n_tiles));
+    const bool ranked = sg.k >= 4 && h->ws_rank8 && h->ws_counts8;      // also rank the tokens for the bucketing that follows
     if (launch_chain(h, fff::k_descent_umma<NP>, (unsigned)grid, fff::kUmmaThreads, (size_t)L::smem_bytes(stages), st, 1, tm,
-                     (const __nv_bfloat16*)sg.wimg, (const float*)sg.bimg, pos_out, h->D, (int)B, sg.k, stages,
-                     h->d_status) != cudaSuccess)
+                     (const __nv_bfloat16*)sg.wimg, (const float*)sg.bimg, pos_out, ranked ? h->ws_rank8 : (uint8_t*)nullptr,
+                     ranked ? h->ws_counts8 : (uint8_t*)nullptr, h->D, (int)B, sg.k, stages, h->d_status) != cudaSuccess)
         return cudaGetLastError(), FFF_ERR_CUDA;
     return launched(h, st, "tree_descent_umma");
 }
@@ -471,7 +494,9 @@ fff_status_t run_descent(fff_handle_s* h, const void* x, int32_t* leaf_out, Coar
             // bucket by the node reached so far; buffers alternate so that the previous level stays readable
             int32_t* perm_out = (i & 1) ? h->ws_perm2 : h->ws_perm;
             int32_t* off_out = h->ws_offsets2[i & 1];
+            prev.ranked = i == 1 && plan[0].umma && plan[0].k >= 4 && h->ws_rank8 != nullptr;
             s = run_bucket(h, pos, 1 << level, prev, off_out, perm_out, B, st, fff::kDTM, "node_bucketing");
+            prev.ranked = false;
             if (s != FFF_OK) return s;
             prev.perm = perm_out;
             prev.offsets = off_out;
@@ -488,6 +513,8 @@ fff_status_t run_descent(fff_handle_s* h, const void* x, int32_t* leaf_out, Coar
         s = h->dtype == FFF_DTYPE_F32 ? run_descent_warp<float>(h, x, level, h->depth - level, pos, leaf_out, B, st)
                                       : run_descent_warp<__nv_bfloat16>(h, x, level, h->depth - level, pos, leaf_out, B, st);
     }
+    // one tcgen05 stage was the whole descent: the leaf indices come with its ranks and counts
+    prev.ranked = n_dense == 1 && level == h->depth && plan[0].umma && plan[0].k >= 4 && h->ws_rank8 != nullptr;
     if (coarse) *coarse = prev;
     return s;
 }
@@ -596,7 +623,7 @@ fff_status_t launch_leaf_mma(fff_handle_s* h, const void* x, const int32_t* perm
     return launched(h, st, "grouped_leaf_ff_mma");
 }
 
-template <int LP>
+template <int LP, bool kFold>
 fff_status_t launch_leaf_umma(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, int tile_rows,
                               cudaStream_t st) {
     using L = fff::LeafUmmaLayout<LP>;
@@ -605,7 +632,7 @@ fff_status_t launch_leaf_umma(fff_handle_s* h, const void* x, const int32_t* per
     if (stages < 2) return FFF_ERR_UNSUPPORTED;
     static bool attr_set[64] = {};
     if (h->device < 64 && !attr_set[h->device]) {
-        cudaFuncSetAttribute(fff::k_leaf_umma<LP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+        cudaFuncSetAttribute(fff::k_leaf_umma<LP, kFold>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
         attr_set[h->device] = true;
     }
     CUtensorMap tm;
@@ -613,7 +640,7 @@ fff_status_t launch_leaf_umma(fff_handle_s* h, const void* x, const int32_t* per
     const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(h->sm_count, n_tiles));
     const int wide = (reinterpret_cast<uintptr_t>(y) & 31u) == 0 ? 1 : 0;
     const int passes = 1;      // two passes (full tiles first) measured slightly slower
-    if (launch_chain(h, fff::k_leaf_umma<LP>, (unsigned)grid, fff::kLUThreads, (size_t)L::smem_bytes(stages), st, 1, tm, perm,
+    if (launch_chain(h, fff::k_leaf_umma<LP, kFold>, (unsigned)grid, fff::kLUThreads, (size_t)L::smem_bytes(stages), st, 1, tm, perm,
                      (const fff::Tile*)h->ws_tiles, n_tiles, (const __nv_bfloat16*)h->w1img, (const float*)h->b1img,
                      (const unsigned char*)h->w2uimg, (__nv_bfloat16*)y, h->D, h->O, h->l, h->act, stages, wide, passes, h->ws_sched,
                      h->d_status) != cudaSuccess)
@@ -627,9 +654,12 @@ fff_status_t run_leaf_mma(fff_handle_s* h, const void* x, const int32_t* perm, v
     const int tile_rows = plan.tile_rows;
     if (plan.umma && h->w2uimg) {
         switch (h->LP) {
-            case 16: return launch_leaf_umma<16>(h, x, perm, y, B, tile_rows, st);
-            case 32: return launch_leaf_umma<32>(h, x, perm, y, B, tile_rows, st);
-            case 64: return launch_leaf_umma<64>(h, x, perm, y, B, tile_rows, st);
+            case 16: return h->l < 16 ? launch_leaf_umma<16, true>(h, x, perm, y, B, tile_rows, st)
+                                      : launch_leaf_umma<16, false>(h, x, perm, y, B, tile_rows, st);
+            case 32: return h->l < 32 ? launch_leaf_umma<32, true>(h, x, perm, y, B, tile_rows, st)
+                                      : launch_leaf_umma<32, false>(h, x, perm, y, B, tile_rows, st);
+            case 64: return h->l < 64 ? launch_leaf_umma<64, true>(h, x, perm, y, B, tile_rows, st)
+                                      : launch_leaf_umma<64, false>(h, x, perm, y, B, tile_rows, st);
         }
     }
     if (tile_rows == 32) {

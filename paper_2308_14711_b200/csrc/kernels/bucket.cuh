@@ -614,6 +614,146 @@ k_bucket_coop(const int32_t* __restrict__ keys, int32_t* __restrict__ offsets_ou
     }
 }
 
+// ---- bucketing from per-tile ranks and counts --------------------------------------------------------
+// The first descent stage already has every token's key in a register, 128 consecutive tokens per tile.
+// It leaves, besides the keys, rank8[t] = number of earlier tokens of t's own tile with the same key, and
+// counts8[tile][bin] = tokens of the tile with that key (both fit a byte).  What remains of the stable
+// counting sort is then a sum over tiles and a scatter, with no barrier across CTAs: CTA c takes a
+// contiguous range of tiles, adds up the count rows of all tiles (bin totals) and of the tiles before its
+// own (its starting position inside every bin), scans the totals, and places its tokens at
+//     start[bin] + tokens of the bin in earlier tiles + rank8[t].
+// Same result as the other bucketing kernels.  Needs 16 <= nbins <= 256 (a multiple of 16) and at most
+// kRankedMaxTilesPerCta tiles per CTA.
+constexpr int kRankTile = 128;
+constexpr int kRankedThreads = 256;
+constexpr int kRankedWarps = kRankedThreads / 32;
+constexpr int kRankedMaxTilesPerCta = 8;
+
+// Dynamic shared memory: (3 + kRankedMaxTilesPerCta) * nbins ints.
+__global__ void __launch_bounds__(kRankedThreads)
+k_bucket_ranked(const int32_t* __restrict__ keys, const uint8_t* __restrict__ rank8, const uint8_t* __restrict__ counts8,
+                int32_t* __restrict__ offsets_out, int32_t* __restrict__ perm_out, int B, int nbins, int tile_rows,
+                Tile* __restrict__ tiles, int n_tiles_total)
+{
+    extern __shared__ int s_dyn[];
+    __shared__ int s_warp[32];
+    int* s_total = s_dyn;                     // [nbins] tokens in the bin
+    int* s_before = s_total + nbins;          // [nbins] of which in tiles before this CTA's
+    int* s_start = s_before + nbins;          // [nbins] first position of the bin
+    int* s_tile = s_start + nbins;            // [own tiles][nbins] position of the tile's first token of the bin
+    const int tid = threadIdx.x;
+    const int G = gridDim.x, c = blockIdx.x;
+    const int n_src = (B + kRankTile - 1) / kRankTile;
+    const int t0 = (int)((int64_t)c * n_src / G), t1 = (int)((int64_t)(c + 1) * n_src / G);
+
+    pdl_trigger();
+    for (int i = tid; i < 2 * nbins; i += kRankedThreads) s_dyn[i] = 0;
+    __syncthreads();
+    pdl_wait();
+
+    // everything this thread will need later is requested now, so that the L2 round trips overlap:
+    // its tokens' keys and ranks, and (thread = bin) the counts of the CTA's own tiles
+    constexpr int kTok = kRankedMaxTilesPerCta * kRankTile / kRankedThreads;
+    const int64_t first = (int64_t)t0 * kRankTile, last = min((int64_t)t1 * kRankTile, (int64_t)B);
+    int my_key[kTok];
+    int my_rank[kTok];
+#pragma unroll
+    for (int i = 0; i < kTok; ++i) {
+        const int64_t t = first + tid + i * kRankedThreads;
+        my_key[i] = t < last ? __ldg(keys + t) : -1;
+        my_rank[i] = t < last ? (int)rank8[t] : 0;
+    }
+    int own[kRankedMaxTilesPerCta];
+#pragma unroll
+    for (int i = 0; i < kRankedMaxTilesPerCta; ++i)
+        own[i] = (tid < nbins && t0 + i < t1) ? (int)counts8[(int64_t)(t0 + i) * nbins + tid] : 0;
+
+    // column sums of the count matrix, 16 bins per 16-byte load; bytes are added up in 16-bit lanes and
+    // flushed to shared memory before they can overflow
+    {
+        const int V = nbins >> 4;                         // 16-byte columns
+        const int P = kRankedThreads / V;                 // threads per column
+        const int vb = tid % V, part = tid / V;
+        const uint4* m = reinterpret_cast<const uint4*>(counts8);
+        for (int r0 = part; r0 < n_src && part < P; r0 += 256 * P) {
+            uint32_t tot[8] = {0, 0, 0, 0, 0, 0, 0, 0}, bef[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+            const int r_end = min(n_src, r0 + 256 * P);
+            for (int r = r0; r < r_end; r += 8 * P) {
+                uint4 v[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) v[j] = r + j * P < r_end ? __ldcg(m + (int64_t)(r + j * P) * V + vb) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
+                    const uint32_t mask = r + j * P < t0 ? 0xFFFFFFFFu : 0u;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const uint32_t lo = w[q] & 0x00FF00FFu, hi = (w[q] >> 8) & 0x00FF00FFu;
+                        tot[2 * q] += lo; tot[2 * q + 1] += hi;
+                        bef[2 * q] += lo & mask; bef[2 * q + 1] += hi & mask;
+                    }
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int b = 16 * vb + 4 * q;            // word q holds bins b .. b+3: lanes (b, b+2) and (b+1, b+3)
+                atomicAdd(&s_total[b], (int)(tot[2 * q] & 0xFFFFu));      atomicAdd(&s_total[b + 2], (int)(tot[2 * q] >> 16));
+                atomicAdd(&s_total[b + 1], (int)(tot[2 * q + 1] & 0xFFFFu)); atomicAdd(&s_total[b + 3], (int)(tot[2 * q + 1] >> 16));
+                atomicAdd(&s_before[b], (int)(bef[2 * q] & 0xFFFFu));     atomicAdd(&s_before[b + 2], (int)(bef[2 * q] >> 16));
+                atomicAdd(&s_before[b + 1], (int)(bef[2 * q + 1] & 0xFFFFu)); atomicAdd(&s_before[b + 3], (int)(bef[2 * q + 1] >> 16));
+            }
+        }
+    }
+    __syncthreads();
+
+    // exclusive scan of the totals over the bins (nbins <= kRankedThreads)
+    {
+        const int v = tid < nbins ? s_total[tid] : 0;
+        int all = 0;
+        const int ex = block_exclusive_scan_nw<kRankedWarps>(v, s_warp, &all);
+        if (tid < nbins) {
+            s_start[tid] = ex;
+            if (c == 0) {
+                offsets_out[tid] = ex;
+                if (tid == nbins - 1) offsets_out[nbins] = ex + v;
+            }
+            // positions of this CTA's tiles inside the bin
+            int run = ex + s_before[tid];
+#pragma unroll
+            for (int i = 0; i < kRankedMaxTilesPerCta; ++i) {
+                if (t0 + i < t1) s_tile[i * nbins + tid] = run;
+                run += own[i];
+            }
+        }
+    }
+    __syncthreads();
+    if (tile_rows > 0 && c == 0) {
+        const int total = tid < nbins ? s_total[tid] : 0;
+        const int nt = (total + tile_rows - 1) / tile_rows;
+        int n_all = 0;
+        const int tl0 = block_exclusive_scan_nw<kRankedWarps>(nt, s_warp, &n_all);
+        for (int i = 0; i < nt; ++i) {
+            Tile tl;
+            tl.bin = tid;
+            tl.start = s_start[tid] + i * tile_rows;
+            tl.rows = min(tile_rows, total - i * tile_rows);
+            tl.pad = 0;
+            tiles[tl0 + i] = tl;
+        }
+        Tile empty;
+        empty.bin = 0; empty.start = 0; empty.rows = 0; empty.pad = 0;
+        for (int i = n_all + tid; i < n_tiles_total; i += kRankedThreads) tiles[i] = empty;
+    }
+
+    // place
+#pragma unroll
+    for (int i = 0; i < kTok; ++i) {
+        const int64_t t = first + tid + i * kRankedThreads;
+        const int k = my_key[i];
+        if (t < last && k >= 0 && k < nbins) perm_out[s_tile[(int)((t - first) / kRankTile) * nbins + k] + my_rank[i]] = (int32_t)t;
+    }
+}
+
 // Tile list from an existing offsets array (one CTA; used when the caller supplies the bucketing),
 // padded with empty tiles up to n_tiles_total = floor(B / tile_rows) + nbins.
 __global__ void __launch_bounds__(kBucketThreads)

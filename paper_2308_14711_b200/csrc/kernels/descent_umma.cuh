@@ -19,6 +19,10 @@
 //            subtree on the bits.
 // The tensor pipe, the copy engine and the epilogue overlap across tiles through the two accumulators.
 //
+// The epilogue can also prepare the bucketing by the position just computed (k_bucket_ranked): with the
+// 128 keys of a tile in registers, the rank of every token among the equal keys of its tile and the tile's
+// count per key cost a few ballots and one pass over a 1 KB table in shared memory.
+//
 // Every wait is bounded (see ptx.cuh); tensor memory is released on every exit path.
 //
 // Requirements: bf16, D % 64 == 0, x 16-byte aligned.
@@ -26,6 +30,7 @@
 
 #include <cuda.h>      // CUtensorMap
 
+#include "bucket.cuh"
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -44,16 +49,19 @@ template <int NP> struct DescentUmmaLayout {
     static constexpr int kStageBytes = kXStageBytes + kWStageBytes;          // a multiple of 1024
     static constexpr int kBarrierBytes = 256;                                // 2 * kUmmaMaxStages + 4 mbarriers, tmem slot
     static constexpr int kTmemCols = 2 * NP;                                 // two accumulators
-    static constexpr int smem_bytes(int stages) { return 1024 + stages * kStageBytes + kBarrierBytes + NP * 4; }
+    static constexpr int kCountBytes = kUmmaEpilogueWarps * 256;              // per-warp counts of up to 256 keys, one byte each
+    static constexpr int smem_bytes(int stages) { return 1024 + stages * kStageBytes + kBarrierBytes + NP * 4 + kCountBytes; }
 };
 
 // wimg: [D / 64][NP rows][64 columns] 128-byte swizzled (the single-group image of k_pack_nodes),
 // bimg: [NP] float32.  pos_out[t] = position reached at level k.
+// rank8 / counts8 (both or neither, k >= 4): rank8[t] = earlier tokens of t's 128-token tile at the same
+// position, counts8[tile][2^k] = tokens of the tile per position.
 template <int NP>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 k_descent_umma(const __grid_constant__ CUtensorMap tmap_x, const __nv_bfloat16* __restrict__ wimg,
-               const float* __restrict__ bimg, int32_t* __restrict__ pos_out, int D, int B, int k, int kStages,
-               int* __restrict__ status)
+               const float* __restrict__ bimg, int32_t* __restrict__ pos_out, uint8_t* __restrict__ rank8,
+               uint8_t* __restrict__ counts8, int D, int B, int k, int kStages, int* __restrict__ status)
 {
     using L = DescentUmmaLayout<NP>;
     extern __shared__ unsigned char smem_raw[];
@@ -64,6 +72,7 @@ k_descent_umma(const __grid_constant__ CUtensorMap tmap_x, const __nv_bfloat16* 
     uint64_t* acc_empty = acc_full + 2;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
     float* bias = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(full) + L::kBarrierBytes);
+    uint8_t* s_cnt = reinterpret_cast<uint8_t*>(bias + NP);                   // [epilogue warp][256]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_tiles = (B + kUM - 1) / kUM;
@@ -86,6 +95,7 @@ k_descent_umma(const __grid_constant__ CUtensorMap tmap_x, const __nv_bfloat16* 
         ptx::tmem_relinquish_alloc_permit();
     }
     for (int i = threadIdx.x; i < NP; i += kUmmaThreads) bias[i] = bimg[i];    // a parameter image, not a predecessor's output
+    for (int i = threadIdx.x; i < L::kCountBytes / 4; i += kUmmaThreads) reinterpret_cast<uint32_t*>(s_cnt)[i] = 0;
     ptx::tc_fence_before_sync();
     pdl_trigger();
     __syncthreads();
@@ -166,7 +176,31 @@ k_descent_umma(const __grid_constant__ CUtensorMap tmap_x, const __nv_bfloat16* 
                 p = 2 * p + 1 + (int)((w >> (p & 31)) & 1u);
             }
             const int tok = tile * kUM + warp * 32 + lane;
-            if (tok < B) pos_out[tok] = p - ((1 << k) - 1);
+            const int key = p - ((1 << k) - 1);
+            if (tok < B) pos_out[tok] = key;
+            if (rank8) {
+                const int nbins = 1 << k;
+                const bool in = tok < B;
+                const unsigned peers = peers_by_ballot(in, key, k);
+                if (in && lane == __ffs(peers) - 1) s_cnt[warp * 256 + key] = (uint8_t)__popc(peers);
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (in) {
+                    int before = __popc(peers & ((1u << lane) - 1u));
+                    for (int w = 0; w < warp; ++w) before += s_cnt[w * 256 + key];
+                    rank8[tok] = (uint8_t)before;
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                for (int b = warp * 32 + lane; b < nbins; b += kUmmaEpilogueWarps * 32) {
+                    int total = 0;
+#pragma unroll
+                    for (int w = 0; w < kUmmaEpilogueWarps; ++w) {
+                        total += s_cnt[w * 256 + b];
+                        s_cnt[w * 256 + b] = 0;
+                    }
+                    counts8[(int64_t)tile * nbins + b] = (uint8_t)total;
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+            }
         }
     }
     if (timed_out) {

@@ -125,7 +125,8 @@ __global__ void k_pack_w2_umma(const T* __restrict__ w2, const T* __restrict__ b
 
 // sched: two ints, both zero before the first launch and again after every launch: [0] list entries
 // handed out so far, [1] CTAs that have finished.
-template <int LP>
+// kFold: l < LP, the spare hidden column l carries the output bias (see k_pack_w2_umma).
+template <int LP, bool kFold>
 __global__ void __launch_bounds__(kLUThreads, 1)
 k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restrict__ perm,
             const Tile* __restrict__ tiles, int n_tiles_total,
@@ -396,8 +397,8 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                     for (int j = 0; j < HC; j += 2) {
                         float h0 = activate_bf16(act, __uint_as_float(v[j]) + b1r[j]);
                         float h1 = activate_bf16(act, __uint_as_float(v[j + 1]) + b1r[j + 1]);
-                        if (part * HC + j == l) h0 = 1.0f;           // the bias column (only when l < LP)
-                        if (part * HC + j + 1 == l) h1 = 1.0f;
+                        if (kFold && part * HC + j == l) h0 = 1.0f;          // the bias column
+                        if (kFold && part * HC + j + 1 == l) h1 = 1.0f;
                         hp[j / 2] = ptx::pack_bf16(h0, h1);
                     }
                 }
@@ -432,7 +433,7 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                         ptx::tmem_ld_wait();
                         const int o0 = p * kLUPiece + c0;
                         uint32_t out[16];
-                        if (l < LP) {                                // bias already added by GEMM2
+                        if (kFold) {                                 // bias already added by GEMM2
 #pragma unroll
                             for (int e = 0; e < 16; ++e)
                                 out[e] = ptx::pack_bf16(__uint_as_float(v[2 * e]), __uint_as_float(v[2 * e + 1]));
