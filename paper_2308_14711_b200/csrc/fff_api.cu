@@ -448,6 +448,38 @@ fff_status_t run_descent_umma(fff_handle_s* h, const fff_handle_s::DenseStage& s
     return FFF_ERR_UNSUPPORTED;
 }
 
+template <int NP>
+fff_status_t launch_descent_umma_grouped(fff_handle_s* h, const fff_handle_s::DenseStage& sg, const void* x, const int32_t* perm,
+                                         int32_t* pos_out, int64_t B, cudaStream_t st) {
+    using L = fff::DescentUmmaGroupedLayout<NP>;
+    const int stages = std::min((int)fff::kUmmaMaxStages, (kSmemBudget - L::smem_bytes(0)) / L::kStageBytes);
+    if (stages < 2) return FFF_ERR_UNSUPPORTED;
+    static bool attr_set[64] = {};
+    if (h->device < 64 && !attr_set[h->device]) {
+        cudaFuncSetAttribute(fff::k_descent_umma_grouped<NP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+        attr_set[h->device] = true;
+    }
+    CUtensorMap tm;
+    if (!make_x_tensor_map(&tm, x, B, h->D, 1)) return FFF_ERR_CUDA;       // one-row boxes: rows are gathered four at a time
+    const int n_tiles = tile_list_len(B, fff::kUM, 1 << sg.L0);
+    const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(h->sm_count, n_tiles));
+    if (launch_chain(h, fff::k_descent_umma_grouped<NP>, (unsigned)grid, fff::kUGThreads, (size_t)L::smem_bytes(stages), st, 1, tm,
+                     perm, (const fff::Tile*)h->ws_tiles, n_tiles, (const __nv_bfloat16*)sg.wimg, (const float*)sg.bimg, pos_out,
+                     h->D, sg.k, stages, h->d_status) != cudaSuccess)
+        return cudaGetLastError(), FFF_ERR_CUDA;
+    return launched(h, st, "tree_descent_umma_grouped");
+}
+
+fff_status_t run_descent_umma_grouped(fff_handle_s* h, const fff_handle_s::DenseStage& sg, const void* x, const int32_t* perm,
+                                      int32_t* pos_out, int64_t B, cudaStream_t st) {
+    switch (sg.NP) {
+        case 16: return launch_descent_umma_grouped<16>(h, sg, x, perm, pos_out, B, st);
+        case 32: return launch_descent_umma_grouped<32>(h, sg, x, perm, pos_out, B, st);
+        case 64: return launch_descent_umma_grouped<64>(h, sg, x, perm, pos_out, B, st);
+    }
+    return FFF_ERR_UNSUPPORTED;
+}
+
 template <typename T>
 fff_status_t run_descent_warp(fff_handle_s* h, const void* x, int level0, int levels, const int32_t* pos_in,
                               int32_t* pos_out, int64_t B, cudaStream_t st) {
@@ -490,12 +522,14 @@ fff_status_t run_descent(fff_handle_s* h, const void* x, int32_t* leaf_out, Coar
     const auto& plan = stage_plan(h);
     for (int i = 0; i < n_dense; ++i) {
         const auto& sg = plan[i];
+        // later stages: the tcgen05 kernel on 128-row tiles when the groups fill them reasonably, else mma.sync on 64-row tiles
+        const bool grouped_umma = i > 0 && sg.umma && (B >> sg.L0) >= 64;
         if (i > 0) {
             // bucket by the node reached so far; buffers alternate so that the previous level stays readable
             int32_t* perm_out = (i & 1) ? h->ws_perm2 : h->ws_perm;
             int32_t* off_out = h->ws_offsets2[i & 1];
             prev.ranked = i == 1 && plan[0].umma && plan[0].k >= 4 && h->ws_rank8 != nullptr;
-            s = run_bucket(h, pos, 1 << level, prev, off_out, perm_out, B, st, fff::kDTM, "node_bucketing");
+            s = run_bucket(h, pos, 1 << level, prev, off_out, perm_out, B, st, grouped_umma ? fff::kUM : fff::kDTM, "node_bucketing");
             prev.ranked = false;
             if (s != FFF_OK) return s;
             prev.perm = perm_out;
@@ -504,7 +538,9 @@ fff_status_t run_descent(fff_handle_s* h, const void* x, int32_t* leaf_out, Coar
         }
         const bool last = level + sg.k == h->depth;
         int32_t* out = last ? leaf_out : h->ws_pos[i & 1];
-        s = sg.umma ? run_descent_umma(h, sg, x, out, B, st) : run_descent_mma(h, sg, x, prev.perm, i > 0, out, B, st);
+        s = i == 0 && sg.umma ? run_descent_umma(h, sg, x, out, B, st)
+            : grouped_umma    ? run_descent_umma_grouped(h, sg, x, prev.perm, out, B, st)
+                              : run_descent_mma(h, sg, x, prev.perm, i > 0, out, B, st);
         if (s != FFF_OK) return s;
         level += sg.k;
         pos = out;
@@ -579,7 +615,8 @@ fff_status_t pack_node_images(fff_handle_s* h) {
         L0 = 0;
         for (size_t i = 0; i < ks.size(); ++i) {
             const int np = i == 0 ? std::max(32, 1 << ks[i]) : std::max(16, 1 << ks[i]);
-            if ((s = pack_stage<T>(h, h->ustages, L0, ks[i], np, i == 0)) != FFF_OK) return s;
+            static const bool no_grouped = std::getenv("FFF_NO_UMMA_GROUPED") != nullptr;        // tuning aid
+            if ((s = pack_stage<T>(h, h->ustages, L0, ks[i], np, i == 0 || (!no_grouped && h->D % 128 == 0))) != FFF_OK) return s;
             L0 += ks[i];
         }
         cudaFuncSetAttribute(fff::k_descent_umma<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);

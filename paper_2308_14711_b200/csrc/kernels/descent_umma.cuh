@@ -215,4 +215,198 @@ k_descent_umma(const __grid_constant__ CUtensorMap tmap_x, const __nv_bfloat16* 
     }
 }
 
+// ---- later stages: tokens grouped by the node they have reached -------------------------------------
+// The same dense evaluation for a stage that starts at level L0 > 0: the tokens have been bucketed by their
+// node at level L0 (perm, and a list of tiles of up to 128 consecutive entries of one bucket), every bucket
+// has its own subtree image, and the rows of a tile are gathered through the permutation with tile::gather4
+// tensor-map loads (4 rows x 128 bytes per request, 128-byte swizzled by the copy engine).
+//   warps 0-3  epilogue, as above; pos_out[token] = (node << k) + position inside the subtree;
+//   warp 4     MMA issuer;
+//   warps 5-8  gathers, the 4-row groups of a tile dealt round-robin to the four warps; the first of them
+//              also starts the bulk copy of the bucket's weight K-blocks.
+// A ring stage holds two K-blocks of 64 columns.  CTAs walk the tile list with a static stride and skip its
+// empty entries; rows of a ragged tile beyond its length are not loaded and their logits never used.
+constexpr int kUGGatherWarps = 4;
+constexpr int kUGThreads = (kUmmaEpilogueWarps + 1 + kUGGatherWarps) * 32;
+constexpr int kUGSub = 2;                                  // K-blocks per ring stage
+
+template <int NP> struct DescentUmmaGroupedLayout {
+    static_assert(NP == 16 || NP == 32 || NP == 64, "accumulator width");
+    static constexpr int kXSubBytes = kUM * kUKB * 2;
+    static constexpr int kWSubBytes = NP * kUKB * 2;
+    static constexpr int kXStageBytes = kUGSub * kXSubBytes;
+    static constexpr int kWStageBytes = kUGSub * kWSubBytes;
+    static constexpr int kStageBytes = kXStageBytes + kWStageBytes;          // a multiple of 1024
+    static constexpr int kBarrierBytes = 256;
+    static constexpr int kTmemCols = 2 * NP < 64 ? 64 : 2 * NP;              // two accumulators; the epilogue always loads 32 columns
+    static constexpr int smem_bytes(int stages) { return 1024 + stages * kStageBytes + kBarrierBytes + 2 * NP * 4; }
+};
+
+// wimg: [group][D / 64][NP rows][64 columns] swizzled, bimg: [group][NP] float32 (k_pack_nodes).
+template <int NP>
+__global__ void __launch_bounds__(kUGThreads, 1)
+k_descent_umma_grouped(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restrict__ perm,
+                       const Tile* __restrict__ tiles, int n_tiles_total, const __nv_bfloat16* __restrict__ wimg,
+                       const float* __restrict__ bimg, int32_t* __restrict__ pos_out, int D, int k, int kStages,
+                       int* __restrict__ status)
+{
+    using L = DescentUmmaGroupedLayout<NP>;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* full = reinterpret_cast<uint64_t*>(ring + kStages * L::kStageBytes);
+    uint64_t* empty = full + kUmmaMaxStages;
+    uint64_t* acc_full = empty + kUmmaMaxStages;
+    uint64_t* acc_empty = acc_full + 2;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    float* bias = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(full) + L::kBarrierBytes);     // [2][NP]
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int KB = D / (kUKB * kUGSub);                    // ring stages per tile
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            ptx::mbar_init(full + s, kUGGatherWarps);      // one arrival per gather warp
+            ptx::mbar_init(empty + s, 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            ptx::mbar_init(acc_full + a, 1);
+            ptx::mbar_init(acc_empty + a, kUmmaEpilogueWarps * 32);
+        }
+        ptx::fence_mbar_init();
+        ptx::prefetch_tensormap(&tmap_x);
+    }
+    if (warp == 4) {
+        ptx::tmem_alloc(tmem_slot, L::kTmemCols);
+        ptx::tmem_relinquish_alloc_permit();
+    }
+    ptx::tc_fence_before_sync();
+    pdl_trigger();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    pdl_wait();
+    const uint32_t tmem_base = *tmem_slot;
+
+    bool timed_out = false;
+    if (warp > 4) {
+        // ------------------------------------------------------------------ row gathers (+ weight copies)
+        const int gw = warp - 5;
+        int stage = 0;
+        uint32_t phase = 0;
+        for (int tile = blockIdx.x; tile < n_tiles_total; tile += gridDim.x) {
+            const Tile tl = tiles[tile];
+            if (tl.rows <= 0) continue;
+            const int total_groups = (tl.rows + 3) >> 2;
+            const int groups = max((total_groups - gw + kUGGatherWarps - 1) / kUGGatherWarps, 0);
+            const int first = (lane * kUGGatherWarps + gw) * 4;
+            int r[4] = {0, 0, 0, 0};
+            if (lane < groups) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) r[i] = perm[tl.start + min(first + i, tl.rows - 1)];
+            }
+            for (int kb = 0; kb < KB; ++kb) {
+                if (!timed_out && !ptx::mbar_wait_relaxed(empty + stage, phase ^ 1)) timed_out = true;
+                unsigned char* st = ring + stage * L::kStageBytes;
+                if (lane == 0) {
+                    const uint32_t bytes = (uint32_t)groups * (512u * kUGSub) + (gw == 0 ? (uint32_t)L::kWStageBytes : 0u);
+                    if (bytes > 0) ptx::mbar_arrive_expect_tx(full + stage, bytes);
+                    else ptx::mbar_arrive(full + stage);
+                    if (gw == 0)
+                        ptx::bulk_g2s(st + L::kXStageBytes, wimg + ((int64_t)tl.bin * KB + kb) * (kUGSub * NP * kUKB), L::kWStageBytes,
+                                      full + stage);
+                }
+                __syncwarp();
+                if (lane < groups) {
+#pragma unroll
+                    for (int sb = 0; sb < kUGSub; ++sb)
+                        ptx::tma_gather4(st + sb * L::kXSubBytes + first * 128, &tmap_x, (kb * kUGSub + sb) * kUKB, r[0], r[1], r[2], r[3],
+                                         full + stage);
+                }
+                if (++stage == kStages) { stage = 0; phase ^= 1; }
+            }
+        }
+    } else if (warp == 4) {
+        // ------------------------------------------------------------------ MMA issuer
+        constexpr uint32_t idesc = ptx::umma_idesc_bf16(kUM, NP);
+        int stage = 0;
+        uint32_t phase = 0;
+        int it = 0;
+        for (int tile = blockIdx.x; tile < n_tiles_total; tile += gridDim.x) {
+            if (tiles[tile].rows <= 0) continue;
+            const int a = it & 1;
+            if (!timed_out && !ptx::mbar_wait(acc_empty + a, ((it >> 1) & 1) ^ 1)) timed_out = true;
+            ptx::tc_fence_after_sync();
+            for (int kb = 0; kb < KB; ++kb) {
+                if (!timed_out && !ptx::mbar_wait(full + stage, phase)) timed_out = true;
+                ptx::tc_fence_after_sync();
+                if (lane == 0) {
+                    const uint32_t xs = ptx::smem_addr(ring + stage * L::kStageBytes);
+#pragma unroll
+                    for (int sb = 0; sb < kUGSub; ++sb) {
+                        const uint64_t ad = ptx::umma_desc_k128(xs + sb * L::kXSubBytes);
+                        const uint64_t bd = ptx::umma_desc_k128(xs + L::kXStageBytes + sb * L::kWSubBytes);
+#pragma unroll
+                        for (int j = 0; j < kUKB / 16; ++j)
+                            ptx::umma_bf16(tmem_base + a * NP, ad + 2 * j, bd + 2 * j, idesc, (kb | sb | j) != 0 ? 1u : 0u);
+                    }
+                    ptx::umma_commit(empty + stage);
+                    if (kb == KB - 1) ptx::umma_commit(acc_full + a);
+                }
+                __syncwarp();
+                if (++stage == kStages) { stage = 0; phase ^= 1; }
+            }
+            ++it;
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue: one token per thread
+        int it = 0;
+        for (int tile = blockIdx.x; tile < n_tiles_total; tile += gridDim.x) {
+            const Tile tl = tiles[tile];
+            if (tl.rows <= 0) continue;
+            const int a = it & 1;
+            const int row = warp * 32 + lane;
+            const int64_t tok = row < tl.rows ? perm[tl.start + row] : -1;
+            // this bucket's biases; the buffer of two tiles ago is free: its readers have passed the barrier
+            // of the previous tile
+            float* tb = bias + a * NP;
+            if (row < NP) tb[row] = __ldg(bimg + (int64_t)tl.bin * NP + row);
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (!timed_out && !ptx::mbar_wait(acc_full + a, (it >> 1) & 1)) timed_out = true;
+            ptx::tc_fence_after_sync();
+            uint32_t bits = 0, bits_hi = 0;
+            {
+                uint32_t v[32];
+                ptx::tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + a * NP, v);      // columns past NP are not used
+                ptx::tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 32 && j < NP; ++j) bits |= (__uint_as_float(v[j]) + tb[j] >= 0.0f ? 1u : 0u) << j;
+                if (NP == 64) {
+                    ptx::tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + a * NP + 32, v);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) bits_hi |= (__uint_as_float(v[j]) + tb[32 + j] >= 0.0f ? 1u : 0u) << j;
+                }
+            }
+            ptx::tc_fence_before_sync();
+            ptx::mbar_arrive(acc_empty + a);
+            int p = 0;
+            for (int r = 0; r < k; ++r) {
+                const uint32_t w = (NP == 64 && p >= 32) ? bits_hi : bits;
+                p = 2 * p + 1 + (int)((w >> (p & 31)) & 1u);
+            }
+            if (tok >= 0) pos_out[tok] = (tl.bin << k) + (p - ((1 << k) - 1));
+            ++it;
+        }
+    }
+    if (timed_out) {
+        if (lane == 0) atomicExch(status, kDevTimeout);
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);     // let copies and MMAs still in flight finish before exit
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 4) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, L::kTmemCols);
+    }
+}
+
 }  // namespace fff
