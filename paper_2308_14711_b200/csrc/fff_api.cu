@@ -609,9 +609,18 @@ fff_status_t pack_node_images(fff_handle_s* h) {
             for (size_t i = 1; i < ks.size(); ++i) ok = ok && ks[i] >= 1 && ks[i] <= 6;
             if (!ok) ks.clear();
         }
-        // Up to 8 levels in one stage when that is the whole tree (no node bucketing at all); deeper
-        // trees measured best with the usual cut into stages of at most 6 levels.
-        if (ks.empty()) ks = d <= 8 ? std::vector<int>{d} : cut_levels(d);
+        // Measured: up to 8 levels in one stage when that is the whole tree (no node bucketing at all); two
+        // balanced stages up to depth 12 ([6,5] beats [8,3]: 64 bins instead of 256 and fatter groups);
+        // deeper trees as few stages as possible, 8 levels first and then 6 at a time ([8,6,1] beats [5,5,5]:
+        // one pass over x and one bucketing less, the last thin levels go to the warp kernel anyway).
+        if (ks.empty()) {
+            if (d <= 8) ks = {d};
+            else if (d <= 12) ks = cut_levels(d);
+            else {
+                ks.push_back(8);
+                for (int rest = d - 8; rest > 0; rest -= 6) ks.push_back(std::min(rest, 6));
+            }
+        }
         L0 = 0;
         for (size_t i = 0; i < ks.size(); ++i) {
             const int np = i == 0 ? std::max(32, 1 << ks[i]) : std::max(16, 1 << ks[i]);
