@@ -29,6 +29,10 @@
 // GEMM1 of the next tile runs while the epilogue of the current one drains, and the row gathers never
 // stop in between: loads and stores overlap across tiles.
 //
+// When the hidden width is padded (l < LP) the spare column l of H is set to 1 and the same column of the W2
+// image holds b2, so GEMM2 adds the output bias itself and the epilogue only converts and stores; with
+// l == LP the biases ride behind the W2 pieces and are added in the epilogue.
+//
 // Rows of a ragged tile beyond its length are not loaded: their accumulator rows hold garbage that is
 // never stored (rows of an MMA are independent).
 //
