@@ -112,7 +112,13 @@ fff_status_t fff_forward_infer(fff_handle_t h, const void *x, void *y, int32_t *
 /*
  * The same computation for buffers in HOST memory (pinned or pageable):
  * copies x to the device, runs fff_forward_infer, copies y (and leaf_idx when
- * not NULL) back, and returns after `cuda_stream` has completed.
+ * not NULL) back, and returns after `cuda_stream` has completed.  Batches of
+ * 16384 tokens or more are cut into up to 16 chunks whose copies (on two
+ * library-owned streams, ordered after what `cuda_stream` already holds) and
+ * kernels overlap; with pinned host buffers this takes about the time of the
+ * slower copy direction.  Results do not depend on the chunking.  After a
+ * chunked call fff_debug_get_bucketing has nothing to report
+ * (FFF_ERR_INVALID_ARG) until the next fff_forward_infer.
  */
 fff_status_t fff_forward_infer_host(fff_handle_t h, const void *x_host, void *y_host,
                                     int32_t *leaf_idx_host, int64_t B, void *cuda_stream);

@@ -92,6 +92,10 @@ struct fff_handle_s {
     int64_t cap_host_B = 0;
     void *st_x = nullptr, *st_y = nullptr;
     int32_t *st_leaf = nullptr;
+    // copy streams and events of the chunked host-buffer pipeline (created on first use)
+    static constexpr int kMaxHostChunks = 16;
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    cudaEvent_t ev_in[kMaxHostChunks] = {}, ev_done[kMaxHostChunks] = {}, ev_start = nullptr, ev_end = nullptr;
 
     int path = FFF_PATH_AUTO;
     bool pdl = true;              // launch every kernel of a forward but the first as a programmatic dependent
@@ -184,6 +188,14 @@ void release(fff_handle_s* h) {
     for (auto& sg : h->ustages) { dfree(sg.wimg); dfree(sg.bimg); }
     dfree(h->ws_pos[0]); dfree(h->ws_pos[1]);
     dfree(h->w1img); dfree(h->b1img); dfree(h->w2img); dfree(h->w2uimg); dfree(h->ws_sched); dfree(h->ws_tiles); dfree(h->ws_rank); dfree(h->ws_rank8); dfree(h->ws_counts8); dfree(h->ws_matrix);
+    if (h->copy_in) cudaStreamDestroy(h->copy_in);
+    if (h->copy_out) cudaStreamDestroy(h->copy_out);
+    for (int i = 0; i < fff_handle_s::kMaxHostChunks; ++i) {
+        if (h->ev_in[i]) cudaEventDestroy(h->ev_in[i]);
+        if (h->ev_done[i]) cudaEventDestroy(h->ev_done[i]);
+    }
+    if (h->ev_start) cudaEventDestroy(h->ev_start);
+    if (h->ev_end) cudaEventDestroy(h->ev_end);
     prof_free(h);
     h->magic = 0;
     delete h;
@@ -1065,16 +1077,60 @@ fff_status_t fff_forward_infer_host(fff_handle_t h, const void* x_host, void* y_
         h->cap_host_B = B;
     }
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    if (cudaMemcpyAsync(h->st_x, x_host, (size_t)B * h->D * h->esize, cudaMemcpyHostToDevice, st) != cudaSuccess)
-        return cudaGetLastError(), FFF_ERR_CUDA;
-    if ((s = fff_forward_infer(h, h->st_x, h->st_y, h->st_leaf, B, cuda_stream)) != FFF_OK) return s;
-    if (cudaMemcpyAsync(y_host, h->st_y, (size_t)B * h->O * h->esize, cudaMemcpyDeviceToHost, st) != cudaSuccess)
-        return cudaGetLastError(), FFF_ERR_CUDA;
-    if (leaf_idx_host &&
-        cudaMemcpyAsync(leaf_idx_host, h->st_leaf, (size_t)B * sizeof(int32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess)
-        return cudaGetLastError(), FFF_ERR_CUDA;
-    if (cudaStreamSynchronize(st) != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
-    return FFF_OK;
+    // Large batches go through in chunks so that the copy of chunk i+1 to the device, the kernels of chunk i
+    // and the copy of chunk i-1 back overlap (tokens are independent, so chunking does not change any result).
+    const int n_chunks = (int)std::max<int64_t>(1, std::min<int64_t>(fff_handle_s::kMaxHostChunks, B / 8192));
+    if (n_chunks == 1) {
+        if (cudaMemcpyAsync(h->st_x, x_host, (size_t)B * h->D * h->esize, cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return cudaGetLastError(), FFF_ERR_CUDA;
+        if ((s = fff_forward_infer(h, h->st_x, h->st_y, h->st_leaf, B, cuda_stream)) != FFF_OK) return s;
+        if (cudaMemcpyAsync(y_host, h->st_y, (size_t)B * h->O * h->esize, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            return cudaGetLastError(), FFF_ERR_CUDA;
+        if (leaf_idx_host &&
+            cudaMemcpyAsync(leaf_idx_host, h->st_leaf, (size_t)B * sizeof(int32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            return cudaGetLastError(), FFF_ERR_CUDA;
+        if (cudaStreamSynchronize(st) != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
+        return FFF_OK;
+    }
+    if (!h->copy_in) {
+        bool ok = cudaStreamCreateWithFlags(&h->copy_in, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&h->copy_out, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&h->ev_start, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&h->ev_end, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; ok && i < fff_handle_s::kMaxHostChunks; ++i)
+            ok = cudaEventCreateWithFlags(&h->ev_in[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&h->ev_done[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) return cudaGetLastError(), FFF_ERR_CUDA;
+    }
+    const int64_t chunk = (((B + n_chunks - 1) / n_chunks) + 127) & ~int64_t(127);
+    const size_t xrow = (size_t)h->D * h->esize, yrow = (size_t)h->O * h->esize;
+    bool ok = cudaEventRecord(h->ev_start, st) == cudaSuccess &&              // the copies come after what the caller enqueued
+              cudaStreamWaitEvent(h->copy_in, h->ev_start, 0) == cudaSuccess &&
+              cudaStreamWaitEvent(h->copy_out, h->ev_start, 0) == cudaSuccess;
+    for (int c = 0; ok && c < n_chunks; ++c) {
+        const int64_t b0 = c * chunk, n = std::min(chunk, B - b0);
+        if (n <= 0) break;
+        ok = cudaMemcpyAsync((char*)h->st_x + b0 * xrow, (const char*)x_host + b0 * xrow, (size_t)n * xrow, cudaMemcpyHostToDevice,
+                             h->copy_in) == cudaSuccess &&
+             cudaEventRecord(h->ev_in[c], h->copy_in) == cudaSuccess;
+    }
+    for (int c = 0; ok && c < n_chunks; ++c) {
+        const int64_t b0 = c * chunk, n = std::min(chunk, B - b0);
+        if (n <= 0) break;
+        ok = cudaStreamWaitEvent(st, h->ev_in[c], 0) == cudaSuccess;
+        if (!ok) break;
+        if ((s = fff_forward_infer(h, (char*)h->st_x + b0 * xrow, (char*)h->st_y + b0 * yrow, h->st_leaf + b0, n, cuda_stream)) != FFF_OK)
+            return s;
+        ok = cudaEventRecord(h->ev_done[c], st) == cudaSuccess && cudaStreamWaitEvent(h->copy_out, h->ev_done[c], 0) == cudaSuccess &&
+             cudaMemcpyAsync((char*)y_host + b0 * yrow, (char*)h->st_y + b0 * yrow, (size_t)n * yrow, cudaMemcpyDeviceToHost,
+                             h->copy_out) == cudaSuccess &&
+             (!leaf_idx_host || cudaMemcpyAsync(leaf_idx_host + b0, h->st_leaf + b0, (size_t)n * sizeof(int32_t),
+                                                cudaMemcpyDeviceToHost, h->copy_out) == cudaSuccess);
+    }
+    ok = ok && cudaEventRecord(h->ev_end, h->copy_out) == cudaSuccess && cudaStreamWaitEvent(st, h->ev_end, 0) == cudaSuccess &&
+         cudaStreamSynchronize(st) == cudaSuccess;
+    h->last_B = -1;        // the workspace holds the last chunk only: no bucketing of the whole batch to report
+    return ok ? FFF_OK : (cudaGetLastError(), FFF_ERR_CUDA);
 }
 
 fff_status_t fff_debug_get_bucketing(fff_handle_t h, int32_t* perm, int32_t* offsets, void* cuda_stream) {

@@ -155,6 +155,29 @@ def test_host_buffer_entry_point(small_case):
     layer.close()
 
 
+@pytest.mark.parametrize("B", [16384, 40001])
+def test_host_buffer_entry_point_chunked(B):
+    """Batches of 16384 tokens or more go through the host entry point in overlapping chunks."""
+    cfg = wl.FFFConfig("bf16_host_chunks", 128, 144, 4, 16, "gelu", "bf16", B, "normal")
+    case = util.make_case(cfg, seed=3)
+    y_ref, leaf_ref = orc.forward_i(case.net, case.x, threads=util.ORACLE_THREADS)
+    layer = util.make_layer(case)
+    xh = torch.from_numpy(case.x).to(torch.bfloat16).pin_memory()
+    yh = torch.empty((B, cfg.O), dtype=torch.bfloat16).pin_memory()
+    lh = torch.empty((B,), dtype=torch.int32).pin_memory()
+    for _ in range(2):                                   # the second call reuses streams, events and staging
+        yh.zero_()
+        lh.fill_(-1)
+        layer.forward_infer_host(xh, yh, lh)
+        np.testing.assert_array_equal(lh.numpy(), leaf_ref)
+        util.check_outputs(yh, y_ref, cfg.dtype)
+    # the same rows through the device entry point, unchunked: identical bits (a row's result depends on no other row)
+    y_dev, leaf_dev = layer.forward_infer(xh.cuda())
+    torch.cuda.synchronize()
+    assert torch.equal(y_dev.cpu(), yh)
+    layer.close()
+
+
 def test_gpu_argument_errors_are_reported_not_faulted():
     from paper_2308_14711_b200 import binding
     cfg = wl.FFFConfig("e", 16, 8, 2, 4, "relu", "f32", 8)
