@@ -371,7 +371,10 @@ def cpu_baseline(cfg, w_host, x_host, budget_s: float = 20.0) -> dict:
     per_tok = (time.perf_counter() - t) / probe
     n = int(max(probe, min(cfg.B, budget_s / max(per_tok, 1e-9))))
     # about 10 s of CPU work: the whole batch (or the prefix that fits the budget), as many passes as that takes
-    passes = int(max(1, min(200, 10.0 / max(per_tok * n, 1e-9))))
+    # (sized from one untimed pass: the short probe above overestimates the per-token cost)
+    t = time.perf_counter()
+    orc.forward_i(net, x_host[:n], threads=cores)
+    passes = int(max(1, min(500, 10.0 / max(time.perf_counter() - t, 1e-6))))
     t = time.perf_counter()
     for _ in range(passes):
         orc.forward_i(net, x_host[:n], threads=cores)
