@@ -419,7 +419,7 @@ EncodeTiledFn encode_tiled_fn() {
 
 // Tensor map of the bf16 token matrix x[B, D] for boxes of box_rows x 64 columns, 128-byte swizzled;
 // rows past B read as zeros.
-bool make_x_tensor_map(CUtensorMap* tm, const void* x, int64_t B, int D, int box_rows) {
+bool make_x_tensor_map(CUtensorMap* tm, const void* x, int64_t B, int D, int box_rows, bool swizzle = true) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return false;
     const cuuint64_t gdim[2] = {(cuuint64_t)D, (cuuint64_t)B};
@@ -427,7 +427,8 @@ bool make_x_tensor_map(CUtensorMap* tm, const void* x, int64_t B, int D, int box
     const cuuint32_t box[2] = {(cuuint32_t)fff::kUKB, (cuuint32_t)box_rows};
     const cuuint32_t estride[2] = {1, 1};
     return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(x), gdim, gstride, box, estride,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+               CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -449,8 +450,40 @@ fff_status_t launch_descent_umma(fff_handle_s* h, const fff_handle_s::DenseStage
     return launched(h, st, "tree_descent_umma");
 }
 
+// The same on CTA pairs that share the weight K-blocks (NP >= 128, where re-streaming them binds the kernel).
+template <int NP>
+fff_status_t launch_descent_umma_pair(fff_handle_s* h, const fff_handle_s::DenseStage& sg, const void* x, int32_t* pos_out,
+                                      int64_t B, cudaStream_t st) {
+    using L = fff::DescentUmmaPairLayout<NP>;
+    const int stages = std::min((int)fff::kUmmaMaxStages, (kSmemBudget - L::smem_bytes(0)) / L::kStageBytes);
+    if (stages < 2) return FFF_ERR_UNSUPPORTED;
+    static bool attr_set[64] = {};
+    if (h->device < 64 && !attr_set[h->device]) {
+        cudaFuncSetAttribute(fff::k_descent_umma_pair<NP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+        attr_set[h->device] = true;
+    }
+    CUtensorMap tm, tw;
+    if (!make_x_tensor_map(&tm, x, B, h->D, fff::kUM)) return FFF_ERR_CUDA;
+    // the weight image as (D/64) * NP rows of 64 columns, stored pre-swizzled: copied as it is
+    if (!make_x_tensor_map(&tw, sg.wimg, (int64_t)(h->D / fff::kUKB) * NP, fff::kUKB, NP / 2, false)) return FFF_ERR_CUDA;
+    const int64_t n_pairs = ((B + fff::kUM - 1) / fff::kUM + 1) / 2;
+    const int64_t grid = 2 * std::max<int64_t>(1, std::min<int64_t>(h->sm_count / 2, n_pairs));
+    const bool ranked = sg.k >= 4 && h->ws_rank8 && h->ws_counts8;
+    if (launch_chain(h, fff::k_descent_umma_pair<NP>, (unsigned)grid, fff::kUmmaThreads, (size_t)L::smem_bytes(stages), st, 2, tm,
+                     tw, (const float*)sg.bimg, pos_out, ranked ? h->ws_rank8 : (uint8_t*)nullptr,
+                     ranked ? h->ws_counts8 : (uint8_t*)nullptr, h->D, (int)B, sg.k, stages, h->d_status) != cudaSuccess)
+        return cudaGetLastError(), FFF_ERR_CUDA;
+    return launched(h, st, "tree_descent_umma");
+}
+
 fff_status_t run_descent_umma(fff_handle_s* h, const fff_handle_s::DenseStage& sg, const void* x, int32_t* pos_out, int64_t B,
                               cudaStream_t st) {
+    static const bool no_pair = std::getenv("FFF_NO_UMMA_PAIR") != nullptr;      // tuning aid
+    // pairs pay once there is more than one round of tiles (measured: 29.1 vs 31.2 us at 394 tiles, 18.7 vs 17.0 at 128)
+    if (!no_pair && (B + fff::kUM - 1) / fff::kUM > h->sm_count && h->sm_count >= 2) {
+        if (sg.NP == 128) return launch_descent_umma_pair<128>(h, sg, x, pos_out, B, st);
+        if (sg.NP == 256) return launch_descent_umma_pair<256>(h, sg, x, pos_out, B, st);
+    }
     switch (sg.NP) {
         case 32: return launch_descent_umma<32>(h, sg, x, pos_out, B, st);
         case 64: return launch_descent_umma<64>(h, sg, x, pos_out, B, st);

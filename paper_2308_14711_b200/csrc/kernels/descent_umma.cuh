@@ -42,6 +42,54 @@ constexpr int kUmmaEpilogueWarps = 4;
 constexpr int kUmmaThreads = (kUmmaEpilogueWarps + 2) * 32;
 constexpr int kUmmaMaxStages = 8;
 
+// Decision bits of one token: bit p of bits[] says whether logit[p] + bias[p] >= 0 (a logit of zero goes right,
+// NaN left).  The NP logits are this thread's tensor-memory lane, read 32 columns at a time with the next load
+// already in flight.
+template <int NP>
+__device__ __forceinline__ void umma_decision_bits(uint32_t taddr, const float* __restrict__ bias, uint32_t (&bits)[NP / 32])
+{
+    uint32_t v[2][32];
+    ptx::tmem_ld32(taddr, v[0]);
+#pragma unroll
+    for (int c = 0; c < NP / 32; ++c) {
+        ptx::tmem_ld_wait();
+        if (c + 1 < NP / 32) ptx::tmem_ld32(taddr + (c + 1) * 32, v[(c + 1) & 1]);
+        uint32_t m = 0;
+#pragma unroll
+        for (int j = 0; j < 32; j += 4) {
+            const float4 b = *reinterpret_cast<const float4*>(bias + c * 32 + j);     // same address in every lane
+            m |= (__uint_as_float(v[c & 1][j]) + b.x >= 0.0f ? 1u : 0u) << j;
+            m |= (__uint_as_float(v[c & 1][j + 1]) + b.y >= 0.0f ? 1u : 0u) << (j + 1);
+            m |= (__uint_as_float(v[c & 1][j + 2]) + b.z >= 0.0f ? 1u : 0u) << (j + 2);
+            m |= (__uint_as_float(v[c & 1][j + 3]) + b.w >= 0.0f ? 1u : 0u) << (j + 3);
+        }
+        bits[c] = m;
+    }
+}
+
+// The walk p <- 2p + 1 + bit[p] over k levels, p in the subtree's breadth-first numbering.  Level r lives at
+// positions 2^r - 1 .. 2^(r+1) - 2, i.e. in words (2^r - 1) / 32 .. (2^(r+1) - 2) / 32 only, so the word is picked
+// with as few selects as the level needs (none up to level 4).
+template <int NP>
+__device__ __forceinline__ int umma_walk(const uint32_t (&bits)[NP / 32], int k)
+{
+    int p = 0;
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+        if (r < k && ((1 << r) - 1) < NP) {
+            constexpr int kWords = NP / 32;
+            const int w_lo = ((1 << r) - 1) >> 5;
+            const int w_hi = min(((2 << r) - 2) >> 5, kWords - 1);
+            uint32_t w = bits[w_lo < kWords ? w_lo : 0];
+#pragma unroll
+            for (int c = 1; c < kWords; ++c)
+                if (c > w_lo && c <= w_hi) w = (p >> 5) == c ? bits[c] : w;
+            p = 2 * p + 1 + (int)((w >> (p & 31)) & 1u);
+        }
+    }
+    return p;
+}
+
 template <int NP> struct DescentUmmaLayout {
     static_assert(NP == 32 || NP == 64 || NP == 128 || NP == 256, "accumulator width");
     static constexpr int kXStageBytes = kUM * kUKB * 2;
@@ -155,26 +203,11 @@ k_descent_umma(const __grid_constant__ CUtensorMap tmap_x, const __nv_bfloat16* 
             if (!timed_out && !ptx::mbar_wait(acc_full + a, (it >> 1) & 1)) timed_out = true;
             ptx::tc_fence_after_sync();
             uint32_t bits[NP / 32];
-#pragma unroll
-            for (int c = 0; c < NP / 32; ++c) {
-                uint32_t v[32];
-                ptx::tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + a * NP + c * 32, v);
-                ptx::tmem_ld_wait();
-                uint32_t m = 0;
-#pragma unroll
-                for (int j = 0; j < 32; ++j) m |= (__uint_as_float(v[j]) + bias[c * 32 + j] >= 0.0f ? 1u : 0u) << j;
-                bits[c] = m;
-            }
+            umma_decision_bits<NP>(tmem_base + ((uint32_t)(warp * 32) << 16) + a * NP, bias, bits);
             ptx::tc_fence_before_sync();
             ptx::mbar_arrive(acc_empty + a);
 
-            int p = 0;
-            for (int r = 0; r < k; ++r) {
-                uint32_t w = bits[0];
-#pragma unroll
-                for (int c = 1; c < NP / 32; ++c) w = (p >> 5) == c ? bits[c] : w;
-                p = 2 * p + 1 + (int)((w >> (p & 31)) & 1u);
-            }
+            const int p = umma_walk<NP>(bits, k);
             const int tok = tile * kUM + warp * 32 + lane;
             const int key = p - ((1 << k) - 1);
             if (tok < B) pos_out[tok] = key;
@@ -212,6 +245,195 @@ k_descent_umma(const __grid_constant__ CUtensorMap tmap_x, const __nv_bfloat16* 
     if (warp == 5) {
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, L::kTmemCols);
+    }
+}
+
+// ---- the first stage on CTA pairs ----------------------------------------------------------------------
+// With NP = 128 or 256 the weight K-blocks (16-32 KB each) are re-streamed from L2 for every 128-token tile,
+// and that traffic, not DRAM, bounds the kernel above.  Here two CTAs (a cluster of two, cta_group::2) share
+// every weight K-block: each loads its own 128-token tile of x and HALF of the NP weight rows, the pair's first
+// CTA issues one MMA over 256 rows that reads A and B from both CTAs' shared memory, and each CTA keeps the
+// accumulator rows of its own tokens in its own tensor memory.  Roles per CTA as above; differences:
+//   * the "stage full" and "accumulator free" barriers that the MMA issuer waits on live in the first CTA; the
+//     second CTA's producer and epilogue arrive on them through the shared::cluster window, and its tensor-map
+//     loads (cta_group::2 form) count their bytes there;
+//   * tcgen05.commit frees a stage / publishes an accumulator in both CTAs (one commit per CTA);
+//   * the weight image is read through a tensor map of its own (rows of 64 columns, no swizzle mode: the image
+//     is stored pre-swizzled), because only tensor-map loads can signal the other CTA's barrier;
+//   * cluster barriers order barrier initialisation before the first remote arrival, and the last remote
+//     operation before either CTA leaves.
+template <int NP> struct DescentUmmaPairLayout {
+    static_assert(NP == 128 || NP == 256, "accumulator width");
+    static constexpr int kXStageBytes = kUM * kUKB * 2;
+    static constexpr int kWStageBytes = (NP / 2) * kUKB * 2;                 // this CTA's half of the weight rows
+    static constexpr int kStageBytes = kXStageBytes + kWStageBytes;          // a multiple of 1024
+    static constexpr int kBarrierBytes = 256;
+    static constexpr int kTmemCols = 2 * NP;                                 // two accumulators (per CTA)
+    static constexpr int kCountBytes = kUmmaEpilogueWarps * 256;
+    static constexpr int smem_bytes(int stages) { return 1024 + stages * kStageBytes + kBarrierBytes + NP * 4 + kCountBytes; }
+};
+
+// tmap_w: the single-group image as a matrix of (D/64) * NP rows of 64 columns, boxes of NP/2 rows.
+template <int NP>
+__global__ void __launch_bounds__(kUmmaThreads, 1)
+k_descent_umma_pair(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+                    const float* __restrict__ bimg, int32_t* __restrict__ pos_out, uint8_t* __restrict__ rank8,
+                    uint8_t* __restrict__ counts8, int D, int B, int k, int kStages, int* __restrict__ status)
+{
+    namespace cg = cooperative_groups;
+    using L = DescentUmmaPairLayout<NP>;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* full = reinterpret_cast<uint64_t*>(ring + kStages * L::kStageBytes);     // used in the first CTA only
+    uint64_t* empty = full + kUmmaMaxStages;
+    uint64_t* acc_full = empty + kUmmaMaxStages;
+    uint64_t* acc_empty = acc_full + 2;                                                 // used in the first CTA only
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    float* bias = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(full) + L::kBarrierBytes);
+    uint8_t* s_cnt = reinterpret_cast<uint8_t*>(bias + NP);
+
+    cg::cluster_group cluster = cg::this_cluster();
+    const uint32_t rank = cluster.block_rank();            // 0: issues the MMAs
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_tiles = (B + kUM - 1) / kUM;
+    const int n_pairs = (n_tiles + 1) / 2;
+    const int pair0 = blockIdx.x >> 1, pair_stride = gridDim.x >> 1;
+    const int KB = D / kUKB;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            ptx::mbar_init(full + s, 2);                   // one arrival (with its byte count) per CTA
+            ptx::mbar_init(empty + s, 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            ptx::mbar_init(acc_full + a, 1);
+            ptx::mbar_init(acc_empty + a, 2 * kUmmaEpilogueWarps * 32);
+        }
+        ptx::fence_mbar_init();
+        ptx::prefetch_tensormap(&tmap_x);
+        ptx::prefetch_tensormap(&tmap_w);
+    }
+    if (warp == 5) {
+        ptx::tmem_alloc_pair(tmem_slot, L::kTmemCols);
+        ptx::tmem_relinquish_alloc_permit_pair();
+    }
+    for (int i = threadIdx.x; i < NP; i += kUmmaThreads) bias[i] = bimg[i];
+    for (int i = threadIdx.x; i < L::kCountBytes / 4; i += kUmmaThreads) reinterpret_cast<uint32_t*>(s_cnt)[i] = 0;
+    ptx::tc_fence_before_sync();
+    pdl_trigger();
+    cluster.sync();                                        // both CTAs' barriers exist before anything arrives on them
+    ptx::tc_fence_after_sync();
+    pdl_wait();
+    const uint32_t tmem_base = *tmem_slot;
+
+    bool timed_out = false;
+    if (warp == 4) {
+        // ------------------------------------------------------------------ producer (each CTA: its tile, its half of W)
+        int stage = 0;
+        uint32_t phase = 0;
+        for (int pair = pair0; pair < n_pairs; pair += pair_stride) {
+            const int tile = 2 * pair + (int)rank;         // may be one past the end: such rows read as zeros
+            for (int kb = 0; kb < KB; ++kb) {
+                if (!timed_out && !ptx::mbar_wait_relaxed(empty + stage, phase ^ 1)) timed_out = true;
+                if (lane == 0) {
+                    unsigned char* st = ring + stage * L::kStageBytes;
+                    const uint32_t bar = ptx::map_to_cta(ptx::smem_addr(full + stage), 0);
+                    ptx::mbar_arrive_expect_tx_cluster(bar, (uint32_t)L::kStageBytes);
+                    ptx::tma_load_2d_pair(st, &tmap_x, kb * kUKB, tile * kUM, bar);
+                    ptx::tma_load_2d_pair(st + L::kXStageBytes, &tmap_w, 0, kb * NP + (int)rank * (NP / 2), bar);
+                }
+                __syncwarp();
+                if (++stage == kStages) { stage = 0; phase ^= 1; }
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------------------------ MMA issuer (first CTA only)
+        if (rank == 0) {
+            constexpr uint32_t idesc = ptx::umma_idesc_bf16(2 * kUM, NP);
+            int stage = 0;
+            uint32_t phase = 0;
+            int it = 0;
+            for (int pair = pair0; pair < n_pairs; pair += pair_stride, ++it) {
+                const int a = it & 1;
+                if (!timed_out && !ptx::mbar_wait(acc_empty + a, ((it >> 1) & 1) ^ 1)) timed_out = true;
+                ptx::tc_fence_after_sync();
+                for (int kb = 0; kb < KB; ++kb) {
+                    if (!timed_out && !ptx::mbar_wait(full + stage, phase)) timed_out = true;
+                    ptx::tc_fence_after_sync();
+                    if (lane == 0) {
+                        const uint32_t xs = ptx::smem_addr(ring + stage * L::kStageBytes);
+                        const uint64_t ad = ptx::umma_desc_k128(xs), bd = ptx::umma_desc_k128(xs + L::kXStageBytes);
+#pragma unroll
+                        for (int j = 0; j < kUKB / 16; ++j)
+                            ptx::umma_bf16_pair(tmem_base + a * NP, ad + 2 * j, bd + 2 * j, idesc, (kb | j) != 0 ? 1u : 0u);
+                        const uint32_t e0 = ptx::smem_addr(empty + stage);
+                        ptx::umma_commit_pair(ptx::map_to_cta(e0, 0));
+                        ptx::umma_commit_pair(ptx::map_to_cta(e0, 1));
+                        if (kb == KB - 1) {
+                            const uint32_t f0 = ptx::smem_addr(acc_full + a);
+                            ptx::umma_commit_pair(ptx::map_to_cta(f0, 0));
+                            ptx::umma_commit_pair(ptx::map_to_cta(f0, 1));
+                        }
+                    }
+                    __syncwarp();
+                    if (++stage == kStages) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue: one token per thread
+        int it = 0;
+        for (int pair = pair0; pair < n_pairs; pair += pair_stride, ++it) {
+            const int tile = 2 * pair + (int)rank;
+            const int a = it & 1;
+            if (!timed_out && !ptx::mbar_wait(acc_full + a, (it >> 1) & 1)) timed_out = true;
+            ptx::tc_fence_after_sync();
+            uint32_t bits[NP / 32];
+            umma_decision_bits<NP>(tmem_base + ((uint32_t)(warp * 32) << 16) + a * NP, bias, bits);
+            ptx::tc_fence_before_sync();
+            // (relaxed: the loads above have completed, there is nothing else of this thread to publish)
+            ptx::mbar_arrive_cluster_relaxed(ptx::map_to_cta(ptx::smem_addr(acc_empty + a), 0));
+
+            const int p = umma_walk<NP>(bits, k);
+            const int tok = tile * kUM + warp * 32 + lane;
+            const int key = p - ((1 << k) - 1);
+            if (tok < B) pos_out[tok] = key;
+            if (rank8) {
+                const int nbins = 1 << k;
+                const bool in = tok < B;
+                const unsigned peers = peers_by_ballot(in, key, k);
+                if (in && lane == __ffs(peers) - 1) s_cnt[warp * 256 + key] = (uint8_t)__popc(peers);
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (in) {
+                    int before = __popc(peers & ((1u << lane) - 1u));
+                    for (int w = 0; w < warp; ++w) before += s_cnt[w * 256 + key];
+                    rank8[tok] = (uint8_t)before;
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (tile < n_tiles) {
+                    for (int b = warp * 32 + lane; b < nbins; b += kUmmaEpilogueWarps * 32) {
+                        int total = 0;
+#pragma unroll
+                        for (int w = 0; w < kUmmaEpilogueWarps; ++w) {
+                            total += s_cnt[w * 256 + b];
+                            s_cnt[w * 256 + b] = 0;
+                        }
+                        counts8[(int64_t)tile * nbins + b] = (uint8_t)total;
+                    }
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+            }
+        }
+    }
+    if (timed_out) {
+        if (lane == 0) atomicExch(status, kDevTimeout);
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+    }
+    ptx::tc_fence_before_sync();
+    cluster.sync();                                        // nothing of the pair is in flight any more
+    if (warp == 5) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc_pair(tmem_base, L::kTmemCols);
     }
 }
 
