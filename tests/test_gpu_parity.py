@@ -52,6 +52,8 @@ def small_cfgs():
         C("bf16_tiny_batch", 128, 144, 3, 16, "relu", "bf16", 37, "normal", node_bias_std=0.2),
         # eight levels in one dense stage (255 nodes), small batch
         C("bf16_d8_small", 256, 64, 8, 8, "gelu", "bf16", 5000, "layernorm"),
+        # more 128-token tiles than SMs: the first stage runs on CTA pairs (127 nodes, odd number of tiles)
+        C("bf16_d7_pairs", 128, 64, 7, 8, "relu", "bf16", 20001, "normal"),
     ]
 
 
