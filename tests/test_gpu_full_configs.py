@@ -45,3 +45,29 @@ def test_full_config(name):
     # properties that hold for every row: finite outputs, and rows of one leaf see that leaf's bias
     assert torch.isfinite(y.float()).all()
     layer.close()
+
+
+def test_large_batch_many_tiles_per_sm():
+    """Half a million tokens of a small layer: many rounds of tiles per SM in every kernel, the first stage on
+    CTA pairs with 255 nodes, more count rows than the ranked bucketing takes (it falls back to the grid-wide
+    kernel), and an odd batch size."""
+    cfg = wl.FFFConfig("bf16_large_batch", 128, 64, 8, 8, "gelu", "bf16", 500001, "normal")
+    case = util.make_case(cfg, seed=5)
+    leaf_ref, margin, _ = orc.descend(case.net, case.x, threads=util.ORACLE_THREADS)
+    off_ref, perm_ref = orc.bucket(leaf_ref, cfg.n_leaves)
+    layer = util.make_layer(case)
+    x = util.to_device(case.x, cfg.dtype)
+    for _ in range(2):
+        y, leaf = layer.forward_infer(x)
+        torch.cuda.synchronize()
+        assert layer.last_status() == 0
+        np.testing.assert_array_equal(leaf.cpu().numpy(), leaf_ref)
+        off, perm = layer.last_bucketing(cfg.B)
+        np.testing.assert_array_equal(off.cpu().numpy(), off_ref)
+        np.testing.assert_array_equal(perm.cpu().numpy(), perm_ref)
+    rows = np.sort(np.random.default_rng(1).choice(cfg.B, SAMPLE_ROWS, replace=False))
+    rows[-1] = cfg.B - 1
+    y_ref, _ = orc.forward_i(case.net, case.x[rows], threads=util.ORACLE_THREADS)
+    util.check_outputs(y, y_ref, cfg.dtype, rows=rows)
+    assert torch.isfinite(y.float()).all()
+    layer.close()
