@@ -558,7 +558,15 @@ int dense_stage_count(const fff_handle_s* h, int64_t B) {
 // The whole descent: tensor-core stages (with a bucketing by current node between them), then the
 // remaining levels, if any, one warp per token.  leaf_out receives the leaf index.  *coarse describes
 // the last node bucketing made on the way (the leaf bucketing can refine it instead of starting over).
-fff_status_t run_descent(fff_handle_s* h, const void* x, int32_t* leaf_out, Coarse* coarse, int64_t B, cudaStream_t st) {
+// Levels of the descent that the caller's leaf kernel will walk itself (k_leaf_warp), instead of a launch of
+// k_descent_warp: the walk starts at level `level0` from the positions `pos` (NULL = the root).
+struct DescentTail {
+    int level0 = 0, levels = 0;
+    const int32_t* pos = nullptr;
+};
+
+fff_status_t run_descent(fff_handle_s* h, const void* x, int32_t* leaf_out, Coarse* coarse, int64_t B, cudaStream_t st,
+                         DescentTail* defer_tail = nullptr) {
     fff_status_t s = FFF_OK;
     const int n_dense = dense_stage_count(h, B);
     int level = 0;
@@ -590,7 +598,11 @@ fff_status_t run_descent(fff_handle_s* h, const void* x, int32_t* leaf_out, Coar
         level += sg.k;
         pos = out;
     }
-    if (level < h->depth || h->depth == 0) {
+    if (level < h->depth && defer_tail) {
+        defer_tail->level0 = level;
+        defer_tail->levels = h->depth - level;
+        defer_tail->pos = pos;
+    } else if (level < h->depth || h->depth == 0) {
         s = h->dtype == FFF_DTYPE_F32 ? run_descent_warp<float>(h, x, level, h->depth - level, pos, leaf_out, B, st)
                                       : run_descent_warp<__nv_bfloat16>(h, x, level, h->depth - level, pos, leaf_out, B, st);
     }
@@ -686,14 +698,15 @@ fff_status_t pack_node_images(fff_handle_s* h) {
 
 template <typename T>
 fff_status_t run_leaf(fff_handle_s* h, const void* x, const int32_t* leaf_idx, const int32_t* perm, void* y,
-                      int64_t B, cudaStream_t st) {
+                      int64_t B, cudaStream_t st, const DescentTail& tail = DescentTail(), int32_t* leaf_out = nullptr) {
     const int64_t blocks = std::min<int64_t>((B + fff::kLeafWarps - 1) / fff::kLeafWarps, (int64_t)h->sm_count * 8);
     const size_t smem = sizeof(float) * (size_t)fff::kLeafWarps * h->l;
     if (launch_chain(h, fff::k_leaf_warp<T>, (unsigned)blocks, fff::kLeafWarps * 32, smem, st, 1, (const T*)x, leaf_idx, perm,
                      (const T*)h->w1, (const T*)h->b1, (const T*)h->w2, (const T*)h->b2, (T*)y, h->D, h->O, h->l, h->act, B,
-                     h->vec_ok && aligned16(x)) != cudaSuccess)
+                     h->vec_ok && aligned16(x), (const T*)h->node_w, (const T*)h->node_b, tail.level0, tail.levels, tail.pos,
+                     leaf_out) != cudaSuccess)
         return cudaGetLastError(), FFF_ERR_CUDA;
-    return launched(h, st, "grouped_leaf_ff_warp");
+    return launched(h, st, tail.levels > 0 ? "descent_tail+leaf_ff_warp" : "grouped_leaf_ff_warp");
 }
 
 template <int LP, int TM, int S>
@@ -1065,17 +1078,19 @@ fff_status_t fff_forward_infer(fff_handle_t h, const void* x, void* y, int32_t* 
     const bool lazy_bucketing = !tensor_leaf && B < 4 * h->n_leaves;
     if (lazy_bucketing) leaf = h->ws_leaf;
     Coarse coarse;
-    s = run_descent(h, x, leaf, &coarse, B, st);
+    DescentTail tail;
+    // without a bucketing in between, the warp leaf kernel also walks the levels the staged descent leaves over
+    s = run_descent(h, x, leaf, &coarse, B, st, lazy_bucketing ? &tail : nullptr);
     const LeafPlan plan = tensor_leaf ? leaf_plan(h, B) : LeafPlan{};
     const int tile_rows = plan.tile_rows;
     // the final permutation goes to whichever buffer the last node bucketing did not use
     h->last_perm = coarse.perm == h->ws_perm ? h->ws_perm2 : h->ws_perm;
     h->bucketing_pending = lazy_bucketing;
     if (lazy_bucketing) {
+        if (s == FFF_OK) s = FFF_DISPATCH(h, run_leaf, h, x, leaf, nullptr, y, B, st, tail, leaf);
         if (s == FFF_OK && leaf_idx &&
             cudaMemcpyAsync(leaf_idx, leaf, sizeof(int32_t) * (size_t)B, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
             s = (cudaGetLastError(), FFF_ERR_CUDA);
-        if (s == FFF_OK) s = FFF_DISPATCH(h, run_leaf, h, x, leaf, nullptr, y, B, st);
     } else {
         if (s == FFF_OK)
             s = run_bucket(h, leaf, (int)h->n_leaves, coarse, h->ws_offsets, h->last_perm, B, st, tile_rows, "leaf_bucketing");

@@ -8,6 +8,11 @@
 // weights through L1/L2.  The row of y is written straight to the token's
 // original position, which is the un-permute step.
 //
+// The kernel can also finish the descent first (tail_levels > 0): the warp walks the last levels of the tree
+// from the position the staged descent reached, exactly as k_descent_warp would (same dot product, same
+// comparison), records the leaf index and goes on with that leaf.  With a token per warp and no bucketing in
+// between, this saves a kernel and one pass over x.
+//
 // General path: any D, l, O, both element types, float32 accumulation.  It is
 // the path for float32 layers, for very thin leaves and for buckets of a few
 // tokens, where the work is a gather of weights rather than a contraction.
@@ -25,7 +30,9 @@ template <typename T>
 __global__ void __launch_bounds__(kLeafWarps * 32)
 k_leaf_warp(const T* __restrict__ x, const int32_t* __restrict__ leaf_idx, const int32_t* __restrict__ perm,
             const T* __restrict__ w1, const T* __restrict__ b1, const T* __restrict__ w2, const T* __restrict__ b2,
-            T* __restrict__ y, int D, int O, int l, int act, int64_t B, bool vec)
+            T* __restrict__ y, int D, int O, int l, int act, int64_t B, bool vec,
+            const T* __restrict__ node_w, const T* __restrict__ node_b, int tail_level0, int tail_levels,
+            const int32_t* __restrict__ tail_pos, int32_t* __restrict__ leaf_out)
 {
     extern __shared__ float s_h[];
     pdl_trigger();
@@ -39,8 +46,21 @@ k_leaf_warp(const T* __restrict__ x, const int32_t* __restrict__ leaf_idx, const
 
     for (int64_t i = warp0; i < B; i += nwarps) {
         const int64_t t = perm ? perm[i] : i;
-        const int64_t j = leaf_idx[t];
         const T* xt = x + t * D;
+        int64_t j;
+        if (tail_levels > 0) {
+            // the walk starts at node N_{tail_level0, tail_pos[t]} (position 0 without tail_pos)
+            int64_t n = tail_pos ? tail_pos[t] : 0;
+            for (int m = tail_level0; m < tail_level0 + tail_levels; ++m) {
+                const int64_t row = ((int64_t)1 << m) - 1 + n;
+                const float logit = warp_dot<T>(node_w + row * D, xt, D, vec, lane) + Elem<T>::to_float(node_b[row]);
+                n = 2 * n + (logit >= 0.0f ? 1 : 0);
+            }
+            j = n;
+            if (lane == 0) leaf_out[t] = (int32_t)n;
+        } else {
+            j = leaf_idx[t];
+        }
         const T* w1j = w1 + j * (int64_t)l * D;
         const T* b1j = b1 + j * (int64_t)l;
 
