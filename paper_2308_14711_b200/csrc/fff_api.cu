@@ -701,10 +701,13 @@ fff_status_t run_leaf(fff_handle_s* h, const void* x, const int32_t* leaf_idx, c
                       int64_t B, cudaStream_t st, const DescentTail& tail = DescentTail(), int32_t* leaf_out = nullptr) {
     const int64_t blocks = std::min<int64_t>((B + fff::kLeafWarps - 1) / fff::kLeafWarps, (int64_t)h->sm_count * 8);
     const size_t smem = sizeof(float) * (size_t)fff::kLeafWarps * h->l;
-    if (launch_chain(h, fff::k_leaf_warp<T>, (unsigned)blocks, fff::kLeafWarps * 32, smem, st, 1, (const T*)x, leaf_idx, perm,
-                     (const T*)h->w1, (const T*)h->b1, (const T*)h->w2, (const T*)h->b2, (T*)y, h->D, h->O, h->l, h->act, B,
-                     h->vec_ok && aligned16(x), (const T*)h->node_w, (const T*)h->node_b, tail.level0, tail.levels, tail.pos,
-                     leaf_out) != cudaSuccess)
+    auto launch = [&](auto kern) {
+        return launch_chain(h, kern, (unsigned)blocks, fff::kLeafWarps * 32, smem, st, 1, (const T*)x, leaf_idx, perm,
+                            (const T*)h->w1, (const T*)h->b1, (const T*)h->w2, (const T*)h->b2, (T*)y, h->D, h->O, h->l, h->act, B,
+                            h->vec_ok && aligned16(x), (const T*)h->node_w, (const T*)h->node_b, tail.level0, tail.levels, tail.pos,
+                            leaf_out);
+    };
+    if ((tail.levels > 0 ? launch(fff::k_leaf_warp<T, true>) : launch(fff::k_leaf_warp<T, false>)) != cudaSuccess)
         return cudaGetLastError(), FFF_ERR_CUDA;
     return launched(h, st, tail.levels > 0 ? "descent_tail+leaf_ff_warp" : "grouped_leaf_ff_warp");
 }

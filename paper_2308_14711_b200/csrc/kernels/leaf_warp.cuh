@@ -26,7 +26,8 @@ constexpr int kLeafWarps = 8;
 constexpr int kLeafHiddenUnroll = 4;
 
 // Dynamic shared memory: kLeafWarps * l floats (hidden activations per warp).
-template <typename T>
+// kTail: walk tail_levels levels of the descent first (a separate instantiation keeps the plain kernel lean).
+template <typename T, bool kTail>
 __global__ void __launch_bounds__(kLeafWarps * 32)
 k_leaf_warp(const T* __restrict__ x, const int32_t* __restrict__ leaf_idx, const int32_t* __restrict__ perm,
             const T* __restrict__ w1, const T* __restrict__ b1, const T* __restrict__ w2, const T* __restrict__ b2,
@@ -48,7 +49,7 @@ k_leaf_warp(const T* __restrict__ x, const int32_t* __restrict__ leaf_idx, const
         const int64_t t = perm ? perm[i] : i;
         const T* xt = x + t * D;
         int64_t j;
-        if (tail_levels > 0) {
+        if (kTail) {
             // the walk starts at node N_{tail_level0, tail_pos[t]} (position 0 without tail_pos)
             int64_t n = tail_pos ? tail_pos[t] : 0;
             for (int m = tail_level0; m < tail_level0 + tail_levels; ++m) {
