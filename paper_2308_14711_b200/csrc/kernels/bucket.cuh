@@ -3,19 +3,26 @@
 //   offsets[j]          = number of tokens whose bin is < j      (offsets[nbins] = B)
 //   perm[offsets[j]+r]  = r-th smallest token id with bin j
 //
-// The result is unique, so it is reproduced bit for bit.  No float, no
-// order-dependent atomics: the only atomics are the integer histogram counts,
-// whose sums do not depend on arrival order.
+// The result is unique (tokens of a bin stay in token order), so every kernel here reproduces it bit for
+// bit.  No float, and no atomics whose arrival order could show in the result: the integer sums that
+// some variants accumulate atomically do not depend on it.
 //
-// Decomposition: the bins are split into contiguous ranges, one CTA per range.
-// Every CTA reads all B keys (B * 4 bytes, L2-resident) and places the tokens
-// of its own bins.  Inside the CTA each of the 32 warps owns a contiguous slice
-// of the token ids, so "earlier token" means "earlier warp, or earlier step of
-// the same warp, or lower lane of the same step" -- three orders that are all
-// resolved without communication between CTAs:
-//   pass 1  per-warp, per-bin counts in shared memory;
-//   scan    bin starts from the global histogram, warp starts from the counts;
-//   pass 2  each warp re-reads its slice in order and writes perm.
+// Four implementations of the same sort, chosen by the caller:
+//   k_histogram + k_bucket    two launches; the bins are split into contiguous ranges, one CTA per range
+//                             reads all keys and places the tokens of its bins (the allocation-free
+//                             entry point uses these: their only scratch is the histogram);
+//   k_bucket_cluster          one launch, clusters of 8 CTAs exchange per-CTA counts through distributed
+//                             shared memory; global mode (every cluster scans all keys for its bin range)
+//                             or segmented mode (one cluster per bucket of a previous, coarser bucketing);
+//   k_bucket_coop             one cooperative launch for up to 1024 bins: every CTA ranks one slice of the
+//                             tokens, one grid-wide barrier, column sums over the per-CTA counts;
+//   k_bucket_ranked           after the first descent stage, whose epilogue has already ranked the tokens of
+//                             each 128-token tile: sum of the per-tile counts, scan, scatter; no barrier
+//                             across CTAs.
+// In all of them "earlier token" is resolved hierarchically: earlier slice (tile, CTA, warp), earlier step of
+// the same warp, lower lane of the same step (ballot masks of equal keys).
+// Each can also write the tile list of the grouped kernel that follows: the tiles of bin 0 first, each bin
+// cut into tiles of at most tile_rows consecutive entries, padded with empty tiles to a length the host knows.
 #pragma once
 
 #include <cooperative_groups.h>
