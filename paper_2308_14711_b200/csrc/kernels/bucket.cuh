@@ -636,27 +636,26 @@ constexpr int kRankedThreads = 256;
 constexpr int kRankedWarps = kRankedThreads / 32;
 constexpr int kRankedMaxTilesPerCta = 8;
 
-// Dynamic shared memory: (3 + kRankedMaxTilesPerCta) * nbins ints.
-__global__ void __launch_bounds__(kRankedThreads)
-k_bucket_ranked(const int32_t* __restrict__ keys, const uint8_t* __restrict__ rank8, const uint8_t* __restrict__ counts8,
-                int32_t* __restrict__ offsets_out, int32_t* __restrict__ perm_out, int B, int nbins, int tile_rows,
-                Tile* __restrict__ tiles, int n_tiles_total)
+// The work of one CTA (c of G) of that bucketing, callable from a kernel of its own or as the prologue of a
+// larger one: the first kRankedThreads threads of the CTA work, all its threads must call.
+// s_dyn: (3 + kRankedMaxTilesPerCta) * nbins ints of shared memory, s_warp: 32 ints.
+__device__ __forceinline__ void bucket_ranked_cta(const int32_t* __restrict__ keys, const uint8_t* __restrict__ rank8,
+                                                  const uint8_t* __restrict__ counts8, int32_t* offsets_out, int32_t* perm_out,
+                                                  int B, int nbins, int tile_rows, Tile* tiles, int n_tiles_total, int* s_dyn,
+                                                  int* s_warp, int G, int c)
 {
-    extern __shared__ int s_dyn[];
-    __shared__ int s_warp[32];
     int* s_total = s_dyn;                     // [nbins] tokens in the bin
     int* s_before = s_total + nbins;          // [nbins] of which in tiles before this CTA's
     int* s_start = s_before + nbins;          // [nbins] first position of the bin
     int* s_tile = s_start + nbins;            // [own tiles][nbins] position of the tile's first token of the bin
     const int tid = threadIdx.x;
-    const int G = gridDim.x, c = blockIdx.x;
+    const bool on = tid < kRankedThreads;                  // a larger CTA may call this: its other threads only join the barriers
     const int n_src = (B + kRankTile - 1) / kRankTile;
     const int t0 = (int)((int64_t)c * n_src / G), t1 = (int)((int64_t)(c + 1) * n_src / G);
 
-    pdl_trigger();
-    for (int i = tid; i < 2 * nbins; i += kRankedThreads) s_dyn[i] = 0;
+    if (on)
+        for (int i = tid; i < 2 * nbins; i += kRankedThreads) s_dyn[i] = 0;
     __syncthreads();
-    pdl_wait();
 
     // everything this thread will need later is requested now, so that the L2 round trips overlap:
     // its tokens' keys and ranks, and (thread = bin) the counts of the CTA's own tiles
@@ -667,8 +666,8 @@ k_bucket_ranked(const int32_t* __restrict__ keys, const uint8_t* __restrict__ ra
 #pragma unroll
     for (int i = 0; i < kTok; ++i) {
         const int64_t t = first + tid + i * kRankedThreads;
-        my_key[i] = t < last ? __ldg(keys + t) : -1;
-        my_rank[i] = t < last ? (int)rank8[t] : 0;
+        my_key[i] = on && t < last ? __ldg(keys + t) : -1;
+        my_rank[i] = on && t < last ? (int)rank8[t] : 0;
     }
     int own[kRankedMaxTilesPerCta];
 #pragma unroll
@@ -749,7 +748,8 @@ k_bucket_ranked(const int32_t* __restrict__ keys, const uint8_t* __restrict__ ra
         }
         Tile empty;
         empty.bin = 0; empty.start = 0; empty.rows = 0; empty.pad = 0;
-        for (int i = n_all + tid; i < n_tiles_total; i += kRankedThreads) tiles[i] = empty;
+        if (on)
+            for (int i = n_all + tid; i < n_tiles_total; i += kRankedThreads) tiles[i] = empty;
     }
 
     // place
@@ -759,6 +759,20 @@ k_bucket_ranked(const int32_t* __restrict__ keys, const uint8_t* __restrict__ ra
         const int k = my_key[i];
         if (t < last && k >= 0 && k < nbins) perm_out[s_tile[(int)((t - first) / kRankTile) * nbins + k] + my_rank[i]] = (int32_t)t;
     }
+}
+
+// Dynamic shared memory: (3 + kRankedMaxTilesPerCta) * nbins ints.
+__global__ void __launch_bounds__(kRankedThreads)
+k_bucket_ranked(const int32_t* __restrict__ keys, const uint8_t* __restrict__ rank8, const uint8_t* __restrict__ counts8,
+                int32_t* __restrict__ offsets_out, int32_t* __restrict__ perm_out, int B, int nbins, int tile_rows,
+                Tile* __restrict__ tiles, int n_tiles_total)
+{
+    extern __shared__ int s_dyn[];
+    __shared__ int s_warp[32];
+    pdl_trigger();
+    pdl_wait();
+    bucket_ranked_cta(keys, rank8, counts8, offsets_out, perm_out, B, nbins, tile_rows, tiles, n_tiles_total, s_dyn, s_warp,
+                      (int)gridDim.x, (int)blockIdx.x);
 }
 
 // Tile list from an existing offsets array (one CTA; used when the caller supplies the bucketing),
