@@ -166,9 +166,11 @@ def kernel_bytes(name: str, cfg: wl.FFFConfig, B: int, leaves_touched: int) -> f
     e = cfg.elem_bytes
     if name.startswith("tree_descent"):
         return B * cfg.D * e + cfg.n_nodes * (cfg.D + 1) * e + 4 * B
+    if name.startswith("leaf_bucketing+grouped_leaf_ff"):      # bucketing done by the leaf kernel's prologue
+        return 8 * B + 8 * cfg.n_leaves + kernel_bytes("grouped_leaf_ff", cfg, B, leaves_touched)
     if name.startswith("leaf_bucketing") or name.startswith("leaf_histogram"):
         return 8 * B + 8 * cfg.n_leaves
-    if name.startswith("grouped_leaf_ff"):
+    if name.startswith("grouped_leaf_ff") or name.startswith("descent_tail+leaf_ff"):   # the tail's node rows: O(B) more
         return B * (cfg.D + cfg.O) * e + leaves_touched * leaf_param_bytes(cfg) + 8 * B
     return 0.0
 

@@ -730,16 +730,16 @@ fff_status_t launch_leaf_mma(fff_handle_s* h, const void* x, const int32_t* perm
     return launched(h, st, "grouped_leaf_ff_mma");
 }
 
-template <int LP, bool kFold, bool kFused>
+template <int LP, bool kFold>
 fff_status_t launch_leaf_umma(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, int tile_rows,
-                              cudaStream_t st, const fff::FusedBucketArgs& fb) {
+                              cudaStream_t st) {
     using L = fff::LeafUmmaLayout<LP>;
     const int n_tiles = tile_list_len(B, tile_rows, (int)h->n_leaves);
     const int stages = std::min((int)fff::kLUMaxStages, (kSmemBudget - L::smem_bytes(0)) / L::kStageBytes);
     if (stages < 2) return FFF_ERR_UNSUPPORTED;
     static bool attr_set[64] = {};
     if (h->device < 64 && !attr_set[h->device]) {
-        cudaFuncSetAttribute(fff::k_leaf_umma<LP, kFold, kFused>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+        cudaFuncSetAttribute(fff::k_leaf_umma<LP, kFold>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
         attr_set[h->device] = true;
     }
     CUtensorMap tm;
@@ -747,7 +747,7 @@ fff_status_t launch_leaf_umma(fff_handle_s* h, const void* x, const int32_t* per
     const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(h->sm_count, n_tiles));
     const int wide = (reinterpret_cast<uintptr_t>(y) & 31u) == 0 ? 1 : 0;
     const int passes = 1;      // two passes (full tiles first) measured slightly slower
-    if (launch_chain(h, fff::k_leaf_umma<LP, kFold, kFused>, (unsigned)grid, fff::kLUThreads, (size_t)L::smem_bytes(stages), st, 1, tm, fb, perm,
+    if (launch_chain(h, fff::k_leaf_umma<LP, kFold>, (unsigned)grid, fff::kLUThreads, (size_t)L::smem_bytes(stages), st, 1, tm, perm,
                      (const fff::Tile*)h->ws_tiles, n_tiles, (const __nv_bfloat16*)h->w1img, (const float*)h->b1img,
                      (const unsigned char*)h->w2uimg, (__nv_bfloat16*)y, h->D, h->O, h->l, h->act, stages, wide, passes, h->ws_sched,
                      h->d_status) != cudaSuccess)
@@ -755,27 +755,18 @@ fff_status_t launch_leaf_umma(fff_handle_s* h, const void* x, const int32_t* per
     return launched(h, st, "grouped_leaf_ff_umma");
 }
 
-template <int LP>
-fff_status_t leaf_umma_variant(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, int tile_rows,
-                               cudaStream_t st, const fff::FusedBucketArgs* fused) {
-    const fff::FusedBucketArgs none = {};
-    if (fused)
-        return h->l < LP ? launch_leaf_umma<LP, true, true>(h, x, perm, y, B, tile_rows, st, *fused)
-                         : launch_leaf_umma<LP, false, true>(h, x, perm, y, B, tile_rows, st, *fused);
-    return h->l < LP ? launch_leaf_umma<LP, true, false>(h, x, perm, y, B, tile_rows, st, none)
-                     : launch_leaf_umma<LP, false, false>(h, x, perm, y, B, tile_rows, st, none);
-}
-
 // Ring depth per (LP, TM): what fits twice into an SM's shared memory (once for LP = 64).
-// fused != NULL: the tcgen05 kernel makes the leaf bucketing itself (see fused_bucket_ok).
 fff_status_t run_leaf_mma(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, const LeafPlan& plan,
-                          cudaStream_t st, const fff::FusedBucketArgs* fused = nullptr) {
+                          cudaStream_t st) {
     const int tile_rows = plan.tile_rows;
     if (plan.umma && h->w2uimg) {
         switch (h->LP) {
-            case 16: return leaf_umma_variant<16>(h, x, perm, y, B, tile_rows, st, fused);
-            case 32: return leaf_umma_variant<32>(h, x, perm, y, B, tile_rows, st, fused);
-            case 64: return leaf_umma_variant<64>(h, x, perm, y, B, tile_rows, st, fused);
+            case 16: return h->l < 16 ? launch_leaf_umma<16, true>(h, x, perm, y, B, tile_rows, st)
+                                      : launch_leaf_umma<16, false>(h, x, perm, y, B, tile_rows, st);
+            case 32: return h->l < 32 ? launch_leaf_umma<32, true>(h, x, perm, y, B, tile_rows, st)
+                                      : launch_leaf_umma<32, false>(h, x, perm, y, B, tile_rows, st);
+            case 64: return h->l < 64 ? launch_leaf_umma<64, true>(h, x, perm, y, B, tile_rows, st)
+                                      : launch_leaf_umma<64, false>(h, x, perm, y, B, tile_rows, st);
         }
     }
     if (tile_rows == 32) {
@@ -813,7 +804,7 @@ fff_status_t pack_leaf_images(fff_handle_s* h) {
     if (encode_tiled_fn() && h->O % 16 == 0 && h->D % fff::kLUKB == 0 && std::getenv("FFF_NO_UMMA_LEAF") == nullptr) {
         const size_t P = (size_t)(h->O + fff::kLUPiece - 1) / fff::kLUPiece;
         if ((s = dmalloc((void**)&h->w2uimg, nl * P * ((size_t)fff::kLUPiece * LP * 2 + fff::kLUPiece * 4))) != FFF_OK) return s;
-        if ((s = clone((void**)&h->ws_sched, nullptr, 4 * sizeof(int))) != FFF_OK) return s;
+        if ((s = clone((void**)&h->ws_sched, nullptr, 2 * sizeof(int))) != FFF_OK) return s;
         fff::k_pack_w2_umma<T><<<blocks, 256>>>((const T*)h->w2, (const T*)h->b2, h->w2uimg, (int)nl, h->l, LP, h->O);
         if (cudaGetLastError() != cudaSuccess) return FFF_ERR_CUDA;
     }
@@ -1104,19 +1095,10 @@ fff_status_t fff_forward_infer(fff_handle_t h, const void* x, void* y, int32_t* 
             cudaMemcpyAsync(leaf_idx, leaf, sizeof(int32_t) * (size_t)B, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
             s = (cudaGetLastError(), FFF_ERR_CUDA);
     } else {
-        // After a one-stage tcgen05 descent the leaf kernel can do the (ranked) bucketing as its own prologue.
-        static const bool no_fused = std::getenv("FFF_NO_FUSED_BUCKET") != nullptr;      // tuning aid
-        const int64_t n_src = (B + fff::kRankTile - 1) / fff::kRankTile;
-        const int64_t leaf_ctas = std::min<int64_t>(h->sm_count, tile_list_len(B, fff::kLUM, (int)h->n_leaves));
-        const bool fuse = !no_fused && !h->prof_active && tensor_leaf && plan.umma && plan.tile_rows == fff::kLUM && coarse.ranked &&
-                          !coarse.perm && h->n_leaves >= 16 && h->n_leaves <= 256 &&
-                          (n_src + leaf_ctas - 1) / leaf_ctas <= fff::kRankedMaxTilesPerCta;
-        const fff::FusedBucketArgs fb = {leaf, h->ws_rank8, h->ws_counts8, h->ws_offsets, h->last_perm, h->ws_tiles, (int)B,
-                                         (int)h->n_leaves};
-        if (s == FFF_OK && !fuse)
+        if (s == FFF_OK)
             s = run_bucket(h, leaf, (int)h->n_leaves, coarse, h->ws_offsets, h->last_perm, B, st, tile_rows, "leaf_bucketing");
         if (s == FFF_OK)
-            s = tensor_leaf ? run_leaf_mma(h, x, h->last_perm, y, B, plan, st, fuse ? &fb : nullptr)
+            s = tensor_leaf ? run_leaf_mma(h, x, h->last_perm, y, B, plan, st)
                             : FFF_DISPATCH(h, run_leaf, h, x, leaf, h->last_perm, y, B, st);
     }
     if (h->prof_active) {

@@ -43,7 +43,6 @@
 
 #include <cuda.h>      // CUtensorMap
 
-#include "bucket.cuh"
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -128,29 +127,13 @@ __global__ void k_pack_w2_umma(const T* __restrict__ w2, const T* __restrict__ b
     }
 }
 
-// What the kernel needs to make the leaf bucketing itself (kFusedBucket): the first descent stage's keys, ranks
-// and per-tile counts, and where offsets, permutation and tile list go.
-struct FusedBucketArgs {
-    const int32_t* keys;
-    const uint8_t* rank8;
-    const uint8_t* counts8;
-    int32_t* offsets_out;
-    int32_t* perm_out;
-    Tile* tiles_out;
-    int B, nbins;
-};
-
-// sched: three ints, all zero before the first launch and again after every launch: [0] list entries
-// handed out so far, [1] CTAs that have finished, [2] CTAs that have finished the bucketing prologue.
+// sched: two ints, both zero before the first launch and again after every launch: [0] list entries
+// handed out so far, [1] CTAs that have finished.
 // kFold: l < LP, the spare hidden column l carries the output bias (see k_pack_w2_umma).
-// kFusedBucket: the kernel first does the work of k_bucket_ranked (every CTA its share, then one barrier across
-// the grid: all CTAs are resident, one per SM, and the wait is bounded like every other), which saves a launch
-// and the latency of a kernel that moves a few hundred kilobytes.  perm and tiles are then this kernel's own
-// output (fb.perm_out, fb.tiles_out) and are read with ordinary, coherent loads.
-template <int LP, bool kFold, bool kFusedBucket>
+template <int LP, bool kFold>
 __global__ void __launch_bounds__(kLUThreads, 1)
-k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const FusedBucketArgs fb, const int32_t* __restrict__ perm_in,
-            const Tile* __restrict__ tiles_in, int n_tiles_total,
+k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restrict__ perm,
+            const Tile* __restrict__ tiles, int n_tiles_total,
             const __nv_bfloat16* __restrict__ w1img, const float* __restrict__ b1img,
             const unsigned char* __restrict__ w2img, __nv_bfloat16* __restrict__ y,
             int D, int O, int l, int act, int kStages, int wide_stores, int passes, int* __restrict__ sched,
@@ -217,30 +200,6 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const FusedBucketArgs fb
 
     bool timed_out = false;
     const int max_iters = n_tiles_total + kLUQueue + 1;     // no role loops longer than this, whatever it reads
-    const int32_t* perm = kFusedBucket ? static_cast<const int32_t*>(fb.perm_out) : perm_in;
-    const Tile* tiles = kFusedBucket ? static_cast<const Tile*>(fb.tiles_out) : tiles_in;
-    if (kFusedBucket) {
-        __shared__ int s_warp[32];
-        // the ring is idle until the gathers start: its first kilobytes serve as the bucketing's scratch
-        bucket_ranked_cta(fb.keys, fb.rank8, fb.counts8, fb.offsets_out, fb.perm_out, fb.B, fb.nbins, kLUM, fb.tiles_out,
-                          n_tiles_total, reinterpret_cast<int*>(ring), s_warp, (int)gridDim.x, (int)blockIdx.x);
-        __threadfence();
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            unsigned* bar = reinterpret_cast<unsigned*>(sched + 2);
-            atomicAdd(bar, 1u);
-            const long long t0 = clock64();
-            while (ptx::ld_acquire_gpu(bar) < gridDim.x) {
-                __nanosleep(100);
-                if (clock64() - t0 > ptx::kWaitCycles) {
-                    atomicExch(status, kDevTimeout);
-                    break;
-                }
-            }
-            __threadfence();
-        }
-        __syncthreads();
-    }
 
     // Consumers take the tiles in the order the scheduler published them; rows < 0 ends the sequence.
     int q_slot = 0;
@@ -528,7 +487,6 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const FusedBucketArgs fb
         if (atomicAdd(sched + 1, 1) == (int)gridDim.x - 1) {
             sched[0] = 0;
             sched[1] = 0;
-            sched[2] = 0;
             __threadfence();
         }
     }
