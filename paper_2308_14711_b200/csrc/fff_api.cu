@@ -22,6 +22,7 @@
 #include "kernels/descent_warp.cuh"
 #include "kernels/leaf_mma.cuh"
 #include "kernels/leaf_umma.cuh"
+#include "kernels/leaf_umma_packed.cuh"
 #include "kernels/leaf_warp.cuh"
 
 namespace {
@@ -57,6 +58,7 @@ struct fff_handle_s {
     __nv_bfloat16* w1img = nullptr;
     float* b1img = nullptr;
     unsigned char* w2img = nullptr;
+    bool w2_finite = false;            // every W2 and b2 entry is finite (leaves may then share a tile, see leaf_umma_packed.cuh)
     unsigned char* w2uimg = nullptr;   // W2 pieces (+ biases) of the tcgen05 leaf kernel (nullptr = kernel not available)
     int* ws_sched = nullptr;           // its tile counter and finished-CTA counter (zero between launches)
     fff::Tile* ws_tiles = nullptr;
@@ -213,7 +215,10 @@ size_t max_tiles(const fff_handle_s* h, int64_t B) { return (size_t)(B / kMinTil
 struct LeafPlan {
     int tile_rows = 0;
     bool umma = false;
+    int pack = 1;          // leaves per 128-row tile of the tcgen05 kernel (tile_rows = 128 / pack)
 };
+
+bool leaf_pack_fits(int LP, int pack);
 
 LeafPlan leaf_plan(const fff_handle_s* h, int64_t B) {
     static const int forced = [] {
@@ -230,10 +235,22 @@ LeafPlan leaf_plan(const fff_handle_s* h, int64_t B) {
             const int v = e ? std::atoi(e) : 0;
             return (v >= 4 && v <= fff::kLUM && v % 4 == 0) ? v : 0;
         }();
-        return LeafPlan{umma_rows ? umma_rows : fff::kLUM, true};
+        // Thin buckets: several leaves share the rows of a tile.  Sub-tiles of 64 rows while most buckets fit into
+        // one, of 32 rows below that.
+        static const int forced_pack = [] {
+            const char* e = std::getenv("FFF_LEAF_PACK");       // tuning aid: 1, 2 or 4
+            const int v = e ? std::atoi(e) : 0;
+            return (v == 1 || v == 2 || v == 4) ? v : 0;
+        }();
+        const int64_t avg = B / h->n_leaves;
+        int pack = forced_pack ? forced_pack : avg >= 96 ? 1 : avg >= 24 ? 2 : 4;
+        if (!h->w2_finite || umma_rows) pack = 1;
+        while (pack > 1 && !leaf_pack_fits(h->LP, pack)) pack >>= 1;
+        if (pack > 1) return LeafPlan{fff::kLUM / pack, true, pack};
+        return LeafPlan{umma_rows ? umma_rows : fff::kLUM, true, 1};
     }
-    if (forced) return LeafPlan{forced, false};
-    return LeafPlan{B / h->n_leaves <= 40 ? 32 : 64, false};
+    if (forced) return LeafPlan{forced, false, 1};
+    return LeafPlan{B / h->n_leaves <= 40 ? 32 : 64, false, 1};
 }
 
 bool use_tensor_leaf(const fff_handle_s* h) {
@@ -755,10 +772,69 @@ fff_status_t launch_leaf_umma(fff_handle_s* h, const void* x, const int32_t* per
     return launched(h, st, "grouped_leaf_ff_umma");
 }
 
+template <int LP, int G>
+int leaf_pack_stages() {
+    using L = fff::LeafPackLayout<LP, G>;
+    return std::min((int)fff::kLUMaxStages, (kSmemBudget - L::smem_bytes(0)) / L::kStageBytes);
+}
+
+// Whether the kernel that packs `pack` leaves into a tile has room for a ring of at least three stages.
+bool leaf_pack_fits(int LP, int pack) {
+    int st = 0;
+    switch (LP * 8 + pack) {
+        case 16 * 8 + 2: st = leaf_pack_stages<16, 2>(); break;
+        case 16 * 8 + 4: st = leaf_pack_stages<16, 4>(); break;
+        case 32 * 8 + 2: st = leaf_pack_stages<32, 2>(); break;
+        case 32 * 8 + 4: st = leaf_pack_stages<32, 4>(); break;
+        case 64 * 8 + 2: st = leaf_pack_stages<64, 2>(); break;
+        default: break;                                        // (64, 4) does not fit
+    }
+    return st >= 3;
+}
+
+template <int LP, bool kFold, int G>
+fff_status_t launch_leaf_umma_packed(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, cudaStream_t st) {
+    using L = fff::LeafPackLayout<LP, G>;
+    const int n_tiles = tile_list_len(B, L::kSubRows, (int)h->n_leaves);
+    const int stages = leaf_pack_stages<LP, G>();
+    if (stages < 3) return FFF_ERR_UNSUPPORTED;
+    static bool attr_set[64] = {};
+    if (h->device < 64 && !attr_set[h->device]) {
+        cudaFuncSetAttribute(fff::k_leaf_umma_packed<LP, kFold, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+        attr_set[h->device] = true;
+    }
+    CUtensorMap tm;
+    if (!make_x_tensor_map(&tm, x, B, h->D, 1)) return FFF_ERR_CUDA;       // one-row boxes: rows are gathered four at a time
+    const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(h->sm_count, (n_tiles + G - 1) / G));
+    const int wide = (reinterpret_cast<uintptr_t>(y) & 31u) == 0 ? 1 : 0;
+    if (launch_chain(h, fff::k_leaf_umma_packed<LP, kFold, G>, (unsigned)grid, fff::kLUThreads, (size_t)L::smem_bytes(stages), st, 1, tm,
+                     perm, (const fff::Tile*)h->ws_tiles, n_tiles, (const __nv_bfloat16*)h->w1img, (const float*)h->b1img,
+                     (const unsigned char*)h->w2uimg, (__nv_bfloat16*)y, h->D, h->O, h->l, h->act, stages, wide, h->ws_sched,
+                     h->d_status) != cudaSuccess)
+        return cudaGetLastError(), FFF_ERR_CUDA;
+    return launched(h, st, "grouped_leaf_ff_umma_packed");
+}
+
+template <int LP, int G>
+fff_status_t leaf_umma_packed_variant(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, cudaStream_t st) {
+    return h->l < LP ? launch_leaf_umma_packed<LP, true, G>(h, x, perm, y, B, st)
+                     : launch_leaf_umma_packed<LP, false, G>(h, x, perm, y, B, st);
+}
+
 // Ring depth per (LP, TM): what fits twice into an SM's shared memory (once for LP = 64).
 fff_status_t run_leaf_mma(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, const LeafPlan& plan,
                           cudaStream_t st) {
     const int tile_rows = plan.tile_rows;
+    if (plan.umma && h->w2uimg && plan.pack > 1) {
+        switch (h->LP * 8 + plan.pack) {
+            case 16 * 8 + 2: return leaf_umma_packed_variant<16, 2>(h, x, perm, y, B, st);
+            case 16 * 8 + 4: return leaf_umma_packed_variant<16, 4>(h, x, perm, y, B, st);
+            case 32 * 8 + 2: return leaf_umma_packed_variant<32, 2>(h, x, perm, y, B, st);
+            case 32 * 8 + 4: return leaf_umma_packed_variant<32, 4>(h, x, perm, y, B, st);
+            case 64 * 8 + 2: return leaf_umma_packed_variant<64, 2>(h, x, perm, y, B, st);
+        }
+        return FFF_ERR_UNSUPPORTED;
+    }
     if (plan.umma && h->w2uimg) {
         switch (h->LP) {
             case 16: return h->l < 16 ? launch_leaf_umma<16, true>(h, x, perm, y, B, tile_rows, st)
@@ -804,9 +880,12 @@ fff_status_t pack_leaf_images(fff_handle_s* h) {
     if (encode_tiled_fn() && h->O % 16 == 0 && h->D % fff::kLUKB == 0 && std::getenv("FFF_NO_UMMA_LEAF") == nullptr) {
         const size_t P = (size_t)(h->O + fff::kLUPiece - 1) / fff::kLUPiece;
         if ((s = dmalloc((void**)&h->w2uimg, nl * P * ((size_t)fff::kLUPiece * LP * 2 + fff::kLUPiece * 4))) != FFF_OK) return s;
-        if ((s = clone((void**)&h->ws_sched, nullptr, 2 * sizeof(int))) != FFF_OK) return s;
-        fff::k_pack_w2_umma<T><<<blocks, 256>>>((const T*)h->w2, (const T*)h->b2, h->w2uimg, (int)nl, h->l, LP, h->O);
+        if ((s = clone((void**)&h->ws_sched, nullptr, 4 * sizeof(int))) != FFF_OK) return s;
+        fff::k_pack_w2_umma<T><<<blocks, 256>>>((const T*)h->w2, (const T*)h->b2, h->w2uimg, (int)nl, h->l, LP, h->O, h->ws_sched + 3);
         if (cudaGetLastError() != cudaSuccess) return FFF_ERR_CUDA;
+        int nonfinite = 1;
+        if (cudaMemcpy(&nonfinite, h->ws_sched + 3, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
+        h->w2_finite = nonfinite == 0;
     }
     return cudaGetLastError() == cudaSuccess ? FFF_OK : FFF_ERR_CUDA;
 }

@@ -35,6 +35,8 @@
 //
 // Rows of a ragged tile beyond its length are not loaded: their accumulator rows hold garbage that is
 // never stored (rows of an MMA are independent).
+// Thin buckets (a few dozen tokens per leaf) go to k_leaf_umma_packed instead, which stacks several leaves in
+// the rows of one tile.
 //
 // Every wait is bounded (see ptx.cuh); tensor memory is released on every exit path.
 //
@@ -103,7 +105,7 @@ __host__ __device__ __forceinline__ uint32_t swz_rows(uint32_t off, int row_byte
 // then the 128 float32 biases of those features }.
 template <typename T>
 __global__ void k_pack_w2_umma(const T* __restrict__ w2, const T* __restrict__ b2, unsigned char* __restrict__ img,
-                               int n_leaves, int l, int LP, int O)
+                               int n_leaves, int l, int LP, int O, int* __restrict__ nonfinite)
 {
     const int P = (O + kLUPiece - 1) / kLUPiece;
     const int64_t piece_bytes = (int64_t)kLUPiece * LP * 2 + kLUPiece * 4;
@@ -120,9 +122,12 @@ __global__ void k_pack_w2_umma(const T* __restrict__ w2, const T* __restrict__ b
             // b2 by itself and the epilogue has no bias to fetch and add (b2 is bf16 already: exact)
             float v = (o < O && c < l) ? Elem<T>::to_float(w2[(j * O + o) * (int64_t)l + c]) : 0.0f;
             if (c == l && o < O) v = Elem<T>::to_float(b2[j * O + o]);
+            if (!isfinite(v)) atomicOr(nonfinite, 1);            // (the kernel that packs several leaves into a tile needs to know)
             *reinterpret_cast<__nv_bfloat16*>(piece + swz_rows((uint32_t)(n * LP * 2 + c * 2), LP * 2)) = __float2bfloat16_rn(v);
         } else {
-            reinterpret_cast<float*>(piece + (int64_t)kLUPiece * LP * 2)[n] = o < O ? Elem<T>::to_float(b2[j * O + o]) : 0.0f;
+            const float v = o < O ? Elem<T>::to_float(b2[j * O + o]) : 0.0f;
+            if (!isfinite(v)) atomicOr(nonfinite, 1);
+            reinterpret_cast<float*>(piece + (int64_t)kLUPiece * LP * 2)[n] = v;
         }
     }
 }

@@ -200,6 +200,47 @@ def test_gpu_argument_errors_are_reported_not_faulted():
     torch.cuda.synchronize()
 
 
+@pytest.mark.parametrize("B,depth,l", [(3000, 6, 32), (1200, 6, 12), (9000, 7, 64)])
+def test_thin_buckets_share_a_tile(B, depth, l):
+    """A few dozen tokens per leaf: the tcgen05 leaf kernel stacks two or four leaves in the rows of one tile.
+    Two calls (the scheduler words rearm themselves), both GELU-free and GELU paths via the shapes' activations."""
+    cfg = wl.FFFConfig("bf16_packed", 256, 272, depth, l, "gelu" if l != 12 else "relu", "bf16", B, "normal")
+    case = util.make_case(cfg, seed=5)
+    y_ref, leaf_ref = orc.forward_i(case.net, case.x, threads=util.ORACLE_THREADS)
+    layer = util.make_layer(case)
+    x = util.to_device(case.x, "bf16")
+    for _ in range(2):
+        y, leaf = layer.forward_infer(x)
+        torch.cuda.synchronize()
+        np.testing.assert_array_equal(leaf.cpu().numpy(), leaf_ref)
+        util.check_outputs(y, y_ref, "bf16")
+        assert layer.last_status() == 0
+    layer.close()
+
+
+def test_nonfinite_leaf_weights_stay_in_their_leaf():
+    """Infinite output weights in one leaf make that leaf's tokens non-finite and leave every other token's
+    result as the oracle has it (leaves that share a tile must not see each other's weights)."""
+    cfg = wl.FFFConfig("bf16_inf_leaf", 128, 144, 5, 16, "gelu", "bf16", 1500, "normal")
+    case = util.make_case(cfg, seed=2)
+    bad = int(np.bincount(orc.forward_i(case.net, case.x, threads=util.ORACLE_THREADS)[1], minlength=32).argmax())
+    case.weights["w2"][bad, :, :] = np.inf
+    case.net = orc.Net.from_config(cfg, case.weights)
+    with np.errstate(all="ignore"):
+        y_ref, leaf_ref = orc.forward_i(case.net, case.x, threads=util.ORACLE_THREADS)
+    layer = util.make_layer(case)
+    y, leaf = layer.forward_infer(util.to_device(case.x, "bf16"))
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(leaf.cpu().numpy(), leaf_ref)
+    hit = leaf_ref == bad
+    assert hit.any() and not hit.all()
+    assert not np.isfinite(y_ref[hit]).all(axis=1).any()
+    assert not torch.isfinite(y[torch.from_numpy(hit).cuda()].float()).all(dim=1).any()
+    rows = np.nonzero(~hit)[0]
+    util.check_outputs(y, y_ref[rows], "bf16", rows=rows)
+    layer.close()
+
+
 def test_nan_inputs_stay_in_range():
     cfg = wl.FFFConfig("n", 64, 32, 4, 8, "gelu", "bf16", 64)
     case = util.make_case(cfg, 0)
