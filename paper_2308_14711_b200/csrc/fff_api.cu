@@ -58,6 +58,7 @@ struct fff_handle_s {
     __nv_bfloat16* w1img = nullptr;
     float* b1img = nullptr;
     unsigned char* w2img = nullptr;
+    int leaf_pack = 1;                 // fff_set_leaf_packing: 1 off, 2 / 4 leaves per tile, 0 chosen from B / n_leaves
     bool w2_finite = false;            // every W2 and b2 entry is finite (leaves may then share a tile, see leaf_umma_packed.cuh)
     unsigned char* w2uimg = nullptr;   // W2 pieces (+ biases) of the tcgen05 leaf kernel (nullptr = kernel not available)
     int* ws_sched = nullptr;           // its tile counter and finished-CTA counter (zero between launches)
@@ -235,15 +236,16 @@ LeafPlan leaf_plan(const fff_handle_s* h, int64_t B) {
             const int v = e ? std::atoi(e) : 0;
             return (v >= 4 && v <= fff::kLUM && v % 4 == 0) ? v : 0;
         }();
-        // Thin buckets: several leaves share the rows of a tile.  Sub-tiles of 64 rows while most buckets fit into
-        // one, of 32 rows below that.
+        // Thin buckets: several leaves may share the rows of a tile (fff_set_leaf_packing; off unless asked for,
+        // because it loses when a few buckets hold most tokens, which the host cannot know here).
         static const int forced_pack = [] {
             const char* e = std::getenv("FFF_LEAF_PACK");       // tuning aid: 1, 2 or 4
             const int v = e ? std::atoi(e) : 0;
             return (v == 1 || v == 2 || v == 4) ? v : 0;
         }();
         const int64_t avg = B / h->n_leaves;
-        int pack = forced_pack ? forced_pack : avg >= 96 ? 1 : avg >= 24 ? 2 : 4;
+        const int by_size = avg >= 96 ? 1 : avg >= 24 ? 2 : 4;
+        int pack = forced_pack ? forced_pack : h->leaf_pack == 0 ? by_size : h->leaf_pack;
         if (!h->w2_finite || umma_rows) pack = 1;
         while (pack > 1 && !leaf_pack_fits(h->LP, pack)) pack >>= 1;
         if (pack > 1) return LeafPlan{fff::kLUM / pack, true, pack};
@@ -1092,6 +1094,13 @@ fff_status_t fff_set_path(fff_handle_t h, fff_path_t path) {
     if (path != FFF_PATH_AUTO && path != FFF_PATH_WARP && path != FFF_PATH_TENSOR) return FFF_ERR_INVALID_ARG;
     if (path == FFF_PATH_TENSOR && h->LP == 0 && h->stages.empty()) return FFF_ERR_UNSUPPORTED;
     h->path = path;
+    return FFF_OK;
+}
+
+fff_status_t fff_set_leaf_packing(fff_handle_t h, int leaves) {
+    if (!live(h)) return FFF_ERR_BAD_HANDLE;
+    if (leaves != 0 && leaves != 1 && leaves != 2 && leaves != 4) return FFF_ERR_INVALID_ARG;
+    h->leaf_pack = leaves;
     return FFF_OK;
 }
 

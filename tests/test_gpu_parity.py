@@ -200,21 +200,30 @@ def test_gpu_argument_errors_are_reported_not_faulted():
     torch.cuda.synchronize()
 
 
-@pytest.mark.parametrize("B,depth,l", [(3000, 6, 32), (1200, 6, 12), (9000, 7, 64)])
-def test_thin_buckets_share_a_tile(B, depth, l):
-    """A few dozen tokens per leaf: the tcgen05 leaf kernel stacks two or four leaves in the rows of one tile.
-    Two calls (the scheduler words rearm themselves), both GELU-free and GELU paths via the shapes' activations."""
-    cfg = wl.FFFConfig("bf16_packed", 256, 272, depth, l, "gelu" if l != 12 else "relu", "bf16", B, "normal")
+@pytest.mark.parametrize("B,depth,l,x_kind", [(3000, 6, 32, "normal"), (1200, 6, 12, "normal"), (9000, 7, 64, "normal"),
+                                              (6000, 7, 16, "clusters")])
+@pytest.mark.parametrize("leaves", [0, 2, 4])
+def test_thin_buckets_share_a_tile(B, depth, l, x_kind, leaves):
+    """Leaf packing: two or four leaves in the rows of one tcgen05 tile (0: chosen from the average bucket size).
+    Same results as with one leaf per tile, bit for bit; two calls each (the scheduler words rearm themselves).
+    The clustered inputs give buckets of several sub-tiles next to empty ones."""
+    cfg = wl.FFFConfig("bf16_packed", 256, 272, depth, l, "gelu" if l != 12 else "relu", "bf16", B, x_kind)
     case = util.make_case(cfg, seed=5)
     y_ref, leaf_ref = orc.forward_i(case.net, case.x, threads=util.ORACLE_THREADS)
     layer = util.make_layer(case)
     x = util.to_device(case.x, "bf16")
+    y_one, _ = layer.forward_infer(x)
+    layer.set_leaf_packing(leaves)
     for _ in range(2):
         y, leaf = layer.forward_infer(x)
         torch.cuda.synchronize()
         np.testing.assert_array_equal(leaf.cpu().numpy(), leaf_ref)
         util.check_outputs(y, y_ref, "bf16")
+        assert torch.equal(y, y_one)
         assert layer.last_status() == 0
+    layer.set_leaf_packing(1)
+    with pytest.raises(Exception):
+        layer.set_leaf_packing(3)
     layer.close()
 
 
@@ -229,6 +238,7 @@ def test_nonfinite_leaf_weights_stay_in_their_leaf():
     with np.errstate(all="ignore"):
         y_ref, leaf_ref = orc.forward_i(case.net, case.x, threads=util.ORACLE_THREADS)
     layer = util.make_layer(case)
+    layer.set_leaf_packing(2)                       # asked for, but not taken: the weights are not all finite
     y, leaf = layer.forward_infer(util.to_device(case.x, "bf16"))
     torch.cuda.synchronize()
     np.testing.assert_array_equal(leaf.cpu().numpy(), leaf_ref)
