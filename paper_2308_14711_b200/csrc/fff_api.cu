@@ -70,6 +70,9 @@ struct fff_handle_s {
     int32_t* ws_rank = nullptr;   // per-token rank scratch of the bucketing kernel (large batches only)
     uint8_t* ws_rank8 = nullptr;  // rank of every token inside its 128-token tile, left by the first descent stage
     uint8_t* ws_counts8 = nullptr;   // and that stage's per-tile counts, [ceil(B/128)][<= 256]
+    int32_t* ws_blocksum = nullptr;  // [4] CTA counter of k_bucket_ranked, then the counts summed over blocks of 16 tiles
+    size_t blocksum_bytes = 0;
+    bool blocksum_dirty = false;     // a descent has added to the table and no ranked bucketing has cleared it since
     int max_bucket_clusters = 8;
     int32_t* last_perm = nullptr; // where the most recent forward left its leaf permutation
     bool bucketing_pending = false;   // the last forward skipped the leaf bucketing; ws_leaf holds its leaf indices
@@ -190,7 +193,7 @@ void release(fff_handle_s* h) {
     for (auto& sg : h->stages) { dfree(sg.wimg); dfree(sg.bimg); }
     for (auto& sg : h->ustages) { dfree(sg.wimg); dfree(sg.bimg); }
     dfree(h->ws_pos[0]); dfree(h->ws_pos[1]);
-    dfree(h->w1img); dfree(h->b1img); dfree(h->w2img); dfree(h->w2uimg); dfree(h->ws_sched); dfree(h->ws_tiles); dfree(h->ws_rank); dfree(h->ws_rank8); dfree(h->ws_counts8); dfree(h->ws_matrix);
+    dfree(h->w1img); dfree(h->b1img); dfree(h->w2img); dfree(h->w2uimg); dfree(h->ws_sched); dfree(h->ws_tiles); dfree(h->ws_rank); dfree(h->ws_rank8); dfree(h->ws_counts8); dfree(h->ws_blocksum); dfree(h->ws_matrix);
     if (h->copy_in) cudaStreamDestroy(h->copy_in);
     if (h->copy_out) cudaStreamDestroy(h->copy_out);
     for (int i = 0; i < fff_handle_s::kMaxHostChunks; ++i) {
@@ -264,8 +267,9 @@ fff_status_t grow_workspace(fff_handle_s* h, int64_t B) {
     if (B <= h->cap_B) return FFF_OK;
     if (cudaDeviceSynchronize() != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
     dfree(h->ws_leaf); dfree(h->ws_perm); dfree(h->ws_perm2); dfree(h->ws_tiles); dfree(h->ws_rank); dfree(h->ws_pos[0]);
-    dfree(h->ws_rank8); dfree(h->ws_counts8);
+    dfree(h->ws_rank8); dfree(h->ws_counts8); dfree(h->ws_blocksum);
     h->ws_rank8 = h->ws_counts8 = nullptr;
+    h->ws_blocksum = nullptr;
     dfree(h->ws_pos[1]);
     h->ws_leaf = h->ws_perm = h->ws_perm2 = h->ws_rank = h->ws_pos[0] = h->ws_pos[1] = nullptr;
     h->ws_tiles = nullptr;
@@ -278,6 +282,9 @@ fff_status_t grow_workspace(fff_handle_s* h, int64_t B) {
     if (!h->ustages.empty()) {
         if ((s = dmalloc((void**)&h->ws_rank8, (size_t)B)) != FFF_OK) return s;
         if ((s = dmalloc((void**)&h->ws_counts8, (size_t)((B + 127) / 128) * 256)) != FFF_OK) return s;
+        h->blocksum_bytes = sizeof(int32_t) * (4 + (size_t)(((B + 127) / 128 + fff::kRankBlock - 1) / fff::kRankBlock) * 256);
+        if ((s = clone((void**)&h->ws_blocksum, nullptr, h->blocksum_bytes)) != FFF_OK) return s;      // zeroed
+        h->blocksum_dirty = false;
     }
     if (h->stages.size() > 1 || h->ustages.size() > 1) {
         if ((s = dmalloc((void**)&h->ws_pos[0], sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
@@ -300,6 +307,26 @@ fff_status_t launched(fff_handle_s* h, cudaStream_t st, const char* name) {
 
 
 // ---- stage launchers -------------------------------------------------------
+
+// Whether k_bucket_ranked can follow a first descent stage over B tokens (few enough 128-token tiles per CTA).
+bool ranked_bucketing_fits(const fff_handle_s* h, int64_t B) {
+    const int64_t n_src = (B + fff::kRankTile - 1) / fff::kRankTile;
+    const int64_t ctas = std::min<int64_t>(h->sm_count, n_src);
+    return B > 0 && h->ws_rank8 && h->ws_counts8 && h->ws_blocksum &&
+           (n_src + ctas - 1) / ctas <= fff::kRankedMaxTilesPerCta;
+}
+
+// The block-sum table the first descent stage adds to, ready for use: null when no ranked bucketing can follow,
+// cleared first if an earlier descent was not followed by one.
+fff_status_t blocksum_for_descent(fff_handle_s* h, int64_t B, bool ranked, cudaStream_t st, int32_t** table) {
+    *table = nullptr;
+    if (!ranked || !ranked_bucketing_fits(h, B)) return FFF_OK;
+    if (h->blocksum_dirty && cudaMemsetAsync(h->ws_blocksum, 0, h->blocksum_bytes, st) != cudaSuccess)
+        return cudaGetLastError(), FFF_ERR_CUDA;
+    h->blocksum_dirty = true;
+    *table = h->ws_blocksum + 4;
+    return FFF_OK;
+}
 
 // What a bucketing refines: nothing (all tokens in natural order), or the previous bucketing.
 struct Coarse {
@@ -329,14 +356,14 @@ fff_status_t run_bucket(fff_handle_s* h, const int32_t* keys, int nbins, const C
     cudaError_t e;
     const int64_t n_src = (B + fff::kRankTile - 1) / fff::kRankTile;
     const int64_t ranked_ctas = std::min<int64_t>(h->sm_count, n_src);
-    if (coarse.ranked && !coarse.perm && nbins >= 16 && nbins <= 256 && B > 0 &&
-        (n_src + ranked_ctas - 1) / ranked_ctas <= fff::kRankedMaxTilesPerCta) {
+    if (coarse.ranked && !coarse.perm && nbins >= 16 && nbins <= 256 && ranked_bucketing_fits(h, B)) {
         // the descent kernel has done the ranking: sum its per-tile counts and scatter
         if (launch_chain(h, fff::k_bucket_ranked, (unsigned)ranked_ctas, fff::kRankedThreads,
                          sizeof(int) * (size_t)(3 + fff::kRankedMaxTilesPerCta) * nbins, st, 1, keys, (const uint8_t*)h->ws_rank8,
-                         (const uint8_t*)h->ws_counts8, offsets, perm, (int)B, nbins, tile_rows, h->ws_tiles,
-                         n_tiles_total) != cudaSuccess)
+                         (const uint8_t*)h->ws_counts8, h->ws_blocksum + 4, (int*)h->ws_blocksum, offsets, perm, (int)B, nbins,
+                         tile_rows, h->ws_tiles, n_tiles_total) != cudaSuccess)
             return cudaGetLastError(), FFF_ERR_CUDA;
+        h->blocksum_dirty = false;          // the kernel clears the table when all its CTAs have read it
         return launched(h, st, name);
     }
     // Refining pays while the coarse buckets are few and large; thousands of tiny buckets would mean
@@ -462,9 +489,11 @@ fff_status_t launch_descent_umma(fff_handle_s* h, const fff_handle_s::DenseStage
     const int64_t n_tiles = (B + fff::kUM - 1) / fff::kUM;
     const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(h->sm_count, n_tiles));
     const bool ranked = sg.k >= 4 && h->ws_rank8 && h->ws_counts8;      // also rank the tokens for the bucketing that follows
+    int32_t* sums = nullptr;
+    if (blocksum_for_descent(h, B, ranked, st, &sums) != FFF_OK) return FFF_ERR_CUDA;
     if (launch_chain(h, fff::k_descent_umma<NP>, (unsigned)grid, fff::kUmmaThreads, (size_t)L::smem_bytes(stages), st, 1, tm,
                      (const __nv_bfloat16*)sg.wimg, (const float*)sg.bimg, pos_out, ranked ? h->ws_rank8 : (uint8_t*)nullptr,
-                     ranked ? h->ws_counts8 : (uint8_t*)nullptr, h->D, (int)B, sg.k, stages, h->d_status) != cudaSuccess)
+                     ranked ? h->ws_counts8 : (uint8_t*)nullptr, sums, h->D, (int)B, sg.k, stages, h->d_status) != cudaSuccess)
         return cudaGetLastError(), FFF_ERR_CUDA;
     return launched(h, st, "tree_descent_umma");
 }
@@ -488,9 +517,11 @@ fff_status_t launch_descent_umma_pair(fff_handle_s* h, const fff_handle_s::Dense
     const int64_t n_pairs = ((B + fff::kUM - 1) / fff::kUM + 1) / 2;
     const int64_t grid = 2 * std::max<int64_t>(1, std::min<int64_t>(h->sm_count / 2, n_pairs));
     const bool ranked = sg.k >= 4 && h->ws_rank8 && h->ws_counts8;
+    int32_t* sums = nullptr;
+    if (blocksum_for_descent(h, B, ranked, st, &sums) != FFF_OK) return FFF_ERR_CUDA;
     if (launch_chain(h, fff::k_descent_umma_pair<NP>, (unsigned)grid, fff::kUmmaThreads, (size_t)L::smem_bytes(stages), st, 2, tm,
                      tw, (const float*)sg.bimg, pos_out, ranked ? h->ws_rank8 : (uint8_t*)nullptr,
-                     ranked ? h->ws_counts8 : (uint8_t*)nullptr, h->D, (int)B, sg.k, stages, h->d_status) != cudaSuccess)
+                     ranked ? h->ws_counts8 : (uint8_t*)nullptr, sums, h->D, (int)B, sg.k, stages, h->d_status) != cudaSuccess)
         return cudaGetLastError(), FFF_ERR_CUDA;
     return launched(h, st, "tree_descent_umma");
 }

@@ -626,23 +626,30 @@ k_bucket_coop(const int32_t* __restrict__ keys, int32_t* __restrict__ offsets_ou
 // It leaves, besides the keys, rank8[t] = number of earlier tokens of t's own tile with the same key, and
 // counts8[tile][bin] = tokens of the tile with that key (both fit a byte).  What remains of the stable
 // counting sort is then a sum over tiles and a scatter, with no barrier across CTAs: CTA c takes a
-// contiguous range of tiles, adds up the count rows of all tiles (bin totals) and of the tiles before its
+// contiguous range of tiles, adds up the counts of all tiles (bin totals) and of the tiles before its
 // own (its starting position inside every bin), scans the totals, and places its tokens at
 //     start[bin] + tokens of the bin in earlier tiles + rank8[t].
+// Every CTA needs those sums over all tiles, so reading the byte matrix row by row made 148 CTAs pull the
+// whole matrix through L2 each (6 of the kernel's 8 microseconds at 394 tiles x 256 bins).  The descent
+// kernel therefore also adds every tile's counts to block_sums[tile / kRankBlock][bin] (int32 atomics), and a
+// CTA here reads that table plus the few byte rows between the last block boundary and its first tile.  The
+// table must be zero when the descent kernel starts: the last CTA of this kernel to have read it clears it
+// (`done` counts the CTAs; zero before and after every launch).
 // Same result as the other bucketing kernels.  Needs 16 <= nbins <= 256 (a multiple of 16) and at most
 // kRankedMaxTilesPerCta tiles per CTA.
 constexpr int kRankTile = 128;
 constexpr int kRankedThreads = 256;
 constexpr int kRankedWarps = kRankedThreads / 32;
 constexpr int kRankedMaxTilesPerCta = 8;
+constexpr int kRankBlock = 16;             // tiles per row of the block-sum table
 
 // The work of one CTA (c of G) of that bucketing, callable from a kernel of its own or as the prologue of a
 // larger one: the first kRankedThreads threads of the CTA work, all its threads must call.
 // s_dyn: (3 + kRankedMaxTilesPerCta) * nbins ints of shared memory, s_warp: 32 ints.
 __device__ __forceinline__ void bucket_ranked_cta(const int32_t* __restrict__ keys, const uint8_t* __restrict__ rank8,
-                                                  const uint8_t* __restrict__ counts8, int32_t* offsets_out, int32_t* perm_out,
-                                                  int B, int nbins, int tile_rows, Tile* tiles, int n_tiles_total, int* s_dyn,
-                                                  int* s_warp, int G, int c)
+                                                  const uint8_t* __restrict__ counts8, int32_t* block_sums, int* done,
+                                                  int32_t* offsets_out, int32_t* perm_out, int B, int nbins, int tile_rows,
+                                                  Tile* tiles, int n_tiles_total, int* s_dyn, int* s_warp, int G, int c)
 {
     int* s_total = s_dyn;                     // [nbins] tokens in the bin
     int* s_before = s_total + nbins;          // [nbins] of which in tiles before this CTA's
@@ -674,43 +681,64 @@ __device__ __forceinline__ void bucket_ranked_cta(const int32_t* __restrict__ ke
     for (int i = 0; i < kRankedMaxTilesPerCta; ++i)
         own[i] = (tid < nbins && t0 + i < t1) ? (int)counts8[(int64_t)(t0 + i) * nbins + tid] : 0;
 
-    // column sums of the count matrix, 16 bins per 16-byte load; bytes are added up in 16-bit lanes and
-    // flushed to shared memory before they can overflow
+    // Column sums of the count matrix.  Whole blocks of kRankBlock tiles come from the block-sum table the descent
+    // kernel accumulated (4 bins per 16-byte load), the tiles between the last block boundary and this CTA's first
+    // tile from the byte matrix (16 bins per load): one round of loads instead of a pass over every tile's row.
+    __shared__ int s_last;
     {
-        const int V = nbins >> 4;                         // 16-byte columns
-        const int P = kRankedThreads / V;                 // threads per column
-        const int vb = tid % V, part = tid / V;
-        const uint4* m = reinterpret_cast<const uint4*>(counts8);
-        for (int r0 = part; r0 < n_src && part < P; r0 += 256 * P) {
-            uint32_t tot[8] = {0, 0, 0, 0, 0, 0, 0, 0}, bef[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-            const int r_end = min(n_src, r0 + 256 * P);
-            for (int r = r0; r < r_end; r += 8 * P) {
-                uint4 v[8];
+        const int nb = (n_src + kRankBlock - 1) / kRankBlock;
+        const int bb = t0 / kRankBlock;                   // blocks that lie entirely before this CTA's tiles
+        const int V4 = nbins >> 2;                        // 16-byte columns of the table
+        const int P = kRankedThreads / V4;                // threads per column
+        const int vb = tid % V4, part = tid / V4;
+        const int4* m4 = reinterpret_cast<const int4*>(block_sums);
+        int4 tot = make_int4(0, 0, 0, 0), bef = make_int4(0, 0, 0, 0);
+        for (int r = part; on && part < P && r < nb; r += 8 * P) {
+            int4 v[8];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) v[j] = r + j * P < r_end ? __ldcg(m + (int64_t)(r + j * P) * V + vb) : make_uint4(0, 0, 0, 0);
+            for (int j = 0; j < 8; ++j) v[j] = r + j * P < nb ? __ldcg(m4 + (int64_t)(r + j * P) * V4 + vb) : make_int4(0, 0, 0, 0);
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
-                    const uint32_t mask = r + j * P < t0 ? 0xFFFFFFFFu : 0u;
+            for (int j = 0; j < 8; ++j) {
+                tot.x += v[j].x; tot.y += v[j].y; tot.z += v[j].z; tot.w += v[j].w;
+                if (r + j * P < bb) { bef.x += v[j].x; bef.y += v[j].y; bef.z += v[j].z; bef.w += v[j].w; }
+            }
+        }
+        // (the byte row of a tile: nbins / 16 loads; at most kRankBlock - 1 such rows, one load per thread)
+        const int V = nbins >> 4;
+        const int prow = bb * kRankBlock + tid / V;
+        uint4 pv = make_uint4(0, 0, 0, 0);
+        const bool partial = on && prow < t0;
+        if (partial) pv = __ldcg(reinterpret_cast<const uint4*>(counts8) + (int64_t)prow * V + tid % V);
+        if (on && part < P) {
+            const int b = 4 * vb;
+            if (tot.x) atomicAdd(&s_total[b], tot.x);
+            if (tot.y) atomicAdd(&s_total[b + 1], tot.y);
+            if (tot.z) atomicAdd(&s_total[b + 2], tot.z);
+            if (tot.w) atomicAdd(&s_total[b + 3], tot.w);
+            if (bef.x) atomicAdd(&s_before[b], bef.x);
+            if (bef.y) atomicAdd(&s_before[b + 1], bef.y);
+            if (bef.z) atomicAdd(&s_before[b + 2], bef.z);
+            if (bef.w) atomicAdd(&s_before[b + 3], bef.w);
+        }
+        if (partial) {
+            const uint32_t w[4] = {pv.x, pv.y, pv.z, pv.w};
+            const int b = 16 * (tid % V);
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const uint32_t lo = w[q] & 0x00FF00FFu, hi = (w[q] >> 8) & 0x00FF00FFu;
-                        tot[2 * q] += lo; tot[2 * q + 1] += hi;
-                        bef[2 * q] += lo & mask; bef[2 * q + 1] += hi & mask;
-                    }
+            for (int q = 0; q < 4; ++q)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int cnt = (int)((w[q] >> (8 * e)) & 0xFFu);
+                    if (cnt) atomicAdd(&s_before[b + 4 * q + e], cnt);
                 }
-            }
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const int b = 16 * vb + 4 * q;            // word q holds bins b .. b+3: lanes (b, b+2) and (b+1, b+3)
-                atomicAdd(&s_total[b], (int)(tot[2 * q] & 0xFFFFu));      atomicAdd(&s_total[b + 2], (int)(tot[2 * q] >> 16));
-                atomicAdd(&s_total[b + 1], (int)(tot[2 * q + 1] & 0xFFFFu)); atomicAdd(&s_total[b + 3], (int)(tot[2 * q + 1] >> 16));
-                atomicAdd(&s_before[b], (int)(bef[2 * q] & 0xFFFFu));     atomicAdd(&s_before[b + 2], (int)(bef[2 * q] >> 16));
-                atomicAdd(&s_before[b + 1], (int)(bef[2 * q + 1] & 0xFFFFu)); atomicAdd(&s_before[b + 3], (int)(bef[2 * q + 1] >> 16));
-            }
         }
     }
     __syncthreads();
+    // The table has served this CTA.  The last CTA to get here clears it for the next descent (which adds to it)
+    // and rearms the counter.
+    if (tid == 0) {
+        __threadfence();
+        s_last = atomicAdd(done, 1) == G - 1 ? 1 : 0;
+    }
 
     // exclusive scan of the totals over the bins (nbins <= kRankedThreads)
     {
@@ -733,6 +761,11 @@ __device__ __forceinline__ void bucket_ranked_cta(const int32_t* __restrict__ ke
         }
     }
     __syncthreads();
+    if (s_last) {
+        const int n = (n_src + kRankBlock - 1) / kRankBlock * nbins;
+        for (int i = tid; i < n; i += blockDim.x) block_sums[i] = 0;
+        if (tid == 0) *done = 0;
+    }
     if (tile_rows > 0 && c == 0) {
         const int total = tid < nbins ? s_total[tid] : 0;
         const int nt = (total + tile_rows - 1) / tile_rows;
@@ -764,6 +797,7 @@ __device__ __forceinline__ void bucket_ranked_cta(const int32_t* __restrict__ ke
 // Dynamic shared memory: (3 + kRankedMaxTilesPerCta) * nbins ints.
 __global__ void __launch_bounds__(kRankedThreads)
 k_bucket_ranked(const int32_t* __restrict__ keys, const uint8_t* __restrict__ rank8, const uint8_t* __restrict__ counts8,
+                int32_t* __restrict__ block_sums, int* __restrict__ done,
                 int32_t* __restrict__ offsets_out, int32_t* __restrict__ perm_out, int B, int nbins, int tile_rows,
                 Tile* __restrict__ tiles, int n_tiles_total)
 {
@@ -771,7 +805,8 @@ k_bucket_ranked(const int32_t* __restrict__ keys, const uint8_t* __restrict__ ra
     __shared__ int s_warp[32];
     pdl_trigger();
     pdl_wait();
-    bucket_ranked_cta(keys, rank8, counts8, offsets_out, perm_out, B, nbins, tile_rows, tiles, n_tiles_total, s_dyn, s_warp,
+    bucket_ranked_cta(keys, rank8, counts8, block_sums, done, offsets_out, perm_out, B, nbins, tile_rows, tiles, n_tiles_total,
+                      s_dyn, s_warp,
                       (int)gridDim.x, (int)blockIdx.x);
 }
 

@@ -104,12 +104,15 @@ template <int NP> struct DescentUmmaLayout {
 // wimg: [D / 64][NP rows][64 columns] 128-byte swizzled (the single-group image of k_pack_nodes),
 // bimg: [NP] float32.  pos_out[t] = position reached at level k.
 // rank8 / counts8 (both or neither, k >= 4): rank8[t] = earlier tokens of t's 128-token tile at the same
-// position, counts8[tile][2^k] = tokens of the tile per position.
+// position, counts8[tile][2^k] = tokens of the tile per position.  block_sums (optional, with them):
+// [ceil(tiles / kRankBlock)][2^k] int32, zero on entry, to which the counts of every block of kRankBlock
+// consecutive tiles are added (integer atomics: the sums do not depend on the order).
 template <int NP>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 k_descent_umma(const __grid_constant__ CUtensorMap tmap_x, const __nv_bfloat16* __restrict__ wimg,
                const float* __restrict__ bimg, int32_t* __restrict__ pos_out, uint8_t* __restrict__ rank8,
-               uint8_t* __restrict__ counts8, int D, int B, int k, int kStages, int* __restrict__ status)
+               uint8_t* __restrict__ counts8, int32_t* __restrict__ block_sums, int D, int B, int k, int kStages,
+               int* __restrict__ status)
 {
     using L = DescentUmmaLayout<NP>;
     extern __shared__ unsigned char smem_raw[];
@@ -231,6 +234,7 @@ k_descent_umma(const __grid_constant__ CUtensorMap tmap_x, const __nv_bfloat16* 
                         s_cnt[w * 256 + b] = 0;
                     }
                     counts8[(int64_t)tile * nbins + b] = (uint8_t)total;
+                    if (block_sums && total > 0) atomicAdd(block_sums + (int64_t)(tile / kRankBlock) * nbins + b, total);
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");
             }
@@ -278,7 +282,8 @@ template <int NP>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 k_descent_umma_pair(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                     const float* __restrict__ bimg, int32_t* __restrict__ pos_out, uint8_t* __restrict__ rank8,
-                    uint8_t* __restrict__ counts8, int D, int B, int k, int kStages, int* __restrict__ status)
+                    uint8_t* __restrict__ counts8, int32_t* __restrict__ block_sums, int D, int B, int k, int kStages,
+               int* __restrict__ status)
 {
     namespace cg = cooperative_groups;
     using L = DescentUmmaPairLayout<NP>;
@@ -419,6 +424,7 @@ k_descent_umma_pair(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                             s_cnt[w * 256 + b] = 0;
                         }
                         counts8[(int64_t)tile * nbins + b] = (uint8_t)total;
+                        if (block_sums && total > 0) atomicAdd(block_sums + (int64_t)(tile / kRankBlock) * nbins + b, total);
                     }
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");
