@@ -733,12 +733,10 @@ __device__ __forceinline__ void bucket_ranked_cta(const int32_t* __restrict__ ke
         }
     }
     __syncthreads();
-    // The table has served this CTA.  The last CTA to get here clears it for the next descent (which adds to it)
-    // and rearms the counter.
-    if (tid == 0) {
-        __threadfence();
-        s_last = atomicAdd(done, 1) == G - 1 ? 1 : 0;
-    }
+    // The table has served this CTA (its values have been used above).  The last CTA to get here clears it for the
+    // next descent, at the end of the kernel; the ticket is only looked at there, so nobody waits for it now.
+    int ticket = -1;
+    if (tid == 0) ticket = atomicAdd(done, 1);
 
     // exclusive scan of the totals over the bins (nbins <= kRankedThreads)
     {
@@ -761,36 +759,44 @@ __device__ __forceinline__ void bucket_ranked_cta(const int32_t* __restrict__ ke
         }
     }
     __syncthreads();
-    if (s_last) {
-        const int n = (n_src + kRankBlock - 1) / kRankBlock * nbins;
-        for (int i = tid; i < n; i += blockDim.x) block_sums[i] = 0;
-        if (tid == 0) *done = 0;
-    }
-    if (tile_rows > 0 && c == 0) {
-        const int total = tid < nbins ? s_total[tid] : 0;
-        const int nt = (total + tile_rows - 1) / tile_rows;
-        int n_all = 0;
-        const int tl0 = block_exclusive_scan_nw<kRankedWarps>(nt, s_warp, &n_all);
-        for (int i = 0; i < nt; ++i) {
-            Tile tl;
-            tl.bin = tid;
-            tl.start = s_start[tid] + i * tile_rows;
-            tl.rows = min(tile_rows, total - i * tile_rows);
-            tl.pad = 0;
-            tiles[tl0 + i] = tl;
-        }
-        Tile empty;
-        empty.bin = 0; empty.start = 0; empty.rows = 0; empty.pad = 0;
-        if (on)
-            for (int i = n_all + tid; i < n_tiles_total; i += kRankedThreads) tiles[i] = empty;
-    }
-
     // place
 #pragma unroll
     for (int i = 0; i < kTok; ++i) {
         const int64_t t = first + tid + i * kRankedThreads;
         const int k = my_key[i];
         if (t < last && k >= 0 && k < nbins) perm_out[s_tile[(int)((t - first) / kRankTile) * nbins + k] + my_rank[i]] = (int32_t)t;
+    }
+
+    // tile list: every CTA knows all totals, so each writes the tiles of its share of the bins (bin % G == c) and
+    // of the padding
+    if (tile_rows > 0) {
+        const int total = tid < nbins ? s_total[tid] : 0;
+        const int nt = (total + tile_rows - 1) / tile_rows;
+        int n_all = 0;
+        const int tl0 = block_exclusive_scan_nw<kRankedWarps>(nt, s_warp, &n_all);
+        if (tid < nbins && tid % G == c) {
+            for (int i = 0; i < nt; ++i) {
+                Tile tl;
+                tl.bin = tid;
+                tl.start = s_start[tid] + i * tile_rows;
+                tl.rows = min(tile_rows, total - i * tile_rows);
+                tl.pad = 0;
+                tiles[tl0 + i] = tl;
+            }
+        }
+        Tile empty;
+        empty.bin = 0; empty.start = 0; empty.rows = 0; empty.pad = 0;
+        if (on)
+            for (int i = n_all + c * kRankedThreads + tid; i < n_tiles_total; i += G * kRankedThreads) tiles[i] = empty;
+    }
+
+    // the last CTA to have read the block-sum table clears it and rearms the counter
+    if (tid == 0) s_last = ticket == G - 1 ? 1 : 0;
+    __syncthreads();
+    if (s_last) {
+        const int n = (n_src + kRankBlock - 1) / kRankBlock * nbins;
+        for (int i = tid; i < n; i += blockDim.x) block_sums[i] = 0;
+        if (tid == 0) *done = 0;
     }
 }
 
