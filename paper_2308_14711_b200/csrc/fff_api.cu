@@ -73,6 +73,7 @@ struct fff_handle_s {
     int32_t* ws_blocksum = nullptr;  // [4] CTA counter of k_bucket_ranked, then the counts summed over blocks of 16 tiles
     size_t blocksum_bytes = 0;
     bool blocksum_dirty = false;     // a descent has added to the table and no ranked bucketing has cleared it since
+    bool blocksum_wanted = false;    // k_bucket_ranked follows the first descent stage of the call in progress
     int max_bucket_clusters = 8;
     int32_t* last_perm = nullptr; // where the most recent forward left its leaf permutation
     bool bucketing_pending = false;   // the last forward skipped the leaf bucketing; ws_leaf holds its leaf indices
@@ -320,7 +321,7 @@ bool ranked_bucketing_fits(const fff_handle_s* h, int64_t B) {
 // cleared first if an earlier descent was not followed by one.
 fff_status_t blocksum_for_descent(fff_handle_s* h, int64_t B, bool ranked, cudaStream_t st, int32_t** table) {
     *table = nullptr;
-    if (!ranked || !ranked_bucketing_fits(h, B)) return FFF_OK;
+    if (!ranked || !h->blocksum_wanted || !ranked_bucketing_fits(h, B)) return FFF_OK;
     if (h->blocksum_dirty && cudaMemsetAsync(h->ws_blocksum, 0, h->blocksum_bytes, st) != cudaSuccess)
         return cudaGetLastError(), FFF_ERR_CUDA;
     h->blocksum_dirty = true;
@@ -615,10 +616,15 @@ struct DescentTail {
     const int32_t* pos = nullptr;
 };
 
+// leaf_bucketing_follows: the caller buckets by leaf right after (run_bucket with *coarse).
 fff_status_t run_descent(fff_handle_s* h, const void* x, int32_t* leaf_out, Coarse* coarse, int64_t B, cudaStream_t st,
-                         DescentTail* defer_tail = nullptr) {
+                         DescentTail* defer_tail = nullptr, bool leaf_bucketing_follows = false) {
     fff_status_t s = FFF_OK;
     const int n_dense = dense_stage_count(h, B);
+    // the first stage's counts are summed per block of tiles only if the bucketing kernel that reads (and clears)
+    // the sums comes next: a node bucketing before the second stage, or the caller's leaf bucketing
+    h->blocksum_wanted = n_dense > 1 || (n_dense == 1 && leaf_bucketing_follows && coarse != nullptr &&
+                                         stage_plan(h)[0].k == h->depth);
     int level = 0;
     const int32_t* pos = nullptr;
     Coarse prev;
@@ -1202,7 +1208,7 @@ fff_status_t fff_forward_infer(fff_handle_t h, const void* x, void* y, int32_t* 
     Coarse coarse;
     DescentTail tail;
     // without a bucketing in between, the warp leaf kernel also walks the levels the staged descent leaves over
-    s = run_descent(h, x, leaf, &coarse, B, st, lazy_bucketing ? &tail : nullptr);
+    s = run_descent(h, x, leaf, &coarse, B, st, lazy_bucketing ? &tail : nullptr, !lazy_bucketing);
     const LeafPlan plan = tensor_leaf ? leaf_plan(h, B) : LeafPlan{};
     const int tile_rows = plan.tile_rows;
     // the final permutation goes to whichever buffer the last node bucketing did not use

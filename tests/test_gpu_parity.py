@@ -251,6 +251,39 @@ def test_nonfinite_leaf_weights_stay_in_their_leaf():
     layer.close()
 
 
+def test_descent_alone_then_forward():
+    """The stage entry point for the descent, then whole forwards on the same handle: scratch that the descent
+    leaves for the bucketing kernel must not leak from one call into the next."""
+    cfg = wl.FFFConfig("bf16_d8_mixed_calls", 256, 64, 8, 8, "gelu", "bf16", 5000, "layernorm")
+    case = util.make_case(cfg, seed=4)
+    y_ref, leaf_ref = orc.forward_i(case.net, case.x, threads=util.ORACLE_THREADS)
+    off_ref, perm_ref = orc.bucket(leaf_ref, cfg.n_leaves)
+    layer = util.make_layer(case)
+    x = util.to_device(case.x, "bf16")
+    for _ in range(2):
+        np.testing.assert_array_equal(layer.tree_descent(x).cpu().numpy(), leaf_ref)
+        for _ in range(2):
+            y, leaf = layer.forward_infer(x)
+            torch.cuda.synchronize()
+            np.testing.assert_array_equal(leaf.cpu().numpy(), leaf_ref)
+            off, perm = layer.last_bucketing(cfg.B)
+            np.testing.assert_array_equal(off.cpu().numpy(), off_ref)
+            np.testing.assert_array_equal(perm.cpu().numpy(), perm_ref)
+            util.check_outputs(y, y_ref, "bf16")
+    # a smaller batch afterwards: fewer tiles and blocks than the table has seen
+    small = 700
+    y, leaf = layer.forward_infer(x[:small])
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(leaf.cpu().numpy(), leaf_ref[:small])
+    off, perm = layer.last_bucketing(small)
+    off_s, perm_s = orc.bucket(leaf_ref[:small], cfg.n_leaves)
+    np.testing.assert_array_equal(off.cpu().numpy(), off_s)
+    np.testing.assert_array_equal(perm.cpu().numpy(), perm_s)
+    util.check_outputs(y, y_ref[:small], "bf16")
+    assert layer.last_status() == 0
+    layer.close()
+
+
 def test_nan_inputs_stay_in_range():
     cfg = wl.FFFConfig("n", 64, 32, 4, 8, "gelu", "bf16", 64)
     case = util.make_case(cfg, 0)
