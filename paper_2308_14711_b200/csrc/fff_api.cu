@@ -74,6 +74,13 @@ struct fff_handle_s {
     size_t blocksum_bytes = 0;
     bool blocksum_dirty = false;     // a descent has added to the table and no ranked bucketing has cleared it since
     bool blocksum_wanted = false;    // k_bucket_ranked follows the first descent stage of the call in progress
+    // direct lists (slot_tokens in descent_umma.cuh): when one tcgen05 stage is the whole descent and the tcgen05
+    // leaf kernel follows, the descent files every token under its leaf itself and no bucketing kernel runs
+    int32_t* ws_slots = nullptr;     // [n_leaves][slot_cap] token numbers
+    int32_t* ws_cursor = nullptr;    // [n_leaves] entries used; zero between calls (the leaf kernel clears it)
+    int64_t slot_cap = 0;
+    bool cursor_dirty = false;       // a descent has filled the lists and no leaf kernel has cleared the counts since
+    bool slots_now = false;          // the call in progress uses the direct lists
     int max_bucket_clusters = 8;
     int32_t* last_perm = nullptr; // where the most recent forward left its leaf permutation
     bool bucketing_pending = false;   // the last forward skipped the leaf bucketing; ws_leaf holds its leaf indices
@@ -194,7 +201,7 @@ void release(fff_handle_s* h) {
     for (auto& sg : h->stages) { dfree(sg.wimg); dfree(sg.bimg); }
     for (auto& sg : h->ustages) { dfree(sg.wimg); dfree(sg.bimg); }
     dfree(h->ws_pos[0]); dfree(h->ws_pos[1]);
-    dfree(h->w1img); dfree(h->b1img); dfree(h->w2img); dfree(h->w2uimg); dfree(h->ws_sched); dfree(h->ws_tiles); dfree(h->ws_rank); dfree(h->ws_rank8); dfree(h->ws_counts8); dfree(h->ws_blocksum); dfree(h->ws_matrix);
+    dfree(h->w1img); dfree(h->b1img); dfree(h->w2img); dfree(h->w2uimg); dfree(h->ws_sched); dfree(h->ws_tiles); dfree(h->ws_rank); dfree(h->ws_rank8); dfree(h->ws_counts8); dfree(h->ws_blocksum); dfree(h->ws_matrix); dfree(h->ws_slots); dfree(h->ws_cursor);
     if (h->copy_in) cudaStreamDestroy(h->copy_in);
     if (h->copy_out) cudaStreamDestroy(h->copy_out);
     for (int i = 0; i < fff_handle_s::kMaxHostChunks; ++i) {
@@ -212,6 +219,8 @@ constexpr int kMinTileRows = 32;
 
 // Length of a tile list: floor(B / tile_rows) + nbins entries, some of them empty (see k_bucket_cluster).
 int tile_list_len(int64_t B, int tile_rows, int nbins) { return (int)(B / tile_rows) + nbins; }
+
+constexpr size_t kMaxSlotBytes = (size_t)1 << 30;      // largest table of direct lists a handle allocates
 
 // Capacity of the tile buffer: the longest list any stage can ask for.
 size_t max_tiles(const fff_handle_s* h, int64_t B) { return (size_t)(B / kMinTileRows + h->n_leaves + 1); }
@@ -268,7 +277,9 @@ fff_status_t grow_workspace(fff_handle_s* h, int64_t B) {
     if (B <= h->cap_B) return FFF_OK;
     if (cudaDeviceSynchronize() != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
     dfree(h->ws_leaf); dfree(h->ws_perm); dfree(h->ws_perm2); dfree(h->ws_tiles); dfree(h->ws_rank); dfree(h->ws_pos[0]);
-    dfree(h->ws_rank8); dfree(h->ws_counts8); dfree(h->ws_blocksum);
+    dfree(h->ws_rank8); dfree(h->ws_counts8); dfree(h->ws_blocksum); dfree(h->ws_slots); dfree(h->ws_cursor);
+    h->ws_slots = h->ws_cursor = nullptr;
+    h->slot_cap = 0;
     h->ws_rank8 = h->ws_counts8 = nullptr;
     h->ws_blocksum = nullptr;
     dfree(h->ws_pos[1]);
@@ -292,6 +303,15 @@ fff_status_t grow_workspace(fff_handle_s* h, int64_t B) {
         if ((s = dmalloc((void**)&h->ws_pos[1], sizeof(int32_t) * (size_t)B)) != FFF_OK) return s;
     }
     if ((s = dmalloc((void**)&h->ws_tiles, sizeof(fff::Tile) * max_tiles(h, B))) != FFF_OK) return s;
+    // direct lists: every leaf's list can take the whole batch, so their size grows with n_leaves * B; beyond
+    // kMaxSlotBytes the forward keeps the bucketing kernel instead
+    if (h->ustages.size() == 1 && h->ustages[0].umma && h->ustages[0].k == h->depth && h->w2uimg &&
+        (size_t)h->n_leaves * (size_t)B * sizeof(int32_t) <= kMaxSlotBytes) {
+        if ((s = dmalloc((void**)&h->ws_slots, sizeof(int32_t) * (size_t)h->n_leaves * (size_t)B)) != FFF_OK) return s;
+        if ((s = clone((void**)&h->ws_cursor, nullptr, sizeof(int32_t) * (size_t)h->n_leaves)) != FFF_OK) return s;
+        h->slot_cap = B;
+        h->cursor_dirty = false;
+    }
     h->cap_B = B;
     return FFF_OK;
 }
@@ -479,6 +499,22 @@ bool make_x_tensor_map(CUtensorMap* tm, const void* x, int64_t B, int D, int box
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Arguments of the first descent stage for the direct lists (all null unless the call in progress uses them);
+// the positions are also kept in the workspace, from which a bucketing can be made on demand afterwards.
+struct SlotArgs {
+    int32_t *pos2 = nullptr, *cursor = nullptr, *slots = nullptr;
+    int cap = 0;
+};
+SlotArgs slot_args(const fff_handle_s* h, const int32_t* pos_out) {
+    SlotArgs a;
+    if (!h->slots_now) return a;
+    a.pos2 = pos_out == h->ws_leaf ? nullptr : h->ws_leaf;
+    a.cursor = h->ws_cursor;
+    a.slots = h->ws_slots;
+    a.cap = (int)h->slot_cap;
+    return a;
+}
+
 template <int NP>
 fff_status_t launch_descent_umma(fff_handle_s* h, const fff_handle_s::DenseStage& sg, const void* x, int32_t* pos_out,
                                  int64_t B, cudaStream_t st) {
@@ -492,9 +528,11 @@ fff_status_t launch_descent_umma(fff_handle_s* h, const fff_handle_s::DenseStage
     const bool ranked = sg.k >= 4 && h->ws_rank8 && h->ws_counts8;      // also rank the tokens for the bucketing that follows
     int32_t* sums = nullptr;
     if (blocksum_for_descent(h, B, ranked, st, &sums) != FFF_OK) return FFF_ERR_CUDA;
+    const SlotArgs sl = slot_args(h, pos_out);
     if (launch_chain(h, fff::k_descent_umma<NP>, (unsigned)grid, fff::kUmmaThreads, (size_t)L::smem_bytes(stages), st, 1, tm,
                      (const __nv_bfloat16*)sg.wimg, (const float*)sg.bimg, pos_out, ranked ? h->ws_rank8 : (uint8_t*)nullptr,
-                     ranked ? h->ws_counts8 : (uint8_t*)nullptr, sums, h->D, (int)B, sg.k, stages, h->d_status) != cudaSuccess)
+                     ranked ? h->ws_counts8 : (uint8_t*)nullptr, sums, sl.pos2, sl.cursor, sl.slots, sl.cap, h->D, (int)B, sg.k,
+                     stages, h->d_status) != cudaSuccess)
         return cudaGetLastError(), FFF_ERR_CUDA;
     return launched(h, st, "tree_descent_umma");
 }
@@ -520,9 +558,11 @@ fff_status_t launch_descent_umma_pair(fff_handle_s* h, const fff_handle_s::Dense
     const bool ranked = sg.k >= 4 && h->ws_rank8 && h->ws_counts8;
     int32_t* sums = nullptr;
     if (blocksum_for_descent(h, B, ranked, st, &sums) != FFF_OK) return FFF_ERR_CUDA;
+    const SlotArgs sl = slot_args(h, pos_out);
     if (launch_chain(h, fff::k_descent_umma_pair<NP>, (unsigned)grid, fff::kUmmaThreads, (size_t)L::smem_bytes(stages), st, 2, tm,
                      tw, (const float*)sg.bimg, pos_out, ranked ? h->ws_rank8 : (uint8_t*)nullptr,
-                     ranked ? h->ws_counts8 : (uint8_t*)nullptr, sums, h->D, (int)B, sg.k, stages, h->d_status) != cudaSuccess)
+                     ranked ? h->ws_counts8 : (uint8_t*)nullptr, sums, sl.pos2, sl.cursor, sl.slots, sl.cap, h->D, (int)B, sg.k,
+                     stages, h->d_status) != cudaSuccess)
         return cudaGetLastError(), FFF_ERR_CUDA;
     return launched(h, st, "tree_descent_umma");
 }
@@ -803,10 +843,12 @@ fff_status_t launch_leaf_umma(fff_handle_s* h, const void* x, const int32_t* per
     const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(h->sm_count, n_tiles));
     const int wide = (reinterpret_cast<uintptr_t>(y) & 31u) == 0 ? 1 : 0;
     const int passes = 1;      // two passes (full tiles first) measured slightly slower
+    // direct lists: perm is the table of lists, the tiles come from its counts
+    int32_t* counts = h->slots_now && perm == h->ws_slots ? h->ws_cursor : nullptr;
     if (launch_chain(h, fff::k_leaf_umma<LP, kFold>, (unsigned)grid, fff::kLUThreads, (size_t)L::smem_bytes(stages), st, 1, tm, perm,
                      (const fff::Tile*)h->ws_tiles, n_tiles, (const __nv_bfloat16*)h->w1img, (const float*)h->b1img,
                      (const unsigned char*)h->w2uimg, (__nv_bfloat16*)y, h->D, h->O, h->l, h->act, stages, wide, passes, h->ws_sched,
-                     h->d_status) != cudaSuccess)
+                     counts, (int)h->n_leaves, (int)h->slot_cap, h->d_status) != cudaSuccess)
         return cudaGetLastError(), FFF_ERR_CUDA;
     return launched(h, st, "grouped_leaf_ff_umma");
 }
@@ -1207,10 +1249,35 @@ fff_status_t fff_forward_infer(fff_handle_t h, const void* x, void* y, int32_t* 
     if (lazy_bucketing) leaf = h->ws_leaf;
     Coarse coarse;
     DescentTail tail;
-    // without a bucketing in between, the warp leaf kernel also walks the levels the staged descent leaves over
-    s = run_descent(h, x, leaf, &coarse, B, st, lazy_bucketing ? &tail : nullptr, !lazy_bucketing);
     const LeafPlan plan = tensor_leaf ? leaf_plan(h, B) : LeafPlan{};
     const int tile_rows = plan.tile_rows;
+    // One tcgen05 stage is the whole descent and the tcgen05 leaf kernel takes whole 128-row tiles of one leaf:
+    // the descent files the tokens under their leaves itself and the leaf kernel follows at once.
+    static const bool no_slots = std::getenv("FFF_NO_DIRECT_LISTS") != nullptr;      // tuning aid
+    h->slots_now = !no_slots && tensor_leaf && plan.umma && plan.pack <= 1 && tile_rows == fff::kLUM && h->ws_slots &&
+                   B <= h->slot_cap && h->n_leaves * h->slot_cap <= INT32_MAX && dense_stage_count(h, B) == 1 &&
+                   h->ustages.size() == 1;
+    if (h->slots_now) {
+        if (h->cursor_dirty && cudaMemsetAsync(h->ws_cursor, 0, sizeof(int32_t) * (size_t)h->n_leaves, st) != cudaSuccess)
+            return h->slots_now = false, cudaGetLastError(), FFF_ERR_CUDA;
+        h->cursor_dirty = true;
+        s = run_descent(h, x, leaf, nullptr, B, st);
+        h->last_perm = h->ws_perm;
+        h->bucketing_pending = true;          // the stable permutation is made on demand from ws_leaf
+        if (s == FFF_OK) s = run_leaf_mma(h, x, h->ws_slots, y, B, plan, st);
+        if (s == FFF_OK) h->cursor_dirty = false;
+        h->slots_now = false;
+        if (h->prof_active) {
+            h->prof_active = false;
+            if (s == FFF_OK && (h->prof_steps == 0 || h->prof_nlaunch == h->launches)) {
+                h->prof_nlaunch = std::min(h->launches, (int)fff_handle_s::kMaxProfLaunches);
+                ++h->prof_steps;
+            }
+        }
+        return s;
+    }
+    // without a bucketing in between, the warp leaf kernel also walks the levels the staged descent leaves over
+    s = run_descent(h, x, leaf, &coarse, B, st, lazy_bucketing ? &tail : nullptr, !lazy_bucketing);
     // the final permutation goes to whichever buffer the last node bucketing did not use
     h->last_perm = coarse.perm == h->ws_perm ? h->ws_perm2 : h->ws_perm;
     h->bucketing_pending = lazy_bucketing;

@@ -90,6 +90,24 @@ __device__ __forceinline__ int umma_walk(const uint32_t (&bits)[NP / 32], int k)
     return p;
 }
 
+// Direct slotting by the position just computed, for a leaf kernel that follows at once: the tokens of a warp
+// that reached the same key reserve a run of entries of that key's list with one atomic add on its cursor and
+// write their token numbers there: slots[key * cap + cursor .. ), cap >= B.  The order of a list depends on the
+// order in which warps arrive, which is harmless for the leaf kernel (the rows of a tile are independent: a
+// token's output does not depend on its neighbours) but is not the stable order of the bucketing, so no
+// permutation is reported from these lists.  cursor[] is zero on entry and holds the counts per key afterwards.
+__device__ __forceinline__ void slot_tokens(bool in, int key, int nbits, int tok, int32_t* __restrict__ cursor,
+                                            int32_t* __restrict__ slots, int cap)
+{
+    const int lane = threadIdx.x & 31;
+    const unsigned peers = peers_by_ballot(in, key, nbits);
+    const int leader = in ? __ffs(peers) - 1 : lane;
+    int base = 0;
+    if (in && lane == leader) base = atomicAdd(cursor + key, __popc(peers));
+    base = __shfl_sync(kFullMask, base, leader);
+    if (in) slots[(int64_t)key * cap + base + __popc(peers & ((1u << lane) - 1u))] = tok;
+}
+
 template <int NP> struct DescentUmmaLayout {
     static_assert(NP == 32 || NP == 64 || NP == 128 || NP == 256, "accumulator width");
     static constexpr int kXStageBytes = kUM * kUKB * 2;
@@ -107,11 +125,14 @@ template <int NP> struct DescentUmmaLayout {
 // position, counts8[tile][2^k] = tokens of the tile per position.  block_sums (optional, with them):
 // [ceil(tiles / kRankBlock)][2^k] int32, zero on entry, to which the counts of every block of kRankBlock
 // consecutive tiles are added (integer atomics: the sums do not depend on the order).
+// pos_out2 (optional): a second copy of the positions.  cursor / slots / cap (optional, instead of the ranks):
+// see slot_tokens.
 template <int NP>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 k_descent_umma(const __grid_constant__ CUtensorMap tmap_x, const __nv_bfloat16* __restrict__ wimg,
                const float* __restrict__ bimg, int32_t* __restrict__ pos_out, uint8_t* __restrict__ rank8,
-               uint8_t* __restrict__ counts8, int32_t* __restrict__ block_sums, int D, int B, int k, int kStages,
+               uint8_t* __restrict__ counts8, int32_t* __restrict__ block_sums, int32_t* __restrict__ pos_out2,
+               int32_t* __restrict__ cursor, int32_t* __restrict__ slots, int cap, int D, int B, int k, int kStages,
                int* __restrict__ status)
 {
     using L = DescentUmmaLayout<NP>;
@@ -213,8 +234,13 @@ k_descent_umma(const __grid_constant__ CUtensorMap tmap_x, const __nv_bfloat16* 
             const int p = umma_walk<NP>(bits, k);
             const int tok = tile * kUM + warp * 32 + lane;
             const int key = p - ((1 << k) - 1);
-            if (tok < B) pos_out[tok] = key;
-            if (rank8) {
+            if (tok < B) {
+                pos_out[tok] = key;
+                if (pos_out2) pos_out2[tok] = key;
+            }
+            if (cursor) {
+                slot_tokens(tok < B, key, k, tok, cursor, slots, cap);
+            } else if (rank8) {
                 const int nbins = 1 << k;
                 const bool in = tok < B;
                 const unsigned peers = peers_by_ballot(in, key, k);
@@ -282,8 +308,9 @@ template <int NP>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 k_descent_umma_pair(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                     const float* __restrict__ bimg, int32_t* __restrict__ pos_out, uint8_t* __restrict__ rank8,
-                    uint8_t* __restrict__ counts8, int32_t* __restrict__ block_sums, int D, int B, int k, int kStages,
-               int* __restrict__ status)
+                    uint8_t* __restrict__ counts8, int32_t* __restrict__ block_sums, int32_t* __restrict__ pos_out2,
+                    int32_t* __restrict__ cursor, int32_t* __restrict__ slots, int cap, int D, int B, int k, int kStages,
+                    int* __restrict__ status)
 {
     namespace cg = cooperative_groups;
     using L = DescentUmmaPairLayout<NP>;
@@ -402,8 +429,13 @@ k_descent_umma_pair(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             const int p = umma_walk<NP>(bits, k);
             const int tok = tile * kUM + warp * 32 + lane;
             const int key = p - ((1 << k) - 1);
-            if (tok < B) pos_out[tok] = key;
-            if (rank8) {
+            if (tok < B) {
+                pos_out[tok] = key;
+                if (pos_out2) pos_out2[tok] = key;
+            }
+            if (cursor) {
+                slot_tokens(tok < B, key, k, tok, cursor, slots, cap);
+            } else if (rank8) {
                 const int nbins = 1 << k;
                 const bool in = tok < B;
                 const unsigned peers = peers_by_ballot(in, key, k);

@@ -135,6 +135,10 @@ __global__ void k_pack_w2_umma(const T* __restrict__ w2, const T* __restrict__ b
 // sched: two ints, both zero before the first launch and again after every launch: [0] list entries
 // handed out so far, [1] CTAs that have finished.
 // kFold: l < LP, the spare hidden column l carries the output bias (see k_pack_w2_umma).
+// slot_counts (optional): instead of a tile list, the lists the descent kernel filled directly (slot_tokens):
+// perm[bin * cap + i], i < slot_counts[bin], are the tokens of bin.  The scheduler then derives the tiles itself:
+// every lane owns a run of bins and knows how many tiles precede it; a claimed number is resolved by the lane
+// whose range holds it.  The last CTA to finish clears the counts for the next call.
 template <int LP, bool kFold>
 __global__ void __launch_bounds__(kLUThreads, 1)
 k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restrict__ perm,
@@ -142,7 +146,7 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
             const __nv_bfloat16* __restrict__ w1img, const float* __restrict__ b1img,
             const unsigned char* __restrict__ w2img, __nv_bfloat16* __restrict__ y,
             int D, int O, int l, int act, int kStages, int wide_stores, int passes, int* __restrict__ sched,
-            int* __restrict__ status)
+            int32_t* __restrict__ slot_counts, int n_bins, int cap, int* __restrict__ status)
 {
     using L = LeafUmmaLayout<LP>;
     extern __shared__ unsigned char smem_raw[];
@@ -224,19 +228,60 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
         int published = 0;
         Tile last;
         last.bin = 0; last.start = 0; last.rows = -1; last.pad = 0;
+        // direct lists: tiles of this lane's bins, and of all lanes before it
+        const int per_lane = (n_bins + 31) >> 5;
+        const int bin0 = min(lane * per_lane, n_bins), bin1 = min(bin0 + per_lane, n_bins);
+        int tiles_incl = 0, tiles_mine = 0, tiles_all = 0;
+        if (slot_counts) {
+            for (int b = bin0; b < bin1; ++b) tiles_mine += (__ldcg(slot_counts + b) + kLUM - 1) / kLUM;
+            tiles_incl = tiles_mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(kFullMask, tiles_incl, o);
+                if (lane >= o) tiles_incl += v;
+            }
+            tiles_all = __shfl_sync(kFullMask, tiles_incl, 31);
+        }
         for (;;) {
             // tile n >= 2 is claimed once the gathers have started tile n - 1
             if (published >= 2 && !timed_out && !ptx::mbar_wait_relaxed(want, (uint32_t)(published - 1) & 1u)) timed_out = true;
             int idx = 0;
             if (lane == 0) idx = atomicAdd(sched, 1);
             idx = __shfl_sync(kFullMask, idx, 0);
+            Tile c;
+            if (slot_counts) {
+                if (idx >= tiles_all || ++fetched > max_iters) break;
+                int bin = 0, start = 0, rows = 0;
+                if (idx >= tiles_incl - tiles_mine && idx < tiles_incl) {       // exactly one lane
+                    int rem = idx - (tiles_incl - tiles_mine);
+                    for (int b = bin0; b < bin1; ++b) {
+                        const int cnt = __ldcg(slot_counts + b);
+                        const int t = (cnt + kLUM - 1) / kLUM;
+                        if (rem < t) {
+                            bin = b;
+                            start = b * cap + rem * kLUM;
+                            rows = min(kLUM, cnt - rem * kLUM);
+                            break;
+                        }
+                        rem -= t;
+                    }
+                }
+                const unsigned owner = __ballot_sync(kFullMask, rows > 0);
+                if (owner == 0) continue;
+                const int src = __ffs(owner) - 1;
+                c.bin = __shfl_sync(kFullMask, bin, src);
+                c.start = __shfl_sync(kFullMask, start, src);
+                c.rows = __shfl_sync(kFullMask, rows, src);
+                c.pad = 0;
+            } else {
             if (idx >= passes * n_tiles_total || ++fetched > passes * max_iters) break;
             // with two passes the full tiles go first and the ragged ones last, so that the work handed out
             // at the end comes in small pieces
             const int second = idx >= n_tiles_total ? 1 : 0;
-            const Tile c = tiles[idx - second * n_tiles_total];
+            c = tiles[idx - second * n_tiles_total];
+            }
             if (c.rows <= 0 || c.rows > kLUM) continue;          // empty list entry
-            if (passes == 2 && (c.rows == kLUM) != (second == 0)) continue;
+            if (!slot_counts && passes == 2 && (c.rows == kLUM) != (idx < n_tiles_total)) continue;
             if (!timed_out && !ptx::mbar_wait_relaxed(q_empty + q_slot, q_phase ^ 1)) timed_out = true;
             if (lane == 0) {
                 queue[q_slot] = c;
@@ -486,12 +531,21 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, kLUTmemCols);
     }
-    // the last CTA to finish rearms the scheduler words for the next launch
-    if (threadIdx.x == 0) {
-        __threadfence();
-        if (atomicAdd(sched + 1, 1) == (int)gridDim.x - 1) {
-            sched[0] = 0;
-            sched[1] = 0;
+    // the last CTA to finish rearms the scheduler words (and the direct lists' counts) for the next launch
+    if (warp == 0) {
+        int is_last = 0;
+        if (lane == 0) {
+            __threadfence();
+            is_last = atomicAdd(sched + 1, 1) == (int)gridDim.x - 1 ? 1 : 0;
+        }
+        is_last = __shfl_sync(kFullMask, is_last, 0);
+        if (is_last) {
+            if (slot_counts)
+                for (int b = lane; b < n_bins; b += 32) slot_counts[b] = 0;
+            if (lane == 0) {
+                sched[0] = 0;
+                sched[1] = 0;
+            }
             __threadfence();
         }
     }

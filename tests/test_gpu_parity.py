@@ -284,6 +284,42 @@ def test_descent_alone_then_forward():
     layer.close()
 
 
+@pytest.mark.parametrize("routing", ["spread", "one_leaf"])
+def test_forward_without_bucketing_kernel(routing):
+    """A tree of at most eight levels in front of the tensor-core leaf kernel: the descent files the tokens under
+    their leaves itself, so a forward is two launches.  With zero node weights every logit is 0, which goes right
+    (Algorithm 1: c >= 1/2), and the last leaf receives the whole batch: one list of many tiles, all others empty.
+    The stable bucketing is still reported afterwards, and repeated calls start from cleared lists."""
+    cfg = wl.FFFConfig("bf16_d5_direct", 256, 128, 5, 16, "gelu", "bf16", 3000, "normal")
+    weights = wl.make_weights(cfg, 6)
+    if routing == "one_leaf":
+        weights["node_w"] = np.zeros_like(weights["node_w"])
+        weights["node_b"] = np.zeros_like(weights["node_b"])
+    net = orc.Net.from_config(cfg, weights)
+    src = wl.TokenSource(cfg, 6)
+    if routing == "spread":
+        wl.enforce_margin(src, lambda rows: orc.path_margin(net, rows, threads=util.ORACLE_THREADS))
+    case = util.Case(cfg, weights, net, src.x, 0)
+    y_ref, leaf_ref = orc.forward_i(net, case.x, threads=util.ORACLE_THREADS)
+    if routing == "one_leaf":
+        assert (leaf_ref == cfg.n_leaves - 1).all()
+    off_ref, perm_ref = orc.bucket(leaf_ref, cfg.n_leaves)
+    layer = util.make_layer(case)
+    x = util.to_device(case.x, "bf16")
+    for B in (cfg.B, 1000, cfg.B):
+        y, leaf = layer.forward_infer(x[:B])
+        torch.cuda.synchronize()
+        assert layer.last_launch_count() == 2
+        np.testing.assert_array_equal(leaf.cpu().numpy(), leaf_ref[:B])
+        util.check_outputs(y, y_ref[:B], "bf16")
+        off, perm = layer.last_bucketing(B)
+        off_b, perm_b = (off_ref, perm_ref) if B == cfg.B else orc.bucket(leaf_ref[:B], cfg.n_leaves)
+        np.testing.assert_array_equal(off.cpu().numpy(), off_b)
+        np.testing.assert_array_equal(perm.cpu().numpy(), perm_b)
+    assert layer.last_status() == 0
+    layer.close()
+
+
 def test_nan_inputs_stay_in_range():
     cfg = wl.FFFConfig("n", 64, 32, 4, 8, "gelu", "bf16", 64)
     case = util.make_case(cfg, 0)
