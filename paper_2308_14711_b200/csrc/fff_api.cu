@@ -81,6 +81,7 @@ struct fff_handle_s {
     int64_t slot_cap = 0;
     bool cursor_dirty = false;       // a descent has filled the lists and no leaf kernel has cleared the counts since
     bool slots_now = false;          // the call in progress uses the direct lists
+    bool slots_here = false;         // ... and the descent stage being launched is the one that fills them (the last)
     int max_bucket_clusters = 8;
     int32_t* last_perm = nullptr; // where the most recent forward left its leaf permutation
     bool bucketing_pending = false;   // the last forward skipped the leaf bucketing; ws_leaf holds its leaf indices
@@ -305,7 +306,7 @@ fff_status_t grow_workspace(fff_handle_s* h, int64_t B) {
     if ((s = dmalloc((void**)&h->ws_tiles, sizeof(fff::Tile) * max_tiles(h, B))) != FFF_OK) return s;
     // direct lists: every leaf's list can take the whole batch, so their size grows with n_leaves * B; beyond
     // kMaxSlotBytes the forward keeps the bucketing kernel instead
-    if (h->ustages.size() == 1 && h->ustages[0].umma && h->ustages[0].k == h->depth && h->w2uimg &&
+    if (!h->ustages.empty() && h->ustages.back().umma && h->ustages.back().L0 + h->ustages.back().k == h->depth && h->w2uimg &&
         (size_t)h->n_leaves * (size_t)B * sizeof(int32_t) <= kMaxSlotBytes) {
         if ((s = dmalloc((void**)&h->ws_slots, sizeof(int32_t) * (size_t)h->n_leaves * (size_t)B)) != FFF_OK) return s;
         if ((s = clone((void**)&h->ws_cursor, nullptr, sizeof(int32_t) * (size_t)h->n_leaves)) != FFF_OK) return s;
@@ -507,7 +508,7 @@ struct SlotArgs {
 };
 SlotArgs slot_args(const fff_handle_s* h, const int32_t* pos_out) {
     SlotArgs a;
-    if (!h->slots_now) return a;
+    if (!h->slots_here) return a;
     a.pos2 = pos_out == h->ws_leaf ? nullptr : h->ws_leaf;
     a.cursor = h->ws_cursor;
     a.slots = h->ws_slots;
@@ -599,9 +600,10 @@ fff_status_t launch_descent_umma_grouped(fff_handle_s* h, const fff_handle_s::De
     if (!make_x_tensor_map(&tm, x, B, h->D, 1)) return FFF_ERR_CUDA;       // one-row boxes: rows are gathered four at a time
     const int n_tiles = tile_list_len(B, fff::kUM, 1 << sg.L0);
     const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(h->sm_count, n_tiles));
+    const SlotArgs sl = slot_args(h, pos_out);
     if (launch_chain(h, fff::k_descent_umma_grouped<NP>, (unsigned)grid, fff::kUGThreads, (size_t)L::smem_bytes(stages), st, 1, tm,
                      perm, (const fff::Tile*)h->ws_tiles, n_tiles, (const __nv_bfloat16*)sg.wimg, (const float*)sg.bimg, pos_out,
-                     h->D, sg.k, stages, h->d_status) != cudaSuccess)
+                     sl.pos2, sl.cursor, sl.slots, sl.cap, h->D, sg.k, stages, h->d_status) != cudaSuccess)
         return cudaGetLastError(), FFF_ERR_CUDA;
     return launched(h, st, "tree_descent_umma_grouped");
 }
@@ -687,9 +689,11 @@ fff_status_t run_descent(fff_handle_s* h, const void* x, int32_t* leaf_out, Coar
         }
         const bool last = level + sg.k == h->depth;
         int32_t* out = last ? leaf_out : h->ws_pos[i & 1];
+        h->slots_here = h->slots_now && last;
         s = i == 0 && sg.umma ? run_descent_umma(h, sg, x, out, B, st)
             : grouped_umma    ? run_descent_umma_grouped(h, sg, x, prev.perm, out, B, st)
                               : run_descent_mma(h, sg, x, prev.perm, i > 0, out, B, st);
+        h->slots_here = false;
         if (s != FFF_OK) return s;
         level += sg.k;
         pos = out;
@@ -1251,12 +1255,13 @@ fff_status_t fff_forward_infer(fff_handle_t h, const void* x, void* y, int32_t* 
     DescentTail tail;
     const LeafPlan plan = tensor_leaf ? leaf_plan(h, B) : LeafPlan{};
     const int tile_rows = plan.tile_rows;
-    // One tcgen05 stage is the whole descent and the tcgen05 leaf kernel takes whole 128-row tiles of one leaf:
-    // the descent files the tokens under their leaves itself and the leaf kernel follows at once.
+    // The descent ends with a tcgen05 stage and the tcgen05 leaf kernel takes whole 128-row tiles of one leaf:
+    // that stage files the tokens under their leaves itself and the leaf kernel follows at once.
     static const bool no_slots = std::getenv("FFF_NO_DIRECT_LISTS") != nullptr;      // tuning aid
     h->slots_now = !no_slots && tensor_leaf && plan.umma && plan.pack <= 1 && tile_rows == fff::kLUM && h->ws_slots &&
-                   B <= h->slot_cap && h->n_leaves * h->slot_cap <= INT32_MAX && dense_stage_count(h, B) == 1 &&
-                   h->ustages.size() == 1;
+                   B <= h->slot_cap && h->n_leaves * h->slot_cap <= INT32_MAX &&
+                   dense_stage_count(h, B) == (int)h->ustages.size() &&
+                   (h->ustages.size() == 1 || (B >> h->ustages.back().L0) >= 64);
     if (h->slots_now) {
         if (h->cursor_dirty && cudaMemsetAsync(h->ws_cursor, 0, sizeof(int32_t) * (size_t)h->n_leaves, st) != cudaSuccess)
             return h->slots_now = false, cudaGetLastError(), FFF_ERR_CUDA;

@@ -503,11 +503,13 @@ template <int NP> struct DescentUmmaGroupedLayout {
 };
 
 // wimg: [group][D / 64][NP rows][64 columns] swizzled, bimg: [group][NP] float32 (k_pack_nodes).
+// pos_out2 / cursor / slots / cap (optional): as in the first stage (slot_tokens).
 template <int NP>
 __global__ void __launch_bounds__(kUGThreads, 1)
 k_descent_umma_grouped(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restrict__ perm,
                        const Tile* __restrict__ tiles, int n_tiles_total, const __nv_bfloat16* __restrict__ wimg,
-                       const float* __restrict__ bimg, int32_t* __restrict__ pos_out, int D, int k, int kStages,
+                       const float* __restrict__ bimg, int32_t* __restrict__ pos_out, int32_t* __restrict__ pos_out2,
+                       int32_t* __restrict__ cursor, int32_t* __restrict__ slots, int cap, int D, int k, int kStages,
                        int* __restrict__ status)
 {
     using L = DescentUmmaGroupedLayout<NP>;
@@ -653,7 +655,13 @@ k_descent_umma_grouped(const __grid_constant__ CUtensorMap tmap_x, const int32_t
                 const uint32_t w = (NP == 64 && p >= 32) ? bits_hi : bits;
                 p = 2 * p + 1 + (int)((w >> (p & 31)) & 1u);
             }
-            if (tok >= 0) pos_out[tok] = (tl.bin << k) + (p - ((1 << k) - 1));
+            const int key = (tl.bin << k) + (p - ((1 << k) - 1));
+            if (tok >= 0) {
+                pos_out[tok] = key;
+                if (pos_out2) pos_out2[tok] = key;
+            }
+            // (the keys of a tile differ in their low k bits only)
+            if (cursor) slot_tokens(tok >= 0, key, k, (int)tok, cursor, slots, cap);
             ++it;
         }
     }

@@ -232,8 +232,18 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
         const int per_lane = (n_bins + 31) >> 5;
         const int bin0 = min(lane * per_lane, n_bins), bin1 = min(bin0 + per_lane, n_bins);
         int tiles_incl = 0, tiles_mine = 0, tiles_all = 0;
+        // (the counts are read with ordinary loads, so that the repeated walks below hit in L1; nothing writes them
+        // while any CTA still reads them)
+        const bool vec4 = (per_lane & 3) == 0;               // whole 16-byte groups of counts per lane
         if (slot_counts) {
-            for (int b = bin0; b < bin1; ++b) tiles_mine += (__ldcg(slot_counts + b) + kLUM - 1) / kLUM;
+            if (vec4) {
+                for (int b = bin0; b < bin1; b += 4) {
+                    const int4 c4 = *reinterpret_cast<const int4*>(slot_counts + b);
+                    tiles_mine += (c4.x + kLUM - 1) / kLUM + (c4.y + kLUM - 1) / kLUM + (c4.z + kLUM - 1) / kLUM + (c4.w + kLUM - 1) / kLUM;
+                }
+            } else {
+                for (int b = bin0; b < bin1; ++b) tiles_mine += (slot_counts[b] + kLUM - 1) / kLUM;
+            }
             tiles_incl = tiles_mine;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -254,16 +264,24 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                 int bin = 0, start = 0, rows = 0;
                 if (idx >= tiles_incl - tiles_mine && idx < tiles_incl) {       // exactly one lane
                     int rem = idx - (tiles_incl - tiles_mine);
-                    for (int b = bin0; b < bin1; ++b) {
-                        const int cnt = __ldcg(slot_counts + b);
+                    // branch-free walk over this lane's bins (the loads do not depend on the running search)
+                    auto visit = [&](int b, int cnt) {
                         const int t = (cnt + kLUM - 1) / kLUM;
-                        if (rem < t) {
+                        if (rows == 0 && rem < t) {
                             bin = b;
                             start = b * cap + rem * kLUM;
                             rows = min(kLUM, cnt - rem * kLUM);
-                            break;
                         }
                         rem -= t;
+                    };
+                    if (vec4) {
+#pragma unroll 4
+                        for (int b = bin0; b < bin1; b += 4) {
+                            const int4 c4 = *reinterpret_cast<const int4*>(slot_counts + b);
+                            visit(b, c4.x); visit(b + 1, c4.y); visit(b + 2, c4.z); visit(b + 3, c4.w);
+                        }
+                    } else {
+                        for (int b = bin0; b < bin1; ++b) visit(b, slot_counts[b]);
                     }
                 }
                 const unsigned owner = __ballot_sync(kFullMask, rows > 0);
