@@ -320,6 +320,31 @@ def test_forward_without_bucketing_kernel(routing):
     layer.close()
 
 
+def test_two_stage_descent_without_leaf_bucketing_kernel():
+    """Ten levels as two tensor-core stages in front of the tensor-core leaf kernel: a node bucketing between the
+    stages, then the second stage files the tokens under their leaves itself: four launches, no leaf bucketing
+    kernel.  The descent entry point alone is three launches and must leave nothing behind for the next forward."""
+    cfg = wl.FFFConfig("bf16_d10_direct", 128, 64, 10, 16, "gelu", "bf16", 20000, "clusters")
+    case = util.make_case(cfg, seed=8)
+    y_ref, leaf_ref = orc.forward_i(case.net, case.x, threads=util.ORACLE_THREADS)
+    layer = util.make_layer(case)
+    x = util.to_device(case.x, "bf16")
+    for B in (cfg.B, 17000, cfg.B):
+        y, leaf = layer.forward_infer(x[:B])
+        torch.cuda.synchronize()
+        assert layer.last_launch_count() == 4
+        np.testing.assert_array_equal(leaf.cpu().numpy(), leaf_ref[:B])
+        util.check_outputs(y, y_ref[:B], "bf16")
+        off, perm = layer.last_bucketing(B)
+        off_b, perm_b = orc.bucket(leaf_ref[:B], cfg.n_leaves)
+        np.testing.assert_array_equal(off.cpu().numpy(), off_b)
+        np.testing.assert_array_equal(perm.cpu().numpy(), perm_b)
+        np.testing.assert_array_equal(layer.tree_descent(x[:B]).cpu().numpy(), leaf_ref[:B])
+        assert layer.last_launch_count() == 3
+    assert layer.last_status() == 0
+    layer.close()
+
+
 def test_nan_inputs_stay_in_range():
     cfg = wl.FFFConfig("n", 64, 32, 4, 8, "gelu", "bf16", 64)
     case = util.make_case(cfg, 0)
