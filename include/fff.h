@@ -215,10 +215,12 @@ fff_status_t fff_grouped_leaf_ff(fff_handle_t h, const void *x, const int32_t *l
                                  int64_t B, void *cuda_stream);
 
 /* Copy the bucketing of the handle's most recent forward into caller buffers
- * (device): perm [B], offsets [2^depth + 1].  Enqueued on `cuda_stream`.  When the
- * forward had fewer than about 4 tokens per leaf and evaluated the leaves one
- * token at a time, it did not need the bucketing; it is then computed here, from
- * the leaf indices the forward kept in the handle's workspace. */
+ * (device): perm [B], offsets [2^depth + 1].  Enqueued on `cuda_stream`.  Two kinds
+ * of forward do not make the stable bucketing themselves: one with fewer than
+ * about 4 tokens per leaf, which evaluates the leaves one token at a time, and one
+ * whose descent files the tokens under their leaves directly for the tensor-core
+ * leaf kernel (in an order that is not the stable one).  The bucketing is then
+ * computed here, from the leaf indices the forward kept in the handle's workspace. */
 fff_status_t fff_debug_get_bucketing(fff_handle_t h, int32_t *perm, int32_t *offsets,
                                      void *cuda_stream);
 
