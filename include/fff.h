@@ -106,6 +106,9 @@ fff_status_t fff_create(fff_handle_t *out, int D, int O, int depth, int leaf_wid
  *
  * B == 0 is FFF_OK and enqueues nothing.  If B exceeds what fff_reserve was
  * given, the workspace is grown first (this allocates and synchronises).
+ * Otherwise the call only enqueues kernels (and at most a small memset) and
+ * returns: after fff_reserve(B) and one ordinary call of the same size, it may
+ * be captured into a CUDA graph and replayed on new contents of x (tested).
  */
 fff_status_t fff_forward_infer(fff_handle_t h, const void *x, void *y, int32_t *leaf_idx,
                                int64_t B, void *cuda_stream);

@@ -345,6 +345,46 @@ def test_two_stage_descent_without_leaf_bucketing_kernel():
     layer.close()
 
 
+@pytest.mark.parametrize("cfg", [
+    wl.FFFConfig("graph_bf16_d6", 256, 128, 6, 16, "gelu", "bf16", 3000, "normal"),       # tensor kernels, direct leaf lists
+    wl.FFFConfig("graph_bf16_d10", 128, 64, 10, 16, "gelu", "bf16", 20000, "clusters"),   # two descent stages, node bucketing
+    wl.FFFConfig("graph_f32_d3", 784, 10, 3, 32, "relu", "f32", 517, "normal"),           # warp kernels
+], ids=lambda c: c.name)
+def test_forward_replayed_from_a_cuda_graph(cfg):
+    """A forward enqueues kernels (and at most a small memset) on the caller's stream and, once the workspace has its
+    size, neither allocates nor synchronises: it can be captured into a CUDA graph and replayed on new contents of
+    the same buffers."""
+    case = util.make_case(cfg, seed=9)
+    y_ref, leaf_ref = orc.forward_i(case.net, case.x, threads=util.ORACLE_THREADS)
+    layer = util.make_layer(case)
+    layer.reserve(cfg.B)
+    td = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
+    x_all = util.to_device(case.x, cfg.dtype)
+    x = torch.zeros_like(x_all)
+    y = torch.empty((cfg.B, cfg.O), dtype=td, device="cuda")
+    leaf = torch.empty((cfg.B,), dtype=torch.int32, device="cuda")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        layer.forward_infer(x, y=y, leaf_idx=leaf, stream=side)          # warm-up outside the capture
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        layer.forward_infer(x, y=y, leaf_idx=leaf, stream=torch.cuda.current_stream())
+    for _ in range(2):
+        y.zero_()
+        leaf.fill_(-1)
+        x.copy_(x_all)
+        graph.replay()
+        torch.cuda.synchronize()
+        np.testing.assert_array_equal(leaf.cpu().numpy(), leaf_ref)
+        util.check_outputs(y, y_ref, cfg.dtype)
+    assert layer.last_status() == 0
+    del graph
+    layer.close()
+
+
 def test_nan_inputs_stay_in_range():
     cfg = wl.FFFConfig("n", 64, 32, 4, 8, "gelu", "bf16", 64)
     case = util.make_case(cfg, 0)
