@@ -320,6 +320,39 @@ def test_forward_without_bucketing_kernel(routing):
     layer.close()
 
 
+@pytest.mark.parametrize("routing", ["spread", "one_leaf"])
+def test_warp_kernels_changing_batch_sizes(routing):
+    """float32 layer with eight leaves (the warp kernels: descent, bucketing, leaf), also with every token in the last
+    leaf (zero node weights: a logit of 0 goes right), and with batch sizes that change from call to call."""
+    cfg = wl.FFFConfig("f32_d3_batches", 784, 10, 3, 32, "relu", "f32", 2048, "normal")
+    weights = wl.make_weights(cfg, 3)
+    if routing == "one_leaf":
+        weights["node_w"] = np.zeros_like(weights["node_w"])
+        weights["node_b"] = np.zeros_like(weights["node_b"])
+    net = orc.Net.from_config(cfg, weights)
+    src = wl.TokenSource(cfg, 3)
+    if routing == "spread":
+        wl.enforce_margin(src, lambda rows: orc.path_margin(net, rows, threads=util.ORACLE_THREADS))
+    case = util.Case(cfg, weights, net, src.x, 0)
+    y_ref, leaf_ref = orc.forward_i(net, case.x, threads=util.ORACLE_THREADS)
+    if routing == "one_leaf":
+        assert (leaf_ref == cfg.n_leaves - 1).all()
+    layer = util.make_layer(case)
+    x = util.to_device(case.x, "f32")
+    for B in (cfg.B, 33, 1500, cfg.B):
+        y, leaf = layer.forward_infer(x[:B])
+        torch.cuda.synchronize()
+        assert layer.last_launch_count() == 3
+        np.testing.assert_array_equal(leaf.cpu().numpy(), leaf_ref[:B])
+        util.check_outputs(y, y_ref[:B], "f32")
+        off, perm = layer.last_bucketing(B)
+        off_b, perm_b = orc.bucket(leaf_ref[:B], cfg.n_leaves)
+        np.testing.assert_array_equal(off.cpu().numpy(), off_b)
+        np.testing.assert_array_equal(perm.cpu().numpy(), perm_b)
+    assert layer.last_status() == 0
+    layer.close()
+
+
 def test_two_stage_descent_without_leaf_bucketing_kernel():
     """Ten levels as two tensor-core stages in front of the tensor-core leaf kernel: a node bucketing between the
     stages, then the second stage files the tokens under their leaves itself: four launches, no leaf bucketing
