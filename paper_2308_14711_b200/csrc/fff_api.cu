@@ -516,6 +516,18 @@ SlotArgs slot_args(const fff_handle_s* h, const int32_t* pos_out) {
     return a;
 }
 
+// CTAs for `units` equal work units walked with a static stride on at most `max_ctas` CTAs: the fewest CTAs that
+// still need no more rounds, so that all of them finish together (512 tiles on 148 SMs: 128 CTAs with 4 tiles
+// each instead of 68 with 4 and 80 with 3; the memory system is shared, so the idle SMs cost nothing).
+int64_t balanced_grid(int64_t max_ctas, int64_t units) {
+    static const bool off = std::getenv("FFF_NO_BALANCED_GRID") != nullptr;      // tuning aid
+    max_ctas = std::max<int64_t>(1, max_ctas);
+    if (units <= max_ctas) return std::max<int64_t>(1, units);
+    if (off) return max_ctas;
+    const int64_t rounds = (units + max_ctas - 1) / max_ctas;
+    return (units + rounds - 1) / rounds;
+}
+
 template <int NP>
 fff_status_t launch_descent_umma(fff_handle_s* h, const fff_handle_s::DenseStage& sg, const void* x, int32_t* pos_out,
                                  int64_t B, cudaStream_t st) {
@@ -525,7 +537,7 @@ fff_status_t launch_descent_umma(fff_handle_s* h, const fff_handle_s::DenseStage
     CUtensorMap tm;
     if (!make_x_tensor_map(&tm, x, B, h->D, fff::kUM)) return FFF_ERR_CUDA;
     const int64_t n_tiles = (B + fff::kUM - 1) / fff::kUM;
-    const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(h->sm_count, n_tiles));
+    const int64_t grid = balanced_grid(h->sm_count, n_tiles);
     const bool ranked = sg.k >= 4 && h->ws_rank8 && h->ws_counts8;      // also rank the tokens for the bucketing that follows
     int32_t* sums = nullptr;
     if (blocksum_for_descent(h, B, ranked, st, &sums) != FFF_OK) return FFF_ERR_CUDA;
@@ -555,7 +567,7 @@ fff_status_t launch_descent_umma_pair(fff_handle_s* h, const fff_handle_s::Dense
     // the weight image as (D/64) * NP rows of 64 columns, stored pre-swizzled: copied as it is
     if (!make_x_tensor_map(&tw, sg.wimg, (int64_t)(h->D / fff::kUKB) * NP, fff::kUKB, NP / 2, false)) return FFF_ERR_CUDA;
     const int64_t n_pairs = ((B + fff::kUM - 1) / fff::kUM + 1) / 2;
-    const int64_t grid = 2 * std::max<int64_t>(1, std::min<int64_t>(h->sm_count / 2, n_pairs));
+    const int64_t grid = 2 * balanced_grid(h->sm_count / 2, n_pairs);
     const bool ranked = sg.k >= 4 && h->ws_rank8 && h->ws_counts8;
     int32_t* sums = nullptr;
     if (blocksum_for_descent(h, B, ranked, st, &sums) != FFF_OK) return FFF_ERR_CUDA;
