@@ -132,7 +132,10 @@ fff_status_t fff_forward_infer_host(fff_handle_t h, const void *x_host, void *y_
 fff_status_t fff_destroy(fff_handle_t h);
 
 /* Size the workspace for batches of up to max_B tokens so that later forwards
- * allocate nothing.  Allocates and synchronises. */
+ * allocate nothing.  Allocates and synchronises.  The workspace is a few
+ * int32 per token, plus, on the tensor-core path, a table of per-leaf token
+ * lists of 2^depth * max_B int32 (only while that is at most 1 GiB; larger
+ * layers run a bucketing kernel instead), of which a forward touches B entries. */
 fff_status_t fff_reserve(fff_handle_t h, int64_t max_B);
 
 /* Pin the handle to one kernel family (FFF_PATH_*).  FFF_ERR_UNSUPPORTED if
