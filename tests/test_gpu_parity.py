@@ -378,6 +378,33 @@ def test_two_stage_descent_without_leaf_bucketing_kernel():
     layer.close()
 
 
+def test_leaf_lists_too_large_fall_back_to_the_bucketing_kernel():
+    """2048 leaves x 140 000 tokens x 4 bytes is more than the table of per-leaf lists may take (1 GiB): the forward
+    then buckets by leaf with a kernel again (five launches) and reports that stable bucketing directly."""
+    cfg = wl.FFFConfig("bf16_d11_big_batch", 128, 64, 11, 16, "gelu", "bf16", 140000, "normal")
+    case = util.make_case(cfg, seed=11)
+    y_ref, leaf_ref = orc.forward_i(case.net, case.x, threads=util.ORACLE_THREADS)
+    off_ref, perm_ref = orc.bucket(leaf_ref, cfg.n_leaves)
+    layer = util.make_layer(case)
+    x = util.to_device(case.x, "bf16")
+    for _ in range(2):
+        y, leaf = layer.forward_infer(x)
+        torch.cuda.synchronize()
+        assert layer.last_launch_count() == 5
+        np.testing.assert_array_equal(leaf.cpu().numpy(), leaf_ref)
+        util.check_outputs(y, y_ref, "bf16")
+        off, perm = layer.last_bucketing(cfg.B)
+        np.testing.assert_array_equal(off.cpu().numpy(), off_ref)
+        np.testing.assert_array_equal(perm.cpu().numpy(), perm_ref)
+    # a batch small enough for the lists on the same handle (the workspace keeps its size: still no lists)
+    y, leaf = layer.forward_infer(x[:40000])
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(leaf.cpu().numpy(), leaf_ref[:40000])
+    util.check_outputs(y, y_ref[:40000], "bf16")
+    assert layer.last_status() == 0
+    layer.close()
+
+
 @pytest.mark.parametrize("cfg", [
     wl.FFFConfig("graph_bf16_d6", 256, 128, 6, 16, "gelu", "bf16", 3000, "normal"),       # tensor kernels, direct leaf lists
     wl.FFFConfig("graph_bf16_d10", 128, 64, 10, 16, "gelu", "bf16", 20000, "clusters"),   # two descent stages, node bucketing
