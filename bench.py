@@ -6,7 +6,9 @@
 One step = one pass of the whole path (tree descent, leaf bucketing, grouped leaf evaluation with
 un-permuting write-back) over one batch of synthetic tokens.  Prints ONE JSON line (rank 0).
 
-  value      tokens/s with inputs resident in HBM (CUDA events around K steps, max over ranks)
+  value      tokens/s with inputs resident in HBM: CUDA events around a region of exactly K steps, max over
+             ranks; the region is repeated back to back (R times, at least 0.25 s in all) and the median
+             region is the headline, the fastest one is reported beside it
   e2e        tokens/s through fff_forward_infer_host: pinned host x -> device, forward, y and leaf_idx -> host
   roofline   dominant kernel: algorithmic bytes per launch / mean launch time (events recorded by the library
              on the launching stream inside the timed region) against the measured HBM copy bandwidth
@@ -39,7 +41,8 @@ from paper_2308_14711_b200 import replicas, workloads as wl  # noqa: E402
 DEFAULT_CONFIG = "vit_d8_l12_bf16"
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
-L2_BYTES = 126 * 1024 * 1024
+L2_BYTES_NOMINAL = 126 * 1024 * 1024      # used only when the device attribute cannot be read
+MIN_TIMED_SECONDS = 0.25                  # the K-step region is repeated until the timed span is at least this long
 METRIC = "FFF hard-inference tokens/sec"
 UNIT = "tokens/s"
 
@@ -194,13 +197,23 @@ def make_device_case(cfg: wl.FFFConfig, seed: int, n_sets: int):
     return layer, w, xs_host, xs, ys, ls, td
 
 
+def l2_bytes() -> int:
+    try:
+        import torch
+        return int(torch.cuda.get_device_properties(torch.cuda.current_device()).L2_cache_size)
+    except Exception:
+        return L2_BYTES_NOMINAL
+
+
 def n_buffer_sets(cfg: wl.FFFConfig) -> int:
     per_set = cfg.B * (cfg.D + cfg.O) * cfg.elem_bytes
-    return max(2, min(64, int(np.ceil(2.5 * L2_BYTES / per_set))))
+    return max(2, min(64, int(np.ceil(2.5 * l2_bytes() / per_set))))
 
 
-def time_device(layer, xs, ys, ls, steps: int, warmup: int, profile: bool):
-    """K forwards on resident inputs, rotating buffer sets. Returns (ms total, launches, profile, t0, t1)."""
+def time_device(layer, xs, ys, ls, steps: int, warmup: int, profile: bool, min_seconds: float = 0.0):
+    """Regions of exactly `steps` forwards on resident inputs, rotating buffer sets, each between two CUDA
+    events on the launching stream; repeated back to back until the span lasts min_seconds.
+    Returns (list of ms per region, launches of one region, profile, t0, t1)."""
     import torch
     n = len(xs)
     for i in range(warmup):
@@ -208,19 +221,41 @@ def time_device(layer, xs, ys, ls, steps: int, warmup: int, profile: bool):
     torch.cuda.synchronize()
     if profile:
         layer.profile_begin(steps)
-    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    launches = 0
+    regions, launches = [], 0
     torch.cuda.synchronize()
     t0 = time.perf_counter()
-    start.record()
-    for i in range(steps):
-        layer.forward_infer(xs[i % n], ys[i % n], ls[i % n])
-        launches += layer.last_launch_count()
-    stop.record()
+    while True:
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        launches = 0
+        start.record()
+        for i in range(steps):
+            layer.forward_infer(xs[i % n], ys[i % n], ls[i % n])
+            launches += layer.last_launch_count()
+        stop.record()
+        regions.append((start, stop))
+        if profile or len(regions) >= 4096 or time.perf_counter() - t0 >= min_seconds:
+            break
     torch.cuda.synchronize()
     t1 = time.perf_counter()
     prof = layer.profile_end() if profile else None
-    return start.elapsed_time(stop), launches, prof, t0, t1
+    return [a.elapsed_time(b) for a, b in regions], launches, prof, t0, t1
+
+
+def dominant_kernel_roofline(prof, cfg, B, leaves_touched, peaks, steps, ms_prof):
+    """The roofline object of the launch that takes longest, from the per-launch events of a profiled pass."""
+    kernels, prof_steps = prof
+    if not kernels:
+        return None
+    name, kms = max(kernels, key=lambda kv: kv[1])
+    kb = kernel_bytes(name, cfg, B, leaves_touched)
+    achieved = kb / (kms * 1e-3) / 1e9
+    traffic, traffic_note = ncu_traffic(name, cfg.name)
+    return {"bound": "hbm", "kernel": name, "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"],
+            "unit": "GB/s", "frac": round(achieved / peaks["hbm_gbs"], 4), "traffic": traffic,
+            "peak_source": peaks["source"], "kernel_ms": round(kms, 5), "algorithmic_bytes": int(kb),
+            "launches_ms": {f"{i}:{n}": round(m, 5) for i, (n, m) in enumerate(kernels)},
+            "profiled_steps": prof_steps, "profiled_ms_per_step": round(ms_prof / steps, 5),
+            "traffic_note": traffic_note}
 
 
 def run_ours(args, rank: int, world: int, local_rank: int):
@@ -248,32 +283,23 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     sampler = ClockSampler(local_rank)
     sampler.start()
     barrier()
-    ms, launches, _, t0, t1 = time_device(layer, xs, ys, ls, args.steps, args.warmup, profile=False)
+    region_ms, launches, _, t0, t1 = time_device(layer, xs, ys, ls, args.steps, args.warmup, profile=False,
+                                                 min_seconds=MIN_TIMED_SECONDS)
     barrier()
     clocks = sampler.stop(t0, t1)
-    ms = max_over_ranks(ms)
+    # every rank ran its own number of regions; the median region of each rank, then the max over ranks
+    ms = max_over_ranks(statistics.median(region_ms))
+    ms_min = max_over_ranks(min(region_ms))
     # the same K steps once more with one CUDA event after every launch (recorded by the library on the
     # launching stream): per-kernel durations for the roofline.  Kept out of the headline region because
     # the extra events lengthen the gaps between these short kernels.
-    ms_prof, _, prof, _, _ = time_device(layer, xs, ys, ls, args.steps, 3, profile=True)
+    prof_ms, _, prof, _, _ = time_device(layer, xs, ys, ls, args.steps, 3, profile=True)
     status = layer.last_status()
     ms_per_step = ms / args.steps
     value = replicas.whole_job_throughput(B, args.steps, world, ms)
 
     leaves_touched = int(torch.unique(ls[0]).numel())
-    kernels, prof_steps = prof
-    roofline = None
-    if kernels:
-        name, kms = max(kernels, key=lambda kv: kv[1])
-        kb = kernel_bytes(name, cfg, B, leaves_touched)
-        achieved = kb / (kms * 1e-3) / 1e9
-        traffic, traffic_note = ncu_traffic(name, cfg.name)
-        roofline = {"bound": "hbm", "kernel": name, "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"],
-                    "unit": "GB/s", "frac": round(achieved / peaks["hbm_gbs"], 4), "traffic": traffic,
-                    "peak_source": peaks["source"], "kernel_ms": round(kms, 5), "algorithmic_bytes": int(kb),
-                    "launches_ms": {f"{i}:{n}": round(m, 5) for i, (n, m) in enumerate(kernels)},
-                    "profiled_steps": prof_steps, "profiled_ms_per_step": round(ms_prof / args.steps, 5),
-                    "traffic_note": traffic_note}
+    roofline = dominant_kernel_roofline(prof, cfg, B, leaves_touched, peaks, args.steps, prof_ms[0])
     pb, pf = path_bytes(cfg, B, leaves_touched), path_flops(cfg, B)
     t_roof_ms = max(pf / (peaks["bf16_tflops"] * 1e12), pb / (peaks["hbm_gbs"] * 1e9)) * 1e3
     path_roofline = {"bound": "hbm" if pb / (peaks["hbm_gbs"] * 1e9) >= pf / (peaks["bf16_tflops"] * 1e12) else "tensor",
@@ -309,12 +335,14 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                       "l2": f"inputs larger than L2: {n_sets} rotating x/y buffer sets of "
                             f"{B * (cfg.D + cfg.O) * cfg.elem_bytes / 1e6:.0f} MB",
                       "parallelism": "replicas only" if world > 1 else "single GPU"},
-           "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "device_status": status,
-           "roofline": roofline, "path_roofline": path_roofline}
+           "path_roofline": path_roofline, "roofline": roofline,
+           "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "device_status": status}
 
     if rank == 0 and world == 1:
         if not args.no_cpu_baseline:
             out["cpu_baseline"] = cpu_baseline(cfg, w_host, xs_host[0], budget_s=args.cpu_budget)
+            # the oracle's own count of distinct leaves reached by buffer set 0 (the GPU's count sizes path_roofline)
+            path_roofline["leaves_touched_oracle"] = out["cpu_baseline"].pop("leaves_touched")
         if not args.no_per_config:
             out["per_config"] = per_config_table(args, peaks, skip={cfg.name: (ms_per_step, path_roofline)})
     layer.close()
@@ -337,20 +365,27 @@ def per_config_table(args, peaks, skip):
             n_sets = n_buffer_sets(cfg)
             layer, _, _, xs, ys, ls, _ = make_device_case(cfg, seed=0, n_sets=n_sets)
             steps = max(5, min(args.steps, 200))
-            ms, _, _, _, _ = time_device(layer, xs, ys, ls, steps, max(3, min(args.warmup, 10)), profile=False)
-            ms_step = ms / steps
+            region_ms, _, _, _, _ = time_device(layer, xs, ys, ls, steps, max(3, min(args.warmup, 10)), profile=False,
+                                                min_seconds=MIN_TIMED_SECONDS / 2)
+            ms_step = statistics.median(region_ms) / steps
             touched = int(torch.unique(ls[0]).numel())
             pb, pf = path_bytes(cfg, cfg.B, touched), path_flops(cfg, cfg.B)
             t_roof = max(pf / (peaks["bf16_tflops"] * 1e12), pb / (peaks["hbm_gbs"] * 1e9)) * 1e3
             pr = {"algorithmic_bytes": int(pb), "leaves_touched": touched, "roofline_ms": round(t_roof, 5),
                   "frac": round(t_roof / ms_step, 4),
                   "frac_at_8TBs": round(max(pf / 2.25e15, pb / 8e12) * 1e3 / ms_step, 4)}
+            # the per-launch split and the dominant kernel's roofline, as for the headline workload
+            psteps = min(steps, 50)
+            prof_ms, _, prof, _, _ = time_device(layer, xs, ys, ls, psteps, 3, profile=True)
+            pr["roofline"] = dominant_kernel_roofline(prof, cfg, cfg.B, touched, peaks, psteps, prof_ms[0])
             layer.close()
             del layer, xs, ys, ls
             torch.cuda.empty_cache()
         rows[name] = {"tokens_per_s": cfg.B / (ms_step * 1e-3), "ms_per_step": round(ms_step, 5),
                       "roofline_frac": pr["frac"], "roofline_frac_at_8TBs": pr["frac_at_8TBs"],
                       "leaves_touched": pr["leaves_touched"], "algorithmic_bytes": pr["algorithmic_bytes"]}
+        if pr.get("roofline"):
+            rows[name]["roofline"] = pr["roofline"]
     return rows
 
 
@@ -385,7 +420,8 @@ def cpu_baseline(cfg, w_host, x_host, budget_s: float = 20.0) -> dict:
     t = time.perf_counter()
     orc.forward_i(net, x_host[:n1], threads=1)
     dt1 = time.perf_counter() - t
-    return {"value": n * passes / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+    touched = int(np.unique(orc.descend(net, x_host, threads=cores)[0]).size)
+    return {"leaves_touched": touched, "value": n * passes / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"first {n} of {cfg.B} tokens of {cfg.name}, {passes} passes, float64 C oracle, {cores} threads",
             "seconds": round(dt, 3), "single_thread_value": n1 / dt1, "single_thread_sample_tokens": n1}
 
@@ -399,12 +435,15 @@ def run_reference(args, rank: int, world: int):
     cores = n_cores()
     w = wl.make_weights(cfg, 0)
     net = orc.Net.from_config(cfg, w)
-    x = wl.TokenSource(cfg, 0, B=min(cfg.B, 8192)).x
-    probe = min(x.shape[0], 256)
+    x = wl.TokenSource(cfg, 0).x
+    # per-token cost from one untimed pass over a few thousand tokens (a shorter probe overestimates it: thread start-up)
+    probe = min(x.shape[0], 4096)
+    orc.forward_i(net, x[:probe], threads=cores)
     t = time.perf_counter()
     orc.forward_i(net, x[:probe], threads=cores)
     per_tok = (time.perf_counter() - t) / probe
     total_steps = args.steps + args.warmup
+    # the GPU arm's batch when all steps then fit about two minutes, else the prefix that does
     n = int(max(32, min(x.shape[0], (120.0 / total_steps) / max(per_tok, 1e-9))))
     for _ in range(args.warmup):
         orc.forward_i(net, x[:n], threads=cores)

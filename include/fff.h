@@ -45,7 +45,7 @@ typedef struct fff_handle_s *fff_handle_t;
 typedef enum {
     FFF_OK = 0,
     FFF_ERR_INVALID_ARG = 1,     /* NULL / misaligned pointer, non-positive size, unknown enum, B < 0 */
-    FFF_ERR_UNSUPPORTED = 2,     /* valid request this build cannot serve (e.g. depth > FFF_MAX_DEPTH) */
+    FFF_ERR_UNSUPPORTED = 2,     /* valid request this build cannot serve (e.g. depth > FFF_MAX_DEPTH, B > FFF_MAX_TOKENS) */
     FFF_ERR_ALLOC = 3,           /* device or host allocation failed */
     FFF_ERR_CUDA = 4,            /* a CUDA runtime call failed */
     FFF_ERR_DEVICE_TIMEOUT = 5,  /* a bounded device-side wait ran out (read by fff_get_last_status) */
@@ -65,6 +65,8 @@ typedef enum {
 } fff_dtype_t;
 
 #define FFF_MAX_DEPTH 20
+/* Largest batch any call accepts (2^31 - 4096: token numbers and slice bounds are int32). */
+#define FFF_MAX_TOKENS 2147479552
 
 /* Kernel families a handle may be pinned to with fff_set_path (testing / tuning). */
 typedef enum {
@@ -142,6 +144,19 @@ fff_status_t fff_reserve(fff_handle_t h, int64_t max_B);
  * the shapes of this handle cannot run on it. */
 fff_status_t fff_set_path(fff_handle_t h, fff_path_t path);
 
+/* Switches between kernels that compute the same thing, for A/B timing and tests.  Every switch is on (1) by
+ * default, which is the measured best; results never depend on them.  The paper describes no such choices.
+ * FFF_ERR_INVALID_ARG for an unknown key or a value other than 0 or 1. */
+typedef enum {
+    FFF_TUNE_TCGEN05_DESCENT = 0, /* first descent stage of up to 8 levels on tcgen05 (0: stages of <= 6 levels on mma.sync) */
+    FFF_TUNE_TCGEN05_GROUPED = 1, /* later descent stages on tcgen05 when their groups fill 128-row tiles (0: mma.sync) */
+    FFF_TUNE_TCGEN05_LEAF = 2,    /* leaf evaluation on tcgen05 (0: mma.sync kernel) */
+    FFF_TUNE_CTA_PAIRS = 3,       /* first descent stage with 128 or 256 nodes on pairs of CTAs (0: single CTAs) */
+    FFF_TUNE_DIRECT_LISTS = 4,    /* the last descent stage files tokens under their leaves (0: bucketing kernel) */
+    FFF_TUNE_COUNT = 5
+} fff_tuning_t;
+fff_status_t fff_set_tuning(fff_handle_t h, fff_tuning_t key, int value);
+
 /* Leaf packing of the tcgen05 leaf kernel (bf16 tensor path): with only a few dozen tokens per leaf, `leaves`
  * = 2 or 4 leaves share the 128 rows of one tile (sub-tiles of 64 or 32 tokens), which shortens the kernel when
  * routing is close to uniform and lengthens it when a few leaves take most tokens (measured: 124 -> 118 us and
@@ -185,15 +200,18 @@ fff_status_t fff_leaf_bucketing(fff_handle_t h, const int32_t *leaf_idx, int32_t
  * memory and forbids cudaMalloc, or latency-critical loops in which an
  * allocation (which may synchronise the device) is unacceptable.  Such callers
  * cannot create an fff handle, whose workspace is allocated.  This entry point
- * computes exactly what fff_leaf_bucketing computes -- same kernels, same
- * result bit for bit -- but takes no handle and keeps its scratch (the
+ * returns exactly what fff_leaf_bucketing returns, bit for bit (the stable
+ * order is unique), through different kernels (a histogram, then a placement
+ * pass over ranges of leaves); it takes no handle and keeps its scratch (the
  * per-leaf token counts) in a fixed array compiled into the library:
  * 2 * FFF_STATIC_MAX_BINS int32 counters = 512 KiB, resident on every GPU
  * that loads the library, for the life of the process.
  *
- *   leaf_idx [B] in, values in [0, 2^depth); ids outside are ignored
+ *   leaf_idx [B] in, values in [0, 2^depth); ids outside are ignored (they
+ *            are not counted in offsets and take no perm entry, so the last
+ *            B - offsets[2^depth] entries of perm stay unwritten)
  *   offsets  [2^depth + 1] out,  perm [B] out      (as for fff_leaf_bucketing)
- *   depth    0 <= depth <= FFF_STATIC_MAX_DEPTH;  B <= 2^31 - 1
+ *   depth    0 <= depth <= FFF_STATIC_MAX_DEPTH;  B <= FFF_MAX_TOKENS
  *
  * Larger requests return FFF_ERR_TOO_LARGE and launch nothing.  The call uses
  * the current device; all pointers are device pointers on it.  It calls no

@@ -71,8 +71,9 @@ static void leaf_eval(int D, int O, int l, int act,
  * Hard descent of Algorithm 1, FORWARD_I, non-leaf branch, for one token: at
  * N_{m,n} take the right child N_{m+1,2n+1} when c >= 1/2, otherwise the left
  * child N_{m+1,2n}.  sigmoid is increasing with sigmoid(0) = 1/2, so c >= 1/2
- * exactly when the logit is >= 0 ("comparison of the logit to 0", paragraph
- * on inference complexity).  Returns n of the leaf N_{d,n} reached.
+ * exactly when the logit is >= 0 (the paper's own implementation note likewise
+ * tests the sign of the logit: Section "Algorithm", paragraph on inference
+ * complexity).  Returns n of the leaf N_{d,n} reached.
  */
 static long descend_one(int D, int depth, const double *node_w, const double *node_b,
                         const double *xt, double *min_abs, long *node_evals)
@@ -95,7 +96,8 @@ static long descend_one(int D, int depth, const double *node_w, const double *no
  * leaf_idx[t]  = n of the leaf N_{d,n} reached.
  * min_abs[t]   = smallest |logit| met on the path (NULL to skip); +inf if d = 0.
  * node_evals   = incremented once per node network executed (NULL to skip).
- * Pinned by: brute-force path enumeration, zero-weight tie case, hand case.
+ * Pinned by: brute-force path enumeration, zero-weight tie case, hand case
+ * (leaf indices and the per-token smallest |logit|).
  */
 void fff_oracle_descend(int D, int depth, const double *node_w, const double *node_b,
                         const double *x, long t0, long t1,

@@ -113,6 +113,7 @@ struct fff_handle_s {
     cudaEvent_t ev_in[kMaxHostChunks] = {}, ev_done[kMaxHostChunks] = {}, ev_start = nullptr, ev_end = nullptr;
 
     int path = FFF_PATH_AUTO;
+    bool tune[FFF_TUNE_COUNT] = {true, true, true, true, true};      // fff_set_tuning; every switch defaults to on
     bool pdl = true;              // launch every kernel of a forward but the first as a programmatic dependent
     int launches = 0;
     int64_t last_B = -1;
@@ -218,6 +219,21 @@ void release(fff_handle_s* h) {
 
 constexpr int kMinTileRows = 32;
 
+constexpr int kMaxDevices = 64;          // device ordinals the per-device tables below cover (fff_create checks)
+std::mutex g_attr_mu;
+
+// Raises a kernel's dynamic shared-memory limit on the handle's device, once per device and kernel
+// (`done` is that kernel's table).  Handles on different host threads may get here at the same time.
+template <typename K>
+bool raise_smem_limit(K kern, int device, int bytes, bool (&done)[kMaxDevices]) {
+    std::lock_guard<std::mutex> lk(g_attr_mu);
+    if (done[device]) return true;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess)
+        return cudaGetLastError(), false;
+    done[device] = true;
+    return true;
+}
+
 // Length of a tile list: floor(B / tile_rows) + nbins entries, some of them empty (see k_bucket_cluster).
 int tile_list_len(int64_t B, int tile_rows, int nbins) { return (int)(B / tile_rows) + nbins; }
 
@@ -236,36 +252,20 @@ struct LeafPlan {
 bool leaf_pack_fits(int LP, int pack);
 
 LeafPlan leaf_plan(const fff_handle_s* h, int64_t B) {
-    static const int forced = [] {
-        const char* e = std::getenv("FFF_LEAF_TILE_ROWS");      // tuning aid: 32 or 64
-        const int v = e ? std::atoi(e) : 0;
-        return (v == 32 || v == 64) ? v : 0;
-    }();
     // The tcgen05 kernel works on 128-row tiles.  Measured against the mma.sync kernel it is far ahead when
     // some buckets are large (skewed routing), about level with uniformly thin buckets of 32 tokens, and is
     // left out only when buckets are thinner still (every tile costs its epilogue a fixed few microseconds).
-    if (h->w2uimg && B >= 16 * h->n_leaves) {
-        static const int umma_rows = [] {
-            const char* e = std::getenv("FFF_UMMA_TILE_ROWS");  // tuning aid: a multiple of 4 up to 128
-            const int v = e ? std::atoi(e) : 0;
-            return (v >= 4 && v <= fff::kLUM && v % 4 == 0) ? v : 0;
-        }();
+    if (h->w2uimg && h->tune[FFF_TUNE_TCGEN05_LEAF] && B >= 16 * h->n_leaves) {
         // Thin buckets: several leaves may share the rows of a tile (fff_set_leaf_packing; off unless asked for,
         // because it loses when a few buckets hold most tokens, which the host cannot know here).
-        static const int forced_pack = [] {
-            const char* e = std::getenv("FFF_LEAF_PACK");       // tuning aid: 1, 2 or 4
-            const int v = e ? std::atoi(e) : 0;
-            return (v == 1 || v == 2 || v == 4) ? v : 0;
-        }();
         const int64_t avg = B / h->n_leaves;
         const int by_size = avg >= 96 ? 1 : avg >= 24 ? 2 : 4;
-        int pack = forced_pack ? forced_pack : h->leaf_pack == 0 ? by_size : h->leaf_pack;
-        if (!h->w2_finite || umma_rows) pack = 1;
+        int pack = h->leaf_pack == 0 ? by_size : h->leaf_pack;
+        if (!h->w2_finite) pack = 1;
         while (pack > 1 && !leaf_pack_fits(h->LP, pack)) pack >>= 1;
         if (pack > 1) return LeafPlan{fff::kLUM / pack, true, pack};
-        return LeafPlan{umma_rows ? umma_rows : fff::kLUM, true, 1};
+        return LeafPlan{fff::kLUM, true, 1};
     }
-    if (forced) return LeafPlan{forced, false, 1};
     return LeafPlan{B / h->n_leaves <= 40 ? 32 : 64, false, 1};
 }
 
@@ -520,10 +520,8 @@ SlotArgs slot_args(const fff_handle_s* h, const int32_t* pos_out) {
 // still need no more rounds, so that all of them finish together (512 tiles on 148 SMs: 128 CTAs with 4 tiles
 // each instead of 68 with 4 and 80 with 3; the memory system is shared, so the idle SMs cost nothing).
 int64_t balanced_grid(int64_t max_ctas, int64_t units) {
-    static const bool off = std::getenv("FFF_NO_BALANCED_GRID") != nullptr;      // tuning aid
     max_ctas = std::max<int64_t>(1, max_ctas);
     if (units <= max_ctas) return std::max<int64_t>(1, units);
-    if (off) return max_ctas;
     const int64_t rounds = (units + max_ctas - 1) / max_ctas;
     return (units + rounds - 1) / rounds;
 }
@@ -557,11 +555,8 @@ fff_status_t launch_descent_umma_pair(fff_handle_s* h, const fff_handle_s::Dense
     using L = fff::DescentUmmaPairLayout<NP>;
     const int stages = std::min((int)fff::kUmmaMaxStages, (kSmemBudget - L::smem_bytes(0)) / L::kStageBytes);
     if (stages < 2) return FFF_ERR_UNSUPPORTED;
-    static bool attr_set[64] = {};
-    if (h->device < 64 && !attr_set[h->device]) {
-        cudaFuncSetAttribute(fff::k_descent_umma_pair<NP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
-        attr_set[h->device] = true;
-    }
+    static bool limit_raised[kMaxDevices] = {};
+    if (!raise_smem_limit(fff::k_descent_umma_pair<NP>, h->device, kSmemBudget, limit_raised)) return FFF_ERR_CUDA;
     CUtensorMap tm, tw;
     if (!make_x_tensor_map(&tm, x, B, h->D, fff::kUM)) return FFF_ERR_CUDA;
     // the weight image as (D/64) * NP rows of 64 columns, stored pre-swizzled: copied as it is
@@ -582,7 +577,7 @@ fff_status_t launch_descent_umma_pair(fff_handle_s* h, const fff_handle_s::Dense
 
 fff_status_t run_descent_umma(fff_handle_s* h, const fff_handle_s::DenseStage& sg, const void* x, int32_t* pos_out, int64_t B,
                               cudaStream_t st) {
-    static const bool no_pair = std::getenv("FFF_NO_UMMA_PAIR") != nullptr;      // tuning aid
+    const bool no_pair = !h->tune[FFF_TUNE_CTA_PAIRS];
     // pairs pay once there is more than one round of tiles (measured: 29.1 vs 31.2 us at 394 tiles, 18.7 vs 17.0 at 128)
     if (!no_pair && (B + fff::kUM - 1) / fff::kUM > h->sm_count && h->sm_count >= 2) {
         if (sg.NP == 128) return launch_descent_umma_pair<128>(h, sg, x, pos_out, B, st);
@@ -603,11 +598,8 @@ fff_status_t launch_descent_umma_grouped(fff_handle_s* h, const fff_handle_s::De
     using L = fff::DescentUmmaGroupedLayout<NP>;
     const int stages = std::min((int)fff::kUmmaMaxStages, (kSmemBudget - L::smem_bytes(0)) / L::kStageBytes);
     if (stages < 2) return FFF_ERR_UNSUPPORTED;
-    static bool attr_set[64] = {};
-    if (h->device < 64 && !attr_set[h->device]) {
-        cudaFuncSetAttribute(fff::k_descent_umma_grouped<NP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
-        attr_set[h->device] = true;
-    }
+    static bool limit_raised[kMaxDevices] = {};
+    if (!raise_smem_limit(fff::k_descent_umma_grouped<NP>, h->device, kSmemBudget, limit_raised)) return FFF_ERR_CUDA;
     CUtensorMap tm;
     if (!make_x_tensor_map(&tm, x, B, h->D, 1)) return FFF_ERR_CUDA;       // one-row boxes: rows are gathered four at a time
     const int n_tiles = tile_list_len(B, fff::kUM, 1 << sg.L0);
@@ -645,7 +637,7 @@ fff_status_t run_descent_warp(fff_handle_s* h, const void* x, int level0, int le
 // groups it works on (tokens that share the node at the stage's first level) hold enough tokens to
 // reuse the subtree's weights.
 const std::vector<fff_handle_s::DenseStage>& stage_plan(const fff_handle_s* h) {
-    return h->ustages.empty() ? h->stages : h->ustages;
+    return h->ustages.empty() || !h->tune[FFF_TUNE_TCGEN05_DESCENT] ? h->stages : h->ustages;
 }
 
 int dense_stage_count(const fff_handle_s* h, int64_t B) {
@@ -686,7 +678,7 @@ fff_status_t run_descent(fff_handle_s* h, const void* x, int32_t* leaf_out, Coar
     for (int i = 0; i < n_dense; ++i) {
         const auto& sg = plan[i];
         // later stages: the tcgen05 kernel on 128-row tiles when the groups fill them reasonably, else mma.sync on 64-row tiles
-        const bool grouped_umma = i > 0 && sg.umma && (B >> sg.L0) >= 64;
+        const bool grouped_umma = i > 0 && sg.umma && h->tune[FFF_TUNE_TCGEN05_GROUPED] && (B >> sg.L0) >= 64;
         if (i > 0) {
             // bucket by the node reached so far; buffers alternate so that the previous level stays readable
             int32_t* perm_out = (i & 1) ? h->ws_perm2 : h->ws_perm;
@@ -746,9 +738,7 @@ fff_status_t pack_stage(fff_handle_s* h, std::vector<fff_handle_s::DenseStage>& 
 std::vector<int> cut_levels(int levels) {
     std::vector<int> ks;
     const int n_st = (levels + 5) / 6;
-    static const bool small_first = std::getenv("FFF_SMALL_STAGE_FIRST") != nullptr;      // tuning aid
-    for (int i = 0; i < n_st; ++i)
-        ks.push_back(levels / n_st + ((small_first ? i >= n_st - levels % n_st : i < levels % n_st) ? 1 : 0));
+    for (int i = 0; i < n_st; ++i) ks.push_back(levels / n_st + (i < levels % n_st ? 1 : 0));
     return ks;
 }
 
@@ -763,38 +753,22 @@ fff_status_t pack_node_images(fff_handle_s* h) {
         L0 += k;
     }
     // plan with a first stage of up to 8 levels on the tcgen05 kernel, the rest as above
-    if (encode_tiled_fn() && h->D % fff::kUKB == 0 && std::getenv("FFF_NO_UMMA") == nullptr) {
+    if (encode_tiled_fn() && h->D % fff::kUKB == 0) {
         std::vector<int> ks;
-        if (const char* e = std::getenv("FFF_STAGE_PLAN")) {       // tuning aid: "8,3" = 8 levels, then 3
-            int sum = 0;
-            for (const char* p = e; *p;) {
-                const int v = std::atoi(p);
-                ks.push_back(v);
-                sum += v;
-                while (*p && *p != ',') ++p;
-                if (*p == ',') ++p;
-            }
-            bool ok = sum == d && !ks.empty() && ks[0] >= 1 && ks[0] <= 8;
-            for (size_t i = 1; i < ks.size(); ++i) ok = ok && ks[i] >= 1 && ks[i] <= 6;
-            if (!ok) ks.clear();
-        }
         // Measured: up to 8 levels in one stage when that is the whole tree (no node bucketing at all); two
         // balanced stages up to depth 12 ([6,5] beats [8,3]: 64 bins instead of 256 and fatter groups);
         // deeper trees as few stages as possible, 8 levels first and then 6 at a time ([8,6,1] beats [5,5,5]:
         // one pass over x and one bucketing less, the last thin levels go to the warp kernel anyway).
-        if (ks.empty()) {
-            if (d <= 8) ks = {d};
-            else if (d <= 12) ks = cut_levels(d);
-            else {
-                ks.push_back(8);
-                for (int rest = d - 8; rest > 0; rest -= 6) ks.push_back(std::min(rest, 6));
-            }
+        if (d <= 8) ks = {d};
+        else if (d <= 12) ks = cut_levels(d);
+        else {
+            ks.push_back(8);
+            for (int rest = d - 8; rest > 0; rest -= 6) ks.push_back(std::min(rest, 6));
         }
         L0 = 0;
         for (size_t i = 0; i < ks.size(); ++i) {
             const int np = i == 0 ? std::max(32, 1 << ks[i]) : std::max(16, 1 << ks[i]);
-            static const bool no_grouped = std::getenv("FFF_NO_UMMA_GROUPED") != nullptr;        // tuning aid
-            if ((s = pack_stage<T>(h, h->ustages, L0, ks[i], np, i == 0 || (!no_grouped && h->D % 128 == 0))) != FFF_OK) return s;
+            if ((s = pack_stage<T>(h, h->ustages, L0, ks[i], np, i == 0 || h->D % 128 == 0)) != FFF_OK) return s;
             L0 += ks[i];
         }
         cudaFuncSetAttribute(fff::k_descent_umma<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
@@ -828,11 +802,8 @@ template <int LP, int TM, int S>
 fff_status_t launch_leaf_mma(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, cudaStream_t st) {
     const int n_tiles = tile_list_len(B, TM, (int)h->n_leaves);
     using L = fff::LeafMmaLayout<LP, TM, S>;
-    static bool attr_set[64] = {};
-    if (h->device < 64 && !attr_set[h->device]) {
-        cudaFuncSetAttribute(fff::k_leaf_mma<LP, TM, S>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kSmemBytes);
-        attr_set[h->device] = true;
-    }
+    static bool limit_raised[kMaxDevices] = {};
+    if (!raise_smem_limit(fff::k_leaf_mma<LP, TM, S>, h->device, L::kSmemBytes, limit_raised)) return FFF_ERR_CUDA;
     const int per_sm = std::max(1, std::min(2, (int)((227 * 1024) / (L::kSmemBytes + 1024))));
     const int64_t grid = std::min<int64_t>((int64_t)h->sm_count * per_sm, n_tiles);
     if (launch_chain(h, fff::k_leaf_mma<LP, TM, S>, (unsigned)grid, L::kThreads, L::kSmemBytes, st, 1,
@@ -849,11 +820,8 @@ fff_status_t launch_leaf_umma(fff_handle_s* h, const void* x, const int32_t* per
     const int n_tiles = tile_list_len(B, tile_rows, (int)h->n_leaves);
     const int stages = std::min((int)fff::kLUMaxStages, (kSmemBudget - L::smem_bytes(0)) / L::kStageBytes);
     if (stages < 2) return FFF_ERR_UNSUPPORTED;
-    static bool attr_set[64] = {};
-    if (h->device < 64 && !attr_set[h->device]) {
-        cudaFuncSetAttribute(fff::k_leaf_umma<LP, kFold>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
-        attr_set[h->device] = true;
-    }
+    static bool limit_raised[kMaxDevices] = {};
+    if (!raise_smem_limit(fff::k_leaf_umma<LP, kFold>, h->device, kSmemBudget, limit_raised)) return FFF_ERR_CUDA;
     CUtensorMap tm;
     if (!make_x_tensor_map(&tm, x, B, h->D, 1)) return FFF_ERR_CUDA;       // one-row boxes: rows are gathered four at a time
     const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(h->sm_count, n_tiles));
@@ -895,11 +863,8 @@ fff_status_t launch_leaf_umma_packed(fff_handle_s* h, const void* x, const int32
     const int n_tiles = tile_list_len(B, L::kSubRows, (int)h->n_leaves);
     const int stages = leaf_pack_stages<LP, G>();
     if (stages < 3) return FFF_ERR_UNSUPPORTED;
-    static bool attr_set[64] = {};
-    if (h->device < 64 && !attr_set[h->device]) {
-        cudaFuncSetAttribute(fff::k_leaf_umma_packed<LP, kFold, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
-        attr_set[h->device] = true;
-    }
+    static bool limit_raised[kMaxDevices] = {};
+    if (!raise_smem_limit(fff::k_leaf_umma_packed<LP, kFold, G>, h->device, kSmemBudget, limit_raised)) return FFF_ERR_CUDA;
     CUtensorMap tm;
     if (!make_x_tensor_map(&tm, x, B, h->D, 1)) return FFF_ERR_CUDA;       // one-row boxes: rows are gathered four at a time
     const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(h->sm_count, (n_tiles + G - 1) / G));
@@ -974,7 +939,7 @@ fff_status_t pack_leaf_images(fff_handle_s* h) {
     fff::k_pack_w2<T><<<blocks, 256>>>((const T*)h->w2, (const T*)h->b2, h->w2img, (int)nl, h->l, LP, h->O);
     if (cudaGetLastError() != cudaSuccess) return FFF_ERR_CUDA;
     // the tcgen05 kernel: W2 in pieces of 128 output features, and its scheduler words
-    if (encode_tiled_fn() && h->O % 16 == 0 && h->D % fff::kLUKB == 0 && std::getenv("FFF_NO_UMMA_LEAF") == nullptr) {
+    if (encode_tiled_fn() && h->O % 16 == 0 && h->D % fff::kLUKB == 0) {
         const size_t P = (size_t)(h->O + fff::kLUPiece - 1) / fff::kLUPiece;
         if ((s = dmalloc((void**)&h->w2uimg, nl * P * ((size_t)fff::kLUPiece * LP * 2 + fff::kLUPiece * 4))) != FFF_OK) return s;
         if ((s = clone((void**)&h->ws_sched, nullptr, 4 * sizeof(int))) != FFF_OK) return s;
@@ -993,7 +958,7 @@ fff_status_t pack_leaf_images(fff_handle_s* h) {
 fff_status_t check_forward_args(fff_handle_t h, int64_t B) {
     if (!live(h)) return FFF_ERR_BAD_HANDLE;
     if (B < 0) return FFF_ERR_INVALID_ARG;
-    if (B > INT32_MAX) return FFF_ERR_UNSUPPORTED;
+    if (B > FFF_MAX_TOKENS) return FFF_ERR_UNSUPPORTED;
     return FFF_OK;
 }
 
@@ -1007,7 +972,6 @@ static __device__ __align__(256) int g_static_bucket_scratch[2 * FFF_STATIC_MAX_
 
 namespace {
 
-constexpr int kMaxDevices = 64;
 std::mutex g_static_mu;
 int* g_static_ptr[kMaxDevices] = {};
 
@@ -1037,7 +1001,7 @@ extern "C" {
 fff_status_t fff_leaf_bucketing_static(const int32_t* leaf_idx, int32_t* offsets, int32_t* perm, int64_t B,
                                        int depth, void* cuda_stream) {
     if (B < 0 || depth < 0) return FFF_ERR_INVALID_ARG;
-    if (depth > FFF_STATIC_MAX_DEPTH || B > INT32_MAX) return FFF_ERR_TOO_LARGE;
+    if (depth > FFF_STATIC_MAX_DEPTH || B > FFF_MAX_TOKENS) return FFF_ERR_TOO_LARGE;
     if (!offsets || (B > 0 && (!leaf_idx || !perm))) return FFF_ERR_INVALID_ARG;
     int* scratch = nullptr;
     fff_status_t s = static_scratch_for_current_device(&scratch);
@@ -1097,6 +1061,7 @@ fff_status_t fff_create(fff_handle_t* out, int D, int O, int depth, int leaf_wid
     fff_handle_s* h = new (std::nothrow) fff_handle_s();
     if (!h) return FFF_ERR_ALLOC;
     if (cudaGetDevice(&h->device) != cudaSuccess) { delete h; return cudaGetLastError(), FFF_ERR_CUDA; }
+    if (h->device < 0 || h->device >= kMaxDevices) { delete h; return FFF_ERR_UNSUPPORTED; }
     cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device);
     {
         const int smem_max = (int)(sizeof(int) * (fff::kBucketWarps + 1) * fff::kBucketMaxBinsPerCta);
@@ -1192,6 +1157,13 @@ fff_status_t fff_set_path(fff_handle_t h, fff_path_t path) {
     return FFF_OK;
 }
 
+fff_status_t fff_set_tuning(fff_handle_t h, fff_tuning_t key, int value) {
+    if (!live(h)) return FFF_ERR_BAD_HANDLE;
+    if ((int)key < 0 || (int)key >= FFF_TUNE_COUNT || (value != 0 && value != 1)) return FFF_ERR_INVALID_ARG;
+    h->tune[key] = value != 0;
+    return FFF_OK;
+}
+
 fff_status_t fff_set_leaf_packing(fff_handle_t h, int leaves) {
     if (!live(h)) return FFF_ERR_BAD_HANDLE;
     if (leaves != 0 && leaves != 1 && leaves != 2 && leaves != 4) return FFF_ERR_INVALID_ARG;
@@ -1269,8 +1241,7 @@ fff_status_t fff_forward_infer(fff_handle_t h, const void* x, void* y, int32_t* 
     const int tile_rows = plan.tile_rows;
     // The descent ends with a tcgen05 stage and the tcgen05 leaf kernel takes whole 128-row tiles of one leaf:
     // that stage files the tokens under their leaves itself and the leaf kernel follows at once.
-    static const bool no_slots = std::getenv("FFF_NO_DIRECT_LISTS") != nullptr;      // tuning aid
-    h->slots_now = !no_slots && tensor_leaf && plan.umma && plan.pack <= 1 && tile_rows == fff::kLUM && h->ws_slots &&
+    h->slots_now = h->tune[FFF_TUNE_DIRECT_LISTS] && h->tune[FFF_TUNE_TCGEN05_DESCENT] && tensor_leaf && plan.umma && plan.pack <= 1 && tile_rows == fff::kLUM && h->ws_slots &&
                    B <= h->slot_cap && h->n_leaves * h->slot_cap <= INT32_MAX &&
                    dense_stage_count(h, B) == (int)h->ustages.size() &&
                    (h->ustages.size() == 1 || (B >> h->ustages.back().L0) >= 64);

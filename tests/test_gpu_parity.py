@@ -458,3 +458,34 @@ def test_nan_inputs_stay_in_range():
     assert torch.isnan(y[::3].float()).all()
     assert torch.isfinite(y[1::3].float()).all()
     layer.close()
+
+
+@pytest.mark.parametrize("switch", ["tcgen05_descent", "tcgen05_grouped", "tcgen05_leaf", "cta_pairs", "direct_lists"])
+def test_every_tuning_switch_off_gives_the_same_results(switch):
+    """fff_set_tuning only chooses between kernels: with any one switch off, leaf indices and the bucketing stay
+    bit-exact against the oracle and y within tolerance, on a two-stage tree (ten levels) and on a one-stage
+    tree with more 128-token tiles than SMs (seven levels; the shape the CTA pairs serve)."""
+    for cfg, seed in ((wl.FFFConfig("tune_d10", 128, 64, 10, 16, "gelu", "bf16", 20000, "clusters"), 8),
+                      (wl.FFFConfig("tune_d7", 128, 64, 7, 8, "relu", "bf16", 20001, "normal"), 3)):
+        case = util.make_case(cfg, seed=seed)
+        y_ref, leaf_ref = orc.forward_i(case.net, case.x, threads=util.ORACLE_THREADS)
+        off_ref, perm_ref = orc.bucket(leaf_ref, cfg.n_leaves)
+        layer = util.make_layer(case)
+        x = util.to_device(case.x, "bf16")
+        y_on, _ = layer.forward_infer(x)
+        launches_on = layer.last_launch_count()
+        layer.set_tuning(switch, False)
+        y, leaf = layer.forward_infer(x)
+        torch.cuda.synchronize()
+        np.testing.assert_array_equal(leaf.cpu().numpy(), leaf_ref)
+        util.check_outputs(y, y_ref, "bf16")
+        off, perm = layer.last_bucketing(cfg.B)
+        np.testing.assert_array_equal(off.cpu().numpy(), off_ref)
+        np.testing.assert_array_equal(perm.cpu().numpy(), perm_ref)
+        if switch == "direct_lists":
+            assert layer.last_launch_count() == launches_on + 1      # the leaf bucketing kernel is back
+        layer.set_tuning(switch, True)
+        y_back, _ = layer.forward_infer(x)
+        assert torch.equal(y_back, y_on)
+        assert layer.last_status() == 0
+        layer.close()

@@ -70,6 +70,12 @@ def test_hand_computed_descent_and_leaf_values():
     # leaf 3 on (-1,-.5): h = relu([-4, 2+1]) = [0,3]; y = [3, 3, 2]
     expect = np.array([[11, 1, 8], [1, 0, -1], [0, 0.25, -0.75], [11, 0, 8], [3, 3, 2]], float)
     np.testing.assert_allclose(y, expect, rtol=0, atol=1e-15)
+    # smallest |logit| on each token's path, from the logits worked out above:
+    # (2.5, 0) -> 0; (-1.5, 1) -> 1; (-0.25, -0.25) -> 0.25; (2.5, -1) -> 1; (0, 3) -> 0
+    leaf_d, margin, _ = orc.descend(net, x)
+    assert leaf_d.tolist() == [3, 1, 0, 2, 3]
+    assert margin.tolist() == [0.0, 1.0, 0.25, 1.0, 0.0]
+    assert orc.path_margin(net, x).tolist() == [0.0, 1.0, 0.25, 1.0, 0.0]
 
 
 def test_tie_goes_right_zero_node_weights_reach_last_leaf():
