@@ -1244,7 +1244,7 @@ fff_status_t fff_forward_infer(fff_handle_t h, const void* x, void* y, int32_t* 
     h->slots_now = h->tune[FFF_TUNE_DIRECT_LISTS] && h->tune[FFF_TUNE_TCGEN05_DESCENT] && tensor_leaf && plan.umma && plan.pack <= 1 && tile_rows == fff::kLUM && h->ws_slots &&
                    B <= h->slot_cap && h->n_leaves * h->slot_cap <= INT32_MAX &&
                    dense_stage_count(h, B) == (int)h->ustages.size() &&
-                   (h->ustages.size() == 1 || (B >> h->ustages.back().L0) >= 64);
+                   (h->ustages.size() == 1 || (h->tune[FFF_TUNE_TCGEN05_GROUPED] && (B >> h->ustages.back().L0) >= 64));
     if (h->slots_now) {
         if (h->cursor_dirty && cudaMemsetAsync(h->ws_cursor, 0, sizeof(int32_t) * (size_t)h->n_leaves, st) != cudaSuccess)
             return h->slots_now = false, cudaGetLastError(), FFF_ERR_CUDA;
