@@ -157,17 +157,6 @@ typedef enum {
 } fff_tuning_t;
 fff_status_t fff_set_tuning(fff_handle_t h, fff_tuning_t key, int value);
 
-/* Leaf packing of the tcgen05 leaf kernel (bf16 tensor path): with only a few dozen tokens per leaf, `leaves`
- * = 2 or 4 leaves share the 128 rows of one tile (sub-tiles of 64 or 32 tokens), which shortens the kernel when
- * routing is close to uniform and lengthens it when a few leaves take most tokens (measured: 124 -> 118 us and
- * 78 -> 87 us on the two 2048-leaf, 32-tokens-per-leaf workloads).  The library cannot tell which holds without
- * waiting for the routing, so the default is 1 (off).  0 lets the library choose from the average bucket size
- * B / 2^depth alone (>= 96: 1, >= 24: 2, below: 4).  Results do not depend on the setting.  The setting is
- * ignored where the packed kernel cannot run (non-finite output weights, shapes without the tcgen05 kernel).
- * The paper describes no such choice: FORWARD_I (Algorithm 1) is the same computation either way.
- * FFF_ERR_INVALID_ARG for other values. */
-fff_status_t fff_set_leaf_packing(fff_handle_t h, int leaves);
-
 /*
  * Stage entry points.  fff_forward_infer computes what these three compute
  * when called in this order.

@@ -26,7 +26,7 @@ TUNING = {"tcgen05_descent": 0, "tcgen05_grouped": 1, "tcgen05_leaf": 2, "cta_pa
 
 # every symbol include/fff.h declares
 EXPORTS = ["fff_create", "fff_forward_infer", "fff_forward_infer_host", "fff_destroy", "fff_reserve",
-           "fff_set_path", "fff_set_tuning", "fff_set_leaf_packing", "fff_tree_descent", "fff_leaf_bucketing", "fff_grouped_leaf_ff",
+           "fff_set_path", "fff_set_tuning", "fff_tree_descent", "fff_leaf_bucketing", "fff_grouped_leaf_ff",
            "fff_debug_get_bucketing", "fff_get_last_status", "fff_last_launch_count", "fff_status_string",
            "fff_profile_begin", "fff_profile_end", "fff_profile_launches", "fff_profile_launch_name",
            "fff_leaf_bucketing_static"]
@@ -57,7 +57,6 @@ def lib():
     L.fff_destroy.argtypes = [vp]
     L.fff_reserve.argtypes = [vp, i64]
     L.fff_set_path.argtypes = [vp, ci]
-    L.fff_set_leaf_packing.argtypes = [vp, ci]
     L.fff_set_tuning.argtypes = [vp, ci, ci]
     L.fff_tree_descent.argtypes = [vp, vp, vp, i64, vp]
     L.fff_leaf_bucketing.argtypes = [vp, vp, vp, vp, i64, vp]
@@ -119,10 +118,6 @@ def fff_set_path(h, path) -> None:
 
 def fff_set_tuning(h, key, value) -> None:
     _check(lib().fff_set_tuning(h, key, value), "fff_set_tuning")
-
-
-def fff_set_leaf_packing(h, leaves) -> None:
-    _check(lib().fff_set_leaf_packing(h, leaves), "fff_set_leaf_packing")
 
 
 def fff_tree_descent(h, x, leaf_idx, B, stream=None) -> None:
@@ -230,10 +225,6 @@ class FFFLayer:
     def set_tuning(self, key: str, on: bool) -> None:
         """Switch between kernels that compute the same thing (keys of TUNING; all on by default)."""
         fff_set_tuning(self._h, TUNING[key], 1 if on else 0)
-
-    def set_leaf_packing(self, leaves: int) -> None:
-        """1 (default): one leaf per tile; 2 or 4: that many thin leaves share a tile; 0: chosen from B / n_leaves."""
-        fff_set_leaf_packing(self._h, leaves)
 
     def forward_infer(self, x, y=None, leaf_idx=None, want_leaf_idx: bool = True, stream=None):
         torch = _torch()

@@ -22,7 +22,6 @@
 #include "kernels/descent_warp.cuh"
 #include "kernels/leaf_mma.cuh"
 #include "kernels/leaf_umma.cuh"
-#include "kernels/leaf_umma_packed.cuh"
 #include "kernels/leaf_warp.cuh"
 
 namespace {
@@ -58,8 +57,6 @@ struct fff_handle_s {
     __nv_bfloat16* w1img = nullptr;
     float* b1img = nullptr;
     unsigned char* w2img = nullptr;
-    int leaf_pack = 1;                 // fff_set_leaf_packing: 1 off, 2 / 4 leaves per tile, 0 chosen from B / n_leaves
-    bool w2_finite = false;            // every W2 and b2 entry is finite (leaves may then share a tile, see leaf_umma_packed.cuh)
     unsigned char* w2uimg = nullptr;   // W2 pieces (+ biases) of the tcgen05 leaf kernel (nullptr = kernel not available)
     int* ws_sched = nullptr;           // its tile counter and finished-CTA counter (zero between launches)
     fff::Tile* ws_tiles = nullptr;
@@ -246,27 +243,17 @@ size_t max_tiles(const fff_handle_s* h, int64_t B) { return (size_t)(B / kMinTil
 struct LeafPlan {
     int tile_rows = 0;
     bool umma = false;
-    int pack = 1;          // leaves per 128-row tile of the tcgen05 kernel (tile_rows = 128 / pack)
 };
-
-bool leaf_pack_fits(int LP, int pack);
 
 LeafPlan leaf_plan(const fff_handle_s* h, int64_t B) {
     // The tcgen05 kernel works on 128-row tiles.  Measured against the mma.sync kernel it is far ahead when
     // some buckets are large (skewed routing), about level with uniformly thin buckets of 32 tokens, and is
-    // left out only when buckets are thinner still (every tile costs its epilogue a fixed few microseconds).
+    // left out only when buckets are thinner still (tiles of at most 64 rows are stacked in the MMA rows, so the
+    // epilogue's cost follows the rows; the rest of a tile's cost is fixed).
     if (h->w2uimg && h->tune[FFF_TUNE_TCGEN05_LEAF] && B >= 16 * h->n_leaves) {
-        // Thin buckets: several leaves may share the rows of a tile (fff_set_leaf_packing; off unless asked for,
-        // because it loses when a few buckets hold most tokens, which the host cannot know here).
-        const int64_t avg = B / h->n_leaves;
-        const int by_size = avg >= 96 ? 1 : avg >= 24 ? 2 : 4;
-        int pack = h->leaf_pack == 0 ? by_size : h->leaf_pack;
-        if (!h->w2_finite) pack = 1;
-        while (pack > 1 && !leaf_pack_fits(h->LP, pack)) pack >>= 1;
-        if (pack > 1) return LeafPlan{fff::kLUM / pack, true, pack};
-        return LeafPlan{fff::kLUM, true, 1};
+        return LeafPlan{fff::kLUM, true};
     }
-    return LeafPlan{B / h->n_leaves <= 40 ? 32 : 64, false, 1};
+    return LeafPlan{B / h->n_leaves <= 40 ? 32 : 64, false};
 }
 
 bool use_tensor_leaf(const fff_handle_s* h) {
@@ -837,66 +824,10 @@ fff_status_t launch_leaf_umma(fff_handle_s* h, const void* x, const int32_t* per
     return launched(h, st, "grouped_leaf_ff_umma");
 }
 
-template <int LP, int G>
-int leaf_pack_stages() {
-    using L = fff::LeafPackLayout<LP, G>;
-    return std::min((int)fff::kLUMaxStages, (kSmemBudget - L::smem_bytes(0)) / L::kStageBytes);
-}
-
-// Whether the kernel that packs `pack` leaves into a tile has room for a ring of at least three stages.
-bool leaf_pack_fits(int LP, int pack) {
-    int st = 0;
-    switch (LP * 8 + pack) {
-        case 16 * 8 + 2: st = leaf_pack_stages<16, 2>(); break;
-        case 16 * 8 + 4: st = leaf_pack_stages<16, 4>(); break;
-        case 32 * 8 + 2: st = leaf_pack_stages<32, 2>(); break;
-        case 32 * 8 + 4: st = leaf_pack_stages<32, 4>(); break;
-        case 64 * 8 + 2: st = leaf_pack_stages<64, 2>(); break;
-        default: break;                                        // (64, 4) does not fit
-    }
-    return st >= 3;
-}
-
-template <int LP, bool kFold, int G>
-fff_status_t launch_leaf_umma_packed(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, cudaStream_t st) {
-    using L = fff::LeafPackLayout<LP, G>;
-    const int n_tiles = tile_list_len(B, L::kSubRows, (int)h->n_leaves);
-    const int stages = leaf_pack_stages<LP, G>();
-    if (stages < 3) return FFF_ERR_UNSUPPORTED;
-    static bool limit_raised[kMaxDevices] = {};
-    if (!raise_smem_limit(fff::k_leaf_umma_packed<LP, kFold, G>, h->device, kSmemBudget, limit_raised)) return FFF_ERR_CUDA;
-    CUtensorMap tm;
-    if (!make_x_tensor_map(&tm, x, B, h->D, 1)) return FFF_ERR_CUDA;       // one-row boxes: rows are gathered four at a time
-    const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(h->sm_count, (n_tiles + G - 1) / G));
-    const int wide = (reinterpret_cast<uintptr_t>(y) & 31u) == 0 ? 1 : 0;
-    if (launch_chain(h, fff::k_leaf_umma_packed<LP, kFold, G>, (unsigned)grid, fff::kLUThreads, (size_t)L::smem_bytes(stages), st, 1, tm,
-                     perm, (const fff::Tile*)h->ws_tiles, n_tiles, (const __nv_bfloat16*)h->w1img, (const float*)h->b1img,
-                     (const unsigned char*)h->w2uimg, (__nv_bfloat16*)y, h->D, h->O, h->l, h->act, stages, wide, h->ws_sched,
-                     h->d_status) != cudaSuccess)
-        return cudaGetLastError(), FFF_ERR_CUDA;
-    return launched(h, st, "grouped_leaf_ff_umma_packed");
-}
-
-template <int LP, int G>
-fff_status_t leaf_umma_packed_variant(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, cudaStream_t st) {
-    return h->l < LP ? launch_leaf_umma_packed<LP, true, G>(h, x, perm, y, B, st)
-                     : launch_leaf_umma_packed<LP, false, G>(h, x, perm, y, B, st);
-}
-
 // Ring depth per (LP, TM): what fits twice into an SM's shared memory (once for LP = 64).
 fff_status_t run_leaf_mma(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, const LeafPlan& plan,
                           cudaStream_t st) {
     const int tile_rows = plan.tile_rows;
-    if (plan.umma && h->w2uimg && plan.pack > 1) {
-        switch (h->LP * 8 + plan.pack) {
-            case 16 * 8 + 2: return leaf_umma_packed_variant<16, 2>(h, x, perm, y, B, st);
-            case 16 * 8 + 4: return leaf_umma_packed_variant<16, 4>(h, x, perm, y, B, st);
-            case 32 * 8 + 2: return leaf_umma_packed_variant<32, 2>(h, x, perm, y, B, st);
-            case 32 * 8 + 4: return leaf_umma_packed_variant<32, 4>(h, x, perm, y, B, st);
-            case 64 * 8 + 2: return leaf_umma_packed_variant<64, 2>(h, x, perm, y, B, st);
-        }
-        return FFF_ERR_UNSUPPORTED;
-    }
     if (plan.umma && h->w2uimg) {
         switch (h->LP) {
             case 16: return h->l < 16 ? launch_leaf_umma<16, true>(h, x, perm, y, B, tile_rows, st)
@@ -943,11 +874,8 @@ fff_status_t pack_leaf_images(fff_handle_s* h) {
         const size_t P = (size_t)(h->O + fff::kLUPiece - 1) / fff::kLUPiece;
         if ((s = dmalloc((void**)&h->w2uimg, nl * P * ((size_t)fff::kLUPiece * LP * 2 + fff::kLUPiece * 4))) != FFF_OK) return s;
         if ((s = clone((void**)&h->ws_sched, nullptr, 4 * sizeof(int))) != FFF_OK) return s;
-        fff::k_pack_w2_umma<T><<<blocks, 256>>>((const T*)h->w2, (const T*)h->b2, h->w2uimg, (int)nl, h->l, LP, h->O, h->ws_sched + 3);
+        fff::k_pack_w2_umma<T><<<blocks, 256>>>((const T*)h->w2, (const T*)h->b2, h->w2uimg, (int)nl, h->l, LP, h->O);
         if (cudaGetLastError() != cudaSuccess) return FFF_ERR_CUDA;
-        int nonfinite = 1;
-        if (cudaMemcpy(&nonfinite, h->ws_sched + 3, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
-        h->w2_finite = nonfinite == 0;
     }
     return cudaGetLastError() == cudaSuccess ? FFF_OK : FFF_ERR_CUDA;
 }
@@ -1164,13 +1092,6 @@ fff_status_t fff_set_tuning(fff_handle_t h, fff_tuning_t key, int value) {
     return FFF_OK;
 }
 
-fff_status_t fff_set_leaf_packing(fff_handle_t h, int leaves) {
-    if (!live(h)) return FFF_ERR_BAD_HANDLE;
-    if (leaves != 0 && leaves != 1 && leaves != 2 && leaves != 4) return FFF_ERR_INVALID_ARG;
-    h->leaf_pack = leaves;
-    return FFF_OK;
-}
-
 fff_status_t fff_tree_descent(fff_handle_t h, const void* x, int32_t* leaf_idx, int64_t B, void* cuda_stream) {
     fff_status_t s = check_forward_args(h, B);
     if (s != FFF_OK) return s;
@@ -1241,7 +1162,7 @@ fff_status_t fff_forward_infer(fff_handle_t h, const void* x, void* y, int32_t* 
     const int tile_rows = plan.tile_rows;
     // The descent ends with a tcgen05 stage and the tcgen05 leaf kernel takes whole 128-row tiles of one leaf:
     // that stage files the tokens under their leaves itself and the leaf kernel follows at once.
-    h->slots_now = h->tune[FFF_TUNE_DIRECT_LISTS] && h->tune[FFF_TUNE_TCGEN05_DESCENT] && tensor_leaf && plan.umma && plan.pack <= 1 && tile_rows == fff::kLUM && h->ws_slots &&
+    h->slots_now = h->tune[FFF_TUNE_DIRECT_LISTS] && h->tune[FFF_TUNE_TCGEN05_DESCENT] && tensor_leaf && plan.umma && tile_rows == fff::kLUM && h->ws_slots &&
                    B <= h->slot_cap && h->n_leaves * h->slot_cap <= INT32_MAX &&
                    dense_stage_count(h, B) == (int)h->ustages.size() &&
                    (h->ustages.size() == 1 || (h->tune[FFF_TUNE_TCGEN05_GROUPED] && (B >> h->ustages.back().L0) >= 64));

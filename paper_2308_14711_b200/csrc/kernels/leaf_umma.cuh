@@ -35,8 +35,8 @@
 //
 // Rows of a ragged tile beyond its length are not loaded: their accumulator rows hold garbage that is
 // never stored (rows of an MMA are independent).
-// Thin buckets (a few dozen tokens per leaf) go to k_leaf_umma_packed instead, which stacks several leaves in
-// the rows of one tile.
+// Tiles of at most 64 (32) rows are stacked twice (four times) in the MMA rows of GEMM2 so that every epilogue
+// warp has a share of their columns (see the epilogue).
 //
 // Every wait is bounded (see ptx.cuh); tensor memory is released on every exit path.
 //
@@ -105,7 +105,7 @@ __host__ __device__ __forceinline__ uint32_t swz_rows(uint32_t off, int row_byte
 // then the 128 float32 biases of those features }.
 template <typename T>
 __global__ void k_pack_w2_umma(const T* __restrict__ w2, const T* __restrict__ b2, unsigned char* __restrict__ img,
-                               int n_leaves, int l, int LP, int O, int* __restrict__ nonfinite)
+                               int n_leaves, int l, int LP, int O)
 {
     const int P = (O + kLUPiece - 1) / kLUPiece;
     const int64_t piece_bytes = (int64_t)kLUPiece * LP * 2 + kLUPiece * 4;
@@ -122,11 +122,9 @@ __global__ void k_pack_w2_umma(const T* __restrict__ w2, const T* __restrict__ b
             // b2 by itself and the epilogue has no bias to fetch and add (b2 is bf16 already: exact)
             float v = (o < O && c < l) ? Elem<T>::to_float(w2[(j * O + o) * (int64_t)l + c]) : 0.0f;
             if (c == l && o < O) v = Elem<T>::to_float(b2[j * O + o]);
-            if (!isfinite(v)) atomicOr(nonfinite, 1);            // (the kernel that packs several leaves into a tile needs to know)
             *reinterpret_cast<__nv_bfloat16*>(piece + swz_rows((uint32_t)(n * LP * 2 + c * 2), LP * 2)) = __float2bfloat16_rn(v);
         } else {
             const float v = o < O ? Elem<T>::to_float(b2[j * O + o]) : 0.0f;
-            if (!isfinite(v)) atomicOr(nonfinite, 1);
             reinterpret_cast<float*>(piece + (int64_t)kLUPiece * LP * 2)[n] = v;
         }
     }
@@ -435,19 +433,27 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
         }
     } else {
         // ------------------------------------------------------------------ epilogue: one token row and one column part per thread
+        // A warp can only read the 32 tensor-memory lanes of its quarter, so a tile of at most 32 (64) rows would
+        // leave three quarters (one half) of the epilogue warps without work and cost as much as a full tile.
+        // Short tiles are therefore stacked `rep` = 4 (2) times in the 128 rows of GEMM2: H row r is written to the
+        // rows r, r + 128/rep, ... of the A operand, every copy's accumulator rows then hold the same values (the
+        // rows of an MMA are independent; the extra MMA rows cost nothing), and the quarters of copy c convert and
+        // store only the c-th group of 128/rep columns of each piece.
         const int quarter = warp & 3, part = warp >> 2;
-        const int row = quarter * 32 + lane;
         const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
         constexpr int HC = LP / kLUHParts;                       // H columns of a thread that computes H
-        constexpr int YC = kLUPiece / kLUColParts;               // y columns of this thread per piece
         int pc = 0;
         int w2_slot = 0;
         uint32_t w2_phase = 0;
         for (int it = 0; it < max_iters; ++it) {
             const Tile tl = next_tile();
             if (tl.rows <= 0) break;
-            const bool active = quarter * 32 < tl.rows;          // this warp's lanes hold valid rows
-            const bool h_active = active && part < kLUHParts;
+            const int rep = tl.rows <= 32 ? 4 : tl.rows <= 64 ? 2 : 1;
+            const int qper = 4 / rep;                            // lane quarters per copy
+            const int copy = quarter / qper;                     // the copy this thread's lanes hold = its column group
+            const int row = (quarter % qper) * 32 + lane;        // the token row this thread's lane carries
+            const bool active = (quarter % qper) * 32 < tl.rows; // this warp's lanes hold valid rows
+            const bool h_active = active && copy == 0 && part < kLUHParts;      // the first copy's lanes hold acc1
             const int64_t tok = row < tl.rows ? perm[tl.start + row] : -1;
             float b1r[HC];
 #pragma unroll
@@ -456,7 +462,7 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                 b1r[j] = t.x; b1r[j + 1] = t.y; b1r[j + 2] = t.z; b1r[j + 3] = t.w;
             }
 
-            // H = act(acc1 + b1) -> bf16 -> this thread's part of its row of the A operand of GEMM2
+            // H = act(acc1 + b1) -> bf16 -> this thread's part of its row of the A operand of GEMM2 (every copy of it)
             if (!timed_out && !ptx::mbar_wait(acc1_full, it & 1)) timed_out = true;
             ptx::tc_fence_after_sync();
             {
@@ -477,17 +483,22 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                 ptx::tc_fence_before_sync();
                 ptx::mbar_arrive(acc1_empty);
                 if (h_active) {
+                    for (int cp = 0; cp < rep; ++cp) {
+                        const int hrow = row + cp * (kLUM / rep);
 #pragma unroll
-                    for (int c = 0; c < HC / 8; ++c)
-                        *reinterpret_cast<uint4*>(hbuf + swz_rows((uint32_t)(row * L::kRowBytes + (part * HC / 8 + c) * 16), L::kRowBytes)) =
-                            make_uint4(hp[4 * c], hp[4 * c + 1], hp[4 * c + 2], hp[4 * c + 3]);
+                        for (int c = 0; c < HC / 8; ++c)
+                            *reinterpret_cast<uint4*>(hbuf + swz_rows((uint32_t)(hrow * L::kRowBytes + (part * HC / 8 + c) * 16), L::kRowBytes)) =
+                                make_uint4(hp[4 * c], hp[4 * c + 1], hp[4 * c + 2], hp[4 * c + 3]);
+                    }
                     ptx::fence_proxy_async();
                 }
                 ptx::mbar_arrive(h_full);
             }
 
-            // Y pieces: this thread's share of the 128 columns
+            // Y pieces: this thread's share of the 128 columns: 64 / rep columns of column group `copy`
             __nv_bfloat16* yrow = y + (tok >= 0 ? tok : 0) * O;
+            const int ncw = (kLUPiece / kLUColParts) / rep;          // 64, 32 or 16
+            const int cbase = copy * (kLUPiece / rep) + part * ncw;
             for (int p = 0; p < P; ++p, ++pc) {
                 const int b = pc & 1;
                 if (!timed_out && !ptx::mbar_wait(y_full + b, (pc >> 1) & 1)) timed_out = true;
@@ -495,38 +506,68 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                 ptx::tc_fence_after_sync();
                 const float* bias = reinterpret_cast<const float*>(w2ring + w2_slot * L::kW2SlotStride + L::kW2Bytes);
                 const int ncols = min(kLUPiece, O - p * kLUPiece);
-#pragma unroll
-                for (int cc = 0; cc < YC / 32; ++cc) {
-                    const int c0 = part * YC + cc * 32;
-                    const int nv = min(32, ncols - c0);              // <= 0, 16 or 32
-                    if (active && nv > 0) {
-                        uint32_t v[32];
-                        ptx::tmem_ld32(lane_base + kLUAcc2Col + b * kLUAccStride + c0, v);
+                if (ncw == 16) {
+                    const int c0 = cbase;
+                    if (active && c0 < ncols) {                      // ncols is a multiple of 16
+                        uint32_t v[16];
+                        ptx::tmem_ld16(lane_base + kLUAcc2Col + b * kLUAccStride + c0, v);
                         ptx::tmem_ld_wait();
-                        const int o0 = p * kLUPiece + c0;
-                        uint32_t out[16];
-                        if (kFold) {                                 // bias already added by GEMM2
+                        uint32_t out[8];
+                        if (kFold) {
 #pragma unroll
-                            for (int e = 0; e < 16; ++e)
+                            for (int e = 0; e < 8; ++e)
                                 out[e] = ptx::pack_bf16(__uint_as_float(v[2 * e]), __uint_as_float(v[2 * e + 1]));
                         } else {
 #pragma unroll
-                            for (int e = 0; e < 8; ++e) {
+                            for (int e = 0; e < 4; ++e) {
                                 const float4 bb = *reinterpret_cast<const float4*>(bias + c0 + 4 * e);
                                 out[2 * e] = ptx::pack_bf16(__uint_as_float(v[4 * e]) + bb.x, __uint_as_float(v[4 * e + 1]) + bb.y);
                                 out[2 * e + 1] = ptx::pack_bf16(__uint_as_float(v[4 * e + 2]) + bb.z, __uint_as_float(v[4 * e + 3]) + bb.w);
                             }
                         }
                         if (tok >= 0) {
-                            if (wide_stores && nv == 32) {
+                            const int o0 = p * kLUPiece + c0;
+                            if (wide_stores) {
                                 ptx::st_global_v8(yrow + o0, out);
-                                ptx::st_global_v8(yrow + o0 + 16, out + 8);
+                            } else {
+                                *reinterpret_cast<uint4*>(yrow + o0) = make_uint4(out[0], out[1], out[2], out[3]);
+                                *reinterpret_cast<uint4*>(yrow + o0 + 8) = make_uint4(out[4], out[5], out[6], out[7]);
+                            }
+                        }
+                    }
+                } else {
+                    for (int cc = 0; cc * 32 < ncw; ++cc) {
+                        const int c0 = cbase + cc * 32;
+                        const int nv = min(32, ncols - c0);              // <= 0, 16 or 32
+                        if (active && nv > 0) {
+                            uint32_t v[32];
+                            ptx::tmem_ld32(lane_base + kLUAcc2Col + b * kLUAccStride + c0, v);
+                            ptx::tmem_ld_wait();
+                            const int o0 = p * kLUPiece + c0;
+                            uint32_t out[16];
+                            if (kFold) {                                 // bias already added by GEMM2
+#pragma unroll
+                                for (int e = 0; e < 16; ++e)
+                                    out[e] = ptx::pack_bf16(__uint_as_float(v[2 * e]), __uint_as_float(v[2 * e + 1]));
                             } else {
 #pragma unroll
-                                for (int q = 0; q < 4; ++q)
-                                    if (q * 8 < nv)
-                                        *reinterpret_cast<uint4*>(yrow + o0 + q * 8) =
-                                            make_uint4(out[4 * q], out[4 * q + 1], out[4 * q + 2], out[4 * q + 3]);
+                                for (int e = 0; e < 8; ++e) {
+                                    const float4 bb = *reinterpret_cast<const float4*>(bias + c0 + 4 * e);
+                                    out[2 * e] = ptx::pack_bf16(__uint_as_float(v[4 * e]) + bb.x, __uint_as_float(v[4 * e + 1]) + bb.y);
+                                    out[2 * e + 1] = ptx::pack_bf16(__uint_as_float(v[4 * e + 2]) + bb.z, __uint_as_float(v[4 * e + 3]) + bb.w);
+                                }
+                            }
+                            if (tok >= 0) {
+                                if (wide_stores && nv == 32) {
+                                    ptx::st_global_v8(yrow + o0, out);
+                                    ptx::st_global_v8(yrow + o0 + 16, out + 8);
+                                } else {
+#pragma unroll
+                                    for (int q = 0; q < 4; ++q)
+                                        if (q * 8 < nv)
+                                            *reinterpret_cast<uint4*>(yrow + o0 + q * 8) =
+                                                make_uint4(out[4 * q], out[4 * q + 1], out[4 * q + 2], out[4 * q + 3]);
+                                }
                             }
                         }
                     }
