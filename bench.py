@@ -167,6 +167,8 @@ def path_bytes(cfg: wl.FFFConfig, B: int, leaves_touched: int) -> float:
 def kernel_bytes(name: str, cfg: wl.FFFConfig, B: int, leaves_touched: int) -> float:
     """Algorithmic bytes one launch of the named kernel must move."""
     e = cfg.elem_bytes
+    if name.startswith("fused_forward"):                       # the whole path in one launch
+        return path_bytes(cfg, B, leaves_touched)
     if name.startswith("tree_descent"):
         return B * cfg.D * e + cfg.n_nodes * (cfg.D + 1) * e + 4 * B
     if name.startswith("leaf_bucketing+grouped_leaf_ff"):      # bucketing done by the leaf kernel's prologue

@@ -72,7 +72,8 @@ typedef enum {
 typedef enum {
     FFF_PATH_AUTO = 0,           /* library picks per stage from shapes and B */
     FFF_PATH_WARP = 1,           /* CUDA-core warp kernels for descent and leaf evaluation */
-    FFF_PATH_TENSOR = 2          /* tensor-core kernels wherever the shapes allow them */
+    FFF_PATH_TENSOR = 2,         /* tensor-core kernels wherever the shapes allow them */
+    FFF_PATH_FUSED = 3           /* the one-launch kernel for small trees with leaves of at most 32 neurons */
 } fff_path_t;
 
 /*
@@ -153,7 +154,10 @@ typedef enum {
     FFF_TUNE_TCGEN05_LEAF = 2,    /* leaf evaluation on tcgen05 (0: mma.sync kernel) */
     FFF_TUNE_CTA_PAIRS = 3,       /* first descent stage with 128 or 256 nodes on pairs of CTAs (0: single CTAs) */
     FFF_TUNE_DIRECT_LISTS = 4,    /* the last descent stage files tokens under their leaves (0: bucketing kernel) */
-    FFF_TUNE_COUNT = 5
+    FFF_TUNE_FUSED_SMALL = 5,     /* small trees with thin leaves in one launch: descent, grid barrier, leaf evaluation
+                                     by groups of 32 hidden neurons kept in shared memory (0: descent, bucketing and
+                                     leaf kernels).  Taken by default by layers without a tensor-core leaf path */
+    FFF_TUNE_COUNT = 6
 } fff_tuning_t;
 fff_status_t fff_set_tuning(fff_handle_t h, fff_tuning_t key, int value);
 

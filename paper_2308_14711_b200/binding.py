@@ -21,8 +21,8 @@ STATUS_NAMES = {0: "FFF_OK", 1: "FFF_ERR_INVALID_ARG", 2: "FFF_ERR_UNSUPPORTED",
                 4: "FFF_ERR_CUDA", 5: "FFF_ERR_DEVICE_TIMEOUT", 6: "FFF_ERR_BAD_HANDLE", 7: "FFF_ERR_TOO_LARGE"}
 ACTIVATIONS = {"relu": 0, "gelu": 1}
 DTYPES = {"f32": 0, "bf16": 1}
-PATHS = {"auto": 0, "warp": 1, "tensor": 2}
-TUNING = {"tcgen05_descent": 0, "tcgen05_grouped": 1, "tcgen05_leaf": 2, "cta_pairs": 3, "direct_lists": 4}
+PATHS = {"auto": 0, "warp": 1, "tensor": 2, "fused": 3}
+TUNING = {"tcgen05_descent": 0, "tcgen05_grouped": 1, "tcgen05_leaf": 2, "cta_pairs": 3, "direct_lists": 4, "fused_small": 5}
 
 # every symbol include/fff.h declares
 EXPORTS = ["fff_create", "fff_forward_infer", "fff_forward_infer_host", "fff_destroy", "fff_reserve",

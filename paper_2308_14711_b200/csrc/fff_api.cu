@@ -20,6 +20,7 @@
 #include "kernels/descent_mma.cuh"
 #include "kernels/descent_umma.cuh"
 #include "kernels/descent_warp.cuh"
+#include "kernels/fused_small.cuh"
 #include "kernels/leaf_mma.cuh"
 #include "kernels/leaf_umma.cuh"
 #include "kernels/leaf_warp.cuh"
@@ -87,6 +88,10 @@ struct fff_handle_s {
     int32_t* ws_perm2 = nullptr;  // second permutation buffer: successive bucketings alternate between the two
     int32_t* ws_offsets2[2] = {nullptr, nullptr};   // offsets of the intermediate (node) bucketings
 
+    // one-launch forward for small trees with thin leaves (fused_small.cuh); fs_batch == 0: shapes not eligible
+    float *fs_w1g = nullptr, *fs_b1g = nullptr, *fs_w2g = nullptr, *fs_b2f = nullptr;
+    int fs_G = 0, fs_lp = 0, fs_Dp = 0, fs_batch = 0;
+
     // staged descent on tensor cores: consecutive groups of levels, each with its weight image
     struct DenseStage {
         int L0 = 0, k = 0, NP = 0;
@@ -110,7 +115,7 @@ struct fff_handle_s {
     cudaEvent_t ev_in[kMaxHostChunks] = {}, ev_done[kMaxHostChunks] = {}, ev_start = nullptr, ev_end = nullptr;
 
     int path = FFF_PATH_AUTO;
-    bool tune[FFF_TUNE_COUNT] = {true, true, true, true, true};      // fff_set_tuning; every switch defaults to on
+    bool tune[FFF_TUNE_COUNT] = {true, true, true, true, true, true};      // fff_set_tuning; every switch defaults to on
     bool pdl = true;              // launch every kernel of a forward but the first as a programmatic dependent
     int launches = 0;
     int64_t last_B = -1;
@@ -200,6 +205,7 @@ void release(fff_handle_s* h) {
     for (auto& sg : h->stages) { dfree(sg.wimg); dfree(sg.bimg); }
     for (auto& sg : h->ustages) { dfree(sg.wimg); dfree(sg.bimg); }
     dfree(h->ws_pos[0]); dfree(h->ws_pos[1]);
+    dfree(h->fs_w1g); dfree(h->fs_b1g); dfree(h->fs_w2g); dfree(h->fs_b2f);
     dfree(h->w1img); dfree(h->b1img); dfree(h->w2img); dfree(h->w2uimg); dfree(h->ws_sched); dfree(h->ws_tiles); dfree(h->ws_rank); dfree(h->ws_rank8); dfree(h->ws_counts8); dfree(h->ws_blocksum); dfree(h->ws_matrix); dfree(h->ws_slots); dfree(h->ws_cursor);
     if (h->copy_in) cudaStreamDestroy(h->copy_in);
     if (h->copy_out) cudaStreamDestroy(h->copy_out);
@@ -880,6 +886,64 @@ fff_status_t pack_leaf_images(fff_handle_s* h) {
     return cudaGetLastError() == cudaSuccess ? FFF_OK : FFF_ERR_CUDA;
 }
 
+// The one-launch kernel for small trees: eligibility and its weight images (at creation).
+template <typename T>
+fff_status_t pack_fused_small(fff_handle_s* h) {
+    if (h->l > 32 || h->coop_ctas <= 0) return FFF_OK;
+    int lp = 1;
+    while (lp < h->l) lp <<= 1;
+    const int64_t G = (h->n_leaves * lp + 31) / 32;
+    if (G > h->sm_count) return FFF_OK;
+    const int Dp = (h->D + 3) & ~3;
+    int batch = fff::kFSMaxBatch;
+    while (batch >= 8 && fff::FusedSmallLayout{Dp, h->O, batch}.total() > (size_t)kSmemBudget) batch >>= 1;
+    if (batch < 8) return FFF_OK;
+    fff_status_t s;
+    if ((s = dmalloc((void**)&h->fs_w1g, sizeof(float) * (size_t)G * 32 * Dp)) != FFF_OK) return s;
+    if ((s = dmalloc((void**)&h->fs_b1g, sizeof(float) * (size_t)G * 32)) != FFF_OK) return s;
+    if ((s = dmalloc((void**)&h->fs_w2g, sizeof(float) * (size_t)G * h->O * 32)) != FFF_OK) return s;
+    if ((s = dmalloc((void**)&h->fs_b2f, sizeof(float) * (size_t)h->n_leaves * h->O)) != FFF_OK) return s;
+    fff::k_pack_fused_small<T><<<h->sm_count * 8, 256>>>((const T*)h->w1, (const T*)h->b1, (const T*)h->w2, (const T*)h->b2, h->fs_w1g,
+                                                        h->fs_b1g, h->fs_w2g, h->fs_b2f, (int)h->n_leaves, h->l, lp, h->D, Dp, h->O,
+                                                        (int)G);
+    if (cudaGetLastError() != cudaSuccess) return FFF_ERR_CUDA;
+    if (cudaFuncSetAttribute(fff::k_fused_small<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess)
+        return cudaGetLastError(), FFF_ERR_CUDA;
+    h->fs_G = (int)G;
+    h->fs_lp = lp;
+    h->fs_Dp = Dp;
+    h->fs_batch = batch;
+    return FFF_OK;
+}
+
+// Whether a forward of this handle runs as the one-launch kernel: when pinned to it, or by default for layers
+// that have no tensor-core leaf path (float32, or bf16 shapes outside it) and room for batches of at least 8.
+bool use_fused_small(const fff_handle_s* h) {
+    if (h->fs_batch == 0 || !h->tune[FFF_TUNE_FUSED_SMALL]) return false;
+    if (h->path == FFF_PATH_FUSED) return true;
+    return h->path == FFF_PATH_AUTO && h->LP == 0 && h->fs_batch >= 8;
+}
+
+template <typename T>
+fff_status_t run_fused_small(fff_handle_s* h, const void* x, void* y, int32_t* leaf_out, int32_t* leaf_out2, int64_t B,
+                             cudaStream_t st) {
+    const int G = h->fs_G, S = std::max(1, h->sm_count / G);
+    const fff::FusedSmallLayout L{h->fs_Dp, h->O, h->fs_batch};
+    const T* xp = (const T*)x;
+    const T *nw = (const T*)h->node_w, *nb = (const T*)h->node_b;
+    const float *w1g = h->fs_w1g, *b1g = h->fs_b1g, *w2g = h->fs_w2g, *b2f = h->fs_b2f;
+    T* yp = (T*)y;
+    int D = h->D, Dp = h->fs_Dp, O = h->O, depth = h->depth, l = h->l, lp = h->fs_lp, act = h->act, Bi = (int)B, Gi = G,
+        batch = h->fs_batch, vec = h->vec_ok && aligned16(x) ? 1 : 0, nl = (int)h->n_leaves;
+    int* status = h->d_status;
+    void* args[] = {&xp, &nw, &nb, &w1g, &b1g, &w2g, &b2f, &yp, &leaf_out, &leaf_out2, &D, &Dp, &O, &depth, &l, &lp, &act, &Bi,
+                    &Gi, &batch, &vec, &nl, &status};
+    if (cudaLaunchCooperativeKernel((const void*)fff::k_fused_small<T>, dim3((unsigned)(G * S)), dim3(fff::kFSThreads), args,
+                                    L.total(), st) != cudaSuccess)
+        return cudaGetLastError(), FFF_ERR_CUDA;
+    return launched(h, st, "fused_forward_small");
+}
+
 #define FFF_DISPATCH(h, fn, ...) \
     ((h)->dtype == FFF_DTYPE_F32 ? fn<float>(__VA_ARGS__) : fn<__nv_bfloat16>(__VA_ARGS__))
 
@@ -1049,6 +1113,7 @@ fff_status_t fff_create(fff_handle_t* out, int D, int O, int depth, int leaf_wid
         h->LP = leaf_width <= 16 ? 16 : (leaf_width <= 32 ? 32 : 64);
         s = pack_leaf_images<__nv_bfloat16>(h);
     }
+    if (s == FFF_OK) s = FFF_DISPATCH(h, pack_fused_small, h);
     if (s == FFF_OK && cudaDeviceSynchronize() != cudaSuccess) s = (cudaGetLastError(), FFF_ERR_CUDA);
     if (s != FFF_OK) { release(h); return s; }
     {
@@ -1079,8 +1144,10 @@ fff_status_t fff_reserve(fff_handle_t h, int64_t max_B) {
 
 fff_status_t fff_set_path(fff_handle_t h, fff_path_t path) {
     if (!live(h)) return FFF_ERR_BAD_HANDLE;
-    if (path != FFF_PATH_AUTO && path != FFF_PATH_WARP && path != FFF_PATH_TENSOR) return FFF_ERR_INVALID_ARG;
+    if (path != FFF_PATH_AUTO && path != FFF_PATH_WARP && path != FFF_PATH_TENSOR && path != FFF_PATH_FUSED)
+        return FFF_ERR_INVALID_ARG;
     if (path == FFF_PATH_TENSOR && h->LP == 0 && h->stages.empty()) return FFF_ERR_UNSUPPORTED;
+    if (path == FFF_PATH_FUSED && h->fs_batch == 0) return FFF_ERR_UNSUPPORTED;
     h->path = path;
     return FFF_OK;
 }
@@ -1150,6 +1217,21 @@ fff_status_t fff_forward_infer(fff_handle_t h, const void* x, void* y, int32_t* 
     h->prof_active = h->prof_steps < h->prof_max_steps;
     if (h->prof_active)
         cudaEventRecord(h->prof_events[(size_t)h->prof_steps * (fff_handle_s::kMaxProfLaunches + 1)], st);
+    if (use_fused_small(h)) {
+        // one launch: descent, grid barrier, leaf evaluation by groups of hidden neurons; the stable bucketing is
+        // made on demand from the leaf indices it leaves in the workspace
+        s = FFF_DISPATCH(h, run_fused_small, h, x, y, h->ws_leaf, leaf_idx, B, st);
+        h->last_perm = h->ws_perm;
+        h->bucketing_pending = true;
+        if (h->prof_active) {
+            h->prof_active = false;
+            if (s == FFF_OK && (h->prof_steps == 0 || h->prof_nlaunch == h->launches)) {
+                h->prof_nlaunch = std::min(h->launches, (int)fff_handle_s::kMaxProfLaunches);
+                ++h->prof_steps;
+            }
+        }
+        return s;
+    }
     const bool tensor_leaf = use_tensor_leaf(h);
     // With fewer than about 4 tokens per leaf the warp leaf kernel gains nothing from bucket order (no
     // weights to share), so the bucketing is left out of the forward and made on demand

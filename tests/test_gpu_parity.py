@@ -16,7 +16,7 @@ from tests import util
 
 pytestmark = pytest.mark.gpu
 
-PATHS = ["auto", "warp", "tensor"]
+PATHS = ["auto", "warp", "tensor", "fused"]
 
 
 def layer_on_path(case, path):
@@ -318,10 +318,12 @@ def test_forward_without_bucketing_kernel(routing):
     layer.close()
 
 
+@pytest.mark.parametrize("path,launches", [("warp", 3), ("auto", 1)])
 @pytest.mark.parametrize("routing", ["spread", "one_leaf"])
-def test_warp_kernels_changing_batch_sizes(routing):
-    """float32 layer with eight leaves (the warp kernels: descent, bucketing, leaf), also with every token in the last
-    leaf (zero node weights: a logit of 0 goes right), and with batch sizes that change from call to call."""
+def test_warp_kernels_changing_batch_sizes(routing, path, launches):
+    """float32 layer with eight leaves, on the warp kernels (descent, bucketing, leaf: three launches) and on the default
+    path (the one-launch kernel), also with every token in the last leaf (zero node weights: a logit of 0 goes right:
+    one group of hidden neurons gets every token), and with batch sizes that change from call to call."""
     cfg = wl.FFFConfig("f32_d3_batches", 784, 10, 3, 32, "relu", "f32", 2048, "normal")
     weights = wl.make_weights(cfg, 3)
     if routing == "one_leaf":
@@ -335,12 +337,12 @@ def test_warp_kernels_changing_batch_sizes(routing):
     y_ref, leaf_ref = orc.forward_i(net, case.x, threads=util.ORACLE_THREADS)
     if routing == "one_leaf":
         assert (leaf_ref == cfg.n_leaves - 1).all()
-    layer = util.make_layer(case)
+    layer = util.make_layer(case, path)
     x = util.to_device(case.x, "f32")
     for B in (cfg.B, 33, 1500, cfg.B):
         y, leaf = layer.forward_infer(x[:B])
         torch.cuda.synchronize()
-        assert layer.last_launch_count() == 3
+        assert layer.last_launch_count() == launches
         np.testing.assert_array_equal(leaf.cpu().numpy(), leaf_ref[:B])
         util.check_outputs(y, y_ref[:B], "f32")
         off, perm = layer.last_bucketing(B)
@@ -487,3 +489,37 @@ def test_every_tuning_switch_off_gives_the_same_results(switch):
         assert torch.equal(y_back, y_on)
         assert layer.last_status() == 0
         layer.close()
+
+
+@pytest.mark.parametrize("D", [256, 784])
+@pytest.mark.parametrize("width,l", [(16, 1), (16, 8), (32, 2), (64, 4), (128, 1), (128, 8), (64, 1), (128, 2)])
+def test_one_launch_kernel_on_the_shapes_of_the_papers_timing_tables(D, width, l):
+    """float32 layers of the shape grid of Table 1 and the appendix table of inference times (inputs of 256 or 784,
+    10 outputs, training width 16 to 128, leaves of 1 to 8 neurons, 2048 tokens): the default path is the
+    one-launch kernel (several leaves share a group of 32 hidden neurons), checked against the oracle element by
+    element, with the bucketing made on demand, twice in a row and on a shorter batch."""
+    depth = (width // l).bit_length() - 1
+    cfg = wl.FFFConfig(f"table1_D{D}_w{width}_l{l}", D, 10, depth, l, "relu", "f32", 2048, "normal", node_bias_std=0.1)
+    case = util.make_case(cfg, seed=width + l)
+    y_ref, leaf_ref = orc.forward_i(case.net, case.x, threads=util.ORACLE_THREADS)
+    layer = util.make_layer(case)
+    x = util.to_device(case.x, "f32")
+    for B in (cfg.B, cfg.B, 777):
+        y, leaf = layer.forward_infer(x[:B])
+        torch.cuda.synchronize()
+        assert layer.last_launch_count() == 1
+        np.testing.assert_array_equal(leaf.cpu().numpy(), leaf_ref[:B])
+        util.check_outputs(y, y_ref[:B], "f32")
+        off, perm = layer.last_bucketing(B)
+        off_b, perm_b = orc.bucket(leaf_ref[:B], cfg.n_leaves)
+        np.testing.assert_array_equal(off.cpu().numpy(), off_b)
+        np.testing.assert_array_equal(perm.cpu().numpy(), perm_b)
+    # the three-kernel path gives the same leaves and outputs within the same tolerance
+    layer.set_tuning("fused_small", False)
+    y3, leaf3 = layer.forward_infer(x)
+    torch.cuda.synchronize()
+    assert layer.last_launch_count() > 1
+    np.testing.assert_array_equal(leaf3.cpu().numpy(), leaf_ref)
+    util.check_outputs(y3, y_ref, "f32")
+    assert layer.last_status() == 0
+    layer.close()
