@@ -28,12 +28,25 @@
 #include <stdlib.h>
 #include <string.h>
 
-enum { FFF_ORACLE_RELU = 0, FFF_ORACLE_GELU = 1 };
+enum { FFF_ORACLE_RELU = 0, FFF_ORACLE_GELU = 1, FFF_ORACLE_GELU_TANH = 2, FFF_ORACLE_SILU = 3 };
 
+/*
+ * The leaf's hidden activation.  The paper never names one (Definition: the
+ * leaves are plain <D, l, O> feedforward networks), so it is a parameter:
+ *   RELU       max(v, 0)
+ *   GELU       v * Phi(v), Phi the standard normal CDF (exact erf form)
+ *   GELU_TANH  the published tanh approximation of GELU,
+ *              v/2 * (1 + tanh(sqrt(2/pi) * (v + 0.044715 v^3)))
+ *   SILU       v * sigmoid(v)
+ * Pinned by: library routines (torch), table values of Phi, the identity
+ * f(v) - f(-v) = v that the last three share, values at 0 and far from 0.
+ */
 static double act_fn(int act, double v)
 {
     if (act == FFF_ORACLE_RELU) return v > 0.0 ? v : 0.0;
-    /* exact GELU: v * Phi(v), Phi the standard normal CDF */
+    if (act == FFF_ORACLE_GELU_TANH)
+        return 0.5 * v * (1.0 + tanh(sqrt(2.0 / 3.14159265358979323846) * (v + 0.044715 * v * v * v)));
+    if (act == FFF_ORACLE_SILU) return v / (1.0 + exp(-v));
     return 0.5 * v * (1.0 + erf(v / sqrt(2.0)));
 }
 

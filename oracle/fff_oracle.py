@@ -15,7 +15,7 @@ import numpy as np
 
 from . import build as _build
 
-ACT = {"relu": 0, "gelu": 1}
+ACT = {"relu": 0, "gelu": 1, "gelu_tanh": 2, "silu": 3}
 
 _lib = None
 _dp = C.POINTER(C.c_double)

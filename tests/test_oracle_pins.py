@@ -103,7 +103,7 @@ def test_exactly_d_nodes_and_one_leaf_per_token():
 
 
 # ---------------------------------------------------------------- leaf evaluation
-@pytest.mark.parametrize("act", ["relu", "gelu"])
+@pytest.mark.parametrize("act", ["relu", "gelu", "gelu_tanh", "silu"])
 def test_depth_zero_is_a_plain_feedforward_layer(act):
     """d = 0: no nodes, one leaf -- the network is an ordinary <D, l, O> layer (library ops)."""
     rng = np.random.default_rng(2)
@@ -114,7 +114,8 @@ def test_depth_zero_is_a_plain_feedforward_layer(act):
     assert (leaf == 0).all()
     xt = torch.from_numpy(x)
     h = F.linear(xt, torch.from_numpy(net.w1[0]), torch.from_numpy(net.b1[0]))
-    h = F.relu(h) if act == "relu" else F.gelu(h)       # torch's default GELU is the exact erf form
+    # torch's default GELU is the exact erf form
+    h = {"relu": F.relu, "gelu": F.gelu, "gelu_tanh": lambda v: F.gelu(v, approximate="tanh"), "silu": F.silu}[act](h)
     ref = F.linear(h, torch.from_numpy(net.w2[0]), torch.from_numpy(net.b2[0])).numpy()
     np.testing.assert_allclose(y, ref, rtol=1e-12, atol=1e-13)
 
@@ -127,6 +128,26 @@ def test_gelu_known_values():
     y, _ = orc.forward_i(net, x)
     phi1, phi2 = 0.8413447460685429, 0.9772498680518208
     np.testing.assert_allclose(y[:, 0], [0.0, phi1, 2 * phi2, phi1 - 1.0, 30.0, 0.0], rtol=0, atol=1e-15)
+
+
+@pytest.mark.parametrize("act", ["gelu_tanh", "silu"])
+def test_smooth_activations_known_values_and_identity(act):
+    """Both are v times an increasing function s with s(v) + s(-v) = 1, so f(v) - f(-v) = v, f(0) = 0, f(v) -> v and
+    f(-v) -> 0 far from zero; SiLU(1) = 1 / (1 + e^-1); tanh-GELU(1) = (1 + tanh(sqrt(2/pi) * 1.044715)) / 2; and the
+    tanh form stays within 5e-4 of the exact GELU everywhere, yet is not equal to it."""
+    net = orc.Net(1, 1, 0, 1, act, None, None, [[[1.0]]], [[0.0]], [[[1.0]]], [[0.0]])
+    v = np.array([0.0, 1.0, -1.0, 2.5, -2.5, 40.0, -40.0, 0.3, -0.3])
+    y = orc.forward_i(net, v[:, None])[0][:, 0]
+    assert y[0] == 0.0
+    np.testing.assert_allclose(y[1::2] - y[2::2], v[1::2], rtol=0, atol=1e-14)
+    np.testing.assert_allclose(y[5:7], [40.0, 0.0], rtol=0, atol=1e-15)
+    one = 1.0 / (1.0 + np.exp(-1.0)) if act == "silu" else 0.5 * (1.0 + np.tanh(np.sqrt(2.0 / np.pi) * 1.044715))
+    np.testing.assert_allclose(y[1], one, rtol=1e-15)
+    if act == "gelu_tanh":
+        exact = orc.Net(1, 1, 0, 1, "gelu", None, None, [[[1.0]]], [[0.0]], [[[1.0]]], [[0.0]])
+        grid = np.linspace(-6, 6, 2401)[:, None]
+        diff = np.abs(orc.forward_i(net, grid)[0] - orc.forward_i(exact, grid)[0])
+        assert 1e-5 < diff.max() < 5e-4
 
 
 def test_leaf_biases_and_w2_orientation_matter():
@@ -180,7 +201,7 @@ def test_soft_mixture_follows_the_choice_product_on_a_depth_one_tree():
     np.testing.assert_allclose(y[:, 0], expect, rtol=1e-15)
 
 
-@pytest.mark.parametrize("act", ["relu", "gelu"])
+@pytest.mark.parametrize("act", ["relu", "gelu", "gelu_tanh", "silu"])
 def test_hard_inference_is_the_saturated_limit_of_the_soft_mixture(act):
     """Rescaling node coefficients squashes the sigmoid to a step: FORWARD_T -> FORWARD_I."""
     rng = np.random.default_rng(5)
