@@ -55,9 +55,13 @@ typedef enum {
 
 typedef enum {
     FFF_ACT_RELU = 0,            /* max(v, 0) */
-    FFF_ACT_GELU = 1             /* v * Phi(v), erf form (not the tanh approximation); the bf16 tensor-core
+    FFF_ACT_GELU = 1,            /* v * Phi(v), erf form (not the tanh approximation); the bf16 tensor-core
                                     kernels evaluate erf to 1.5e-7 absolute, below bf16 resolution */
-} fff_activation_t;
+    FFF_ACT_GELU_TANH = 2,       /* v/2 * (1 + tanh(sqrt(2/pi) * (v + 0.044715 v^3))): a different function from
+                                    FFF_ACT_GELU (up to 5e-4 apart), not a cheaper evaluation of it */
+    FFF_ACT_SILU = 3             /* v * sigmoid(v) */
+} fff_activation_t;              /* the leaf networks' hidden activation: the paper's Definition (leaves are
+                                    <dim_I, l, dim_O> feedforward networks) names none */
 
 typedef enum {
     FFF_DTYPE_F32 = 0,

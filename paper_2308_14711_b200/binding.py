@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(HERE, "libfff.so")
 FFF_OK = 0
 STATUS_NAMES = {0: "FFF_OK", 1: "FFF_ERR_INVALID_ARG", 2: "FFF_ERR_UNSUPPORTED", 3: "FFF_ERR_ALLOC",
                 4: "FFF_ERR_CUDA", 5: "FFF_ERR_DEVICE_TIMEOUT", 6: "FFF_ERR_BAD_HANDLE", 7: "FFF_ERR_TOO_LARGE"}
-ACTIVATIONS = {"relu": 0, "gelu": 1}
+ACTIVATIONS = {"relu": 0, "gelu": 1, "gelu_tanh": 2, "silu": 3}
 DTYPES = {"f32": 0, "bf16": 1}
 PATHS = {"auto": 0, "warp": 1, "tensor": 2, "fused": 3}
 TUNING = {"tcgen05_descent": 0, "tcgen05_grouped": 1, "tcgen05_leaf": 2, "cta_pairs": 3, "direct_lists": 4, "fused_small": 5}

@@ -1043,7 +1043,7 @@ fff_status_t fff_create(fff_handle_t* out, int D, int O, int depth, int leaf_wid
     if (!out) return FFF_ERR_INVALID_ARG;
     *out = nullptr;
     if (D < 1 || O < 1 || leaf_width < 1 || depth < 0) return FFF_ERR_INVALID_ARG;
-    if (act != FFF_ACT_RELU && act != FFF_ACT_GELU) return FFF_ERR_INVALID_ARG;
+    if (act != FFF_ACT_RELU && act != FFF_ACT_GELU && act != FFF_ACT_GELU_TANH && act != FFF_ACT_SILU) return FFF_ERR_INVALID_ARG;
     if (dtype != FFF_DTYPE_F32 && dtype != FFF_DTYPE_BF16) return FFF_ERR_INVALID_ARG;
     if (depth > FFF_MAX_DEPTH) return FFF_ERR_UNSUPPORTED;
     if (!leaf_w1 || !leaf_w2 || (depth > 0 && !node_w)) return FFF_ERR_INVALID_ARG;

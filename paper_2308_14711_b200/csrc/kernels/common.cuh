@@ -9,7 +9,7 @@ namespace fff {
 
 constexpr unsigned kFullMask = 0xffffffffu;
 
-enum : int { kActRelu = 0, kActGelu = 1 };
+enum : int { kActRelu = 0, kActGelu = 1, kActGeluTanh = 2, kActSilu = 3 };
 
 // Values written to the per-handle device status word by kernels.
 enum : int { kDevOk = 0, kDevTimeout = 1 };
@@ -60,8 +60,13 @@ __device__ __forceinline__ float warp_sum(float v) {
     return v;
 }
 
+// The leaf's hidden activation (create-time parameter; the paper's Definition leaves it open): ReLU, GELU in
+// the exact erf form, GELU in the published tanh form v/2 (1 + tanh(sqrt(2/pi) (v + 0.044715 v^3))), SiLU
+// v sigmoid(v).  All four map 0 to 0, which the zero-padded hidden units of the tensor-core images rely on.
 __device__ __forceinline__ float activate(int act, float v) {
     if (act == kActRelu) return fmaxf(v, 0.0f);
+    if (act == kActGeluTanh) return 0.5f * v * (1.0f + tanhf(0.79788456080286535588f * (v + 0.044715f * v * v * v)));
+    if (act == kActSilu) return v / (1.0f + expf(-v));
     return 0.5f * v * (1.0f + erff(v * 0.70710678118654752440f));
 }
 
@@ -70,6 +75,13 @@ __device__ __forceinline__ float activate(int act, float v) {
 // GELU value), one exponential and one division instead of the long polynomial of erff.
 __device__ __forceinline__ float activate_bf16(int act, float v) {
     if (act == kActRelu) return fmaxf(v, 0.0f);
+    if (act == kActGeluTanh) {
+        // tanh(u) = 1 - 2 / (1 + e^(2u)), u clamped where tanh is +-1 to float32 anyway (keeps e^(2u) finite)
+        const float u = fminf(fmaxf(0.79788456080286535588f * (v + 0.044715f * v * v * v), -15.0f), 15.0f);
+        const float th = 1.0f - __fdividef(2.0f, 1.0f + __expf(2.0f * u));
+        return 0.5f * v * (1.0f + th);
+    }
+    if (act == kActSilu) return v * __fdividef(1.0f, 1.0f + __expf(-fmaxf(v, -80.0f)));      // e^80 is finite; below, the result is -0
     const float z = fabsf(v) * 0.70710678118654752440f;
     const float t = __fdividef(1.0f, fmaf(0.3275911f, z, 1.0f));
     float poly = fmaf(1.061405429f, t, -1.453152027f);

@@ -53,7 +53,7 @@ class FFFConfig:
     O: int                    # dim_O
     depth: int                # d >= 0
     leaf_width: int           # l
-    activation: str           # "relu" | "gelu"
+    activation: str           # "relu" | "gelu" | "gelu_tanh" | "silu"
     dtype: str                # "f32" | "bf16"
     B: int                    # tokens per batch
     x_kind: str = "normal"    # "normal" | "layernorm" | "clusters"

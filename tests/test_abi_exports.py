@@ -46,7 +46,7 @@ def test_create_rejects_bad_arguments_on_the_host(lib):
         return lib.fff_create(C.byref(h) if out is None else out, a["D"], a["O"], a["depth"], a["l"], a["act"],
                               a["dt"], nw, None, w1, None, w2, None)
     assert create(out=C.POINTER(C.c_void_p)()) == 1
-    for bad in (dict(D=0), dict(O=-1), dict(l=0), dict(depth=-1), dict(act=7), dict(dt=3)):
+    for bad in (dict(D=0), dict(O=-1), dict(l=0), dict(depth=-1), dict(act=4), dict(act=-1), dict(dt=3)):
         assert create(**bad) == 1, bad
         assert h.value is None
     assert create(depth=21) == 2

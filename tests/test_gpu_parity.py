@@ -50,6 +50,12 @@ def small_cfgs():
         # O not a multiple of the 128-column output pieces; fewer tokens than one 128-row tile
         C("bf16_o208", 384, 208, 5, 20, "gelu", "bf16", 2000, "normal"),
         C("bf16_tiny_batch", 128, 144, 3, 16, "relu", "bf16", 37, "normal", node_bias_std=0.2),
+        # the other two leaf activations: float32 (one-launch and warp kernels) and bf16 (tensor-core epilogues, l below
+        # and at the padded width, thin buckets; warp kernels)
+        C("f32_silu", 96, 12, 3, 16, "silu", "f32", 700, "normal", node_bias_std=0.2),
+        C("f32_gelu_tanh", 200, 24, 2, 32, "gelu_tanh", "f32", 450, "normal"),
+        C("bf16_silu_l12", 256, 128, 5, 12, "silu", "bf16", 2500, "normal"),
+        C("bf16_gelu_tanh_l32", 128, 256, 6, 32, "gelu_tanh", "bf16", 3001, "clusters"),
         # eight levels in one dense stage (255 nodes), small batch
         C("bf16_d8_small", 256, 64, 8, 8, "gelu", "bf16", 5000, "layernorm"),
         # more 128-token tiles than SMs: the first stage runs on CTA pairs (127 nodes, odd number of tiles)
