@@ -250,6 +250,14 @@ fff_status_t fff_debug_get_bucketing(fff_handle_t h, int32_t *perm, int32_t *off
  * the last call (the word is cleared). */
 fff_status_t fff_get_last_status(fff_handle_t h);
 
+/* Self-test of the error path behind FFF_ERR_DEVICE_TIMEOUT (no counterpart in the paper).  Enqueues a
+ * one-CTA kernel whose threads wait, with the library's bounded-wait helpers, on a barrier that nothing
+ * ever signals; after limit_cycles (1 .. 2^24 SM clock cycles, i.e. at most about 10 ms) the wait gives
+ * up and the kernel records the timeout in the handle's status word and ends.  The next
+ * fff_get_last_status then returns FFF_ERR_DEVICE_TIMEOUT once, and FFF_OK after that.  Nothing faults
+ * and the context stays usable. */
+fff_status_t fff_selftest_bounded_wait(fff_handle_t h, int64_t limit_cycles, void *cuda_stream);
+
 /* Number of kernels the most recent forward / stage call of this handle enqueued
  * (-1 for a bad handle). */
 int fff_last_launch_count(fff_handle_t h);

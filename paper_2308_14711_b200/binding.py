@@ -27,7 +27,7 @@ TUNING = {"tcgen05_descent": 0, "tcgen05_grouped": 1, "tcgen05_leaf": 2, "cta_pa
 # every symbol include/fff.h declares
 EXPORTS = ["fff_create", "fff_forward_infer", "fff_forward_infer_host", "fff_destroy", "fff_reserve",
            "fff_set_path", "fff_set_tuning", "fff_tree_descent", "fff_leaf_bucketing", "fff_grouped_leaf_ff",
-           "fff_debug_get_bucketing", "fff_get_last_status", "fff_last_launch_count", "fff_status_string",
+           "fff_debug_get_bucketing", "fff_get_last_status", "fff_selftest_bounded_wait", "fff_last_launch_count", "fff_status_string",
            "fff_profile_begin", "fff_profile_end", "fff_profile_launches", "fff_profile_launch_name",
            "fff_leaf_bucketing_static"]
 
@@ -58,6 +58,7 @@ def lib():
     L.fff_reserve.argtypes = [vp, i64]
     L.fff_set_path.argtypes = [vp, ci]
     L.fff_set_tuning.argtypes = [vp, ci, ci]
+    L.fff_selftest_bounded_wait.argtypes = [vp, i64, vp]
     L.fff_tree_descent.argtypes = [vp, vp, vp, i64, vp]
     L.fff_leaf_bucketing.argtypes = [vp, vp, vp, vp, i64, vp]
     L.fff_grouped_leaf_ff.argtypes = [vp, vp, vp, vp, vp, vp, i64, vp]
@@ -138,6 +139,10 @@ def fff_debug_get_bucketing(h, perm, offsets, stream=None) -> None:
 
 def fff_get_last_status(h) -> int:
     return lib().fff_get_last_status(h)
+
+
+def fff_selftest_bounded_wait(h, limit_cycles, stream=None) -> None:
+    _check(lib().fff_selftest_bounded_wait(h, limit_cycles, stream), "fff_selftest_bounded_wait")
 
 
 def fff_last_launch_count(h) -> int:

@@ -956,6 +956,25 @@ fff_status_t check_forward_args(fff_handle_t h, int64_t B) {
 
 }  // namespace
 
+// Self-test of the bounded waits: one CTA waits, through the same helpers as the tensor-core kernels, on a barrier
+// that nothing ever arrives on.  The wait gives up after limit_cycles, the thread records kDevTimeout in the status
+// word, as those kernels do, and the kernel ends; nothing faults and nothing waits longer than the limit.
+namespace fff {
+__global__ void k_selftest_bounded_wait(int* __restrict__ status, long long limit_cycles)
+{
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(&bar, 1);
+        ptx::fence_mbar_init();
+    }
+    __syncthreads();
+    bool timed_out = false;
+    if (threadIdx.x == 0 && !ptx::mbar_wait(&bar, 0, limit_cycles)) timed_out = true;
+    if (threadIdx.x == 32 && !ptx::mbar_wait_relaxed(&bar, 0, limit_cycles)) timed_out = true;
+    if (timed_out) atomicExch(status, kDevTimeout);
+}
+}  // namespace fff
+
 // ---- scratch of fff_leaf_bucketing_static ----------------------------------------------------
 // Two histogram buffers of FFF_STATIC_MAX_BINS counters each, resident on every device that loads the
 // library.  In host code this name only stands for the symbol; the device address comes from
@@ -1405,6 +1424,14 @@ fff_status_t fff_get_last_status(fff_handle_t h) {
         return FFF_ERR_DEVICE_TIMEOUT;
     }
     return FFF_OK;
+}
+
+fff_status_t fff_selftest_bounded_wait(fff_handle_t h, int64_t limit_cycles, void* cuda_stream) {
+    if (!live(h)) return FFF_ERR_BAD_HANDLE;
+    if (limit_cycles < 1 || limit_cycles > (int64_t)1 << 24) return FFF_ERR_INVALID_ARG;
+    DeviceGuard g(h->device);
+    fff::k_selftest_bounded_wait<<<1, 64, 0, (cudaStream_t)cuda_stream>>>(h->d_status, (long long)limit_cycles);
+    return cudaGetLastError() == cudaSuccess ? FFF_OK : FFF_ERR_CUDA;
 }
 
 int fff_last_launch_count(fff_handle_t h) { return live(h) ? h->launches : -1; }

@@ -29,6 +29,7 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 
 template <typename T> struct Elem;
 
+
 template <> struct Elem<float> {
     static constexpr int kVec = 4;   // elements per 16-byte load
     __device__ __forceinline__ static float to_float(float v) { return v; }

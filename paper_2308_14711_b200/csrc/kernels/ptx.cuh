@@ -45,23 +45,23 @@ constexpr long long kWaitCycles = 1ll << 28;   // about 0.14 s at 1.9 GHz
 // Waits for the phase with the given parity.  Returns false if it did not complete within
 // kWaitCycles; callers then stop waiting altogether (sticky flag), so a kernel whose pipeline
 // is broken drains in bounded time instead of hanging.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, long long limit_cycles = kWaitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity))
-        if (clock64() - t0 > kWaitCycles) return false;
+        if (clock64() - t0 > limit_cycles) return false;
     return true;
 }
 
 // The same for waits that are not latency-critical (producers waiting for a free slot): sleeps
 // between polls so that the polling warp leaves the issue slots of its scheduler to the warps that
 // do the arithmetic.
-__device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity, long long limit_cycles = kWaitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
         __nanosleep(200);
-        if (clock64() - t0 > kWaitCycles) return false;
+        if (clock64() - t0 > limit_cycles) return false;
     }
     return true;
 }

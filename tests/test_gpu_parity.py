@@ -529,3 +529,30 @@ def test_one_launch_kernel_on_the_shapes_of_the_papers_timing_tables(D, width, l
     util.check_outputs(y3, y_ref, "f32")
     assert layer.last_status() == 0
     layer.close()
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_once_and_the_handle_stays_usable():
+    """The error path of the tensor-core kernels' waits, exercised by the library's self-test kernel: a wait on a
+    barrier that nothing signals gives up after 100 000 cycles (about 50 microseconds), the status word reports
+    FFF_ERR_DEVICE_TIMEOUT exactly once, and forwards before and after it match the oracle."""
+    from paper_2308_14711_b200 import binding
+    cfg = wl.FFFConfig("timeout_probe", 128, 64, 5, 16, "gelu", "bf16", 1500, "normal")
+    case = util.make_case(cfg, seed=4)
+    y_ref, leaf_ref = orc.forward_i(case.net, case.x, threads=util.ORACLE_THREADS)
+    layer = util.make_layer(case)
+    x = util.to_device(case.x, "bf16")
+    y, leaf = layer.forward_infer(x)
+    assert layer.last_status() == 0
+    binding.fff_selftest_bounded_wait(layer.handle, 100_000, torch.cuda.current_stream().cuda_stream)
+    assert layer.last_status() == 5
+    assert binding.status_string(5) == "device-side wait timed out"
+    assert layer.last_status() == 0
+    y2, leaf2 = layer.forward_infer(x)
+    torch.cuda.synchronize()
+    assert layer.last_status() == 0
+    np.testing.assert_array_equal(leaf2.cpu().numpy(), leaf_ref)
+    util.check_outputs(y2, y_ref, "bf16")
+    assert torch.equal(y, y2)
+    with pytest.raises(Exception):
+        binding.fff_selftest_bounded_wait(layer.handle, 0)
+    layer.close()

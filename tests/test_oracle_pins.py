@@ -272,3 +272,54 @@ def test_mean_bucket_size_is_batch_over_leaves():
     leaf = np.random.default_rng(0).integers(0, 128, size=256).astype(np.int32)
     offsets, _ = orc.bucket(leaf, 128)
     assert np.diff(offsets).mean() == 2.0
+
+
+# ---- the stack oracle (several FFF blocks with layer normalisation and residual connections) ----------------
+
+def test_stack_layer_norm_is_the_library_layer_norm():
+    from oracle import fff_stack_oracle as so
+    rng = np.random.default_rng(7)
+    x = rng.standard_normal((9, 33)) * 3.0 + 1.5
+    g, b = rng.standard_normal(33), rng.standard_normal(33)
+    ref = F.layer_norm(torch.from_numpy(x), (33,), torch.from_numpy(g), torch.from_numpy(b), eps=1e-5).numpy()
+    np.testing.assert_allclose(so.layer_norm(x, g, b, 1e-5), ref, rtol=1e-12, atol=1e-13)
+    plain = F.layer_norm(torch.from_numpy(x), (33,), eps=1e-3).numpy()
+    np.testing.assert_allclose(so.layer_norm(x, None, None, 1e-3), plain, rtol=1e-12, atol=1e-13)
+
+
+def test_stack_storage_rounding_is_the_library_conversion():
+    from oracle import fff_stack_oracle as so
+    rng = np.random.default_rng(8)
+    a = np.concatenate([rng.standard_normal(4000) * 10.0 ** rng.integers(-6, 6, 4000), [0.0, -0.0, 1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8]])
+    ref = torch.from_numpy(a.astype(np.float32)).to(torch.bfloat16).double().numpy()
+    np.testing.assert_array_equal(so.store(a, "bf16"), ref)
+    np.testing.assert_array_equal(so.store(a, "f32"), a.astype(np.float32).astype(np.float64))
+
+
+def test_stack_of_one_plain_block_is_forward_i_and_zero_leaves_make_the_identity():
+    from oracle import fff_stack_oracle as so
+    rng = np.random.default_rng(9)
+    D = 12
+    nets = [rand_net(rng, D, D, 3, 4, "gelu") for _ in range(3)]
+    x = rng.standard_normal((40, D))
+    y1, leaves, margin = so.stack_forward(nets[:1], x, "f32", norms=None, residual=False)
+    y_ref, leaf_ref = orc.forward_i(nets[0], x)
+    np.testing.assert_array_equal(leaves[0], leaf_ref)
+    np.testing.assert_array_equal(y1, y_ref.astype(np.float32).astype(np.float64))
+    np.testing.assert_array_equal(margin, orc.path_margin(nets[0], x))
+    # residual blocks whose leaves output zero leave the token unchanged, whatever the normalisation does
+    for n in nets:
+        n.w2[:] = 0.0
+        n.b2[:] = 0.0
+    norms = [(rng.standard_normal(D), rng.standard_normal(D)), None, (None, None)]
+    x32 = x.astype(np.float32).astype(np.float64)
+    y3, leaves3, _ = so.stack_forward(nets, x32, "f32", norms=norms, residual=True)
+    np.testing.assert_array_equal(y3, x32)
+    assert len(leaves3) == 3
+    # two blocks by hand: x1 = x0 + f0(LN(x0)), x2 = x1 + f1(x1)
+    nets2 = [rand_net(rng, D, D, 2, 3, "relu") for _ in range(2)]
+    z0 = so.layer_norm(x32, norms[0][0], norms[0][1], 1e-5).astype(np.float32).astype(np.float64)
+    x1 = (x32 + orc.forward_i(nets2[0], z0)[0]).astype(np.float32).astype(np.float64)
+    x2 = (x1 + orc.forward_i(nets2[1], x1)[0]).astype(np.float32).astype(np.float64)
+    got, _, _ = so.stack_forward(nets2, x32, "f32", norms=[norms[0], None], residual=True)
+    np.testing.assert_array_equal(got, x2)
