@@ -277,6 +277,42 @@ fff_status_t fff_profile_end(fff_handle_t h, double *mean_ms, int *steps);
 int fff_profile_launches(fff_handle_t h);
 const char *fff_profile_launch_name(fff_handle_t h, int i);
 
+/*
+ * Several FFF layers behind one handle (Section "Fast feedforward layers as building blocks": FFF layers in
+ * place of the feedforward layers of a transformer, each behind a layer normalisation and inside a residual
+ * connection; the attention layers between them are not part of this library).  For token x_0 and K layers:
+ *     z_k     = layer_norm ? (x_k - mean) / sqrt(var + eps) * gamma_k + beta_k : x_k      (over the D features)
+ *     x_{k+1} = residual ? x_k + FFF_k(z_k) : FFF_k(z_k)                                   (FORWARD_I per layer)
+ * and y = x_K.  z_k and x_k are stored in the layers' element type between the kernels.
+ *
+ *   layers     n_layers distinct live handles on one device, one element type, D == O == the same width
+ *   ln_gamma   NULL, or n_layers device pointers to [D] vectors in the element type (an entry may be NULL = ones)
+ *   ln_beta    likewise (NULL = zeros); both are copied.  Ignored when layer_norm == 0
+ * The stack does not own the layers: destroy it before them, and run no other forward on them while one of
+ * the stack's is in flight.  fff_set_path / fff_set_tuning on the layers stay in effect.
+ */
+typedef struct fff_stack_s *fff_stack_t;
+fff_status_t fff_stack_create(fff_stack_t *out, int n_layers, const fff_handle_t *layers, int layer_norm,
+                              const void *const *ln_gamma, const void *const *ln_beta, float eps, int residual);
+
+/* x [B, D] in, y [B, D] out, leaf_idx [n_layers, B] out (may be NULL), all device; enqueued on `cuda_stream`.
+ * The first call of a size allocates the buffers between the layers (and synchronises). */
+fff_status_t fff_stack_forward(fff_stack_t s, const void *x, void *y, int32_t *leaf_idx, int64_t B, void *cuda_stream);
+
+/* on = 1: the stack records its forward into a CUDA graph the second time it is called with the same x, y,
+ * leaf_idx, B and stream, and replays that graph on every later call with those arguments (new contents of x
+ * are read; the addresses are part of the recording).  Other arguments run as plain launches and start a new
+ * recording.  If the forward cannot be recorded (the legacy default stream cannot be captured, for one), plain
+ * launches are used from then on; fff_stack_set_graph(s, 1) again allows another attempt.  Default 0. */
+fff_status_t fff_stack_set_graph(fff_stack_t s, int on);
+
+/* Kernels the most recent plain (not replayed) forward enqueued, and whether the most recent forward was a
+ * replay (-1 for a bad handle). */
+int fff_stack_last_launch_count(fff_stack_t s);
+int fff_stack_last_was_replay(fff_stack_t s);
+
+fff_status_t fff_stack_destroy(fff_stack_t s);
+
 /* Static, never NULL. */
 const char *fff_status_string(fff_status_t s);
 

@@ -29,7 +29,8 @@ EXPORTS = ["fff_create", "fff_forward_infer", "fff_forward_infer_host", "fff_des
            "fff_set_path", "fff_set_tuning", "fff_tree_descent", "fff_leaf_bucketing", "fff_grouped_leaf_ff",
            "fff_debug_get_bucketing", "fff_get_last_status", "fff_selftest_bounded_wait", "fff_last_launch_count", "fff_status_string",
            "fff_profile_begin", "fff_profile_end", "fff_profile_launches", "fff_profile_launch_name",
-           "fff_leaf_bucketing_static"]
+           "fff_leaf_bucketing_static", "fff_stack_create", "fff_stack_forward", "fff_stack_set_graph",
+           "fff_stack_last_launch_count", "fff_stack_last_was_replay", "fff_stack_destroy"]
 
 
 class FFFError(RuntimeError):
@@ -58,6 +59,12 @@ def lib():
     L.fff_reserve.argtypes = [vp, i64]
     L.fff_set_path.argtypes = [vp, ci]
     L.fff_set_tuning.argtypes = [vp, ci, ci]
+    L.fff_stack_create.argtypes = [C.POINTER(vp), ci, C.POINTER(vp), ci, C.POINTER(vp), C.POINTER(vp), C.c_float, ci]
+    L.fff_stack_forward.argtypes = [vp, vp, vp, vp, i64, vp]
+    L.fff_stack_set_graph.argtypes = [vp, ci]
+    L.fff_stack_last_launch_count.argtypes = [vp]
+    L.fff_stack_last_was_replay.argtypes = [vp]
+    L.fff_stack_destroy.argtypes = [vp]
     L.fff_selftest_bounded_wait.argtypes = [vp, i64, vp]
     L.fff_tree_descent.argtypes = [vp, vp, vp, i64, vp]
     L.fff_leaf_bucketing.argtypes = [vp, vp, vp, vp, i64, vp]
@@ -299,3 +306,59 @@ class FFFLayer:
 
     def last_launch_count(self) -> int:
         return fff_last_launch_count(self._h)
+
+
+class FFFStack:
+    """Several FFFLayer objects of one width behind one handle: optional layer normalisation in front of every
+    layer, optional residual connections, optional CUDA-graph replay.  The layers stay alive with the stack."""
+
+    def __init__(self, layers, layer_norm: bool = True, gammas=None, betas=None, eps: float = 1e-5, residual: bool = True):
+        torch = _torch()
+        self._s = None
+        self.layers = list(layers)
+        n = len(self.layers)
+        self.D = self.layers[0].D
+        self.tdtype = self.layers[0].tdtype
+        hs = (C.c_void_p * n)(*[l.handle for l in self.layers])
+
+        def ptrs(vs):
+            if vs is None:
+                return None
+            assert len(vs) == n
+            return (C.c_void_p * n)(*[None if v is None else _ptr(v, self.tdtype, (self.D,), "layer-norm vector") for v in vs])
+        out = C.c_void_p()
+        _check(lib().fff_stack_create(C.byref(out), n, hs, 1 if layer_norm else 0, ptrs(gammas), ptrs(betas), eps,
+                                      1 if residual else 0), "fff_stack_create")
+        self._s = out.value
+
+    def close(self) -> None:
+        if getattr(self, "_s", None):
+            s, self._s = self._s, None
+            _check(lib().fff_stack_destroy(s), "fff_stack_destroy")
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def set_graph(self, on: bool) -> None:
+        _check(lib().fff_stack_set_graph(self._s, 1 if on else 0), "fff_stack_set_graph")
+
+    def forward(self, x, y=None, leaf_idx=None, want_leaf_idx: bool = True, stream=None):
+        torch = _torch()
+        B = x.shape[0]
+        if y is None:
+            y = torch.empty((B, self.D), dtype=self.tdtype, device=x.device)
+        if leaf_idx is None and want_leaf_idx:
+            leaf_idx = torch.empty((len(self.layers), B), dtype=torch.int32, device=x.device)
+        st = (stream if stream is not None else torch.cuda.current_stream()).cuda_stream
+        _check(lib().fff_stack_forward(self._s, _ptr(x, self.tdtype, (B, self.D), "x"), _ptr(y, self.tdtype, (B, self.D), "y"),
+                                       _ptr(leaf_idx, torch.int32, (len(self.layers), B), "leaf_idx"), B, st), "fff_stack_forward")
+        return y, leaf_idx
+
+    def last_launch_count(self) -> int:
+        return lib().fff_stack_last_launch_count(self._s)
+
+    def last_was_replay(self) -> bool:
+        return lib().fff_stack_last_was_replay(self._s) == 1

@@ -24,6 +24,7 @@
 #include "kernels/leaf_mma.cuh"
 #include "kernels/leaf_umma.cuh"
 #include "kernels/leaf_warp.cuh"
+#include "kernels/stack.cuh"
 
 namespace {
 
@@ -129,10 +130,42 @@ struct fff_handle_s {
     std::vector<cudaEvent_t> prof_events;         // [prof_max_steps][kMaxProfLaunches + 1]
 };
 
+// Several layers behind one handle (fff_stack_*): the layers stay the caller's; the stack owns the buffers
+// between them, the normalisation parameters and, when asked to, one instantiated CUDA graph of its forward.
+struct fff_stack_s {
+    uint64_t magic = 0;
+    int device = 0, sm_count = 148;
+    std::vector<fff_handle_s*> layers;
+    std::vector<void*> gamma, beta;       // per layer, library-owned copies (nullptr = 1 / 0)
+    bool layer_norm = false, residual = false;
+    float eps = 1e-5f;
+    int D = 0, dtype = 0;
+    size_t esize = 4;
+    int64_t cap_B = 0;
+    void *buf_z = nullptr, *buf_y = nullptr, *buf_x[2] = {nullptr, nullptr};
+    // graph replay: the key of the forward that the instantiated graph holds, and of the last eager forward
+    bool want_graph = false, graph_failed = false;
+    cudaGraphExec_t exec = nullptr;
+    const void *key_x = nullptr, *key_y = nullptr, *key_leaf = nullptr, *seen_x = nullptr, *seen_y = nullptr, *seen_leaf = nullptr;
+    int64_t key_B = -1, seen_B = -1;
+    cudaStream_t key_stream = nullptr, seen_stream = nullptr;
+    int launches = 0;
+    bool replayed = false;
+};
+
 namespace {
+
+constexpr uint64_t kStackMagic = 0x4646465f53544b31ull;   // "FFF_STK1"
 
 std::mutex g_mu;
 std::set<fff_handle_s*> g_live;
+std::set<fff_stack_s*> g_live_stacks;
+
+bool live_stack(fff_stack_s* s) {
+    if (!s) return false;
+    std::lock_guard<std::mutex> lk(g_mu);
+    return g_live_stacks.count(s) != 0 && s->magic == kStackMagic;
+}
 
 bool live(fff_handle_t h) {
     if (!h) return false;
@@ -1480,6 +1513,200 @@ fff_status_t fff_profile_end(fff_handle_t h, double* mean_ms, int* steps) {
     }
     h->prof_max_steps = 0;      // stop recording; names and counts stay readable until the next begin
     return FFF_OK;
+}
+
+
+}  // extern "C"
+
+// ---- stacks of layers --------------------------------------------------------------------------------------
+
+namespace {
+
+void stack_release(fff_stack_s* s) {
+    if (s->exec) cudaGraphExecDestroy(s->exec);
+    for (void* p : s->gamma) dfree(p);
+    for (void* p : s->beta) dfree(p);
+    dfree(s->buf_z); dfree(s->buf_y); dfree(s->buf_x[0]); dfree(s->buf_x[1]);
+    s->magic = 0;
+    delete s;
+}
+
+template <typename T>
+fff_status_t stack_glue(fff_stack_s* s, const void* x_prev, const void* y_prev, void* x_out, void* z, int layer, int64_t B,
+                        cudaStream_t st) {
+    const int64_t blocks = std::min<int64_t>((B + fff::kStackWarps - 1) / fff::kStackWarps, (int64_t)s->sm_count * 8);
+    const bool vec = s->D % (int)(16 / s->esize) == 0 && aligned16(x_prev) && aligned16(y_prev) && aligned16(x_out) && aligned16(z);
+    fff::k_stack_glue<T><<<(unsigned)blocks, fff::kStackWarps * 32, 0, st>>>(
+        (const T*)x_prev, (const T*)y_prev, (T*)x_out, (T*)z, z ? (const T*)s->gamma[layer] : nullptr,
+        z ? (const T*)s->beta[layer] : nullptr, s->eps, s->D, B, vec);
+    ++s->launches;
+    return cudaGetLastError() == cudaSuccess ? FFF_OK : FFF_ERR_CUDA;
+}
+
+// The forward of the whole stack, enqueued kernel by kernel.
+fff_status_t stack_enqueue(fff_stack_s* s, const void* x, void* y, int32_t* leaf_idx, int64_t B, cudaStream_t st) {
+    const int K = (int)s->layers.size();
+    const void* x_cur = x;           // x_k
+    const void* y_prev = nullptr;    // y_{k-1}, not yet added to x_{k-1} (residual stacks)
+    fff_status_t rc = FFF_OK;
+    s->launches = 0;
+    for (int k = 0; k < K && rc == FFF_OK; ++k) {
+        const void* ffn_in = x_cur;
+        if (s->residual && y_prev) {
+            // x_k = x_{k-1} + y_{k-1}, and its normalisation in the same pass
+            void* x_new = s->buf_x[k & 1];
+            rc = s->dtype == FFF_DTYPE_F32 ? stack_glue<float>(s, x_cur, y_prev, x_new, s->layer_norm ? s->buf_z : nullptr, k, B, st)
+                                           : stack_glue<__nv_bfloat16>(s, x_cur, y_prev, x_new, s->layer_norm ? s->buf_z : nullptr, k, B, st);
+            x_cur = x_new;
+            ffn_in = s->layer_norm ? s->buf_z : x_new;
+        } else if (s->layer_norm) {
+            rc = s->dtype == FFF_DTYPE_F32 ? stack_glue<float>(s, x_cur, nullptr, nullptr, s->buf_z, k, B, st)
+                                           : stack_glue<__nv_bfloat16>(s, x_cur, nullptr, nullptr, s->buf_z, k, B, st);
+            ffn_in = s->buf_z;
+        }
+        if (rc != FFF_OK) break;
+        // without residual connections the last layer writes y itself, the others into the buffer the next one reads
+        void* out = (!s->residual && k == K - 1) ? y : (s->residual ? s->buf_y : s->buf_x[k & 1]);
+        rc = fff_forward_infer(s->layers[k], ffn_in, out, leaf_idx ? leaf_idx + (int64_t)k * B : nullptr, B, (void*)st);
+        s->launches += s->layers[k]->launches;
+        if (s->residual) y_prev = out;
+        else x_cur = out;
+    }
+    if (rc == FFF_OK && s->residual)
+        rc = s->dtype == FFF_DTYPE_F32 ? stack_glue<float>(s, x_cur, y_prev, y, nullptr, 0, B, st)
+                                       : stack_glue<__nv_bfloat16>(s, x_cur, y_prev, y, nullptr, 0, B, st);
+    return rc;
+}
+
+}  // namespace
+
+extern "C" {
+
+fff_status_t fff_stack_create(fff_stack_t* out, int n_layers, const fff_handle_t* layers, int layer_norm, const void* const* ln_gamma,
+                              const void* const* ln_beta, float eps, int residual) {
+    if (!out) return FFF_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (n_layers < 1 || n_layers > 1024 || !layers || !(eps >= 0.0f)) return FFF_ERR_INVALID_ARG;
+    for (int k = 0; k < n_layers; ++k)
+        if (!live(layers[k])) return FFF_ERR_BAD_HANDLE;
+    const fff_handle_s* first = layers[0];
+    for (int k = 0; k < n_layers; ++k) {
+        const fff_handle_s* h = layers[k];
+        if (h->device != first->device || h->dtype != first->dtype) return FFF_ERR_INVALID_ARG;
+        // a layer reads what the one before it wrote; residual connections and shared buffers need one width
+        if (h->D != first->D || h->O != first->D) return FFF_ERR_INVALID_ARG;
+        for (int j = 0; j < k; ++j)
+            if (layers[j] == layers[k]) return FFF_ERR_INVALID_ARG;      // a handle serves one forward at a time
+    }
+    fff_stack_s* s = new (std::nothrow) fff_stack_s();
+    if (!s) return FFF_ERR_ALLOC;
+    s->device = first->device;
+    s->sm_count = first->sm_count;
+    s->D = first->D;
+    s->dtype = first->dtype;
+    s->esize = first->esize;
+    s->layer_norm = layer_norm != 0;
+    s->residual = residual != 0;
+    s->eps = eps;
+    s->layers.assign(layers, layers + n_layers);
+    s->gamma.assign(n_layers, nullptr);
+    s->beta.assign(n_layers, nullptr);
+    DeviceGuard g(s->device);
+    fff_status_t rc = FFF_OK;
+    for (int k = 0; k < n_layers && rc == FFF_OK && s->layer_norm; ++k) {
+        if (ln_gamma && ln_gamma[k]) rc = clone(&s->gamma[k], ln_gamma[k], (size_t)s->D * s->esize);
+        if (rc == FFF_OK && ln_beta && ln_beta[k]) rc = clone(&s->beta[k], ln_beta[k], (size_t)s->D * s->esize);
+    }
+    if (rc == FFF_OK && cudaDeviceSynchronize() != cudaSuccess) rc = (cudaGetLastError(), FFF_ERR_CUDA);
+    if (rc != FFF_OK) { stack_release(s); return rc; }
+    s->magic = kStackMagic;
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        g_live_stacks.insert(s);
+    }
+    *out = s;
+    return FFF_OK;
+}
+
+fff_status_t fff_stack_destroy(fff_stack_t s) {
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        if (!s || g_live_stacks.erase(s) == 0) return FFF_ERR_BAD_HANDLE;
+    }
+    DeviceGuard g(s->device);
+    cudaDeviceSynchronize();
+    stack_release(s);
+    return cudaGetLastError() == cudaSuccess ? FFF_OK : FFF_ERR_CUDA;
+}
+
+fff_status_t fff_stack_set_graph(fff_stack_t s, int on) {
+    if (!live_stack(s)) return FFF_ERR_BAD_HANDLE;
+    if (on != 0 && on != 1) return FFF_ERR_INVALID_ARG;
+    s->want_graph = on != 0;
+    s->graph_failed = false;
+    return FFF_OK;
+}
+
+int fff_stack_last_launch_count(fff_stack_t s) { return live_stack(s) ? s->launches : -1; }
+int fff_stack_last_was_replay(fff_stack_t s) { return live_stack(s) ? (s->replayed ? 1 : 0) : -1; }
+
+fff_status_t fff_stack_forward(fff_stack_t s, const void* x, void* y, int32_t* leaf_idx, int64_t B, void* cuda_stream) {
+    if (!live_stack(s)) return FFF_ERR_BAD_HANDLE;
+    if (B < 0) return FFF_ERR_INVALID_ARG;
+    if (B > FFF_MAX_TOKENS) return FFF_ERR_UNSUPPORTED;
+    for (fff_handle_s* h : s->layers)
+        if (!live(h)) return FFF_ERR_BAD_HANDLE;
+    s->replayed = false;
+    if (B == 0) { s->launches = 0; return FFF_OK; }
+    if (!x || !y || !aligned16(x) || !aligned16(y)) return FFF_ERR_INVALID_ARG;
+    DeviceGuard g(s->device);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (B > s->cap_B) {
+        if (cudaDeviceSynchronize() != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
+        if (s->exec) { cudaGraphExecDestroy(s->exec); s->exec = nullptr; }
+        dfree(s->buf_z); dfree(s->buf_y); dfree(s->buf_x[0]); dfree(s->buf_x[1]);
+        s->buf_z = s->buf_y = s->buf_x[0] = s->buf_x[1] = nullptr;
+        s->cap_B = 0;
+        const size_t bytes = (size_t)B * s->D * s->esize;
+        fff_status_t rc;
+        if ((rc = dmalloc(&s->buf_z, bytes)) != FFF_OK || (rc = dmalloc(&s->buf_y, bytes)) != FFF_OK ||
+            (rc = dmalloc(&s->buf_x[0], bytes)) != FFF_OK || (rc = dmalloc(&s->buf_x[1], bytes)) != FFF_OK)
+            return rc;
+        for (fff_handle_s* h : s->layers)
+            if ((rc = grow_workspace(h, B)) != FFF_OK) return rc;
+        s->cap_B = B;
+    }
+    const bool same_as_graph = s->exec && s->key_x == x && s->key_y == y && s->key_leaf == leaf_idx && s->key_B == B && s->key_stream == st;
+    if (s->want_graph && same_as_graph) {
+        if (cudaGraphLaunch(s->exec, st) != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
+        s->replayed = true;
+        return FFF_OK;
+    }
+    // The second forward with the same arguments is recorded into a graph (the first ran every one-time set-up:
+    // workspaces, kernel attributes); later ones replay it.
+    const bool seen = s->seen_x == x && s->seen_y == y && s->seen_leaf == leaf_idx && s->seen_B == B && s->seen_stream == st;
+    if (s->want_graph && !s->graph_failed && seen) {
+        cudaGraph_t graph = nullptr;
+        if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
+            const fff_status_t rc = stack_enqueue(s, x, y, leaf_idx, B, st);
+            const cudaError_t ce = cudaStreamEndCapture(st, &graph);
+            cudaGraphExec_t exec = nullptr;
+            if (rc == FFF_OK && ce == cudaSuccess && graph && cudaGraphInstantiate(&exec, graph, 0) == cudaSuccess) {
+                cudaGraphDestroy(graph);
+                if (s->exec) cudaGraphExecDestroy(s->exec);
+                s->exec = exec;
+                s->key_x = x; s->key_y = y; s->key_leaf = leaf_idx; s->key_B = B; s->key_stream = st;
+                if (cudaGraphLaunch(s->exec, st) != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
+                s->replayed = true;
+                return FFF_OK;
+            }
+            if (graph) cudaGraphDestroy(graph);
+        }
+        cudaGetLastError();
+        s->graph_failed = true;            // this stack's forward cannot be recorded: plain launches from now on
+    }
+    s->seen_x = x; s->seen_y = y; s->seen_leaf = leaf_idx; s->seen_B = B; s->seen_stream = st;
+    return stack_enqueue(s, x, y, leaf_idx, B, st);
 }
 
 }  // extern "C"
