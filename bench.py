@@ -329,7 +329,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
            "h2d_bytes_per_step": B * cfg.D * cfg.elem_bytes, "d2h_bytes_per_step": B * cfg.O * cfg.elem_bytes + 4 * B}
 
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-           "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+           "ms_per_step": ms_per_step, "ms_per_step_min": ms_min / args.steps, "timed_regions": len(region_ms),
+           "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
            "dtype": cfg.dtype, "data": "synthetic",
            "config": {"workload": cfg.name, "D": cfg.D, "O": cfg.O, "depth": cfg.depth, "leaf_width": cfg.leaf_width,
                       "activation": cfg.activation, "tokens_per_step_per_gpu": B, "x": cfg.x_kind,
@@ -347,6 +348,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
             path_roofline["leaves_touched_oracle"] = out["cpu_baseline"].pop("leaves_touched")
         if not args.no_per_config:
             out["per_config"] = per_config_table(args, peaks, skip={cfg.name: (ms_per_step, path_roofline)})
+            # four layers of the ViT-shaped configuration as one stack (the paper's transformer use of the layer)
+            out["stack"] = stack_bench(wl.CONFIGS["vit_d8_l12_bf16"], 4, max(5, min(args.steps, 50)))
     layer.close()
     if dist is not None:
         dist.barrier()
@@ -389,6 +392,59 @@ def per_config_table(args, peaks, skip):
         if pr.get("roofline"):
             rows[name]["roofline"] = pr["roofline"]
     return rows
+
+
+def stack_bench(cfg: wl.FFFConfig, n_layers: int, steps: int) -> dict:
+    """n_layers layers of one configuration as a stack (layer normalisation + residual connections between them),
+    as plain launches and as a recorded CUDA graph: time per stack forward on resident inputs."""
+    import torch
+    from paper_2308_14711_b200.binding import FFFLayer, FFFStack
+    td = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
+    layers = []
+    for k in range(n_layers):
+        w = wl.make_weights(cfg, 100 + k)
+        dev = {n: torch.from_numpy(v).to(td).cuda() for n, v in w.items()}
+        layers.append(FFFLayer(cfg.D, cfg.O, cfg.depth, cfg.leaf_width, cfg.activation, cfg.dtype, **dev))
+        del dev
+    stack = FFFStack(layers, layer_norm=True, residual=True)
+    n_sets = n_buffer_sets(cfg)
+    xs = [torch.from_numpy(wl.TokenSource(cfg, 200 + i).x).to(td).cuda() for i in range(n_sets)]
+    ys = [torch.empty_like(x) for x in xs]
+    side = torch.cuda.Stream()
+    out = {"layers": n_layers, "workload": cfg.name, "tokens": cfg.B}
+    for mode in ("plain", "graph"):
+        stack.set_graph(mode == "graph")
+        with torch.cuda.stream(side):
+            for _ in range(3):                      # warm-up; with the graph on, the second call of a set records it
+                for i in range(1 if mode == "graph" else n_sets):
+                    stack.forward(xs[i], ys[i], want_leaf_idx=False, stream=side)
+            side.synchronize()
+            regions = []
+            t_begin = time.perf_counter()
+            while True:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(side)
+                for i in range(steps):
+                    # (the recording is tied to one set of addresses: the graph arm re-runs set 0, whose 155 MB
+                    # per layer pair still exceed L2 together with the buffers between the layers)
+                    j = 0 if mode == "graph" else i % n_sets
+                    stack.forward(xs[j], ys[j], want_leaf_idx=False, stream=side)
+                e1.record(side)
+                regions.append((e0, e1))
+                if time.perf_counter() - t_begin >= MIN_TIMED_SECONDS / 2 or len(regions) >= 256:
+                    break
+            side.synchronize()
+        ms = statistics.median(a.elapsed_time(b) for a, b in regions) / steps
+        out[f"ms_per_forward_{mode}"] = round(ms, 5)
+        if mode == "graph":
+            out["replayed"] = bool(stack.last_was_replay())
+        else:
+            out["launches_per_forward"] = stack.last_launch_count()
+    out["tokens_per_s"] = cfg.B / (min(out["ms_per_forward_plain"], out["ms_per_forward_graph"]) * 1e-3)
+    stack.close()
+    for l in layers:
+        l.close()
+    return out
 
 
 # ------------------------------------------------------------------------------------------- CPU oracle legs
