@@ -185,6 +185,58 @@ void fff_oracle_forward_t(int D, int O, int depth, int l, int act,
 }
 
 /*
+ * Mixture weights of FORWARD_T written as products over root paths: unrolling the recursion of Algorithm 1,
+ * leaf N_{d,j} enters the output with weight  prod_m (bit_m ? c_m : 1 - c_m), where the ancestor of leaf j at
+ * level m is N_{m, j >> (d-m)}, c_m its choice and bit_m = (j >> (d-m-1)) & 1 the child on j's path
+ * (1 = right, the child that c weighs).  For each token the 2^d weights form a stochastic vector (Section
+ * "Algorithm", paragraph on the soft mixture).  mix: [B][2^d].
+ * Pinned by: weights sum to 1; sum_j mix_j * leaf_j(x) equals the recursive FORWARD_T; d = 1 by hand.
+ */
+void fff_oracle_mixture_weights(int D, int depth, const double *node_w, const double *node_b,
+                                const double *x, long t0, long t1, double *mix)
+{
+    long nl = (long)1 << depth;
+    for (long t = t0; t < t1; ++t) {
+        const double *xt = x + (size_t)t * D;
+        for (long j = 0; j < nl; ++j) {
+            double p = 1.0;
+            for (long m = 0; m < depth; ++m) {
+                long n = j >> (depth - m);
+                long row = ((long)1 << m) - 1 + n;
+                double c = 1.0 / (1.0 + exp(-node_logit(D, node_w + (size_t)row * D, node_b[row], xt)));
+                long bit = (j >> (depth - m - 1)) & 1;
+                p *= bit ? c : 1.0 - c;
+            }
+            mix[(size_t)t * nl + j] = p;
+        }
+    }
+}
+
+/*
+ * Batch mean of the entropy of every node's choice (Section "Training", hardening: the hardening loss is
+ * the sum over the batch and the nodes of the entropies of the Bernoulli choices, and the batch means are
+ * what the paper monitors):  H(c) = -c ln c - (1 - c) ln(1 - c), with 0 ln 0 = 0, c = N_{m,n}(x) evaluated
+ * for EVERY token at EVERY node (not only along the token's path).  ent: [2^d - 1].
+ * Pinned by: c = 1/2 gives ln 2; saturated nodes give 0; a library entropy routine on a hand case.
+ */
+void fff_oracle_node_entropy(int D, int depth, const double *node_w, const double *node_b,
+                             const double *x, long B, double *ent)
+{
+    long nn = ((long)1 << depth) - 1;
+    for (long r = 0; r < nn; ++r) {
+        double sum = 0.0;
+        for (long t = 0; t < B; ++t) {
+            double c = 1.0 / (1.0 + exp(-node_logit(D, node_w + (size_t)r * D, node_b[r], x + (size_t)t * D)));
+            double h = 0.0;
+            if (c > 0.0) h -= c * log(c);
+            if (c < 1.0) h -= (1.0 - c) * log(1.0 - c);
+            sum += h;
+        }
+        ent[r] = B > 0 ? sum / (double)B : 0.0;
+    }
+}
+
+/*
  * Conditional execution written the wasteful way: evaluate every leaf, keep
  * the one whose region contains the token (each leaf is responsible for
  * exactly one region of the partition).  y = sum_j [j == leaf_idx] * L_j(x).

@@ -42,6 +42,10 @@ def _load():
     L.fff_oracle_forward_i.argtypes = [C.c_int] * 5 + [_dp] * 7 + [C.c_long, C.c_long, _dp, _ip, _lp, _lp]
     L.fff_oracle_forward_i.restype = None
     L.fff_oracle_forward_t.argtypes = [C.c_int] * 5 + [_dp] * 7 + [C.c_long, _dp]
+    L.fff_oracle_mixture_weights.restype = None
+    L.fff_oracle_mixture_weights.argtypes = [C.c_int, C.c_int, _dp, _dp, _dp, C.c_long, C.c_long, _dp]
+    L.fff_oracle_node_entropy.restype = None
+    L.fff_oracle_node_entropy.argtypes = [C.c_int, C.c_int, _dp, _dp, _dp, C.c_long, _dp]
     L.fff_oracle_forward_t.restype = None
     L.fff_oracle_forward_all_leaves_masked.argtypes = [C.c_int] * 5 + [_dp] * 5 + [C.c_long, _ip, _dp]
     L.fff_oracle_forward_all_leaves_masked.restype = None
@@ -158,6 +162,42 @@ def forward_t(net: Net, x) -> np.ndarray:
     y = np.zeros((x.shape[0], net.O))
     lib().fff_oracle_forward_t(*net._head(), *net._params(), _p(x), x.shape[0], _p(y))
     return y
+
+
+def forward_t_rows(net: Net, x, threads: int = 1) -> np.ndarray:
+    """FORWARD_T with the token loop split over threads (tokens are independent)."""
+    x = _d(x).reshape(-1, net.D)
+    B = x.shape[0]
+    y = np.zeros((B, net.O))
+    parts = _split(B, threads)
+
+    def run(i):
+        a, b = parts[i]
+        lib().fff_oracle_forward_t(*net._head(), *net._params(), _p(x[a:b]), b - a, _p(y[a:b]))
+    _run(run, len(parts))
+    return y
+
+
+def mixture_weights(net: Net, x, threads: int = 1) -> np.ndarray:
+    """Weight of every leaf in FORWARD_T's mixture, float64 [B, 2^d]."""
+    x = _d(x).reshape(-1, net.D)
+    B = x.shape[0]
+    mix = np.zeros((B, 1 << net.depth))
+    parts = _split(B, threads)
+
+    def run(i):
+        a, b = parts[i]
+        lib().fff_oracle_mixture_weights(net.D, net.depth, _p(net.node_w), _p(net.node_b), _p(x), a, b, _p(mix))
+    _run(run, len(parts))
+    return mix
+
+
+def node_entropy(net: Net, x) -> np.ndarray:
+    """Batch mean of the entropy (nats) of every node's choice, float64 [2^d - 1]."""
+    x = _d(x).reshape(-1, net.D)
+    ent = np.zeros(max((1 << net.depth) - 1, 1))
+    lib().fff_oracle_node_entropy(net.D, net.depth, _p(net.node_w), _p(net.node_b), _p(x), x.shape[0], _p(ent))
+    return ent[:(1 << net.depth) - 1]
 
 
 def forward_all_leaves_masked(net: Net, x, leaf_idx) -> np.ndarray:

@@ -323,3 +323,52 @@ def test_stack_of_one_plain_block_is_forward_i_and_zero_leaves_make_the_identity
     x2 = (x1 + orc.forward_i(nets2[1], x1)[0]).astype(np.float32).astype(np.float64)
     got, _, _ = so.stack_forward(nets2, x32, "f32", norms=[norms[0], None], residual=True)
     np.testing.assert_array_equal(got, x2)
+
+
+# ---- FORWARD_T by products over paths, and node entropies --------------------------------------------------
+
+def test_mixture_weights_are_stochastic_and_reproduce_the_recursive_forward_t():
+    """The product form and the recursion of Algorithm 1 are two separate pieces of code: sum_j mix_j leaf_j(x)
+    must equal FORWARD_T, each row of weights must sum to 1, and d = 1 is (1 - c, c) by hand."""
+    rng = np.random.default_rng(11)
+    for depth in (1, 2, 4):
+        net = rand_net(rng, 5, 3, depth, 2, "gelu")
+        x = rng.standard_normal((13, 5))
+        mix = orc.mixture_weights(net, x, threads=2)
+        assert mix.shape == (13, 1 << depth) and (mix >= 0).all()
+        np.testing.assert_allclose(mix.sum(axis=1), 1.0, rtol=0, atol=1e-14)
+        leaves = np.stack([orc.forward_all_leaves_masked(net, x, np.full(13, j, np.int32)) for j in range(1 << depth)], axis=1)
+        np.testing.assert_allclose((mix[:, :, None] * leaves).sum(axis=1), orc.forward_t(net, x), rtol=1e-12, atol=1e-13)
+        np.testing.assert_array_equal(orc.forward_t_rows(net, x, threads=3), orc.forward_t(net, x))
+    net = rand_net(rng, 2, 1, 1, 1, "relu")
+    net.node_w[:] = [[2.0, -1.0]]
+    net.node_b[:] = [0.5]
+    c = 1.0 / (1.0 + np.exp(-(2.0 * 0.25 - 1.0 * 3.0 + 0.5)))
+    np.testing.assert_allclose(orc.mixture_weights(net, [[0.25, 3.0]]), [[1.0 - c, c]], rtol=1e-15)
+    # on the path of the hard descent every factor is at least 1/2: that leaf's weight is at least 2^-d
+    net = rand_net(rng, 6, 2, 3, 2, "relu")
+    x = rng.standard_normal((50, 6))
+    mix = orc.mixture_weights(net, x)
+    assert (mix[np.arange(50), orc.descend(net, x)[0]] >= 0.125).all()
+
+
+def test_node_entropy_closed_forms_and_library_routine():
+    """c = 1/2 everywhere gives ln 2 per node; saturated nodes give 0; a hand case against scipy's entropy."""
+    from scipy.stats import entropy
+    rng = np.random.default_rng(12)
+    net = rand_net(rng, 4, 2, 3, 2, "relu")
+    x = rng.standard_normal((20, 4))
+    keep_w, keep_b = net.node_w.copy(), net.node_b.copy()
+    net.node_w[:] = 0.0
+    net.node_b[:] = 0.0
+    np.testing.assert_allclose(orc.node_entropy(net, x), np.log(2.0), rtol=1e-14)
+    net.node_w[:] = keep_w * 1e4
+    net.node_b[:] = keep_b * 1e4
+    assert orc.node_entropy(net, x).max() < 1e-6
+    net.node_w[:], net.node_b[:] = keep_w, keep_b
+    ent = orc.node_entropy(net, x)
+    assert ent.shape == (7,) and (ent > 0).all() and (ent <= np.log(2.0)).all()
+    for r in (0, 3, 6):                         # every node sees every token
+        c = 1.0 / (1.0 + np.exp(-(x @ keep_w[r] + keep_b[r])))
+        ref = np.mean([entropy([ci, 1.0 - ci]) for ci in c])
+        np.testing.assert_allclose(ent[r], ref, rtol=1e-12)
