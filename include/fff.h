@@ -121,6 +121,27 @@ fff_status_t fff_forward_infer(fff_handle_t h, const void *x, void *y, int32_t *
                                int64_t B, void *cuda_stream);
 
 /*
+ * FORWARD_T of Algorithm 1 for B tokens: the training-time forward pass, in which every token is evaluated by
+ * ALL leaves and the outputs are mixed with the node choices, y = sum_j mix_j N_{d,j}(x), where mix_j is the
+ * product over the root path of leaf j of c = sigmoid(<w, x> + b) (where the path goes right) or 1 - c (left).
+ * A dense contraction over all 2^d l hidden neurons, run as three tensor-core GEMMs (bf16 products, float32
+ * accumulation; the weighted hidden activations are rounded to bf16 between the last two).
+ *
+ *   x             [B, D]       in
+ *   y             [B, O]       out
+ *   mixture       [B, 2^d]     out, float32, may be NULL: the weight of every leaf (each row sums to 1)
+ *   node_entropy  [2^d - 1]    out, float32, may be NULL: for every node, the batch mean of the entropy
+ *                 -c ln c - (1 - c) ln(1 - c) of its choice (Section "Training": the hardening loss is B times the
+ *                 sum of these; the batch means are what the paper monitors)
+ *
+ * bf16 layers with D % 64 == 0 only (FFF_ERR_UNSUPPORTED otherwise).  The first call of a size allocates a
+ * workspace of B (2^d l + 2^d) bf16 and B 2^(d+1) float32 and synchronises; later calls only enqueue.
+ * No gradients are computed: this is the forward half of a training step.
+ */
+fff_status_t fff_forward_train(fff_handle_t h, const void *x, void *y, float *mixture, float *node_entropy,
+                               int64_t B, void *cuda_stream);
+
+/*
  * The same computation for buffers in HOST memory (pinned or pageable):
  * copies x to the device, runs fff_forward_infer, copies y (and leaf_idx when
  * not NULL) back, and returns after `cuda_stream` has completed.  Batches of

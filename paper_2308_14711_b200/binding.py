@@ -25,7 +25,7 @@ PATHS = {"auto": 0, "warp": 1, "tensor": 2, "fused": 3}
 TUNING = {"tcgen05_descent": 0, "tcgen05_grouped": 1, "tcgen05_leaf": 2, "cta_pairs": 3, "direct_lists": 4, "fused_small": 5}
 
 # every symbol include/fff.h declares
-EXPORTS = ["fff_create", "fff_forward_infer", "fff_forward_infer_host", "fff_destroy", "fff_reserve",
+EXPORTS = ["fff_create", "fff_forward_infer", "fff_forward_train", "fff_forward_infer_host", "fff_destroy", "fff_reserve",
            "fff_set_path", "fff_set_tuning", "fff_tree_descent", "fff_leaf_bucketing", "fff_grouped_leaf_ff",
            "fff_debug_get_bucketing", "fff_get_last_status", "fff_selftest_bounded_wait", "fff_last_launch_count", "fff_status_string",
            "fff_profile_begin", "fff_profile_end", "fff_profile_launches", "fff_profile_launch_name",
@@ -59,6 +59,7 @@ def lib():
     L.fff_reserve.argtypes = [vp, i64]
     L.fff_set_path.argtypes = [vp, ci]
     L.fff_set_tuning.argtypes = [vp, ci, ci]
+    L.fff_forward_train.argtypes = [vp, vp, vp, vp, vp, i64, vp]
     L.fff_stack_create.argtypes = [C.POINTER(vp), ci, C.POINTER(vp), ci, C.POINTER(vp), C.POINTER(vp), C.c_float, ci]
     L.fff_stack_forward.argtypes = [vp, vp, vp, vp, i64, vp]
     L.fff_stack_set_graph.argtypes = [vp, ci]
@@ -248,6 +249,18 @@ class FFFLayer:
         fff_forward_infer(self._h, _ptr(x, self.tdtype, (B, self.D), "x"), _ptr(y, self.tdtype, (B, self.O), "y"),
                           _ptr(leaf_idx, torch.int32, (B,), "leaf_idx"), B, self._stream(stream))
         return y, leaf_idx
+
+    def forward_train(self, x, want_mixture: bool = True, want_entropy: bool = True, stream=None):
+        """FORWARD_T: returns (y, mixture weights float32 [B, 2^d] or None, node entropies float32 [2^d - 1] or None)."""
+        torch = _torch()
+        B = x.shape[0]
+        y = torch.empty((B, self.O), dtype=self.tdtype, device=x.device)
+        mix = torch.empty((B, self.n_leaves), dtype=torch.float32, device=x.device) if want_mixture else None
+        ent = torch.empty((max(self.n_leaves - 1, 1),), dtype=torch.float32, device=x.device) if want_entropy else None
+        _check(lib().fff_forward_train(self._h, _ptr(x, self.tdtype, (B, self.D), "x"), y.data_ptr(),
+                                       None if mix is None else mix.data_ptr(), None if ent is None else ent.data_ptr(), B,
+                                       self._stream(stream)), "fff_forward_train")
+        return y, mix, (None if ent is None else ent[:self.n_leaves - 1])
 
     def forward_infer_host(self, x_host, y_host, leaf_idx_host=None, stream=None) -> None:
         """x_host / y_host / leaf_idx_host: contiguous CPU tensors (pinned for full copy speed)."""

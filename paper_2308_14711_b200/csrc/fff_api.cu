@@ -21,6 +21,7 @@
 #include "kernels/descent_umma.cuh"
 #include "kernels/descent_warp.cuh"
 #include "kernels/fused_small.cuh"
+#include "kernels/gemm_umma.cuh"
 #include "kernels/leaf_mma.cuh"
 #include "kernels/leaf_umma.cuh"
 #include "kernels/leaf_warp.cuh"
@@ -92,6 +93,14 @@ struct fff_handle_s {
     // one-launch forward for small trees with thin leaves (fused_small.cuh); fs_batch == 0: shapes not eligible
     float *fs_w1g = nullptr, *fs_b1g = nullptr, *fs_w2g = nullptr, *fs_b2f = nullptr;
     int fs_G = 0, fs_lp = 0, fs_Dp = 0, fs_batch = 0;
+
+    // FORWARD_T (fff_forward_train): transposed output weights with the output biases appended along K, and the
+    // workspace of the three GEMMs (allocated on first use)
+    __nv_bfloat16* tr_w2t = nullptr;     // [O][tr_Kp]
+    int tr_Kp = 0;                       // 2^d l + 2^d rounded up to 64 (0 = shapes not eligible)
+    int64_t tr_cap_B = 0;
+    float *tr_c = nullptr, *tr_mix = nullptr, *tr_entpart = nullptr;
+    __nv_bfloat16* tr_hp = nullptr;
 
     // staged descent on tensor cores: consecutive groups of levels, each with its weight image
     struct DenseStage {
@@ -239,6 +248,7 @@ void release(fff_handle_s* h) {
     for (auto& sg : h->ustages) { dfree(sg.wimg); dfree(sg.bimg); }
     dfree(h->ws_pos[0]); dfree(h->ws_pos[1]);
     dfree(h->fs_w1g); dfree(h->fs_b1g); dfree(h->fs_w2g); dfree(h->fs_b2f);
+    dfree(h->tr_w2t); dfree(h->tr_c); dfree(h->tr_mix); dfree(h->tr_entpart); dfree(h->tr_hp);
     dfree(h->w1img); dfree(h->b1img); dfree(h->w2img); dfree(h->w2uimg); dfree(h->ws_sched); dfree(h->ws_tiles); dfree(h->ws_rank); dfree(h->ws_rank8); dfree(h->ws_counts8); dfree(h->ws_blocksum); dfree(h->ws_matrix); dfree(h->ws_slots); dfree(h->ws_cursor);
     if (h->copy_in) cudaStreamDestroy(h->copy_in);
     if (h->copy_out) cudaStreamDestroy(h->copy_out);
@@ -977,6 +987,100 @@ fff_status_t run_fused_small(fff_handle_s* h, const void* x, void* y, int32_t* l
     return launched(h, st, "fused_forward_small");
 }
 
+// FORWARD_T: the transposed output weights (at creation) and the three GEMMs.
+fff_status_t pack_train_images(fff_handle_s* h) {
+    if (h->dtype != FFF_DTYPE_BF16 || h->D % fff::kGKB != 0 || !encode_tiled_fn()) return FFF_OK;
+    const int64_t k_used = h->n_leaves * h->l + h->n_leaves;
+    if (k_used > (1 << 24)) return FFF_OK;
+    const int Kp = (int)((k_used + fff::kGKB - 1) / fff::kGKB * fff::kGKB);
+    fff_status_t s;
+    if ((s = dmalloc((void**)&h->tr_w2t, sizeof(__nv_bfloat16) * (size_t)h->O * Kp)) != FFF_OK) return s;
+    fff::k_pack_w2_transposed<__nv_bfloat16><<<h->sm_count * 8, 256>>>((const __nv_bfloat16*)h->w2, (const __nv_bfloat16*)h->b2,
+                                                                      h->tr_w2t, (int)h->n_leaves, h->l, h->O, Kp);
+    if (cudaGetLastError() != cudaSuccess) return FFF_ERR_CUDA;
+    for (auto kern : {(const void*)fff::k_gemm_umma<fff::kGemmNodes>, (const void*)fff::k_gemm_umma<fff::kGemmHidden>,
+                      (const void*)fff::k_gemm_umma<fff::kGemmOutput>})
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, fff::kGSmemBytes) != cudaSuccess)
+            return cudaGetLastError(), FFF_ERR_CUDA;
+    h->tr_Kp = Kp;
+    return FFF_OK;
+}
+
+template <int MODE>
+fff_status_t launch_gemm(fff_handle_s* h, const void* a, int64_t M, int lda, const void* b, int64_t N, int64_t K,
+                         const fff::GemmEpilogueArgs& ep, cudaStream_t st, const char* name) {
+    CUtensorMap ta, tb;
+    // (row pitch = lda elements; the tensor maps describe K columns of them)
+    EncodeTiledFn enc = encode_tiled_fn();
+    auto encode = [&](CUtensorMap* tm, const void* p, int64_t rows, int64_t pitch, int box_rows) {
+        const cuuint64_t gdim[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+        const cuuint64_t gstride[1] = {(cuuint64_t)pitch * 2};
+        const cuuint32_t box[2] = {(cuuint32_t)fff::kGKB, (cuuint32_t)box_rows};
+        const cuuint32_t estride[2] = {1, 1};
+        return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(p), gdim, gstride, box, estride,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    };
+    if (!enc || !encode(&ta, a, M, lda, fff::kGM) || !encode(&tb, b, N, K, fff::kGN)) return FFF_ERR_CUDA;
+    const int64_t tiles = ((M + fff::kGM - 1) / fff::kGM) * ((N + fff::kGN - 1) / fff::kGN);
+    const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(h->sm_count, tiles));
+    fff::k_gemm_umma<MODE><<<(unsigned)grid, fff::kGThreads, fff::kGSmemBytes, st>>>(ta, tb, (int)M, (int)N, (int)K, ep, h->d_status);
+    return launched(h, st, name);
+}
+
+fff_status_t run_forward_train(fff_handle_s* h, const void* x, void* y, float* mixture, float* node_entropy, int64_t B,
+                               cudaStream_t st) {
+    const int64_t nl = h->n_leaves, nn = h->n_nodes, hidden = nl * h->l;
+    const int ldc = (int)std::max<int64_t>(nn, 1);
+    const int64_t n_mt = (B + fff::kGM - 1) / fff::kGM;
+    if (B > h->tr_cap_B) {
+        if (cudaDeviceSynchronize() != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
+        dfree(h->tr_c); dfree(h->tr_mix); dfree(h->tr_entpart); dfree(h->tr_hp);
+        h->tr_c = h->tr_mix = h->tr_entpart = nullptr;
+        h->tr_hp = nullptr;
+        h->tr_cap_B = 0;
+        fff_status_t s;
+        if ((s = dmalloc((void**)&h->tr_c, sizeof(float) * (size_t)B * ldc)) != FFF_OK) return s;
+        if ((s = dmalloc((void**)&h->tr_mix, sizeof(float) * (size_t)B * nl)) != FFF_OK) return s;
+        if ((s = dmalloc((void**)&h->tr_entpart, sizeof(float) * (size_t)n_mt * 4 * ldc)) != FFF_OK) return s;
+        if ((s = dmalloc((void**)&h->tr_hp, sizeof(__nv_bfloat16) * (size_t)B * h->tr_Kp)) != FFF_OK) return s;
+        h->tr_cap_B = B;
+    }
+    fff_status_t s = FFF_OK;
+    fff::GemmEpilogueArgs ep = {};
+    if (nn > 0) {
+        ep.bias = (const __nv_bfloat16*)h->node_b;
+        ep.out_f32 = h->tr_c;
+        ep.ent_part = node_entropy ? h->tr_entpart : nullptr;
+        ep.ld_out = ldc;
+        if ((s = launch_gemm<fff::kGemmNodes>(h, x, B, h->D, h->node_w, nn, h->D, ep, st, "train_node_choices")) != FFF_OK) return s;
+        if (node_entropy) {
+            fff::k_entropy_reduce<<<(unsigned)((nn + 255) / 256), 256, 0, st>>>(h->tr_entpart, (int)(n_mt * 4), (int)nn, B, node_entropy);
+            if ((s = launched(h, st, "train_node_entropy")) != FFF_OK) return s;
+        }
+    }
+    {
+        const int64_t total = B * (h->tr_Kp - hidden);
+        const int64_t blocks = std::max<int64_t>(1, std::min<int64_t>((total + 255) / 256, (int64_t)h->sm_count * 16));
+        fff::k_mixture_weights<<<(unsigned)blocks, 256, 0, st>>>(h->tr_c, ldc, h->tr_mix, mixture, h->tr_hp, h->tr_Kp, (int)hidden,
+                                                                 h->depth, B);
+        if ((s = launched(h, st, "train_mixture_weights")) != FFF_OK) return s;
+    }
+    ep = {};
+    ep.bias = (const __nv_bfloat16*)h->b1;
+    ep.mix = h->tr_mix;
+    ep.out_bf16 = h->tr_hp;
+    ep.ld_out = h->tr_Kp;
+    ep.n_leaves = (int)nl;
+    ep.l = h->l;
+    ep.act = h->act;
+    if ((s = launch_gemm<fff::kGemmHidden>(h, x, B, h->D, h->w1, hidden, h->D, ep, st, "train_hidden_all_leaves")) != FFF_OK) return s;
+    ep = {};
+    ep.out_bf16 = (__nv_bfloat16*)y;
+    ep.ld_out = h->O;
+    return launch_gemm<fff::kGemmOutput>(h, h->tr_hp, B, h->tr_Kp, h->tr_w2t, h->O, h->tr_Kp, ep, st, "train_output_mixture");
+}
+
 #define FFF_DISPATCH(h, fn, ...) \
     ((h)->dtype == FFF_DTYPE_F32 ? fn<float>(__VA_ARGS__) : fn<__nv_bfloat16>(__VA_ARGS__))
 
@@ -1166,6 +1270,7 @@ fff_status_t fff_create(fff_handle_t* out, int D, int O, int depth, int leaf_wid
         s = pack_leaf_images<__nv_bfloat16>(h);
     }
     if (s == FFF_OK) s = FFF_DISPATCH(h, pack_fused_small, h);
+    if (s == FFF_OK) s = pack_train_images(h);
     if (s == FFF_OK && cudaDeviceSynchronize() != cudaSuccess) s = (cudaGetLastError(), FFF_ERR_CUDA);
     if (s != FFF_OK) { release(h); return s; }
     {
@@ -1344,6 +1449,18 @@ fff_status_t fff_forward_infer(fff_handle_t h, const void* x, void* y, int32_t* 
         }
     }
     return s;
+}
+
+fff_status_t fff_forward_train(fff_handle_t h, const void* x, void* y, float* mixture, float* node_entropy, int64_t B,
+                               void* cuda_stream) {
+    fff_status_t s = check_forward_args(h, B);
+    if (s != FFF_OK) return s;
+    if (h->tr_Kp == 0) return FFF_ERR_UNSUPPORTED;
+    if (B == 0) { h->launches = 0; return FFF_OK; }
+    if (!x || !y || !aligned16(x) || !aligned16(y)) return FFF_ERR_INVALID_ARG;
+    DeviceGuard g(h->device);
+    h->launches = 0;
+    return run_forward_train(h, x, y, mixture, node_entropy, B, (cudaStream_t)cuda_stream);
 }
 
 fff_status_t fff_forward_infer_host(fff_handle_t h, const void* x_host, void* y_host, int32_t* leaf_idx_host,

@@ -1,0 +1,304 @@
+// Dense bf16 GEMM on the fifth-generation tensor cores, C = epilogue(A . B^T), for FORWARD_T.
+//
+// Algorithm 1, FORWARD_T: the training-time forward pass evaluates EVERY node and EVERY leaf for every
+// token and mixes the leaf outputs with the products of the node choices along the root paths.  Unlike
+// hard inference this is a true dense contraction, so it runs as three GEMMs with fused epilogues:
+//   kGemmNodes   c[t, r]   = sigmoid(<x_t, w_r> + b_r)                    for all 2^d - 1 nodes r
+//   kGemmHidden  h'[t, q]  = mix[t, leaf(q)] * act(<x_t, W1_q> + b1_q)    for all 2^d l hidden neurons q
+//   kGemmOutput  y[t, o]   = sum_q h'[t, q] W2[o, q] + sum_j mix[t, j] b2[j, o]
+// (the mixture of the output biases rides in 2^d extra columns of the K dimension of the last GEMM).
+//
+// A is [M, K] and B is [N, K], both row-major with K contiguous, read through tensor maps (128-byte
+// swizzle, rows outside the matrix read as zeros).  One persistent CTA per SM works on 128 x 256 tiles of
+// C: warp 4 issues the tensor-map loads of the K-blocks (64 columns) into a ring of shared-memory stages,
+// warp 5 issues four tcgen05.mma (M = 128, N = 256, K = 16) per stage into one of two accumulators in
+// tensor memory, warps 0-3 read the finished accumulator (one row per thread), apply the epilogue and
+// store.  Tiles that share their rows of A are neighbours in the schedule, so A is read from DRAM once.
+//
+// Every wait is bounded (see ptx.cuh); tensor memory is released on every exit path.
+// Requirements: bf16, K % 64 == 0, A and B 16-byte aligned with row pitches that are multiples of 16 bytes.
+#pragma once
+
+#include <cuda.h>      // CUtensorMap
+
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace fff {
+
+constexpr int kGM = 128;                 // rows of C per tile = rows of one tcgen05.mma
+constexpr int kGN = 256;                 // columns of C per tile
+constexpr int kGKB = 64;                 // K-block: 128 bytes, one swizzle line
+constexpr int kGStages = 4;
+constexpr int kGThreads = 6 * 32;
+constexpr int kGStageBytes = (kGM + kGN) * kGKB * 2;                 // 48 KB
+constexpr int kGSmemBytes = 1024 + kGStages * kGStageBytes + 256;
+constexpr int kGTmemCols = 2 * kGN;
+
+enum : int { kGemmNodes = 0, kGemmHidden = 1, kGemmOutput = 2 };
+
+// Entropy in nats of a Bernoulli choice with probability c, 0 ln 0 = 0.
+__device__ __forceinline__ float bernoulli_entropy(float c) {
+    float h = 0.0f;
+    if (c > 0.0f) h -= c * __logf(c);
+    if (c < 1.0f) h -= (1.0f - c) * __logf(1.0f - c);
+    return h;
+}
+
+struct GemmEpilogueArgs {
+    // kGemmNodes: bias = node biases [N] (bf16), out_f32 = c [M, ld_out]; ent_part (optional) = [m tiles * 4][N]
+    // sums of the entropies over each warp's 32 rows.
+    // kGemmHidden: bias = hidden biases [N] (bf16), mix = [M, n_leaves] float32, l = neurons per leaf,
+    // out_bf16 = h' [M, ld_out].
+    // kGemmOutput: out_bf16 = y [M, ld_out].
+    const __nv_bfloat16* bias;
+    const float* mix;
+    float* out_f32;
+    __nv_bfloat16* out_bf16;
+    float* ent_part;
+    int ld_out, n_leaves, l, act;
+};
+
+template <int MODE>
+__global__ void __launch_bounds__(kGThreads, 1)
+k_gemm_umma(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, int M, int N, int K,
+            GemmEpilogueArgs ep, int* __restrict__ status)
+{
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* full = reinterpret_cast<uint64_t*>(ring + kGStages * kGStageBytes);
+    uint64_t* empty = full + kGStages;
+    uint64_t* acc_full = empty + kGStages;
+    uint64_t* acc_empty = acc_full + 2;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_mt = (M + kGM - 1) / kGM, n_nt = (N + kGN - 1) / kGN;
+    const int n_tiles = n_mt * n_nt;
+    const int KB = K / kGKB;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kGStages; ++s) {
+            ptx::mbar_init(full + s, 1);
+            ptx::mbar_init(empty + s, 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            ptx::mbar_init(acc_full + a, 1);
+            ptx::mbar_init(acc_empty + a, 4 * 32);
+        }
+        ptx::fence_mbar_init();
+        ptx::prefetch_tensormap(&tmap_a);
+        ptx::prefetch_tensormap(&tmap_b);
+    }
+    if (warp == 5) {
+        ptx::tmem_alloc(tmem_slot, kGTmemCols);
+        ptx::tmem_relinquish_alloc_permit();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    bool timed_out = false;
+    if (warp == 4) {
+        // ------------------------------------------------------------------ producer
+        int stage = 0;
+        uint32_t phase = 0;
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+            const int mt = tile / n_nt, nt = tile % n_nt;
+            for (int kb = 0; kb < KB; ++kb) {
+                if (!timed_out && !ptx::mbar_wait_relaxed(empty + stage, phase ^ 1)) timed_out = true;
+                if (lane == 0) {
+                    unsigned char* st = ring + stage * kGStageBytes;
+                    ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)kGStageBytes);
+                    ptx::tma_load_2d(st, &tmap_a, kb * kGKB, mt * kGM, full + stage);
+                    ptx::tma_load_2d(st + kGM * kGKB * 2, &tmap_b, kb * kGKB, nt * kGN, full + stage);
+                }
+                __syncwarp();
+                if (++stage == kGStages) { stage = 0; phase ^= 1; }
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------------------------ MMA issuer
+        constexpr uint32_t idesc = ptx::umma_idesc_bf16(kGM, kGN);
+        int stage = 0;
+        uint32_t phase = 0;
+        int it = 0;
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
+            const int a = it & 1;
+            if (!timed_out && !ptx::mbar_wait(acc_empty + a, ((it >> 1) & 1) ^ 1)) timed_out = true;
+            ptx::tc_fence_after_sync();
+            for (int kb = 0; kb < KB; ++kb) {
+                if (!timed_out && !ptx::mbar_wait(full + stage, phase)) timed_out = true;
+                ptx::tc_fence_after_sync();
+                if (lane == 0) {
+                    const uint32_t xs = ptx::smem_addr(ring + stage * kGStageBytes);
+                    const uint64_t ad = ptx::umma_desc_k128(xs), bd = ptx::umma_desc_k128(xs + kGM * kGKB * 2);
+#pragma unroll
+                    for (int j = 0; j < kGKB / 16; ++j)
+                        ptx::umma_bf16(tmem_base + a * kGN, ad + 2 * j, bd + 2 * j, idesc, (kb | j) != 0 ? 1u : 0u);
+                    ptx::umma_commit(empty + stage);
+                    if (kb == KB - 1) ptx::umma_commit(acc_full + a);
+                }
+                __syncwarp();
+                if (++stage == kGStages) { stage = 0; phase ^= 1; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue: one row of C per thread
+        int it = 0;
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
+            const int mt = tile / n_nt, nt = tile % n_nt;
+            const int a = it & 1;
+            const int row = mt * kGM + warp * 32 + lane;
+            const bool row_ok = row < M;
+            if (!timed_out && !ptx::mbar_wait(acc_full + a, (it >> 1) & 1)) timed_out = true;
+            ptx::tc_fence_after_sync();
+            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + a * kGN;
+            for (int c = 0; c < kGN / 32; ++c) {
+                const int col0 = nt * kGN + c * 32;
+                if (col0 >= N) break;                                  // warp-uniform
+                uint32_t v[32];
+                ptx::tmem_ld32(taddr + c * 32, v);
+                ptx::tmem_ld_wait();
+                const int nv = min(32, N - col0);
+                if (MODE == kGemmNodes) {
+                    float* out = ep.out_f32 + (int64_t)row * ep.ld_out + col0;
+#pragma unroll 4
+                    for (int e = 0; e < 32; ++e) {
+                        float cval = 0.0f;
+                        if (e < nv) {
+                            const float logit = __uint_as_float(v[e]) + __bfloat162float(ep.bias[col0 + e]);
+                            cval = 1.0f / (1.0f + __expf(-logit));
+                            if (row_ok) out[e] = cval;
+                        }
+                        if (ep.ent_part) {
+                            const float h = warp_sum((row_ok && e < nv) ? bernoulli_entropy(cval) : 0.0f);
+                            if (lane == 0 && e < nv) ep.ent_part[((int64_t)mt * 4 + warp) * N + col0 + e] = h;
+                        }
+                    }
+                } else if (MODE == kGemmHidden) {
+                    __nv_bfloat16* out = ep.out_bf16 + (int64_t)row * ep.ld_out + col0;
+                    const float* mrow = ep.mix + (int64_t)(row_ok ? row : 0) * ep.n_leaves;
+                    uint32_t packed[16];
+                    int leaf = col0 / ep.l, u = col0 % ep.l;           // leaf and unit of column col0 + e, stepped along
+                    float mw = leaf < ep.n_leaves ? mrow[leaf] : 0.0f;
+#pragma unroll
+                    for (int e = 0; e < 32; e += 2) {
+                        float h2[2];
+#pragma unroll
+                        for (int q = 0; q < 2; ++q) {
+                            float h = 0.0f;
+                            if (e + q < nv) h = mw * activate_bf16(ep.act, __uint_as_float(v[e + q]) + __bfloat162float(ep.bias[col0 + e + q]));
+                            h2[q] = h;
+                            if (++u == ep.l) {
+                                u = 0;
+                                ++leaf;
+                                mw = leaf < ep.n_leaves ? mrow[leaf] : 0.0f;
+                            }
+                        }
+                        packed[e / 2] = ptx::pack_bf16(h2[0], h2[1]);
+                    }
+                    if (row_ok) {
+                        if (nv == 32 && (ep.ld_out & 7) == 0) {
+#pragma unroll
+                            for (int q = 0; q < 4; ++q)
+                                *reinterpret_cast<uint4*>(out + q * 8) = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                        } else {
+                            for (int e = 0; e < nv; ++e)
+                                out[e] = __ushort_as_bfloat16((unsigned short)((packed[e / 2] >> ((e & 1) * 16)) & 0xffffu));
+                        }
+                    }
+                } else {
+                    __nv_bfloat16* out = ep.out_bf16 + (int64_t)row * ep.ld_out + col0;
+                    uint32_t packed[16];
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) packed[e] = ptx::pack_bf16(__uint_as_float(v[2 * e]), __uint_as_float(v[2 * e + 1]));
+                    if (row_ok) {
+                        if (nv == 32 && (ep.ld_out & 7) == 0) {
+#pragma unroll
+                            for (int q = 0; q < 4; ++q)
+                                *reinterpret_cast<uint4*>(out + q * 8) = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                        } else {
+                            for (int e = 0; e < nv; ++e)
+                                out[e] = __ushort_as_bfloat16((unsigned short)((packed[e / 2] >> ((e & 1) * 16)) & 0xffffu));
+                        }
+                    }
+                }
+            }
+            ptx::tc_fence_before_sync();
+            ptx::mbar_arrive(acc_empty + a);
+        }
+    }
+    if (timed_out) {
+        if (lane == 0) atomicExch(status, kDevTimeout);
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);     // let copies and MMAs still in flight finish before exit
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 5) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, kGTmemCols);
+    }
+}
+
+// Mixture weights of FORWARD_T from the node choices: unrolling the recursion of Algorithm 1, leaf j enters the
+// output with the product over its root path of c (where the path turns right) or 1 - c (left).
+// c: [B, ldc] float32 (node r in column r);  mix: [B, 2^d] float32 (optional: mix_user, a second copy);
+// hp_tail: the same weights as bf16 in the last 2^d used columns of the rows of h' (row pitch ld_hp), where
+// the output GEMM multiplies them with the output biases; the padding columns up to ld_hp are zeroed.
+__global__ void __launch_bounds__(256)
+k_mixture_weights(const float* __restrict__ c, int ldc, float* __restrict__ mix, float* __restrict__ mix_user,
+                  __nv_bfloat16* __restrict__ hp, int ld_hp, int hidden, int depth, int64_t B)
+{
+    const int nl = 1 << depth;
+    const int tail = ld_hp - hidden;                          // >= nl: mixture columns, then zero padding
+    const int64_t total = B * tail;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t t = i / tail;
+        const int j = (int)(i % tail);
+        float p = 0.0f;
+        if (j < nl) {
+            p = 1.0f;
+            const float* ct = c + t * ldc;
+            for (int m = 0; m < depth; ++m) {
+                const int n = j >> (depth - m);
+                const float cv = ct[(1 << m) - 1 + n];
+                p *= ((j >> (depth - m - 1)) & 1) ? cv : 1.0f - cv;
+            }
+            mix[t * nl + j] = p;
+            if (mix_user) mix_user[t * nl + j] = p;
+        }
+        hp[t * ld_hp + hidden + j] = __float2bfloat16_rn(p);
+    }
+}
+
+// Batch means of the node entropies from the per-warp partial sums of the node GEMM, added in a fixed order.
+__global__ void k_entropy_reduce(const float* __restrict__ part, int n_parts, int n_nodes, int64_t B, float* __restrict__ ent)
+{
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= n_nodes) return;
+    float s = 0.0f;
+    for (int p = 0; p < n_parts; ++p) s += part[(int64_t)p * n_nodes + r];
+    ent[r] = s / (float)B;
+}
+
+// B operand of the output GEMM: w2t [O][Kp] bf16 with w2t[o][j l + u] = W2[j][o][u], w2t[o][2^d l + j] = b2[j][o],
+// zero up to Kp.
+template <typename T>
+__global__ void k_pack_w2_transposed(const T* __restrict__ w2, const T* __restrict__ b2, __nv_bfloat16* __restrict__ w2t,
+                                     int n_leaves, int l, int O, int Kp)
+{
+    const int64_t total = (int64_t)O * Kp;
+    const int hidden = n_leaves * l;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t o = i / Kp;
+        const int q = (int)(i % Kp);
+        float v = 0.0f;
+        if (q < hidden) v = Elem<T>::to_float(w2[((int64_t)(q / l) * O + o) * l + q % l]);
+        else if (q < hidden + n_leaves && b2) v = Elem<T>::to_float(b2[(int64_t)(q - hidden) * O + o]);
+        w2t[i] = __float2bfloat16_rn(v);
+    }
+}
+
+}  // namespace fff
