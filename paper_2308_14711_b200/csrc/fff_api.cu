@@ -1031,7 +1031,7 @@ fff_status_t launch_gemm(fff_handle_s* h, const void* a, int64_t M, int lda, con
 fff_status_t run_forward_train(fff_handle_s* h, const void* x, void* y, float* mixture, float* node_entropy, int64_t B,
                                cudaStream_t st) {
     const int64_t nl = h->n_leaves, nn = h->n_nodes, hidden = nl * h->l;
-    const int ldc = (int)std::max<int64_t>(nn, 1);
+    const int ldc = (int)std::max<int64_t>((nn + 3) & ~(int64_t)3, 4);      // rows of c start on 16-byte boundaries
     const int64_t n_mt = (B + fff::kGM - 1) / fff::kGM;
     if (B > h->tr_cap_B) {
         if (cudaDeviceSynchronize() != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
@@ -1055,7 +1055,7 @@ fff_status_t run_forward_train(fff_handle_s* h, const void* x, void* y, float* m
         ep.ld_out = ldc;
         if ((s = launch_gemm<fff::kGemmNodes>(h, x, B, h->D, h->node_w, nn, h->D, ep, st, "train_node_choices")) != FFF_OK) return s;
         if (node_entropy) {
-            fff::k_entropy_reduce<<<(unsigned)((nn + 255) / 256), 256, 0, st>>>(h->tr_entpart, (int)(n_mt * 4), (int)nn, B, node_entropy);
+            fff::k_entropy_reduce<<<(unsigned)((nn + 7) / 8), 256, 0, st>>>(h->tr_entpart, (int)(n_mt * 4), (int)nn, B, node_entropy);
             if ((s = launched(h, st, "train_node_entropy")) != FFF_OK) return s;
         }
     }

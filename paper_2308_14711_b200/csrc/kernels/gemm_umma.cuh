@@ -10,10 +10,11 @@
 //
 // A is [M, K] and B is [N, K], both row-major with K contiguous, read through tensor maps (128-byte
 // swizzle, rows outside the matrix read as zeros).  One persistent CTA per SM works on 128 x 256 tiles of
-// C: warp 4 issues the tensor-map loads of the K-blocks (64 columns) into a ring of shared-memory stages,
-// warp 5 issues four tcgen05.mma (M = 128, N = 256, K = 16) per stage into one of two accumulators in
-// tensor memory, warps 0-3 read the finished accumulator (one row per thread), apply the epilogue and
-// store.  Tiles that share their rows of A are neighbours in the schedule, so A is read from DRAM once.
+// C: one warp issues the tensor-map loads of the K-blocks (64 columns) into a ring of shared-memory stages,
+// another issues four tcgen05.mma (M = 128, N = 256, K = 16) per stage into one of two accumulators in
+// tensor memory, the others read the finished accumulator (one row per thread), apply the epilogue and
+// store (sixteen epilogue warps: four per lane quarter, 64 columns each).  Tiles that share their rows of A are
+// neighbours in the schedule, so A is read from DRAM once.
 //
 // Every wait is bounded (see ptx.cuh); tensor memory is released on every exit path.
 // Requirements: bf16, K % 64 == 0, A and B 16-byte aligned with row pitches that are multiples of 16 bytes.
@@ -30,7 +31,11 @@ constexpr int kGM = 128;                 // rows of C per tile = rows of one tcg
 constexpr int kGN = 256;                 // columns of C per tile
 constexpr int kGKB = 64;                 // K-block: 128 bytes, one swizzle line
 constexpr int kGStages = 4;
-constexpr int kGThreads = 6 * 32;
+constexpr int kGEpiWarps = 16;           // four per tensor-memory lane quarter, 64 columns of the tile each: a lone warp per
+                                         // scheduler cannot hide the latency of the epilogue arithmetic
+constexpr int kGColsPerWarp = kGN / (kGEpiWarps / 4);
+constexpr int kGProducerWarp = kGEpiWarps, kGMmaWarp = kGEpiWarps + 1;
+constexpr int kGThreads = (kGEpiWarps + 2) * 32;
 constexpr int kGStageBytes = (kGM + kGN) * kGKB * 2;                 // 48 KB
 constexpr int kGSmemBytes = 1024 + kGStages * kGStageBytes + 256;
 constexpr int kGTmemCols = 2 * kGN;
@@ -84,13 +89,13 @@ k_gemm_umma(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         }
         for (int a = 0; a < 2; ++a) {
             ptx::mbar_init(acc_full + a, 1);
-            ptx::mbar_init(acc_empty + a, 4 * 32);
+            ptx::mbar_init(acc_empty + a, kGEpiWarps * 32);
         }
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(&tmap_a);
         ptx::prefetch_tensormap(&tmap_b);
     }
-    if (warp == 5) {
+    if (warp == kGMmaWarp) {
         ptx::tmem_alloc(tmem_slot, kGTmemCols);
         ptx::tmem_relinquish_alloc_permit();
     }
@@ -100,7 +105,7 @@ k_gemm_umma(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     const uint32_t tmem_base = *tmem_slot;
 
     bool timed_out = false;
-    if (warp == 4) {
+    if (warp == kGProducerWarp) {
         // ------------------------------------------------------------------ producer
         int stage = 0;
         uint32_t phase = 0;
@@ -118,7 +123,7 @@ k_gemm_umma(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                 if (++stage == kGStages) { stage = 0; phase ^= 1; }
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == kGMmaWarp) {
         // ------------------------------------------------------------------ MMA issuer
         constexpr uint32_t idesc = ptx::umma_idesc_bf16(kGM, kGN);
         int stage = 0;
@@ -145,17 +150,19 @@ k_gemm_umma(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue: one row of C per thread
+        // ------------------------------------------------------------------ epilogue: one row of C and one quarter of
+        // the tile's columns per thread (warps w, w + 4, w + 8, w + 12 share the lanes of quarter w % 4)
+        const int quarter = warp & 3, cpart = warp >> 2;
         int it = 0;
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
             const int mt = tile / n_nt, nt = tile % n_nt;
             const int a = it & 1;
-            const int row = mt * kGM + warp * 32 + lane;
+            const int row = mt * kGM + quarter * 32 + lane;
             const bool row_ok = row < M;
             if (!timed_out && !ptx::mbar_wait(acc_full + a, (it >> 1) & 1)) timed_out = true;
             ptx::tc_fence_after_sync();
-            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + a * kGN;
-            for (int c = 0; c < kGN / 32; ++c) {
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + a * kGN;
+            for (int c = cpart * (kGColsPerWarp / 32); c < (cpart + 1) * (kGColsPerWarp / 32); ++c) {
                 const int col0 = nt * kGN + c * 32;
                 if (col0 >= N) break;                                  // warp-uniform
                 uint32_t v[32];
@@ -164,25 +171,52 @@ k_gemm_umma(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                 const int nv = min(32, N - col0);
                 if (MODE == kGemmNodes) {
                     float* out = ep.out_f32 + (int64_t)row * ep.ld_out + col0;
-#pragma unroll 4
+                    float cv[32];
+#pragma unroll
                     for (int e = 0; e < 32; ++e) {
-                        float cval = 0.0f;
-                        if (e < nv) {
-                            const float logit = __uint_as_float(v[e]) + __bfloat162float(ep.bias[col0 + e]);
-                            cval = 1.0f / (1.0f + __expf(-logit));
-                            if (row_ok) out[e] = cval;
+                        const float logit = __uint_as_float(v[e]) + (e < nv ? __bfloat162float(ep.bias[col0 + e]) : 0.0f);
+                        cv[e] = 1.0f / (1.0f + __expf(-logit));
+                    }
+                    if (row_ok) {
+                        if (nv == 32 && (ep.ld_out & 3) == 0) {
+#pragma unroll
+                            for (int q = 0; q < 8; ++q)
+                                *reinterpret_cast<float4*>(out + 4 * q) = make_float4(cv[4 * q], cv[4 * q + 1], cv[4 * q + 2], cv[4 * q + 3]);
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 32; ++e)
+                                if (e < nv) out[e] = cv[e];
                         }
-                        if (ep.ent_part) {
-                            const float h = warp_sum((row_ok && e < nv) ? bernoulli_entropy(cval) : 0.0f);
-                            if (lane == 0 && e < nv) ep.ent_part[((int64_t)mt * 4 + warp) * N + col0 + e] = h;
+                    }
+                    if (ep.ent_part) {
+                        // sums over the warp's 32 rows of all 32 columns at once: in step s every lane hands one half of
+                        // its values to the lane s away and adds what it gets to the half it keeps, so that lane j ends
+                        // with the total of column j (31 shuffles instead of 5 per column); the order is fixed
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) cv[e] = (row_ok && e < nv) ? bernoulli_entropy(cv[e]) : 0.0f;
+#pragma unroll
+                        for (int sft = 16; sft >= 1; sft >>= 1) {
+                            const bool upper = (lane & sft) != 0;
+#pragma unroll
+                            for (int i = 0; i < sft; ++i) {
+                                const float send = upper ? cv[i] : cv[i + sft];
+                                const float keep = upper ? cv[i + sft] : cv[i];
+                                cv[i] = keep + __shfl_xor_sync(kFullMask, send, sft);
+                            }
                         }
+                        if (lane < nv) ep.ent_part[((int64_t)mt * 4 + quarter) * N + col0 + lane] = cv[0];
                     }
                 } else if (MODE == kGemmHidden) {
                     __nv_bfloat16* out = ep.out_bf16 + (int64_t)row * ep.ld_out + col0;
                     const float* mrow = ep.mix + (int64_t)(row_ok ? row : 0) * ep.n_leaves;
                     uint32_t packed[16];
                     int leaf = col0 / ep.l, u = col0 % ep.l;           // leaf and unit of column col0 + e, stepped along
-                    float mw = leaf < ep.n_leaves ? mrow[leaf] : 0.0f;
+                    // the weights of the first leaves of the chunk are fetched together, ahead of their use
+                    float mpre[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) mpre[q] = leaf + q < ep.n_leaves ? mrow[leaf + q] : 0.0f;
+                    int ahead = 0;
+                    float mw = mpre[0];
 #pragma unroll
                     for (int e = 0; e < 32; e += 2) {
                         float h2[2];
@@ -194,7 +228,9 @@ k_gemm_umma(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                             if (++u == ep.l) {
                                 u = 0;
                                 ++leaf;
-                                mw = leaf < ep.n_leaves ? mrow[leaf] : 0.0f;
+                                ++ahead;
+                                mw = ahead == 1 ? mpre[1] : ahead == 2 ? mpre[2] : ahead == 3 ? mpre[3]
+                                                : (leaf < ep.n_leaves ? mrow[leaf] : 0.0f);
                             }
                         }
                         packed[e / 2] = ptx::pack_bf16(h2[0], h2[1]);
@@ -236,7 +272,7 @@ k_gemm_umma(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == kGMmaWarp) {
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, kGTmemCols);
     }
@@ -273,14 +309,18 @@ k_mixture_weights(const float* __restrict__ c, int ldc, float* __restrict__ mix,
     }
 }
 
-// Batch means of the node entropies from the per-warp partial sums of the node GEMM, added in a fixed order.
-__global__ void k_entropy_reduce(const float* __restrict__ part, int n_parts, int n_nodes, int64_t B, float* __restrict__ ent)
+// Batch means of the node entropies from the per-warp partial sums of the node GEMM, added in a fixed order:
+// one warp per node, lane i adds the parts i, i + 32, ... in order, then the lanes' sums are added by a fixed tree.
+// Blocks of 8 warps.
+__global__ void __launch_bounds__(256)
+k_entropy_reduce(const float* __restrict__ part, int n_parts, int n_nodes, int64_t B, float* __restrict__ ent)
 {
-    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    const int r = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (r >= n_nodes) return;
     float s = 0.0f;
-    for (int p = 0; p < n_parts; ++p) s += part[(int64_t)p * n_nodes + r];
-    ent[r] = s / (float)B;
+    for (int p = lane; p < n_parts; p += 32) s += part[(int64_t)p * n_nodes + r];
+    s = warp_sum(s);
+    if (lane == 0) ent[r] = s / (float)B;
 }
 
 // B operand of the output GEMM: w2t [O][Kp] bf16 with w2t[o][j l + u] = W2[j][o][u], w2t[o][2^d l + j] = b2[j][o],
