@@ -350,6 +350,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
             out["per_config"] = per_config_table(args, peaks, skip={cfg.name: (ms_per_step, path_roofline)})
             # four layers of the ViT-shaped configuration as one stack (the paper's transformer use of the layer)
             out["stack"] = stack_bench(wl.CONFIGS["vit_d8_l12_bf16"], 4, max(5, min(args.steps, 50)))
+            out["forward_train"] = train_bench(wl.CONFIGS["vit_d8_l12_bf16"], max(3, min(args.steps, 10)), peaks)
     layer.close()
     if dist is not None:
         dist.barrier()
@@ -445,6 +446,40 @@ def stack_bench(cfg: wl.FFFConfig, n_layers: int, steps: int) -> dict:
     for l in layers:
         l.close()
     return out
+
+
+def train_bench(cfg: wl.FFFConfig, steps: int, peaks) -> dict:
+    """FORWARD_T (all leaves, soft mixture, node entropies) of one configuration: a dense contraction, so its
+    roofline is the tensor peak.  FLOPs = 2 B (nodes D + hidden D + (hidden + leaves, padded to 64) O)."""
+    import torch
+    layer, _, _, xs, _, _, _ = make_device_case(cfg, 0, 2)
+    for i in range(3):
+        layer.forward_train(xs[i % 2], want_mixture=False, want_entropy=True)
+    torch.cuda.synchronize()
+    regions = []
+    t_begin = time.perf_counter()
+    while True:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(steps):
+            layer.forward_train(xs[i % 2], want_mixture=False, want_entropy=True)
+        e1.record()
+        regions.append((e0, e1))
+        if time.perf_counter() - t_begin >= MIN_TIMED_SECONDS / 2 or len(regions) >= 64:
+            break
+    torch.cuda.synchronize()
+    ms = statistics.median(a.elapsed_time(b) for a, b in regions) / steps
+    hidden = cfg.n_leaves * cfg.leaf_width
+    kp = (hidden + cfg.n_leaves + 63) // 64 * 64
+    flops = 2.0 * cfg.B * (cfg.n_nodes * cfg.D + hidden * cfg.D + kp * cfg.O)
+    achieved = flops / (ms * 1e-3) / 1e12
+    status = layer.last_status()
+    layer.close()
+    return {"workload": cfg.name, "tokens": cfg.B, "ms_per_step": round(ms, 5), "tokens_per_s": cfg.B / (ms * 1e-3),
+            "flops": flops, "device_status": status,
+            "roofline": {"bound": "tensor", "achieved": round(achieved, 1), "peak": peaks["bf16_tflops_sustained"],
+                         "unit": "TFLOP/s", "frac": round(achieved / peaks["bf16_tflops_sustained"], 4),
+                         "peak_source": peaks["source"] + " (sustained bf16: several GEMMs back to back)", "traffic": None}}
 
 
 # ------------------------------------------------------------------------------------------- CPU oracle legs
