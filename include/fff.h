@@ -279,6 +279,21 @@ fff_status_t fff_get_last_status(fff_handle_t h);
  * and the context stays usable. */
 fff_status_t fff_selftest_bounded_wait(fff_handle_t h, int64_t limit_cycles, void *cuda_stream);
 
+/* Which kernel families the shapes of this layer admit (a bit set; -1 for a bad handle).  A bf16 layer whose
+ * D is no multiple of 128, whose O is no multiple of 8 or whose leaves are wider than 64 has no tensor-core
+ * kernels: its forward runs on CUDA-core kernels (the one-launch kernel when FFF_CAP_FUSED_SMALL is set, else
+ * one warp per token), which is several times slower per token; float32 layers never have them.  Callers
+ * that depend on tensor-core speed can check here instead of timing. */
+typedef enum {
+    FFF_CAP_TENSOR_DESCENT = 1,   /* staged descent on tensor cores (bf16, D % 128 == 0, depth > 0) */
+    FFF_CAP_TCGEN05_DESCENT = 2,  /* ... its first stage on tcgen05 */
+    FFF_CAP_TENSOR_LEAF = 4,      /* grouped leaf evaluation on tensor cores (also O % 8 == 0, l <= 64) */
+    FFF_CAP_TCGEN05_LEAF = 8,     /* ... on tcgen05 (also O % 16 == 0) */
+    FFF_CAP_FUSED_SMALL = 16,     /* the one-launch kernel (l <= 32, at most one group of 32 neurons per SM) */
+    FFF_CAP_FORWARD_TRAIN = 32    /* fff_forward_train (bf16, D % 64 == 0) */
+} fff_capability_t;
+int fff_capabilities(fff_handle_t h);
+
 /* Number of kernels the most recent forward / stage call of this handle enqueued
  * (-1 for a bad handle). */
 int fff_last_launch_count(fff_handle_t h);

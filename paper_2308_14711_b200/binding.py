@@ -27,7 +27,7 @@ TUNING = {"tcgen05_descent": 0, "tcgen05_grouped": 1, "tcgen05_leaf": 2, "cta_pa
 # every symbol include/fff.h declares
 EXPORTS = ["fff_create", "fff_forward_infer", "fff_forward_train", "fff_forward_infer_host", "fff_destroy", "fff_reserve",
            "fff_set_path", "fff_set_tuning", "fff_tree_descent", "fff_leaf_bucketing", "fff_grouped_leaf_ff",
-           "fff_debug_get_bucketing", "fff_get_last_status", "fff_selftest_bounded_wait", "fff_last_launch_count", "fff_status_string",
+           "fff_debug_get_bucketing", "fff_get_last_status", "fff_capabilities", "fff_selftest_bounded_wait", "fff_last_launch_count", "fff_status_string",
            "fff_profile_begin", "fff_profile_end", "fff_profile_launches", "fff_profile_launch_name",
            "fff_leaf_bucketing_static", "fff_stack_create", "fff_stack_forward", "fff_stack_set_graph",
            "fff_stack_last_launch_count", "fff_stack_last_was_replay", "fff_stack_destroy"]
@@ -59,6 +59,7 @@ def lib():
     L.fff_reserve.argtypes = [vp, i64]
     L.fff_set_path.argtypes = [vp, ci]
     L.fff_set_tuning.argtypes = [vp, ci, ci]
+    L.fff_capabilities.argtypes = [vp]
     L.fff_forward_train.argtypes = [vp, vp, vp, vp, vp, i64, vp]
     L.fff_stack_create.argtypes = [C.POINTER(vp), ci, C.POINTER(vp), ci, C.POINTER(vp), C.POINTER(vp), C.c_float, ci]
     L.fff_stack_forward.argtypes = [vp, vp, vp, vp, i64, vp]
@@ -234,6 +235,10 @@ class FFFLayer:
 
     def set_path(self, path: str) -> None:
         fff_set_path(self._h, PATHS[path])
+
+    def capabilities(self) -> int:
+        """Bit set of FFF_CAP_*: the kernel families this layer's shapes admit."""
+        return lib().fff_capabilities(self._h)
 
     def set_tuning(self, key: str, on: bool) -> None:
         """Switch between kernels that compute the same thing (keys of TUNING; all on by default)."""

@@ -1586,6 +1586,18 @@ fff_status_t fff_selftest_bounded_wait(fff_handle_t h, int64_t limit_cycles, voi
 
 int fff_last_launch_count(fff_handle_t h) { return live(h) ? h->launches : -1; }
 
+int fff_capabilities(fff_handle_t h) {
+    if (!live(h)) return -1;
+    int caps = 0;
+    if (!h->stages.empty() || !h->ustages.empty()) caps |= FFF_CAP_TENSOR_DESCENT;
+    if (!h->ustages.empty()) caps |= FFF_CAP_TCGEN05_DESCENT;
+    if (h->LP != 0) caps |= FFF_CAP_TENSOR_LEAF;
+    if (h->w2uimg) caps |= FFF_CAP_TCGEN05_LEAF;
+    if (h->fs_batch != 0) caps |= FFF_CAP_FUSED_SMALL;
+    if (h->tr_Kp != 0) caps |= FFF_CAP_FORWARD_TRAIN;
+    return caps;
+}
+
 fff_status_t fff_profile_begin(fff_handle_t h, int max_steps) {
     if (!live(h)) return FFF_ERR_BAD_HANDLE;
     if (max_steps < 0 || max_steps > (1 << 20)) return FFF_ERR_INVALID_ARG;

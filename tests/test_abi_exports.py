@@ -62,5 +62,6 @@ def test_calls_reject_dead_handles(lib):
     assert lib.fff_forward_infer(C.c_void_p(0xdead0), None, None, None, 1, None) == 6
     assert lib.fff_reserve(None, 10) == 6
     assert lib.fff_set_tuning(None, 0, 1) == 6
+    assert lib.fff_capabilities(None) == -1
     assert lib.fff_get_last_status(None) == 6
     assert lib.fff_last_launch_count(None) == -1

@@ -556,3 +556,22 @@ def test_a_bounded_wait_that_runs_out_is_reported_once_and_the_handle_stays_usab
     with pytest.raises(Exception):
         binding.fff_selftest_bounded_wait(layer.handle, 0)
     layer.close()
+
+
+def test_capabilities_say_which_kernel_families_a_layer_can_use():
+    def caps(D, O, depth, l, dtype):
+        cfg = wl.FFFConfig("caps", D, O, depth, l, "relu", dtype, 4, "normal")
+        layer = util.make_layer(util.make_case(cfg, seed=1, margin=None))
+        c = layer.capabilities()
+        layer.close()
+        return c
+    full = caps(256, 128, 4, 16, "bf16")
+    assert full & 1 and full & 2 and full & 4 and full & 8 and full & 16 and full & 32
+    odd_d = caps(192, 128, 4, 16, "bf16")              # D no multiple of 128: CUDA cores only, FORWARD_T still runs
+    assert not odd_d & (1 | 2 | 4 | 8) and odd_d & 16 and odd_d & 32
+    odd_o = caps(256, 100, 4, 16, "bf16")              # O no multiple of 8: descent on tensor cores, leaves not
+    assert odd_o & 1 and not odd_o & (4 | 8)
+    f32 = caps(256, 128, 4, 16, "f32")
+    assert f32 == 16
+    wide = caps(256, 128, 2, 48, "f32")                # leaves wider than 32: no one-launch kernel
+    assert wide == 0
