@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of hard-routed FFF inference (FORWARD_I) on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config NAME]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config NAME] [--leg NAME]
 
 One step = one pass of the whole path (tree descent, leaf bucketing, grouped leaf evaluation with
 un-permuting write-back) over one batch of synthetic tokens.  Prints ONE JSON line (rank 0).
@@ -568,6 +568,8 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-config", action="store_true")
+    ap.add_argument("--leg", default="path", choices=["path", "forward_train", "stack"],
+                    help="path: the benchmark line; forward_train / stack: only that extra measurement of --config (for profiling)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", "0"))
@@ -575,6 +577,14 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         run_reference(args, rank, world)
+    elif args.leg != "path":
+        import torch
+        torch.cuda.set_device(local_rank)
+        cfg = wl.CONFIGS[args.config]
+        out = train_bench(cfg, max(1, min(args.steps, 10)), measured_peaks()) if args.leg == "forward_train" else \
+            stack_bench(cfg, 4, max(1, min(args.steps, 50)))
+        if rank == 0:
+            print(json.dumps({"leg": args.leg, **out}), flush=True)
     else:
         run_ours(args, rank, world, local_rank)
 
