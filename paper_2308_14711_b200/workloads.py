@@ -142,6 +142,34 @@ def make_weights(cfg: FFFConfig, seed: int = 0) -> Dict[str, np.ndarray]:
     return {k: _store(cfg, v) for k, v in w.items()}
 
 
+E4M3_MAX = 448.0
+
+
+def e4m3_decode_table() -> np.ndarray:
+    """float32 value of each of the 256 e4m3 codes (the library's conversion; the two NaN codes read as NaN)."""
+    import torch
+    codes = torch.arange(256, dtype=torch.int32).to(torch.uint8)
+    return codes.view(torch.float8_e4m3fn).to(torch.float32).numpy()
+
+
+def quantize_e4m3(w: np.ndarray):
+    """Storage encoding of leaf weights as 8-bit floats with one scale per leaf.
+
+    w: float32 [n_leaves, ...].  Returns (codes uint8 like w, scales float32 [n_leaves], values float64 like w):
+    scale_j = max|w_j| / 448 (1 for an all-zero leaf), code = the library's round-to-nearest-even e4m3 conversion of
+    w / scale, values = decode(code) * scale in float64, i.e. exactly what the stored bytes and scales stand for.
+    Both the oracle and the CUDA library are given these values (as float64 numbers, as codes and scales)."""
+    import torch
+    w = np.ascontiguousarray(w, dtype=np.float32)
+    nl = w.shape[0]
+    amax = np.abs(w.reshape(nl, -1)).max(axis=1)
+    scales = np.where(amax > 0, amax / np.float32(E4M3_MAX), np.float32(1.0)).astype(np.float32)
+    scaled = w / scales.reshape((nl,) + (1,) * (w.ndim - 1))
+    codes = torch.from_numpy(scaled).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    values = e4m3_decode_table().astype(np.float64)[codes] * scales.astype(np.float64).reshape((nl,) + (1,) * (w.ndim - 1))
+    return codes, scales, values
+
+
 def zipf_weights(n: int = N_CLUSTERS, s: float = ZIPF_S) -> np.ndarray:
     w = np.arange(1, n + 1, dtype=np.float64) ** (-s)
     return w / w.sum()

@@ -85,3 +85,34 @@ def test_margin_resampling_with_the_oracle_margin():
     np.testing.assert_array_equal(src.x[keep], before[keep])
     np.testing.assert_array_equal(src.cluster, cl)
     np.testing.assert_array_equal(wl.round_to_bf16(src.x), src.x)
+
+
+def test_e4m3_codes_are_the_published_format_and_quantisation_is_nearest():
+    """The 8-bit weight encoding of the generator: every code decodes to (-1)^s 2^(e-7) (1 + m/8), subnormals
+    m/8 2^-6 (the published e4m3 format: 4 exponent bits with bias 7, 3 mantissa bits, no infinities, largest
+    finite value 448); quantised values are the nearest representable ones and the per-leaf scale maps the largest
+    magnitude of a leaf to 448."""
+    table = wl.e4m3_decode_table()
+    for code in range(256):
+        s, e, m = code >> 7, (code >> 3) & 15, code & 7
+        if e == 15 and m == 7:
+            assert np.isnan(table[code])
+            continue
+        mag = (m / 8.0) * 2.0 ** -6 if e == 0 else 2.0 ** (e - 7) * (1.0 + m / 8.0)
+        assert table[code] == (-mag if s else mag)
+    assert np.nanmax(table) == 448.0
+    rng = np.random.default_rng(0)
+    w = (rng.standard_normal((5, 7, 33)) * rng.uniform(0.01, 3.0, (5, 1, 1))).astype(np.float32)
+    w[3] = 0.0
+    codes, scales, values = wl.quantize_e4m3(w)
+    assert codes.dtype == np.uint8 and codes.shape == w.shape and scales.shape == (5,) and values.dtype == np.float64
+    assert scales[3] == 1.0 and (values[3] == 0).all()
+    finite = np.sort(table[np.isfinite(table)].astype(np.float64))
+    for j in (0, 1, 2, 4):
+        np.testing.assert_allclose(np.abs(values[j]).max(), np.abs(w[j]).max(), rtol=1e-6)
+        target = w[j].astype(np.float64) / float(scales[j])
+        got = values[j] / float(scales[j])
+        # no representable value is closer to the target than the chosen one
+        nearest = np.abs(finite[None, :] - target.reshape(-1, 1)).min(axis=1)
+        np.testing.assert_allclose(np.abs(got - target).reshape(-1), nearest, rtol=0, atol=1e-6)
+        np.testing.assert_array_equal(values[j], table[codes[j]].astype(np.float64) * float(scales[j]))
