@@ -105,6 +105,22 @@ fff_status_t fff_create(fff_handle_t *out, int D, int O, int depth, int leaf_wid
                         const void *leaf_w2, const void *leaf_b2);
 
 /*
+ * The same layer with its leaf weights stored as 8-bit floats: leaf_w1_e4m3 [2^d, l, D] and leaf_w2_e4m3
+ * [2^d, O, l] hold e4m3 codes (4 exponent bits with bias 7, 3 mantissa bits, no infinities), leaf_w1_scale and
+ * leaf_w2_scale [2^d] one float32 scale per leaf: the weight a code stands for is its e4m3 value times the
+ * scale of its leaf.  Everything else (x, y, node weights, biases) is bfloat16; products are accumulated in
+ * float32 and the scales are applied to the sums, so the result is FORWARD_I of the layer with exactly those
+ * weights.  (The paper stores its weights in one floating-point type; this halves the bytes of the leaf
+ * weights, the largest stream of a layer with many thin leaves.)  Runs on the tcgen05 kernels only:
+ * FFF_ERR_UNSUPPORTED unless D % 128 == 0, O % 16 == 0 and l <= 64; fff_forward_train, the warp path and the
+ * one-launch kernel are not available on such a handle.
+ */
+fff_status_t fff_create_w8(fff_handle_t *out, int D, int O, int depth, int leaf_width, fff_activation_t act,
+                           const void *node_w, const void *node_b,
+                           const uint8_t *leaf_w1_e4m3, const float *leaf_w1_scale, const void *leaf_b1,
+                           const uint8_t *leaf_w2_e4m3, const float *leaf_w2_scale, const void *leaf_b2);
+
+/*
  * FORWARD_I of Algorithm 1 for B tokens, enqueued on `cuda_stream`.
  *
  *   x         [B, D]  in

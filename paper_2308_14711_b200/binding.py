@@ -25,7 +25,7 @@ PATHS = {"auto": 0, "warp": 1, "tensor": 2, "fused": 3}
 TUNING = {"tcgen05_descent": 0, "tcgen05_grouped": 1, "tcgen05_leaf": 2, "cta_pairs": 3, "direct_lists": 4, "fused_small": 5}
 
 # every symbol include/fff.h declares
-EXPORTS = ["fff_create", "fff_forward_infer", "fff_forward_train", "fff_forward_infer_host", "fff_destroy", "fff_reserve",
+EXPORTS = ["fff_create", "fff_create_w8", "fff_forward_infer", "fff_forward_train", "fff_forward_infer_host", "fff_destroy", "fff_reserve",
            "fff_set_path", "fff_set_tuning", "fff_tree_descent", "fff_leaf_bucketing", "fff_grouped_leaf_ff",
            "fff_debug_get_bucketing", "fff_get_last_status", "fff_capabilities", "fff_selftest_bounded_wait", "fff_last_launch_count", "fff_status_string",
            "fff_profile_begin", "fff_profile_end", "fff_profile_launches", "fff_profile_launch_name",
@@ -59,6 +59,7 @@ def lib():
     L.fff_reserve.argtypes = [vp, i64]
     L.fff_set_path.argtypes = [vp, ci]
     L.fff_set_tuning.argtypes = [vp, ci, ci]
+    L.fff_create_w8.argtypes = [C.POINTER(vp), ci, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp]
     L.fff_capabilities.argtypes = [vp]
     L.fff_forward_train.argtypes = [vp, vp, vp, vp, vp, i64, vp]
     L.fff_stack_create.argtypes = [C.POINTER(vp), ci, C.POINTER(vp), ci, C.POINTER(vp), C.POINTER(vp), C.c_float, ci]
@@ -196,7 +197,8 @@ class FFFLayer:
     """One FFF layer on the current CUDA device; tensors in, tensors out, all work in libfff.so."""
 
     def __init__(self, D: int, O: int, depth: int, leaf_width: int, activation: str, dtype: str,
-                 node_w, node_b, w1, b1, w2, b2, path: str = "auto"):
+                 node_w, node_b, w1, b1, w2, b2, path: str = "auto", w1_scale=None, w2_scale=None):
+        """With w1_scale / w2_scale (float32 [2^d]) w1 and w2 are uint8 tensors of e4m3 codes (fff_create_w8)."""
         torch = _torch()
         self._h = None
         self.D, self.O, self.depth, self.l = D, O, depth, leaf_width
@@ -204,10 +206,21 @@ class FFFLayer:
         self.tdtype = torch.float32 if dtype == "f32" else torch.bfloat16
         nn, nl = self.n_leaves - 1, self.n_leaves
         td = self.tdtype
-        self._h = fff_create(D, O, depth, leaf_width, ACTIVATIONS[activation], DTYPES[dtype],
-                             _ptr(node_w, td, (nn, D), "node_w"), _ptr(node_b, td, (nn,), "node_b"),
-                             _ptr(w1, td, (nl, leaf_width, D), "w1"), _ptr(b1, td, (nl, leaf_width), "b1"),
-                             _ptr(w2, td, (nl, O, leaf_width), "w2"), _ptr(b2, td, (nl, O), "b2"))
+        if w1_scale is not None:
+            out = C.c_void_p()
+            _check(lib().fff_create_w8(C.byref(out), D, O, depth, leaf_width, ACTIVATIONS[activation],
+                                       _ptr(node_w, td, (nn, D), "node_w"), _ptr(node_b, td, (nn,), "node_b"),
+                                       _ptr(w1, torch.uint8, (nl, leaf_width, D), "w1 codes"),
+                                       _ptr(w1_scale, torch.float32, (nl,), "w1_scale"), _ptr(b1, td, (nl, leaf_width), "b1"),
+                                       _ptr(w2, torch.uint8, (nl, O, leaf_width), "w2 codes"),
+                                       _ptr(w2_scale, torch.float32, (nl,), "w2_scale"), _ptr(b2, td, (nl, O), "b2")),
+                   "fff_create_w8")
+            self._h = out.value
+        else:
+            self._h = fff_create(D, O, depth, leaf_width, ACTIVATIONS[activation], DTYPES[dtype],
+                                 _ptr(node_w, td, (nn, D), "node_w"), _ptr(node_b, td, (nn,), "node_b"),
+                                 _ptr(w1, td, (nl, leaf_width, D), "w1"), _ptr(b1, td, (nl, leaf_width), "b1"),
+                                 _ptr(w2, td, (nl, O, leaf_width), "w2"), _ptr(b2, td, (nl, O), "b2"))
         if path != "auto":
             self.set_path(path)
 

@@ -62,6 +62,10 @@ struct fff_handle_s {
     unsigned char* w2img = nullptr;
     unsigned char* w2uimg = nullptr;   // W2 pieces (+ biases) of the tcgen05 leaf kernel (nullptr = kernel not available)
     int* ws_sched = nullptr;           // its tile counter and finished-CTA counter (zero between launches)
+    // 8-bit leaf weights (fff_create_w8): code images of the tcgen05 leaf kernel and the per-leaf scales
+    bool w8 = false;
+    unsigned char *w1codes = nullptr, *w2codes = nullptr;
+    float *scale1 = nullptr, *scale2 = nullptr;
     fff::Tile* ws_tiles = nullptr;
 
     // workspace
@@ -248,6 +252,7 @@ void release(fff_handle_s* h) {
     for (auto& sg : h->ustages) { dfree(sg.wimg); dfree(sg.bimg); }
     dfree(h->ws_pos[0]); dfree(h->ws_pos[1]);
     dfree(h->fs_w1g); dfree(h->fs_b1g); dfree(h->fs_w2g); dfree(h->fs_b2f);
+    dfree(h->w1codes); dfree(h->w2codes); dfree(h->scale1); dfree(h->scale2);
     dfree(h->tr_w2t); dfree(h->tr_c); dfree(h->tr_mix); dfree(h->tr_entpart); dfree(h->tr_hp);
     dfree(h->w1img); dfree(h->b1img); dfree(h->w2img); dfree(h->w2uimg); dfree(h->ws_sched); dfree(h->ws_tiles); dfree(h->ws_rank); dfree(h->ws_rank8); dfree(h->ws_counts8); dfree(h->ws_blocksum); dfree(h->ws_matrix); dfree(h->ws_slots); dfree(h->ws_cursor);
     if (h->copy_in) cudaStreamDestroy(h->copy_in);
@@ -295,6 +300,7 @@ struct LeafPlan {
 };
 
 LeafPlan leaf_plan(const fff_handle_s* h, int64_t B) {
+    if (h->w8) return LeafPlan{fff::kLUM, true};
     // The tcgen05 kernel works on 128-row tiles.  Measured against the mma.sync kernel it is far ahead when
     // some buckets are large (skewed routing), about level with uniformly thin buckets of 32 tokens, and is
     // left out only when buckets are thinner still (tiles of at most 64 rows are stacked in the MMA rows, so the
@@ -306,6 +312,7 @@ LeafPlan leaf_plan(const fff_handle_s* h, int64_t B) {
 }
 
 bool use_tensor_leaf(const fff_handle_s* h) {
+    if (h->w8) return true;            // 8-bit leaf weights exist for the tcgen05 leaf kernel only
     if (h->LP == 0 || h->path == FFF_PATH_WARP) return false;
     return h->path == FFF_PATH_TENSOR || h->l >= 8;
 }
@@ -342,7 +349,7 @@ fff_status_t grow_workspace(fff_handle_s* h, int64_t B) {
     if ((s = dmalloc((void**)&h->ws_tiles, sizeof(fff::Tile) * max_tiles(h, B))) != FFF_OK) return s;
     // direct lists: every leaf's list can take the whole batch, so their size grows with n_leaves * B; beyond
     // kMaxSlotBytes the forward keeps the bucketing kernel instead
-    if (!h->ustages.empty() && h->ustages.back().umma && h->ustages.back().L0 + h->ustages.back().k == h->depth && h->w2uimg &&
+    if (!h->ustages.empty() && h->ustages.back().umma && h->ustages.back().L0 + h->ustages.back().k == h->depth && (h->w2uimg || h->w2codes) &&
         (size_t)h->n_leaves * (size_t)B * sizeof(int32_t) <= kMaxSlotBytes) {
         if ((s = dmalloc((void**)&h->ws_slots, sizeof(int32_t) * (size_t)h->n_leaves * (size_t)B)) != FFF_OK) return s;
         if ((s = clone((void**)&h->ws_cursor, nullptr, sizeof(int32_t) * (size_t)h->n_leaves)) != FFF_OK) return s;
@@ -849,15 +856,15 @@ fff_status_t launch_leaf_mma(fff_handle_s* h, const void* x, const int32_t* perm
     return launched(h, st, "grouped_leaf_ff_mma");
 }
 
-template <int LP, bool kFold>
+template <int LP, bool kFold, bool kW8 = false>
 fff_status_t launch_leaf_umma(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, int tile_rows,
                               cudaStream_t st) {
-    using L = fff::LeafUmmaLayout<LP>;
+    using L = fff::LeafUmmaLayout<LP, kW8>;
     const int n_tiles = tile_list_len(B, tile_rows, (int)h->n_leaves);
     const int stages = std::min((int)fff::kLUMaxStages, (kSmemBudget - L::smem_bytes(0)) / L::kStageBytes);
     if (stages < 2) return FFF_ERR_UNSUPPORTED;
     static bool limit_raised[kMaxDevices] = {};
-    if (!raise_smem_limit(fff::k_leaf_umma<LP, kFold>, h->device, kSmemBudget, limit_raised)) return FFF_ERR_CUDA;
+    if (!raise_smem_limit(fff::k_leaf_umma<LP, kFold, kW8>, h->device, kSmemBudget, limit_raised)) return FFF_ERR_CUDA;
     CUtensorMap tm;
     if (!make_x_tensor_map(&tm, x, B, h->D, 1)) return FFF_ERR_CUDA;       // one-row boxes: rows are gathered four at a time
     const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(h->sm_count, n_tiles));
@@ -865,18 +872,27 @@ fff_status_t launch_leaf_umma(fff_handle_s* h, const void* x, const int32_t* per
     const int passes = 1;      // two passes (full tiles first) measured slightly slower
     // direct lists: perm is the table of lists, the tiles come from its counts
     int32_t* counts = h->slots_now && perm == h->ws_slots ? h->ws_cursor : nullptr;
-    if (launch_chain(h, fff::k_leaf_umma<LP, kFold>, (unsigned)grid, fff::kLUThreads, (size_t)L::smem_bytes(stages), st, 1, tm, perm,
+    if (launch_chain(h, fff::k_leaf_umma<LP, kFold, kW8>, (unsigned)grid, fff::kLUThreads, (size_t)L::smem_bytes(stages), st, 1, tm, perm,
                      (const fff::Tile*)h->ws_tiles, n_tiles, (const __nv_bfloat16*)h->w1img, (const float*)h->b1img,
-                     (const unsigned char*)h->w2uimg, (__nv_bfloat16*)y, h->D, h->O, h->l, h->act, stages, wide, passes, h->ws_sched,
-                     counts, (int)h->n_leaves, (int)h->slot_cap, h->d_status) != cudaSuccess)
+                     (const unsigned char*)(kW8 ? h->w2codes : h->w2uimg), (__nv_bfloat16*)y, h->D, h->O, h->l, h->act, stages, wide, passes, h->ws_sched,
+                     counts, (int)h->n_leaves, (int)h->slot_cap, h->d_status, (const unsigned char*)h->w1codes, (const float*)h->scale1,
+                     (const float*)h->scale2) != cudaSuccess)
         return cudaGetLastError(), FFF_ERR_CUDA;
-    return launched(h, st, "grouped_leaf_ff_umma");
+    return launched(h, st, kW8 ? "grouped_leaf_ff_umma_w8" : "grouped_leaf_ff_umma");
 }
 
 // Ring depth per (LP, TM): what fits twice into an SM's shared memory (once for LP = 64).
 fff_status_t run_leaf_mma(fff_handle_s* h, const void* x, const int32_t* perm, void* y, int64_t B, const LeafPlan& plan,
                           cudaStream_t st) {
     const int tile_rows = plan.tile_rows;
+    if (h->w8) {
+        switch (h->LP) {
+            case 16: return launch_leaf_umma<16, false, true>(h, x, perm, y, B, tile_rows, st);
+            case 32: return launch_leaf_umma<32, false, true>(h, x, perm, y, B, tile_rows, st);
+            case 64: return launch_leaf_umma<64, false, true>(h, x, perm, y, B, tile_rows, st);
+        }
+        return FFF_ERR_UNSUPPORTED;
+    }
     if (plan.umma && h->w2uimg) {
         switch (h->LP) {
             case 16: return h->l < 16 ? launch_leaf_umma<16, true>(h, x, perm, y, B, tile_rows, st)
@@ -1193,9 +1209,15 @@ const char* fff_status_string(fff_status_t s) {
     return "unknown status";
 }
 
-fff_status_t fff_create(fff_handle_t* out, int D, int O, int depth, int leaf_width, fff_activation_t act,
-                        fff_dtype_t dtype, const void* node_w, const void* node_b, const void* leaf_w1,
-                        const void* leaf_b1, const void* leaf_w2, const void* leaf_b2) {
+}  // extern "C"
+
+namespace {
+
+// fff_create and fff_create_w8: w1_scale != nullptr means leaf_w1 / leaf_w2 are e4m3 codes with per-leaf scales.
+fff_status_t create_common(fff_handle_t* out, int D, int O, int depth, int leaf_width, fff_activation_t act,
+                           fff_dtype_t dtype, const void* node_w, const void* node_b, const void* leaf_w1,
+                           const void* leaf_b1, const void* leaf_w2, const void* leaf_b2, const float* w1_scale,
+                           const float* w2_scale) {
     if (!out) return FFF_ERR_INVALID_ARG;
     *out = nullptr;
     if (D < 1 || O < 1 || leaf_width < 1 || depth < 0) return FFF_ERR_INVALID_ARG;
@@ -1203,8 +1225,12 @@ fff_status_t fff_create(fff_handle_t* out, int D, int O, int depth, int leaf_wid
     if (dtype != FFF_DTYPE_F32 && dtype != FFF_DTYPE_BF16) return FFF_ERR_INVALID_ARG;
     if (depth > FFF_MAX_DEPTH) return FFF_ERR_UNSUPPORTED;
     if (!leaf_w1 || !leaf_w2 || (depth > 0 && !node_w)) return FFF_ERR_INVALID_ARG;
-    for (const void* p : {node_w, node_b, leaf_w1, leaf_b1, leaf_w2, leaf_b2})
+    for (const void* p : {node_w, node_b, leaf_w1, leaf_b1, leaf_w2, leaf_b2, (const void*)w1_scale, (const void*)w2_scale})
         if (p && !aligned16(p)) return FFF_ERR_INVALID_ARG;
+    const bool w8 = w1_scale != nullptr;
+    if (w8 && (!w2_scale || dtype != FFF_DTYPE_BF16)) return FFF_ERR_INVALID_ARG;
+    // 8-bit leaf weights run on the tcgen05 leaf kernel only
+    if (w8 && (D % fff::kKS != 0 || O % 16 != 0 || leaf_width > 64 || !encode_tiled_fn())) return FFF_ERR_UNSUPPORTED;
 
     fff_handle_s* h = new (std::nothrow) fff_handle_s();
     if (!h) return FFF_ERR_ALLOC;
@@ -1241,9 +1267,10 @@ fff_status_t fff_create(fff_handle_t* out, int D, int O, int depth, int leaf_wid
     fff_status_t s = FFF_OK;
     if (s == FFF_OK) s = clone(&h->node_w, node_w, nn * D * e);
     if (s == FFF_OK) s = clone(&h->node_b, node_b, nn * e);
-    if (s == FFF_OK) s = clone(&h->w1, leaf_w1, nl * leaf_width * D * e);
+    h->w8 = w8;
+    if (s == FFF_OK && !w8) s = clone(&h->w1, leaf_w1, nl * leaf_width * D * e);
     if (s == FFF_OK) s = clone(&h->b1, leaf_b1, nl * leaf_width * e);
-    if (s == FFF_OK) s = clone(&h->w2, leaf_w2, nl * O * leaf_width * e);
+    if (s == FFF_OK && !w8) s = clone(&h->w2, leaf_w2, nl * O * leaf_width * e);
     if (s == FFF_OK) s = clone(&h->b2, leaf_b2, nl * O * e);
     if (s == FFF_OK) s = clone((void**)&h->ws_offsets, nullptr, sizeof(int32_t) * (nl + 1));
     if (s == FFF_OK) s = clone((void**)&h->ws_offsets2[0], nullptr, sizeof(int32_t) * (nl + 1));
@@ -1265,12 +1292,30 @@ fff_status_t fff_create(fff_handle_t* out, int D, int O, int depth, int leaf_wid
         }
     }
     if (s == FFF_OK && dtype == FFF_DTYPE_BF16 && D % fff::kKS == 0 && depth > 0) s = pack_node_images<__nv_bfloat16>(h);
-    if (s == FFF_OK && dtype == FFF_DTYPE_BF16 && D % fff::kKS == 0 && O % 8 == 0 && leaf_width <= 64) {
+    if (s == FFF_OK && w8) {
+        h->LP = leaf_width <= 16 ? 16 : (leaf_width <= 32 ? 32 : 64);
+        const int LP = h->LP;
+        const size_t P = (size_t)(O + fff::kLUPiece - 1) / fff::kLUPiece;
+        if (s == FFF_OK) s = dmalloc((void**)&h->w1codes, nl * LP * D);
+        if (s == FFF_OK) s = dmalloc((void**)&h->w2codes, nl * P * ((size_t)fff::kLUPiece * LP + fff::kLUPiece * 4));
+        if (s == FFF_OK) s = dmalloc((void**)&h->b1img, nl * LP * 4);
+        if (s == FFF_OK) s = clone((void**)&h->scale1, w1_scale, nl * sizeof(float));
+        if (s == FFF_OK) s = clone((void**)&h->scale2, w2_scale, nl * sizeof(float));
+        if (s == FFF_OK) s = clone((void**)&h->ws_sched, nullptr, 4 * sizeof(int));
+        if (s == FFF_OK) {
+            // (the caller's code arrays are read directly: nothing else of the library needs a copy of them)
+            fff::k_pack_leaf_codes<__nv_bfloat16><<<h->sm_count * 8, 256>>>((const unsigned char*)leaf_w1, (const unsigned char*)leaf_w2,
+                                                                           (const __nv_bfloat16*)h->b2, h->w1codes, h->w2codes, (int)nl,
+                                                                           leaf_width, LP, D, O);
+            fff::k_pack_b1<__nv_bfloat16><<<h->sm_count * 8, 256>>>((const __nv_bfloat16*)h->b1, h->b1img, (int)nl, leaf_width, LP);
+            if (cudaGetLastError() != cudaSuccess) s = FFF_ERR_CUDA;
+        }
+    } else if (s == FFF_OK && dtype == FFF_DTYPE_BF16 && D % fff::kKS == 0 && O % 8 == 0 && leaf_width <= 64) {
         h->LP = leaf_width <= 16 ? 16 : (leaf_width <= 32 ? 32 : 64);
         s = pack_leaf_images<__nv_bfloat16>(h);
     }
-    if (s == FFF_OK) s = FFF_DISPATCH(h, pack_fused_small, h);
-    if (s == FFF_OK) s = pack_train_images(h);
+    if (s == FFF_OK && !w8) s = FFF_DISPATCH(h, pack_fused_small, h);
+    if (s == FFF_OK && !w8) s = pack_train_images(h);
     if (s == FFF_OK && cudaDeviceSynchronize() != cudaSuccess) s = (cudaGetLastError(), FFF_ERR_CUDA);
     if (s != FFF_OK) { release(h); return s; }
     {
@@ -1279,6 +1324,25 @@ fff_status_t fff_create(fff_handle_t* out, int D, int O, int depth, int leaf_wid
     }
     *out = h;
     return FFF_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+fff_status_t fff_create(fff_handle_t* out, int D, int O, int depth, int leaf_width, fff_activation_t act,
+                        fff_dtype_t dtype, const void* node_w, const void* node_b, const void* leaf_w1,
+                        const void* leaf_b1, const void* leaf_w2, const void* leaf_b2) {
+    return create_common(out, D, O, depth, leaf_width, act, dtype, node_w, node_b, leaf_w1, leaf_b1, leaf_w2, leaf_b2, nullptr,
+                         nullptr);
+}
+
+fff_status_t fff_create_w8(fff_handle_t* out, int D, int O, int depth, int leaf_width, fff_activation_t act,
+                           const void* node_w, const void* node_b, const uint8_t* leaf_w1_e4m3, const float* leaf_w1_scale,
+                           const void* leaf_b1, const uint8_t* leaf_w2_e4m3, const float* leaf_w2_scale, const void* leaf_b2) {
+    if (!leaf_w1_scale || !leaf_w2_scale) return out ? (*out = nullptr, FFF_ERR_INVALID_ARG) : FFF_ERR_INVALID_ARG;
+    return create_common(out, D, O, depth, leaf_width, act, FFF_DTYPE_BF16, node_w, node_b, leaf_w1_e4m3, leaf_b1, leaf_w2_e4m3,
+                         leaf_b2, leaf_w1_scale, leaf_w2_scale);
 }
 
 fff_status_t fff_destroy(fff_handle_t h) {
@@ -1305,6 +1369,7 @@ fff_status_t fff_set_path(fff_handle_t h, fff_path_t path) {
         return FFF_ERR_INVALID_ARG;
     if (path == FFF_PATH_TENSOR && h->LP == 0 && h->stages.empty()) return FFF_ERR_UNSUPPORTED;
     if (path == FFF_PATH_FUSED && h->fs_batch == 0) return FFF_ERR_UNSUPPORTED;
+    if (h->w8 && path != FFF_PATH_AUTO && path != FFF_PATH_TENSOR) return FFF_ERR_UNSUPPORTED;
     h->path = path;
     return FFF_OK;
 }
@@ -1592,7 +1657,7 @@ int fff_capabilities(fff_handle_t h) {
     if (!h->stages.empty() || !h->ustages.empty()) caps |= FFF_CAP_TENSOR_DESCENT;
     if (!h->ustages.empty()) caps |= FFF_CAP_TCGEN05_DESCENT;
     if (h->LP != 0) caps |= FFF_CAP_TENSOR_LEAF;
-    if (h->w2uimg) caps |= FFF_CAP_TCGEN05_LEAF;
+    if (h->w2uimg || h->w2codes) caps |= FFF_CAP_TCGEN05_LEAF;
     if (h->fs_batch != 0) caps |= FFF_CAP_FUSED_SMALL;
     if (h->tr_Kp != 0) caps |= FFF_CAP_FORWARD_TRAIN;
     return caps;

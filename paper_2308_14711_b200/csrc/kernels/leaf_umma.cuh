@@ -70,7 +70,11 @@ constexpr int kLUConsumerWarps = kLUWarps - 1;     // every warp but the schedul
 constexpr int kLUAcc2Col = 64;             // first tensor-memory column of the two GEMM2 accumulators
 constexpr int kLUTmemCols = 512;
 
-template <int LP> struct LeafUmmaLayout {
+// kW8: the leaf weights are stored as 8-bit floats (e4m3 codes, one float32 scale per leaf and matrix).  The MMA wants
+// both operands as bf16, so the codes land in a staging part of their ring slot and the warp that issues the MMAs
+// expands them (every code is exactly a bf16 value) into the operand layout first; the scales multiply the
+// accumulators in the epilogue.
+template <int LP, bool kW8 = false> struct LeafUmmaLayout {
     static_assert(LP == 16 || LP == 32 || LP == 64, "padded hidden width");
     static constexpr int kRowBytes = LP * 2;                                 // row of H and of a W2 piece
     // A ring stage holds kSub K-blocks of 64 columns (each a 128-byte swizzled operand tile of its own):
@@ -81,13 +85,18 @@ template <int LP> struct LeafUmmaLayout {
     static constexpr int kW1SubBytes = LP * kLUKB * 2;
     static constexpr int kXStageBytes = kSub * kXSubBytes;
     static constexpr int kW1StageBytes = kSub * kW1SubBytes;
-    static constexpr int kStageBytes = kXStageBytes + kW1StageBytes;         // a multiple of 1024
-    static constexpr int kW2Bytes = kLUPiece * kRowBytes;                    // weights of a piece
-    static constexpr int kW2PieceBytes = kW2Bytes + kLUPiece * 4;            // + float32 biases
-    static constexpr int kW2SlotStride = (kW2PieceBytes + 1023) & ~1023;
+    static constexpr int kW1CodeBytes = kW8 ? kW1StageBytes / 2 : 0;         // staging for the codes of the stage's W1 K-blocks
+    static constexpr int kW1CopyBytes = kW8 ? kW1CodeBytes : kW1StageBytes;  // what the bulk copy of a stage brings
+    static constexpr int kStageBytes = kXStageBytes + kW1StageBytes + kW1CodeBytes;      // a multiple of 1024
+    static constexpr int kW2Bytes = kLUPiece * kRowBytes;                    // weights of a piece (bf16 operand)
+    static constexpr int kW2CodeBytes = kW8 ? kW2Bytes / 2 : 0;
+    static constexpr int kW2BiasOff = kW2Bytes + kW2CodeBytes;               // the piece's 128 float32 biases inside a slot
+    static constexpr int kW2CopyOff = kW8 ? kW2Bytes : 0;                    // where the bulk copy of a piece lands in its slot
+    static constexpr int kW2PieceBytes = (kW8 ? kW2CodeBytes : kW2Bytes) + kLUPiece * 4;    // a piece in the image: weights + biases
+    static constexpr int kW2SlotStride = (kW2BiasOff + kLUPiece * 4 + 1023) & ~1023;
     static constexpr int kHBytes = kLUM * kRowBytes;
     // W2 ring: a whole tile's pieces (O <= 1024) when they are small, so that no copy waits for an MMA just issued
-    static constexpr int kW2Slots = LP <= 32 ? 8 : 4;
+    static constexpr int kW2Slots = LP <= 16 ? 8 : LP <= 32 ? (kW8 ? 6 : 8) : 4;
     static constexpr int kBarrierBytes = 640;
     static constexpr int smem_bytes(int stages) {
         return 1024 + stages * kStageBytes + kW2Slots * kW2SlotStride + kHBytes + kBarrierBytes;
@@ -130,6 +139,65 @@ __global__ void k_pack_w2_umma(const T* __restrict__ w2, const T* __restrict__ b
     }
 }
 
+// Images of 8-bit leaf weights: w1c [leaf][D / 64][LP][64] codes (rows past l zero = the code of +0);
+// w2c [leaf][ceil(O/128) pieces]{ [128 rows (output features)][LP] codes, then their 128 float32 biases }.
+template <typename T>
+__global__ void k_pack_leaf_codes(const unsigned char* __restrict__ w1, const unsigned char* __restrict__ w2, const T* __restrict__ b2,
+                                  unsigned char* __restrict__ w1c, unsigned char* __restrict__ w2c, int n_leaves, int l, int LP,
+                                  int D, int O)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x, t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int KBn = D / kLUKB;
+    for (int64_t i = t0; i < (int64_t)n_leaves * KBn * LP * kLUKB; i += stride) {
+        const int c = (int)(i % kLUKB), r = (int)((i / kLUKB) % LP);
+        const int64_t kb = (i / ((int64_t)kLUKB * LP)) % KBn, j = i / ((int64_t)kLUKB * LP * KBn);
+        w1c[i] = r < l ? w1[(j * l + r) * D + kb * kLUKB + c] : (unsigned char)0;
+    }
+    const int P = (O + kLUPiece - 1) / kLUPiece;
+    const int64_t piece_bytes = (int64_t)kLUPiece * LP + kLUPiece * 4;
+    for (int64_t i = t0; i < (int64_t)n_leaves * P * kLUPiece * (LP + 1); i += stride) {
+        const int c = (int)(i % (LP + 1)), n = (int)((i / (LP + 1)) % kLUPiece);
+        const int64_t jp = i / ((int64_t)(LP + 1) * kLUPiece), j = jp / P;
+        const int o = (int)(jp % P) * kLUPiece + n;
+        unsigned char* piece = w2c + jp * piece_bytes;
+        if (c < LP) piece[n * LP + c] = (o < O && c < l) ? w2[(j * O + o) * (int64_t)l + c] : (unsigned char)0;
+        else reinterpret_cast<float*>(piece + (int64_t)kLUPiece * LP)[n] = (o < O && b2) ? Elem<T>::to_float(b2[j * O + o]) : 0.0f;
+    }
+}
+
+// Two e4m3 codes (the low and the high byte of `pair`) as two bf16 values: every e4m3 value is exactly a half and
+// exactly a bf16 value, so the published conversions e4m3x2 -> f16x2, f16 -> f32, f32x2 -> bf16x2 lose nothing.
+__device__ __forceinline__ uint32_t e4m3x2_to_bf16x2(uint32_t pair) {
+    uint32_t h2, out;
+    asm("{\n\t.reg .b16 p;\n\tcvt.u16.u32 p, %1;\n\tcvt.rn.f16x2.e4m3x2 %0, p;\n\t}" : "=r"(h2) : "r"(pair));
+    float lo, hi;
+    asm("{\n\t.reg .b16 a, b;\n\tmov.b32 {a, b}, %2;\n\tcvt.f32.f16 %0, a;\n\tcvt.f32.f16 %1, b;\n\t}" : "=f"(lo), "=f"(hi) : "r"(h2));
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(out) : "f"(hi), "f"(lo));
+    return out;
+}
+
+// A tile of e4m3 codes, [rows][COLS] row-major, expanded by one warp into the K-major bf16 operand layout with rows of
+// 2 COLS bytes, swizzled in the mode of that width.  Units of 16 codes (16 bytes in, two 16-byte units out).
+template <int COLS>
+__device__ __forceinline__ void expand_e4m3_tile(const unsigned char* __restrict__ src, unsigned char* __restrict__ dst, int rows,
+                                                 int lane)
+{
+    const int n_units = rows * COLS / 16;
+    for (int u = lane; u < n_units; u += 32) {
+        const uint4 raw = *reinterpret_cast<const uint4*>(src + u * 16);
+        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+        uint32_t o[8];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            o[2 * i] = e4m3x2_to_bf16x2(w[i] & 0xffffu);
+            o[2 * i + 1] = e4m3x2_to_bf16x2(w[i] >> 16);
+        }
+        const uint32_t off = (uint32_t)(u * 16 / COLS) * (COLS * 2) + (uint32_t)(u * 16 % COLS) * 2;
+        *reinterpret_cast<uint4*>(dst + swz_rows(off, COLS * 2)) = make_uint4(o[0], o[1], o[2], o[3]);
+        *reinterpret_cast<uint4*>(dst + swz_rows(off + 16, COLS * 2)) = make_uint4(o[4], o[5], o[6], o[7]);
+    }
+}
+
 // sched: two ints, both zero before the first launch and again after every launch: [0] list entries
 // handed out so far, [1] CTAs that have finished.
 // kFold: l < LP, the spare hidden column l carries the output bias (see k_pack_w2_umma).
@@ -137,16 +205,20 @@ __global__ void k_pack_w2_umma(const T* __restrict__ w2, const T* __restrict__ b
 // perm[bin * cap + i], i < slot_counts[bin], are the tokens of bin.  The scheduler then derives the tiles itself:
 // every lane owns a run of bins and knows how many tiles precede it; a claimed number is resolved by the lane
 // whose range holds it.  The last CTA to finish clears the counts for the next call.
-template <int LP, bool kFold>
+// kW8: w1codes / w2img hold e4m3 codes ([leaf][D / 64][LP][64], and per piece [128][LP] codes + 128 float32 biases),
+// scale1 / scale2 [leaf] the float32 scales of W1 and W2 (kFold must be off: the biases are added in the epilogue).
+template <int LP, bool kFold, bool kW8 = false>
 __global__ void __launch_bounds__(kLUThreads, 1)
 k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restrict__ perm,
             const Tile* __restrict__ tiles, int n_tiles_total,
             const __nv_bfloat16* __restrict__ w1img, const float* __restrict__ b1img,
             const unsigned char* __restrict__ w2img, __nv_bfloat16* __restrict__ y,
             int D, int O, int l, int act, int kStages, int wide_stores, int passes, int* __restrict__ sched,
-            int32_t* __restrict__ slot_counts, int n_bins, int cap, int* __restrict__ status)
+            int32_t* __restrict__ slot_counts, int n_bins, int cap, int* __restrict__ status,
+            const unsigned char* __restrict__ w1codes, const float* __restrict__ scale1, const float* __restrict__ scale2)
 {
-    using L = LeafUmmaLayout<LP>;
+    static_assert(!(kW8 && kFold), "8-bit weights take their biases in the epilogue");
+    using L = LeafUmmaLayout<LP, kW8>;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     unsigned char* w2ring = ring + kStages * L::kStageBytes;
@@ -338,12 +410,17 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
             for (int kb = 0; kb < KB; ++kb) {
                 if (!timed_out && !ptx::mbar_wait_relaxed(empty + stage, phase ^ 1)) timed_out = true;
                 if (lane == 0) {
-                    const uint32_t bytes = (uint32_t)groups * (512u * L::kSub) + (gw == 0 ? (uint32_t)L::kW1StageBytes : 0u);
+                    const uint32_t bytes = (uint32_t)groups * (512u * L::kSub) + (gw == 0 ? (uint32_t)L::kW1CopyBytes : 0u);
                     if (bytes > 0) ptx::mbar_arrive_expect_tx(full + stage, bytes);
                     else ptx::mbar_arrive(full + stage);
-                    if (gw == 0)
-                        ptx::bulk_g2s(ring + stage * L::kStageBytes + L::kXStageBytes,
-                                      w1img + ((int64_t)tl.bin * KB + kb) * (L::kSub * LP * kLUKB), L::kW1StageBytes, full + stage);
+                    if (gw == 0) {
+                        if constexpr (kW8)
+                            ptx::bulk_g2s(ring + stage * L::kStageBytes + L::kXStageBytes + L::kW1StageBytes,
+                                          w1codes + ((int64_t)tl.bin * KB + kb) * L::kW1CodeBytes, L::kW1CodeBytes, full + stage);
+                        else
+                            ptx::bulk_g2s(ring + stage * L::kStageBytes + L::kXStageBytes,
+                                          w1img + ((int64_t)tl.bin * KB + kb) * (L::kSub * LP * kLUKB), L::kW1StageBytes, full + stage);
+                    }
                 }
                 __syncwarp();
                 if (lane < groups) {
@@ -368,6 +445,13 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
             for (int kb = 0; kb < KB; ++kb) {
                 if (!timed_out && !ptx::mbar_wait(full + stage, phase)) timed_out = true;
                 ptx::tc_fence_after_sync();
+                if constexpr (kW8) {
+                    // the stage's W1 codes -> bf16 operand tiles (kSub tiles of LP rows x 64 columns, stacked)
+                    unsigned char* w1s = ring + stage * L::kStageBytes + L::kXStageBytes;
+                    expand_e4m3_tile<kLUKB>(w1s + L::kW1StageBytes, w1s, L::kSub * LP, lane);
+                    ptx::fence_proxy_async();
+                    __syncwarp();
+                }
                 if (lane == 0) {
                     const uint32_t xs = ptx::smem_addr(ring + stage * L::kStageBytes);
 #pragma unroll
@@ -400,8 +484,8 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                 if (!timed_out && !ptx::mbar_wait(w2_empty + ld_slot, ld_phase ^ 1)) timed_out = true;
                 if (lane == 0) {
                     ptx::mbar_arrive_expect_tx(w2_full + ld_slot, (uint32_t)L::kW2PieceBytes);
-                    ptx::bulk_g2s(w2ring + ld_slot * L::kW2SlotStride, w2j + (int64_t)loaded * L::kW2PieceBytes, L::kW2PieceBytes,
-                                  w2_full + ld_slot);
+                    ptx::bulk_g2s(w2ring + ld_slot * L::kW2SlotStride + L::kW2CopyOff, w2j + (int64_t)loaded * L::kW2PieceBytes,
+                                  L::kW2PieceBytes, w2_full + ld_slot);
                 }
                 __syncwarp();
                 ++loaded;
@@ -413,6 +497,13 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
             for (int p = 0; p < P; ++p, ++pc) {
                 const int b = pc & 1;
                 if (!timed_out && !ptx::mbar_wait(w2_full + mm_slot, mm_phase)) timed_out = true;
+                if constexpr (kW8) {
+                    // the piece's codes -> bf16 operand tile (128 output features x LP columns)
+                    unsigned char* slot = w2ring + mm_slot * L::kW2SlotStride;
+                    expand_e4m3_tile<LP>(slot + L::kW2CopyOff, slot, kLUPiece, lane);
+                    ptx::fence_proxy_async();
+                    __syncwarp();
+                }
                 if (!timed_out && !ptx::mbar_wait(y_empty + b, ((pc >> 1) & 1) ^ 1)) timed_out = true;
                 ptx::tc_fence_after_sync();
                 if (lane == 0) {
@@ -455,6 +546,16 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
             const bool active = (quarter % qper) * 32 < tl.rows; // this warp's lanes hold valid rows
             const bool h_active = active && copy == 0 && part < kLUHParts;      // the first copy's lanes hold acc1
             const int64_t tok = row < tl.rows ? perm[tl.start + row] : -1;
+            // accumulator -> pre-activation / output: + bias, and with 8-bit weights the leaf's scale first
+            float s1 = 1.0f, s2 = 1.0f;
+            if constexpr (kW8) {
+                s1 = __ldg(scale1 + tl.bin);
+                s2 = __ldg(scale2 + tl.bin);
+            }
+            auto scaled = [](uint32_t acc, float scale, float bias) {
+                if constexpr (kW8) return fmaf(__uint_as_float(acc), scale, bias);
+                else return __uint_as_float(acc) + bias;
+            };
             float b1r[HC];
 #pragma unroll
             for (int j = 0; j < HC; j += 4) {
@@ -473,8 +574,8 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                     ptx::tmem_ld_wait();
 #pragma unroll
                     for (int j = 0; j < HC; j += 2) {
-                        float h0 = activate_bf16(act, __uint_as_float(v[j]) + b1r[j]);
-                        float h1 = activate_bf16(act, __uint_as_float(v[j + 1]) + b1r[j + 1]);
+                        float h0 = activate_bf16(act, scaled(v[j], s1, b1r[j]));
+                        float h1 = activate_bf16(act, scaled(v[j + 1], s1, b1r[j + 1]));
                         if (kFold && part * HC + j == l) h0 = 1.0f;          // the bias column
                         if (kFold && part * HC + j + 1 == l) h1 = 1.0f;
                         hp[j / 2] = ptx::pack_bf16(h0, h1);
@@ -504,7 +605,7 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                 if (!timed_out && !ptx::mbar_wait(y_full + b, (pc >> 1) & 1)) timed_out = true;
                 if (!timed_out && !ptx::mbar_wait(w2_full + w2_slot, w2_phase)) timed_out = true;     // biases: landed long ago
                 ptx::tc_fence_after_sync();
-                const float* bias = reinterpret_cast<const float*>(w2ring + w2_slot * L::kW2SlotStride + L::kW2Bytes);
+                const float* bias = reinterpret_cast<const float*>(w2ring + w2_slot * L::kW2SlotStride + L::kW2BiasOff);
                 const int ncols = min(kLUPiece, O - p * kLUPiece);
                 if (ncw == 16) {
                     const int c0 = cbase;
@@ -521,8 +622,8 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
 #pragma unroll
                             for (int e = 0; e < 4; ++e) {
                                 const float4 bb = *reinterpret_cast<const float4*>(bias + c0 + 4 * e);
-                                out[2 * e] = ptx::pack_bf16(__uint_as_float(v[4 * e]) + bb.x, __uint_as_float(v[4 * e + 1]) + bb.y);
-                                out[2 * e + 1] = ptx::pack_bf16(__uint_as_float(v[4 * e + 2]) + bb.z, __uint_as_float(v[4 * e + 3]) + bb.w);
+                                out[2 * e] = ptx::pack_bf16(scaled(v[4 * e], s2, bb.x), scaled(v[4 * e + 1], s2, bb.y));
+                                out[2 * e + 1] = ptx::pack_bf16(scaled(v[4 * e + 2], s2, bb.z), scaled(v[4 * e + 3], s2, bb.w));
                             }
                         }
                         if (tok >= 0) {
@@ -553,8 +654,8 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
 #pragma unroll
                                 for (int e = 0; e < 8; ++e) {
                                     const float4 bb = *reinterpret_cast<const float4*>(bias + c0 + 4 * e);
-                                    out[2 * e] = ptx::pack_bf16(__uint_as_float(v[4 * e]) + bb.x, __uint_as_float(v[4 * e + 1]) + bb.y);
-                                    out[2 * e + 1] = ptx::pack_bf16(__uint_as_float(v[4 * e + 2]) + bb.z, __uint_as_float(v[4 * e + 3]) + bb.w);
+                                    out[2 * e] = ptx::pack_bf16(scaled(v[4 * e], s2, bb.x), scaled(v[4 * e + 1], s2, bb.y));
+                                    out[2 * e + 1] = ptx::pack_bf16(scaled(v[4 * e + 2], s2, bb.z), scaled(v[4 * e + 3], s2, bb.w));
                                 }
                             }
                             if (tok >= 0) {
