@@ -351,6 +351,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
             # four layers of the ViT-shaped configuration as one stack (the paper's transformer use of the layer)
             out["stack"] = stack_bench(wl.CONFIGS["vit_d8_l12_bf16"], 4, max(5, min(args.steps, 50)))
             out["forward_train"] = train_bench(wl.CONFIGS["vit_d8_l12_bf16"], max(3, min(args.steps, 10)), peaks)
+            out["w8"] = w8_bench(wl.CONFIGS["wide_d11_l32_bf16"], max(5, min(args.steps, 50)), peaks)
     layer.close()
     if dist is not None:
         dist.barrier()
@@ -446,6 +447,37 @@ def stack_bench(cfg: wl.FFFConfig, n_layers: int, steps: int) -> dict:
     for l in layers:
         l.close()
     return out
+
+
+def w8_bench(cfg: wl.FFFConfig, steps: int, peaks) -> dict:
+    """The hard forward of one configuration with its leaf weights stored as 8-bit floats (fff_create_w8): time per
+    step on resident inputs, and the algorithmic bytes with the leaf weights at one byte each."""
+    import torch
+    from paper_2308_14711_b200.binding import FFFLayer
+    w = wl.make_weights(cfg, 0)
+    c1, s1, _ = wl.quantize_e4m3(w["w1"])
+    c2, s2, _ = wl.quantize_e4m3(w["w2"])
+
+    def bf(a):
+        return torch.from_numpy(a).to(torch.bfloat16).cuda()
+    layer = FFFLayer(cfg.D, cfg.O, cfg.depth, cfg.leaf_width, cfg.activation, "bf16", bf(w["node_w"]), bf(w["node_b"]),
+                     torch.from_numpy(c1).cuda(), bf(w["b1"]), torch.from_numpy(c2).cuda(), bf(w["b2"]),
+                     w1_scale=torch.from_numpy(s1).cuda(), w2_scale=torch.from_numpy(s2).cuda())
+    layer.reserve(cfg.B)
+    n = n_buffer_sets(cfg)
+    xs = [torch.from_numpy(wl.TokenSource(cfg, i).x).to(torch.bfloat16).cuda() for i in range(n)]
+    ys = [torch.empty((cfg.B, cfg.O), dtype=torch.bfloat16, device="cuda") for _ in range(n)]
+    ls = [torch.empty((cfg.B,), dtype=torch.int32, device="cuda") for _ in range(n)]
+    regions, _, _, _, _ = time_device(layer, xs, ys, ls, steps, 5, profile=False, min_seconds=MIN_TIMED_SECONDS / 2)
+    ms = statistics.median(regions) / steps
+    touched = int(torch.unique(ls[0]).numel())
+    l, D, O = cfg.leaf_width, cfg.D, cfg.O
+    pb = cfg.B * (D + O) * 2 + cfg.n_nodes * (D + 1) * 2 + touched * ((l * D + O * l) * 1 + (l + O) * 2 + 8) + 4 * cfg.B
+    status = layer.last_status()
+    layer.close()
+    return {"workload": cfg.name, "leaf_weights": "e4m3 codes + one float32 scale per leaf", "ms_per_step": round(ms, 5),
+            "tokens_per_s": cfg.B / (ms * 1e-3), "algorithmic_bytes": int(pb), "device_status": status,
+            "roofline_frac": round(pb / (peaks["hbm_gbs"] * 1e9) * 1e3 / ms, 4)}
 
 
 def train_bench(cfg: wl.FFFConfig, steps: int, peaks) -> dict:
@@ -568,7 +600,7 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-config", action="store_true")
-    ap.add_argument("--leg", default="path", choices=["path", "forward_train", "stack"],
+    ap.add_argument("--leg", default="path", choices=["path", "forward_train", "stack", "w8"],
                     help="path: the benchmark line; forward_train / stack: only that extra measurement of --config (for profiling)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -581,8 +613,12 @@ def main():
         import torch
         torch.cuda.set_device(local_rank)
         cfg = wl.CONFIGS[args.config]
-        out = train_bench(cfg, max(1, min(args.steps, 10)), measured_peaks()) if args.leg == "forward_train" else \
-            stack_bench(cfg, 4, max(1, min(args.steps, 50)))
+        if args.leg == "forward_train":
+            out = train_bench(cfg, max(1, min(args.steps, 10)), measured_peaks())
+        elif args.leg == "w8":
+            out = w8_bench(cfg, max(1, min(args.steps, 50)), measured_peaks())
+        else:
+            out = stack_bench(cfg, 4, max(1, min(args.steps, 50)))
         if rank == 0:
             print(json.dumps({"leg": args.leg, **out}), flush=True)
     else:

@@ -183,6 +183,7 @@ __device__ __forceinline__ void expand_e4m3_tile(const unsigned char* __restrict
                                                  int lane)
 {
     const int n_units = rows * COLS / 16;
+#pragma unroll 4
     for (int u = lane; u < n_units; u += 32) {
         const uint4 raw = *reinterpret_cast<const uint4*>(src + u * 16);
         const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
