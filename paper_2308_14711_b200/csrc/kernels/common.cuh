@@ -1,6 +1,8 @@
 // Shared device helpers for the FFF inference kernels (sm_100a).
 #pragma once
 
+#include <type_traits>
+
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -91,6 +93,19 @@ __device__ __forceinline__ float activate_bf16(int act, float v) {
     poly = fmaf(poly, t, 0.254829592f);
     const float e = 1.0f - poly * t * __expf(-z * z);          // erf(|v| / sqrt 2)
     return 0.5f * v * (1.0f + copysignf(e, v));
+}
+
+// Calls f(std::integral_constant<int, act>) with the activation as a compile-time constant.  Code that applies the
+// activation to many values in an unrolled loop goes through this: with a run-time `act` every value carries the
+// branches between the four forms, which keeps the values' dependency chains from overlapping.
+template <class F>
+__device__ __forceinline__ void with_activation(int act, F&& f) {
+    switch (act) {
+        case kActRelu: f(std::integral_constant<int, kActRelu>{}); break;
+        case kActGeluTanh: f(std::integral_constant<int, kActGeluTanh>{}); break;
+        case kActSilu: f(std::integral_constant<int, kActSilu>{}); break;
+        default: f(std::integral_constant<int, kActGelu>{}); break;
+    }
 }
 
 // <a, b> over n elements, evaluated by one warp; every lane returns the sum.

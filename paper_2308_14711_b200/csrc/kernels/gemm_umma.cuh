@@ -217,24 +217,27 @@ k_gemm_umma(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                     for (int q = 0; q < 4; ++q) mpre[q] = leaf + q < ep.n_leaves ? mrow[leaf + q] : 0.0f;
                     int ahead = 0;
                     float mw = mpre[0];
+                    with_activation(ep.act, [&](auto a) {
+                        constexpr int kAct = decltype(a)::value;
 #pragma unroll
-                    for (int e = 0; e < 32; e += 2) {
-                        float h2[2];
+                        for (int e = 0; e < 32; e += 2) {
+                            float h2[2];
 #pragma unroll
-                        for (int q = 0; q < 2; ++q) {
-                            float h = 0.0f;
-                            if (e + q < nv) h = mw * activate_bf16(ep.act, __uint_as_float(v[e + q]) + __bfloat162float(ep.bias[col0 + e + q]));
-                            h2[q] = h;
-                            if (++u == ep.l) {
-                                u = 0;
-                                ++leaf;
-                                ++ahead;
-                                mw = ahead == 1 ? mpre[1] : ahead == 2 ? mpre[2] : ahead == 3 ? mpre[3]
-                                                : (leaf < ep.n_leaves ? mrow[leaf] : 0.0f);
+                            for (int q = 0; q < 2; ++q) {
+                                float h = 0.0f;
+                                if (e + q < nv) h = mw * activate_bf16(kAct, __uint_as_float(v[e + q]) + __bfloat162float(ep.bias[col0 + e + q]));
+                                h2[q] = h;
+                                if (++u == ep.l) {
+                                    u = 0;
+                                    ++leaf;
+                                    ++ahead;
+                                    mw = ahead == 1 ? mpre[1] : ahead == 2 ? mpre[2] : ahead == 3 ? mpre[3]
+                                                    : (leaf < ep.n_leaves ? mrow[leaf] : 0.0f);
+                                }
                             }
+                            packed[e / 2] = ptx::pack_bf16(h2[0], h2[1]);
                         }
-                        packed[e / 2] = ptx::pack_bf16(h2[0], h2[1]);
-                    }
+                    });
                     if (row_ok) {
                         if (nv == 32 && (ep.ld_out & 7) == 0) {
 #pragma unroll

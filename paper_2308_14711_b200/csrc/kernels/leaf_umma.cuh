@@ -573,14 +573,17 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                     uint32_t v[32];
                     ptx::tmem_ld32(lane_base + part * HC, v);      // columns past HC are not used
                     ptx::tmem_ld_wait();
+                    with_activation(act, [&](auto a) {
+                        constexpr int kAct = decltype(a)::value;
 #pragma unroll
-                    for (int j = 0; j < HC; j += 2) {
-                        float h0 = activate_bf16(act, scaled(v[j], s1, b1r[j]));
-                        float h1 = activate_bf16(act, scaled(v[j + 1], s1, b1r[j + 1]));
-                        if (kFold && part * HC + j == l) h0 = 1.0f;          // the bias column
-                        if (kFold && part * HC + j + 1 == l) h1 = 1.0f;
-                        hp[j / 2] = ptx::pack_bf16(h0, h1);
-                    }
+                        for (int j = 0; j < HC; j += 2) {
+                            float h0 = activate_bf16(kAct, scaled(v[j], s1, b1r[j]));
+                            float h1 = activate_bf16(kAct, scaled(v[j + 1], s1, b1r[j + 1]));
+                            if (kFold && part * HC + j == l) h0 = 1.0f;          // the bias column
+                            if (kFold && part * HC + j + 1 == l) h1 = 1.0f;
+                            hp[j / 2] = ptx::pack_bf16(h0, h1);
+                        }
+                    });
                 }
                 ptx::tc_fence_before_sync();
                 ptx::mbar_arrive(acc1_empty);
