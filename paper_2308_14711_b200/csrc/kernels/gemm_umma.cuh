@@ -43,11 +43,12 @@ constexpr int kGTmemCols = 2 * kGN;
 enum : int { kGemmNodes = 0, kGemmHidden = 1, kGemmOutput = 2 };
 
 // Entropy in nats of a Bernoulli choice with probability c, 0 ln 0 = 0.
+// (Branch-free: the logarithms take their arguments clamped to the smallest normal float, so that c = 0 and c = 1 give
+// 0 x a finite number = 0; with branches the unrolled epilogue would evaluate its 32 values one after the other.)
 __device__ __forceinline__ float bernoulli_entropy(float c) {
-    float h = 0.0f;
-    if (c > 0.0f) h -= c * __logf(c);
-    if (c < 1.0f) h -= (1.0f - c) * __logf(1.0f - c);
-    return h;
+    const float tiny = 1.17549435e-38f;
+    const float d = 1.0f - c;
+    return -(c * __logf(fmaxf(c, tiny)) + d * __logf(fmaxf(d, tiny)));
 }
 
 struct GemmEpilogueArgs {
@@ -211,31 +212,67 @@ k_gemm_umma(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                     const float* mrow = ep.mix + (int64_t)(row_ok ? row : 0) * ep.n_leaves;
                     uint32_t packed[16];
                     int leaf = col0 / ep.l, u = col0 % ep.l;           // leaf and unit of column col0 + e, stepped along
-                    // the weights of the first leaves of the chunk are fetched together, ahead of their use
+                    // the mixture weights of the first leaves of the chunk are fetched together, ahead of their use
                     float mpre[4];
 #pragma unroll
                     for (int q = 0; q < 4; ++q) mpre[q] = leaf + q < ep.n_leaves ? mrow[leaf + q] : 0.0f;
-                    int ahead = 0;
-                    float mw = mpre[0];
+                    // the chunk's 32 biases: four 16-byte loads (col0 is a multiple of 32, the array 16-byte aligned)
+                    float bs[32];
+                    if (nv == 32) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const uint4 raw = __ldg(reinterpret_cast<const uint4*>(ep.bias + col0) + q);
+                            const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                bs[8 * q + 2 * i] = __uint_as_float(w[i] << 16);
+                                bs[8 * q + 2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) bs[e] = e < nv ? __bfloat162float(ep.bias[col0 + e]) : 0.0f;
+                    }
                     with_activation(ep.act, [&](auto a) {
                         constexpr int kAct = decltype(a)::value;
+                        if (ep.l >= 11) {
+                            // at most four leaves meet in 32 columns: the weight is chosen among the four fetched ones by
+                            // selects, and nothing in the loop branches or loads
+                            int ahead = 0;
 #pragma unroll
-                        for (int e = 0; e < 32; e += 2) {
-                            float h2[2];
+                            for (int e = 0; e < 32; e += 2) {
+                                float h2[2];
 #pragma unroll
-                            for (int q = 0; q < 2; ++q) {
-                                float h = 0.0f;
-                                if (e + q < nv) h = mw * activate_bf16(kAct, __uint_as_float(v[e + q]) + __bfloat162float(ep.bias[col0 + e + q]));
-                                h2[q] = h;
-                                if (++u == ep.l) {
-                                    u = 0;
-                                    ++leaf;
-                                    ++ahead;
-                                    mw = ahead == 1 ? mpre[1] : ahead == 2 ? mpre[2] : ahead == 3 ? mpre[3]
-                                                    : (leaf < ep.n_leaves ? mrow[leaf] : 0.0f);
+                                for (int q = 0; q < 2; ++q) {
+                                    const float mw = ahead == 0 ? mpre[0] : ahead == 1 ? mpre[1] : ahead == 2 ? mpre[2] : mpre[3];
+                                    const float h = mw * activate_bf16(kAct, __uint_as_float(v[e + q]) + bs[e + q]);
+                                    h2[q] = e + q < nv ? h : 0.0f;
+                                    const bool wrap = ++u == ep.l;
+                                    u = wrap ? 0 : u;
+                                    ahead += wrap ? 1 : 0;
                                 }
+                                packed[e / 2] = ptx::pack_bf16(h2[0], h2[1]);
                             }
-                            packed[e / 2] = ptx::pack_bf16(h2[0], h2[1]);
+                        } else {
+                            int ahead = 0;
+                            float mw = mpre[0];
+#pragma unroll
+                            for (int e = 0; e < 32; e += 2) {
+                                float h2[2];
+#pragma unroll
+                                for (int q = 0; q < 2; ++q) {
+                                    const float h = mw * activate_bf16(kAct, __uint_as_float(v[e + q]) + bs[e + q]);
+                                    h2[q] = e + q < nv ? h : 0.0f;
+                                    if (++u == ep.l) {
+                                        u = 0;
+                                        ++leaf;
+                                        ++ahead;
+                                        mw = ahead == 1 ? mpre[1] : ahead == 2 ? mpre[2] : ahead == 3 ? mpre[3]
+                                                        : (leaf < ep.n_leaves ? mrow[leaf] : 0.0f);
+                                    }
+                                }
+                                packed[e / 2] = ptx::pack_bf16(h2[0], h2[1]);
+                            }
                         }
                     });
                     if (row_ok) {
