@@ -198,7 +198,14 @@ typedef enum {
     FFF_TUNE_FUSED_SMALL = 5,     /* small trees with thin leaves in one launch: descent, grid barrier, leaf evaluation
                                      by groups of 32 hidden neurons kept in shared memory (0: descent, bucketing and
                                      leaf kernels).  Taken by default by layers without a tensor-core leaf path */
-    FFF_TUNE_COUNT = 6
+    FFF_TUNE_GROUP_TILES = 6,     /* leaf kernel tiles of tokens that share the node three levels above the leaves: the
+                                     first descent stage stops there, the leaf kernel walks the last three levels from
+                                     7 extra accumulator columns and evaluates the node's 8 leaves side by side, each
+                                     row keeping its own leaf's hidden units (0: tiles of one leaf).  Taken for bf16
+                                     layers with 8 <= leaf_width < 16 and 9 <= depth <= 11 (where it replaces the
+                                     second descent stage and its node bucketing), when those nodes receive at least
+                                     128 tokens each on average */
+    FFF_TUNE_COUNT = 7
 } fff_tuning_t;
 fff_status_t fff_set_tuning(fff_handle_t h, fff_tuning_t key, int value);
 

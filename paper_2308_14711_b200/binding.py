@@ -22,7 +22,7 @@ STATUS_NAMES = {0: "FFF_OK", 1: "FFF_ERR_INVALID_ARG", 2: "FFF_ERR_UNSUPPORTED",
 ACTIVATIONS = {"relu": 0, "gelu": 1, "gelu_tanh": 2, "silu": 3}
 DTYPES = {"f32": 0, "bf16": 1}
 PATHS = {"auto": 0, "warp": 1, "tensor": 2, "fused": 3}
-TUNING = {"tcgen05_descent": 0, "tcgen05_grouped": 1, "tcgen05_leaf": 2, "cta_pairs": 3, "direct_lists": 4, "fused_small": 5}
+TUNING = {"tcgen05_descent": 0, "tcgen05_grouped": 1, "tcgen05_leaf": 2, "cta_pairs": 3, "direct_lists": 4, "fused_small": 5, "group_tiles": 6}
 
 # every symbol include/fff.h declares
 EXPORTS = ["fff_create", "fff_create_w8", "fff_forward_infer", "fff_forward_train", "fff_forward_infer_host", "fff_destroy", "fff_reserve",

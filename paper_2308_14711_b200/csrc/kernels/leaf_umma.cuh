@@ -67,36 +67,46 @@ constexpr int kLUMaxStages = 8;
 constexpr int kLUMaxW2Slots = 12;
 constexpr int kLUQueue = 4;                // tiles published ahead by the scheduler
 constexpr int kLUConsumerWarps = kLUWarps - 1;     // every warp but the scheduler reads the tile queue
-constexpr int kLUAcc2Col = 64;             // first tensor-memory column of the two GEMM2 accumulators
 constexpr int kLUTmemCols = 512;
 
 // kW8: the leaf weights are stored as 8-bit floats (e4m3 codes, one float32 scale per leaf and matrix).  The MMA wants
 // both operands as bf16, so the codes land in a staging part of their ring slot and the warp that issues the MMAs
 // expands them (every code is exactly a bf16 value) into the operand layout first; the scales multiply the
 // accumulators in the epilogue.
-template <int LP, bool kW8 = false> struct LeafUmmaLayout {
+// GL: leaves per tile.  1: a tile holds tokens of one leaf.  8: a tile holds tokens of one node three levels above the
+// leaves; GEMM1 then runs against the hidden units of that node's 8 leaves side by side plus the 7 nodes of its
+// subtree (N = 8 LP + 16 columns, the last 9 zero), the epilogue walks the three levels from the node logits, keeps
+// each row's own leaf's LP columns of H and zeroes the others, and GEMM2 contracts over all 8 LP columns against the
+// 8 leaves' output weights.  The tokens' rows then cross the memory system twice in all (first stage of the descent,
+// then here) instead of being gathered once more per level group, and tiles are as full as the node's share of the batch.
+template <int LP, bool kW8 = false, int GL = 1> struct LeafUmmaLayout {
     static_assert(LP == 16 || LP == 32 || LP == 64, "padded hidden width");
-    static constexpr int kRowBytes = LP * 2;                                 // row of H and of a W2 piece
+    static_assert(GL == 1 || (GL == 8 && LP == 16 && !kW8), "grouped tiles: 8 leaves of padded width 16, bf16 weights");
+    static constexpr int kN1 = GL == 1 ? LP : GL * LP + 16;                  // columns of GEMM1
+    static constexpr int kHCols = GL * LP;                                   // K of GEMM2
+    static constexpr int kRowBytes = GL == 1 ? LP * 2 : 128;                 // row of H and of a W2 piece (per K-block of 64 columns when grouped)
+    static constexpr int kHBlocks = kHCols * 2 / kRowBytes;                  // K-blocks of H and of a W2 piece
     // A ring stage holds kSub K-blocks of 64 columns (each a 128-byte swizzled operand tile of its own):
     // every stage costs each role a fixed few hundred cycles of barrier traffic, so two K-blocks share one
     // where shared memory allows.
-    static constexpr int kSub = LP <= 32 ? 2 : 1;
+    static constexpr int kSub = GL > 1 ? 1 : LP <= 32 ? 2 : 1;
     static constexpr int kXSubBytes = kLUM * kLUKB * 2;
-    static constexpr int kW1SubBytes = LP * kLUKB * 2;
+    static constexpr int kW1SubBytes = kN1 * kLUKB * 2;
     static constexpr int kXStageBytes = kSub * kXSubBytes;
     static constexpr int kW1StageBytes = kSub * kW1SubBytes;
     static constexpr int kW1CodeBytes = kW8 ? kW1StageBytes / 2 : 0;         // staging for the codes of the stage's W1 K-blocks
     static constexpr int kW1CopyBytes = kW8 ? kW1CodeBytes : kW1StageBytes;  // what the bulk copy of a stage brings
     static constexpr int kStageBytes = kXStageBytes + kW1StageBytes + kW1CodeBytes;      // a multiple of 1024
-    static constexpr int kW2Bytes = kLUPiece * kRowBytes;                    // weights of a piece (bf16 operand)
+    static constexpr int kW2Bytes = kLUPiece * kHCols * 2;                   // weights of a piece (bf16 operand)
     static constexpr int kW2CodeBytes = kW8 ? kW2Bytes / 2 : 0;
     static constexpr int kW2BiasOff = kW2Bytes + kW2CodeBytes;               // the piece's 128 float32 biases inside a slot
     static constexpr int kW2CopyOff = kW8 ? kW2Bytes : 0;                    // where the bulk copy of a piece lands in its slot
     static constexpr int kW2PieceBytes = (kW8 ? kW2CodeBytes : kW2Bytes) + kLUPiece * 4;    // a piece in the image: weights + biases
     static constexpr int kW2SlotStride = (kW2BiasOff + kLUPiece * 4 + 1023) & ~1023;
-    static constexpr int kHBytes = kLUM * kRowBytes;
+    static constexpr int kHBytes = kLUM * kHCols * 2;
     // W2 ring: a whole tile's pieces (O <= 1024) when they are small, so that no copy waits for an MMA just issued
-    static constexpr int kW2Slots = LP <= 16 ? 8 : LP <= 32 ? (kW8 ? 6 : 8) : 4;
+    static constexpr int kW2Slots = GL > 1 ? 2 : LP <= 16 ? 8 : LP <= 32 ? (kW8 ? 6 : 8) : 4;
+    static constexpr int kAcc2Col = GL > 1 ? 256 : 64;                       // first tensor-memory column of the two GEMM2 accumulators
     static constexpr int kBarrierBytes = 640;
     static constexpr int smem_bytes(int stages) {
         return 1024 + stages * kStageBytes + kW2Slots * kW2SlotStride + kHBytes + kBarrierBytes;
@@ -136,6 +146,68 @@ __global__ void k_pack_w2_umma(const T* __restrict__ w2, const T* __restrict__ b
             const float v = o < O ? Elem<T>::to_float(b2[j * O + o]) : 0.0f;
             reinterpret_cast<float*>(piece + (int64_t)kLUPiece * LP * 2)[n] = v;
         }
+    }
+}
+
+// Images for grouped tiles (kLUGroup = 8 leaves per tile): bin g is node g of level depth - 3, N1 = 8 LP + 16.
+//   w1g  [bin][D / 64][N1 rows][64 columns] 128-byte swizzled: row j LP + u = hidden unit u of leaf 8 g + j (zero for
+//        u >= l); rows 8 LP + q, q < 7: node q of the subtree below node g, breadth-first; the other rows zero;
+//   g1b  [bin][N1] float32: the biases of those rows;
+//   w2g  [bin][ceil(O / 128) pieces]{ 2 K-blocks of [128 rows (output features)][64 columns] 128-byte swizzled, then 128
+//        float32 (unused, zero) }: column j LP + u of feature o is w2[8 g + j][o][u], and for u == l (the spare hidden
+//        column, which H sets to 1) the output bias b2[8 g + j][o].  The image is zeroed before this kernel runs.
+constexpr int kLUGroup = 8;
+template <typename T>
+__global__ void k_pack_leaf_groups(const T* __restrict__ w1, const T* __restrict__ b1, const T* __restrict__ w2, const T* __restrict__ b2,
+                                   const T* __restrict__ node_w, const T* __restrict__ node_b, __nv_bfloat16* __restrict__ w1g,
+                                   float* __restrict__ g1b, unsigned char* __restrict__ w2g, int n_bins, int depth, int l, int LP, int D,
+                                   int O)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x, t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int HC = kLUGroup * LP, N1 = HC + 16;
+    // node q of the subtree below (level depth - 3, position g), as an index into node_w / node_b
+    auto node_of = [&](int64_t g, int q) {
+        const int r = q == 0 ? 0 : q < 3 ? 1 : 2;
+        return (((int64_t)1 << (depth - 3 + r)) - 1) + (g << r) + (q - ((1 << r) - 1));
+    };
+    for (int64_t i = t0; i < (int64_t)n_bins * N1 * D; i += stride) {
+        const int k = (int)(i % D), n = (int)((i / D) % N1);
+        const int64_t g = i / ((int64_t)D * N1);
+        float v = 0.0f;
+        if (n < HC) {
+            const int j = n / LP, u = n % LP;
+            if (u < l) v = Elem<T>::to_float(w1[((g * kLUGroup + j) * l + u) * (int64_t)D + k]);
+        } else if (n - HC < 7) {
+            v = Elem<T>::to_float(node_w[node_of(g, n - HC) * D + k]);
+        }
+        const int64_t base = (g * (D / kLUKB) + k / kLUKB) * (int64_t)(N1 * kLUKB);       // elements
+        w1g[base + ptx::swz128((uint32_t)(n * 128 + (k % kLUKB) * 2)) / 2] = __float2bfloat16_rn(v);
+    }
+    for (int64_t i = t0; i < (int64_t)n_bins * N1; i += stride) {
+        const int n = (int)(i % N1);
+        const int64_t g = i / N1;
+        float v = 0.0f;
+        if (n < HC) {
+            const int j = n / LP, u = n % LP;
+            if (u < l && b1) v = Elem<T>::to_float(b1[(g * kLUGroup + j) * l + u]);
+        } else if (n - HC < 7 && node_b) {
+            v = Elem<T>::to_float(node_b[node_of(g, n - HC)]);
+        }
+        g1b[i] = v;
+    }
+    const int P = (O + kLUPiece - 1) / kLUPiece;
+    const int64_t piece_bytes = (int64_t)kLUPiece * HC * 2 + kLUPiece * 4;
+    for (int64_t i = t0; i < (int64_t)n_bins * P * kLUPiece * HC; i += stride) {
+        const int c = (int)(i % HC), n = (int)((i / HC) % kLUPiece);
+        const int64_t gp = i / ((int64_t)HC * kLUPiece), g = gp / P;
+        const int o = (int)(gp % P) * kLUPiece + n, j = c / LP, u = c % LP;
+        float v = 0.0f;
+        if (o < O) {
+            if (u < l) v = Elem<T>::to_float(w2[((g * kLUGroup + j) * O + o) * (int64_t)l + u]);
+            else if (u == l && b2) v = Elem<T>::to_float(b2[(g * kLUGroup + j) * O + o]);
+        }
+        unsigned char* blk = w2g + gp * piece_bytes + (int64_t)(c / kLUKB) * (kLUPiece * 128);
+        *reinterpret_cast<__nv_bfloat16*>(blk + ptx::swz128((uint32_t)(n * 128 + (c % kLUKB) * 2))) = __float2bfloat16_rn(v);
     }
 }
 
@@ -208,7 +280,11 @@ __device__ __forceinline__ void expand_e4m3_tile(const unsigned char* __restrict
 // whose range holds it.  The last CTA to finish clears the counts for the next call.
 // kW8: w1codes / w2img hold e4m3 codes ([leaf][D / 64][LP][64], and per piece [128][LP] codes + 128 float32 biases),
 // scale1 / scale2 [leaf] the float32 scales of W1 and W2 (kFold must be off: the biases are added in the epilogue).
-template <int LP, bool kFold, bool kW8 = false>
+// GL = 8 (grouped tiles, see LeafUmmaLayout): a bin is a node three levels above the leaves; w1img holds per bin and
+// K-block the 8 LP + 16 rows (hidden units of the 8 leaves, the 7 nodes of the subtree breadth-first, zeros), g1bias
+// [bin][8 LP + 16] the matching biases, w2img per bin and piece the 128 x 8 LP output weights in two K-blocks (kFold:
+// every leaf's spare column carries its output bias); leaf_out / leaf_out2 (optional) receive every token's leaf.
+template <int LP, bool kFold, bool kW8 = false, int GL = 1>
 __global__ void __launch_bounds__(kLUThreads, 1)
 k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restrict__ perm,
             const Tile* __restrict__ tiles, int n_tiles_total,
@@ -216,10 +292,12 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
             const unsigned char* __restrict__ w2img, __nv_bfloat16* __restrict__ y,
             int D, int O, int l, int act, int kStages, int wide_stores, int passes, int* __restrict__ sched,
             int32_t* __restrict__ slot_counts, int n_bins, int cap, int* __restrict__ status,
-            const unsigned char* __restrict__ w1codes, const float* __restrict__ scale1, const float* __restrict__ scale2)
+            const unsigned char* __restrict__ w1codes, const float* __restrict__ scale1, const float* __restrict__ scale2,
+            const float* __restrict__ g1bias, int32_t* __restrict__ leaf_out, int32_t* __restrict__ leaf_out2)
 {
     static_assert(!(kW8 && kFold), "8-bit weights take their biases in the epilogue");
-    using L = LeafUmmaLayout<LP, kW8>;
+    static_assert(GL == 1 || kFold, "grouped tiles take the output bias through the spare hidden column");
+    using L = LeafUmmaLayout<LP, kW8, GL>;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     unsigned char* w2ring = ring + kStages * L::kStageBytes;
@@ -420,7 +498,7 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                                           w1codes + ((int64_t)tl.bin * KB + kb) * L::kW1CodeBytes, L::kW1CodeBytes, full + stage);
                         else
                             ptx::bulk_g2s(ring + stage * L::kStageBytes + L::kXStageBytes,
-                                          w1img + ((int64_t)tl.bin * KB + kb) * (L::kSub * LP * kLUKB), L::kW1StageBytes, full + stage);
+                                          w1img + ((int64_t)tl.bin * KB + kb) * (L::kW1StageBytes / 2), L::kW1StageBytes, full + stage);
                     }
                 }
                 __syncwarp();
@@ -435,7 +513,7 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
         }
     } else if (warp == kLUGemm1Warp) {
         // ------------------------------------------------------------------ GEMM1 issuer
-        constexpr uint32_t idesc = ptx::umma_idesc_bf16(kLUM, LP);
+        constexpr uint32_t idesc = ptx::umma_idesc_bf16(kLUM, L::kN1);
         int stage = 0;
         uint32_t phase = 0;
         for (int it = 0; it < max_iters; ++it) {
@@ -510,11 +588,17 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                 if (lane == 0) {
                     const int n = min(kLUPiece, O - p * kLUPiece);
                     const uint32_t idesc = ptx::umma_idesc_bf16(kLUM, n);
-                    const uint64_t ad = ptx::umma_desc_rows(hs, L::kRowBytes);
-                    const uint64_t bd = ptx::umma_desc_rows(ptx::smem_addr(w2ring + mm_slot * L::kW2SlotStride), L::kRowBytes);
+                    const uint32_t ws = ptx::smem_addr(w2ring + mm_slot * L::kW2SlotStride);
 #pragma unroll
-                    for (int kk = 0; kk < LP / 16; ++kk)
-                        ptx::umma_bf16(tmem_base + kLUAcc2Col + b * kLUAccStride, ad + 2 * kk, bd + 2 * kk, idesc, kk != 0 ? 1u : 0u);
+                    for (int blk = 0; blk < L::kHBlocks; ++blk) {
+                        // (one K-block of LP columns, or with grouped tiles K-blocks of 64 columns: [128 rows][128 bytes] each)
+                        const uint64_t ad = ptx::umma_desc_rows(hs + blk * (kLUM * L::kRowBytes), L::kRowBytes);
+                        const uint64_t bd = ptx::umma_desc_rows(ws + blk * (kLUPiece * L::kRowBytes), L::kRowBytes);
+#pragma unroll
+                        for (int kk = 0; kk < L::kRowBytes / 32; ++kk)
+                            ptx::umma_bf16(tmem_base + L::kAcc2Col + b * kLUAccStride, ad + 2 * kk, bd + 2 * kk, idesc,
+                                           (blk | kk) != 0 ? 1u : 0u);
+                    }
                     ptx::umma_commit(w2_empty + mm_slot);
                     ptx::umma_commit(y_full + b);
                 }
@@ -540,7 +624,7 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
         for (int it = 0; it < max_iters; ++it) {
             const Tile tl = next_tile();
             if (tl.rows <= 0) break;
-            const int rep = tl.rows <= 32 ? 4 : tl.rows <= 64 ? 2 : 1;
+            const int rep = GL > 1 ? 1 : tl.rows <= 32 ? 4 : tl.rows <= 64 ? 2 : 1;      // (grouped tiles are not stacked)
             const int qper = 4 / rep;                            // lane quarters per copy
             const int copy = quarter / qper;                     // the copy this thread's lanes hold = its column group
             const int row = (quarter % qper) * 32 + lane;        // the token row this thread's lane carries
@@ -557,45 +641,129 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                 if constexpr (kW8) return fmaf(__uint_as_float(acc), scale, bias);
                 else return __uint_as_float(acc) + bias;
             };
-            float b1r[HC];
+            if constexpr (GL == 1) {
+                float b1r[HC];
 #pragma unroll
-            for (int j = 0; j < HC; j += 4) {
-                const float4 t = __ldg(reinterpret_cast<const float4*>(b1img + (int64_t)tl.bin * LP + (part % kLUHParts) * HC + j));
-                b1r[j] = t.x; b1r[j + 1] = t.y; b1r[j + 2] = t.z; b1r[j + 3] = t.w;
-            }
+                for (int j = 0; j < HC; j += 4) {
+                    const float4 t = __ldg(reinterpret_cast<const float4*>(b1img + (int64_t)tl.bin * LP + (part % kLUHParts) * HC + j));
+                    b1r[j] = t.x; b1r[j + 1] = t.y; b1r[j + 2] = t.z; b1r[j + 3] = t.w;
+                }
 
-            // H = act(acc1 + b1) -> bf16 -> this thread's part of its row of the A operand of GEMM2 (every copy of it)
-            if (!timed_out && !ptx::mbar_wait(acc1_full, it & 1)) timed_out = true;
-            ptx::tc_fence_after_sync();
-            {
-                uint32_t hp[HC / 2];
-                if (h_active) {
-                    uint32_t v[32];
-                    ptx::tmem_ld32(lane_base + part * HC, v);      // columns past HC are not used
-                    ptx::tmem_ld_wait();
-                    with_activation(act, [&](auto a) {
-                        constexpr int kAct = decltype(a)::value;
+                // H = act(acc1 + b1) -> bf16 -> this thread's part of its row of the A operand of GEMM2 (every copy of it)
+                if (!timed_out && !ptx::mbar_wait(acc1_full, it & 1)) timed_out = true;
+                ptx::tc_fence_after_sync();
+                {
+                    uint32_t hp[HC / 2];
+                    if (h_active) {
+                        uint32_t v[32];
+                        ptx::tmem_ld32(lane_base + part * HC, v);      // columns past HC are not used
+                        ptx::tmem_ld_wait();
+                        with_activation(act, [&](auto a) {
+                            constexpr int kAct = decltype(a)::value;
 #pragma unroll
-                        for (int j = 0; j < HC; j += 2) {
-                            float h0 = activate_bf16(kAct, scaled(v[j], s1, b1r[j]));
-                            float h1 = activate_bf16(kAct, scaled(v[j + 1], s1, b1r[j + 1]));
-                            if (kFold && part * HC + j == l) h0 = 1.0f;          // the bias column
-                            if (kFold && part * HC + j + 1 == l) h1 = 1.0f;
-                            hp[j / 2] = ptx::pack_bf16(h0, h1);
+                            for (int j = 0; j < HC; j += 2) {
+                                float h0 = activate_bf16(kAct, scaled(v[j], s1, b1r[j]));
+                                float h1 = activate_bf16(kAct, scaled(v[j + 1], s1, b1r[j + 1]));
+                                if (kFold && part * HC + j == l) h0 = 1.0f;          // the bias column
+                                if (kFold && part * HC + j + 1 == l) h1 = 1.0f;
+                                hp[j / 2] = ptx::pack_bf16(h0, h1);
+                            }
+                        });
+                    }
+                    ptx::tc_fence_before_sync();
+                    ptx::mbar_arrive(acc1_empty);
+                    if (h_active) {
+                        for (int cp = 0; cp < rep; ++cp) {
+                            const int hrow = row + cp * (kLUM / rep);
+#pragma unroll
+                            for (int c = 0; c < HC / 8; ++c)
+                                *reinterpret_cast<uint4*>(hbuf + swz_rows((uint32_t)(hrow * L::kRowBytes + (part * HC / 8 + c) * 16), L::kRowBytes)) =
+                                    make_uint4(hp[4 * c], hp[4 * c + 1], hp[4 * c + 2], hp[4 * c + 3]);
                         }
-                    });
+                        ptx::fence_proxy_async();
+                    }
+                    ptx::mbar_arrive(h_full);
+                }
+            } else {
+                // Grouped tile: the row's leaf first (three levels from the subtree's 7 node logits, accumulator columns
+                // 8 LP ..), then H = act(acc1 + b1) for that leaf's LP columns; the row's other 7 LP columns of the
+                // A operand of GEMM2 are zero.  Both column parts walk (the walk is cheap); part p writes K-block p of the
+                // row (the columns of leaves 4p .. 4p + 3).
+                const float* gb = g1bias + (int64_t)tl.bin * L::kN1;
+                float nb[8];
+                {
+                    const float4 q0 = __ldg(reinterpret_cast<const float4*>(gb + GL * LP));
+                    const float4 q1 = __ldg(reinterpret_cast<const float4*>(gb + GL * LP + 4));
+                    nb[0] = q0.x; nb[1] = q0.y; nb[2] = q0.z; nb[3] = q0.w; nb[4] = q1.x; nb[5] = q1.y; nb[6] = q1.z; nb[7] = q1.w;
+                }
+                if (!timed_out && !ptx::mbar_wait(acc1_full, it & 1)) timed_out = true;
+                ptx::tc_fence_after_sync();
+                int j = 0;                                   // the row's leaf among the 8
+                float pre[LP];
+                if (active) {
+                    uint32_t nv[16];
+                    ptx::tmem_ld16(lane_base + GL * LP, nv);
+                    ptx::tmem_ld_wait();
+                    // a logit of zero goes right, NaN left (as in the descent kernels)
+                    const int n0 = __uint_as_float(nv[0]) + nb[0] >= 0.0f ? 1 : 0;
+                    const float l1 = n0 ? __uint_as_float(nv[2]) + nb[2] : __uint_as_float(nv[1]) + nb[1];
+                    const int q = 2 * n0 + (l1 >= 0.0f ? 1 : 0);
+                    const float l2 = q == 0 ? __uint_as_float(nv[3]) + nb[3] : q == 1 ? __uint_as_float(nv[4]) + nb[4]
+                                   : q == 2 ? __uint_as_float(nv[5]) + nb[5] : __uint_as_float(nv[6]) + nb[6];
+                    j = 2 * q + (l2 >= 0.0f ? 1 : 0);
+#pragma unroll
+                    for (int cc = 0; cc < 2; ++cc) {
+                        uint32_t v[32];
+                        ptx::tmem_ld32(lane_base + part * 64 + cc * 32, v);
+                        ptx::tmem_ld_wait();
+                        if (((j & 3) >> 1) == cc) {
+#pragma unroll
+                            for (int i = 0; i < LP; ++i) pre[i] = __uint_as_float((j & 1) ? v[LP + i] : v[i]);
+                        }
+                    }
                 }
                 ptx::tc_fence_before_sync();
                 ptx::mbar_arrive(acc1_empty);
-                if (h_active) {
-                    for (int cp = 0; cp < rep; ++cp) {
-                        const int hrow = row + cp * (kLUM / rep);
+                if (active) {
+                    const bool own = (j >> 2) == part;
+                    uint32_t hp[LP / 2];
 #pragma unroll
-                        for (int c = 0; c < HC / 8; ++c)
-                            *reinterpret_cast<uint4*>(hbuf + swz_rows((uint32_t)(hrow * L::kRowBytes + (part * HC / 8 + c) * 16), L::kRowBytes)) =
-                                make_uint4(hp[4 * c], hp[4 * c + 1], hp[4 * c + 2], hp[4 * c + 3]);
+                    for (int i = 0; i < LP / 2; ++i) hp[i] = 0u;
+                    if (own) {
+                        float b1r[LP];
+#pragma unroll
+                        for (int i = 0; i < LP; i += 4) {
+                            const float4 t = __ldg(reinterpret_cast<const float4*>(gb + j * LP + i));
+                            b1r[i] = t.x; b1r[i + 1] = t.y; b1r[i + 2] = t.z; b1r[i + 3] = t.w;
+                        }
+                        with_activation(act, [&](auto a) {
+                            constexpr int kAct = decltype(a)::value;
+#pragma unroll
+                            for (int i = 0; i < LP; i += 2) {
+                                float h0 = activate_bf16(kAct, pre[i] + b1r[i]);
+                                float h1 = activate_bf16(kAct, pre[i + 1] + b1r[i + 1]);
+                                if (i == l) h0 = 1.0f;                           // the bias column
+                                if (i + 1 == l) h1 = 1.0f;
+                                hp[i / 2] = ptx::pack_bf16(h0, h1);
+                            }
+                        });
+                    }
+                    // the row's 128 bytes of K-block `part`: the leaf's two 16-byte units, zeros elsewhere
+                    const int du = own ? (j & 3) * (LP / 8) : -8;
+                    unsigned char* hb = hbuf + part * (kLUM * L::kRowBytes);
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        uint4 val = make_uint4(0u, 0u, 0u, 0u);
+                        if (u == du) val = make_uint4(hp[0], hp[1], hp[2], hp[3]);
+                        if (u == du + 1) val = make_uint4(hp[4], hp[5], hp[6], hp[7]);
+                        *reinterpret_cast<uint4*>(hb + swz_rows((uint32_t)(row * L::kRowBytes + u * 16), L::kRowBytes)) = val;
                     }
                     ptx::fence_proxy_async();
+                    if (part == 0 && tok >= 0) {
+                        const int32_t leaf = tl.bin * GL + j;
+                        if (leaf_out) leaf_out[tok] = leaf;
+                        if (leaf_out2) leaf_out2[tok] = leaf;
+                    }
                 }
                 ptx::mbar_arrive(h_full);
             }
@@ -615,7 +783,7 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                     const int c0 = cbase;
                     if (active && c0 < ncols) {                      // ncols is a multiple of 16
                         uint32_t v[16];
-                        ptx::tmem_ld16(lane_base + kLUAcc2Col + b * kLUAccStride + c0, v);
+                        ptx::tmem_ld16(lane_base + L::kAcc2Col + b * kLUAccStride + c0, v);
                         ptx::tmem_ld_wait();
                         uint32_t out[8];
                         if (kFold) {
@@ -646,7 +814,7 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                         const int nv = min(32, ncols - c0);              // <= 0, 16 or 32
                         if (active && nv > 0) {
                             uint32_t v[32];
-                            ptx::tmem_ld32(lane_base + kLUAcc2Col + b * kLUAccStride + c0, v);
+                            ptx::tmem_ld32(lane_base + L::kAcc2Col + b * kLUAccStride + c0, v);
                             ptx::tmem_ld_wait();
                             const int o0 = p * kLUPiece + c0;
                             uint32_t out[16];
