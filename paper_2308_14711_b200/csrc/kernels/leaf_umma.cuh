@@ -105,7 +105,7 @@ template <int LP, bool kW8 = false, int GL = 1> struct LeafUmmaLayout {
     static constexpr int kW2SlotStride = (kW2BiasOff + kLUPiece * 4 + 1023) & ~1023;
     static constexpr int kHBytes = kLUM * kHCols * 2;
     // W2 ring: a whole tile's pieces (O <= 1024) when they are small, so that no copy waits for an MMA just issued
-    static constexpr int kW2Slots = GL > 1 ? 2 : LP <= 16 ? 8 : LP <= 32 ? (kW8 ? 6 : 8) : 4;
+    static constexpr int kW2Slots = GL > 1 ? 3 : LP <= 16 ? 8 : LP <= 32 ? (kW8 ? 6 : 8) : 4;
     static constexpr int kAcc2Col = GL > 1 ? 256 : 64;                       // first tensor-memory column of the two GEMM2 accumulators
     static constexpr int kBarrierBytes = 640;
     static constexpr int smem_bytes(int stages) {
@@ -559,8 +559,13 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
             if (tl.rows <= 0) break;
             const unsigned char* w2j = w2img + (int64_t)tl.bin * P * L::kW2PieceBytes;
             int loaded = 0;
-            auto load_piece = [&]() {
-                if (!timed_out && !ptx::mbar_wait(w2_empty + ld_slot, ld_phase ^ 1)) timed_out = true;
+            // the next piece of this tile into the next ring slot; `block`: wait for the slot, else only if it is free
+            auto load_piece = [&](bool block) {
+                if (block) {
+                    if (!timed_out && !ptx::mbar_wait(w2_empty + ld_slot, ld_phase ^ 1)) timed_out = true;
+                } else if (!__any_sync(kFullMask, ptx::mbar_test(w2_empty + ld_slot, ld_phase ^ 1))) {
+                    return false;
+                }
                 if (lane == 0) {
                     ptx::mbar_arrive_expect_tx(w2_full + ld_slot, (uint32_t)L::kW2PieceBytes);
                     ptx::bulk_g2s(w2ring + ld_slot * L::kW2SlotStride + L::kW2CopyOff, w2j + (int64_t)loaded * L::kW2PieceBytes,
@@ -569,12 +574,20 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                 __syncwarp();
                 ++loaded;
                 if (++ld_slot == L::kW2Slots) { ld_slot = 0; ld_phase ^= 1; }
+                return true;
             };
-            while (loaded < P && loaded < L::kW2Slots) load_piece();
+            // Copies run as far ahead as free slots allow, but only the piece that the next MMA needs is waited for: with
+            // fewer slots than pieces (grouped tiles) a wait for the slot of piece p + slots right after the MMA of piece p
+            // would hold back the MMA of piece p + 1, whose operands are already there.
+            auto load_ahead = [&](int needed) {
+                while (loaded < P && load_piece(loaded <= needed)) {}
+            };
+            load_ahead(-1);
             if (!timed_out && !ptx::mbar_wait(h_full, it & 1)) timed_out = true;
             ptx::tc_fence_after_sync();
             for (int p = 0; p < P; ++p, ++pc) {
                 const int b = pc & 1;
+                load_ahead(p);
                 if (!timed_out && !ptx::mbar_wait(w2_full + mm_slot, mm_phase)) timed_out = true;
                 if constexpr (kW8) {
                     // the piece's codes -> bf16 operand tile (128 output features x LP columns)
@@ -604,7 +617,6 @@ k_leaf_umma(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restric
                 }
                 __syncwarp();
                 if (++mm_slot == L::kW2Slots) { mm_slot = 0; mm_phase ^= 1; }
-                if (loaded < P) load_piece();                    // only when a tile has more pieces than ring slots
             }
         }
     } else {

@@ -40,6 +40,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
+// Has the phase with the given parity completed?  Returns at once (mbarrier.try_wait may suspend the thread for a
+// while before it answers "no"), so this is the form for "do this now if it is ready, else later".
+__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_addr(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
 constexpr long long kWaitCycles = 1ll << 28;   // about 0.14 s at 1.9 GHz
 
 // Waits for the phase with the given parity.  Returns false if it did not complete within
