@@ -313,7 +313,8 @@ typedef enum {
     FFF_CAP_TENSOR_LEAF = 4,      /* grouped leaf evaluation on tensor cores (also O % 8 == 0, l <= 64) */
     FFF_CAP_TCGEN05_LEAF = 8,     /* ... on tcgen05 (also O % 16 == 0) */
     FFF_CAP_FUSED_SMALL = 16,     /* the one-launch kernel (l <= 32, at most one group of 32 neurons per SM) */
-    FFF_CAP_FORWARD_TRAIN = 32    /* fff_forward_train (bf16, D % 64 == 0) */
+    FFF_CAP_FORWARD_TRAIN = 32,   /* fff_forward_train (bf16, D % 64 == 0) */
+    FFF_CAP_GROUP_TILES = 64      /* leaf tiles of 8 sibling leaves (FFF_TUNE_GROUP_TILES: 8 <= leaf_width < 16, 9 <= depth <= 11) */
 } fff_capability_t;
 int fff_capabilities(fff_handle_t h);
 

@@ -1756,6 +1756,7 @@ int fff_capabilities(fff_handle_t h) {
     if (h->w2uimg || h->w2codes) caps |= FFF_CAP_TCGEN05_LEAF;
     if (h->fs_batch != 0) caps |= FFF_CAP_FUSED_SMALL;
     if (h->tr_Kp != 0) caps |= FFF_CAP_FORWARD_TRAIN;
+    if (h->g_w1) caps |= FFF_CAP_GROUP_TILES;
     return caps;
 }
 

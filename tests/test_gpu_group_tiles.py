@@ -31,6 +31,7 @@ def test_grouped_tiles_match_the_oracle(cfg):
     y_ref, leaf_ref = orc.forward_i(case.net, case.x, threads=util.ORACLE_THREADS)
     off_ref, perm_ref = orc.bucket(leaf_ref, cfg.n_leaves)
     layer = util.make_layer(case)
+    assert layer.capabilities() & 64                   # FFF_CAP_GROUP_TILES
     x = util.to_device(case.x, "bf16")
     y_first = None
     for _ in range(2):

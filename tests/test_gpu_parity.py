@@ -567,6 +567,8 @@ def test_capabilities_say_which_kernel_families_a_layer_can_use():
         return c
     full = caps(256, 128, 4, 16, "bf16")
     assert full & 1 and full & 2 and full & 4 and full & 8 and full & 16 and full & 32
+    assert not full & 64                               # grouped leaf tiles: thin leaves under deep trees only
+    assert caps(256, 128, 9, 12, "bf16") & 64
     odd_d = caps(192, 128, 4, 16, "bf16")              # D no multiple of 128: CUDA cores only, FORWARD_T still runs
     assert not odd_d & (1 | 2 | 4 | 8) and odd_d & 16 and odd_d & 32
     odd_o = caps(256, 100, 4, 16, "bf16")              # O no multiple of 8: descent on tensor cores, leaves not
