@@ -22,6 +22,7 @@ CASES = [
     C("g_d10", 256, 80, 10, 8, "relu", "bf16", 17000, "normal"),           # O ends in a 16-column piece
     C("g_d10_skew", 128, 272, 10, 15, "silu", "bf16", 20000, "clusters"),  # skewed routing: empty and thin nodes, 3 pieces
     C("g_d11", 128, 64, 11, 8, "gelu", "bf16", 40000, "normal"),           # 256 nodes: first stage of 8 levels on CTA pairs
+    C("g_d11_wide", 1024, 1024, 11, 12, "gelu", "bf16", 65536, "normal"),  # full size: 512 full tiles, every row compared
 ]
 
 
