@@ -30,6 +30,19 @@ def test_header_symbols_are_exported(lib):
     assert sorted(binding.EXPORTS) == names
 
 
+def test_binding_tables_match_the_header_enums():
+    """The binding's name tables carry the header's values (tuning switches, paths, activations)."""
+    text = open(os.path.join(ROOT, "include", "fff.h")).read()
+    enums = {k: int(v) for k, v in re.findall(r"\b(FFF_[A-Z0-9_]+)\s*=\s*(\d+)", text)}
+    tune = {k[len("FFF_TUNE_"):].lower(): v for k, v in enums.items() if k.startswith("FFF_TUNE_") and k != "FFF_TUNE_COUNT"}
+    assert binding.TUNING == tune
+    assert enums["FFF_TUNE_COUNT"] == len(tune) == max(tune.values()) + 1
+    for name, value in binding.ACTIVATIONS.items():
+        assert enums["FFF_ACT_" + name.upper()] == value
+    for name, value in binding.PATHS.items():
+        assert enums["FFF_PATH_" + name.upper()] == value
+
+
 def test_status_strings(lib):
     seen = {binding.status_string(s) for s in range(8)}
     assert len(seen) == 8 and "ok" in seen
