@@ -1157,8 +1157,7 @@ fff_status_t run_forward_train(fff_handle_s* h, const void* x, void* y, float* m
         }
     }
     {
-        const int64_t total = B * (h->tr_Kp - hidden);
-        const int64_t blocks = std::max<int64_t>(1, std::min<int64_t>((total + 255) / 256, (int64_t)h->sm_count * 16));
+        const int64_t blocks = std::max<int64_t>(1, std::min<int64_t>((B + fff::kMixTokens - 1) / fff::kMixTokens, (int64_t)h->sm_count * 16));
         fff::k_mixture_weights<<<(unsigned)blocks, 256, 0, st>>>(h->tr_c, ldc, h->tr_mix, mixture, h->tr_hp, h->tr_Kp, (int)hidden,
                                                                  h->depth, B);
         if ((s = launched(h, st, "train_mixture_weights")) != FFF_OK) return s;

@@ -323,29 +323,84 @@ k_gemm_umma(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
 // c: [B, ldc] float32 (node r in column r);  mix: [B, 2^d] float32 (optional: mix_user, a second copy);
 // hp_tail: the same weights as bf16 in the last 2^d used columns of the rows of h' (row pitch ld_hp), where
 // the output GEMM multiplies them with the output biases; the padding columns up to ld_hp are zeroed.
+// The products along the root path of leaf j for kMixTokens tokens at once, for a tree of DEPTH levels (ct[u] = token
+// u's node choices, nullptr = no token): all loads are independent of each other and are issued before the products
+// start (with a run-time depth the loop stays rolled and every level waits for its own load: DEPTH round trips to L2
+// per value, one token at a time).
+constexpr int kMixTokens = 4;
+template <int DEPTH>
+__device__ __forceinline__ void path_products(const float* const (&ct)[kMixTokens], int j, float (&p)[kMixTokens]) {
+    float cv[kMixTokens][DEPTH];
+#pragma unroll
+    for (int u = 0; u < kMixTokens; ++u)
+#pragma unroll
+        for (int m = 0; m < DEPTH; ++m) cv[u][m] = ct[u] ? ct[u][(1 << m) - 1 + (j >> (DEPTH - m))] : 0.0f;
+#pragma unroll
+    for (int u = 0; u < kMixTokens; ++u) {
+        float q = 1.0f;
+#pragma unroll
+        for (int m = 0; m < DEPTH; ++m) q *= ((j >> (DEPTH - m - 1)) & 1) ? cv[u][m] : 1.0f - cv[u][m];
+        p[u] = q;
+    }
+}
+
+// Mixture weights of FORWARD_T from the node choices: unrolling the recursion of Algorithm 1, leaf j enters the
+// output with the product over its root path of c (where the path turns right) or 1 - c (left).
+// c: [B, ldc] float32 (node r in column r);  mix: [B, 2^d] float32 (optional: mix_user, a second copy);
+// hp_tail: the same weights as bf16 in the last 2^d used columns of the rows of h' (row pitch ld_hp), where
+// the output GEMM multiplies them with the output biases; the padding columns up to ld_hp are zeroed.
+// A block takes kMixTokens tokens at a time, a thread one column of each (no 64-bit divisions in the loop).
 __global__ void __launch_bounds__(256)
 k_mixture_weights(const float* __restrict__ c, int ldc, float* __restrict__ mix, float* __restrict__ mix_user,
                   __nv_bfloat16* __restrict__ hp, int ld_hp, int hidden, int depth, int64_t B)
 {
     const int nl = 1 << depth;
     const int tail = ld_hp - hidden;                          // >= nl: mixture columns, then zero padding
-    const int64_t total = B * tail;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t t = i / tail;
-        const int j = (int)(i % tail);
-        float p = 0.0f;
+    for (int64_t t0 = (int64_t)blockIdx.x * kMixTokens; t0 < B; t0 += (int64_t)gridDim.x * kMixTokens)
+    for (int j = threadIdx.x; j < tail; j += blockDim.x) {
+        float p[kMixTokens];
+#pragma unroll
+        for (int u = 0; u < kMixTokens; ++u) p[u] = 0.0f;
         if (j < nl) {
-            p = 1.0f;
-            const float* ct = c + t * ldc;
-            for (int m = 0; m < depth; ++m) {
-                const int n = j >> (depth - m);
-                const float cv = ct[(1 << m) - 1 + n];
-                p *= ((j >> (depth - m - 1)) & 1) ? cv : 1.0f - cv;
+            const float* ct[kMixTokens];
+#pragma unroll
+            for (int u = 0; u < kMixTokens; ++u) ct[u] = t0 + u < B ? c + (t0 + u) * ldc : nullptr;
+            switch (depth) {            // (the same multiplications in the same order in every case)
+                case 1: path_products<1>(ct, j, p); break;
+                case 2: path_products<2>(ct, j, p); break;
+                case 3: path_products<3>(ct, j, p); break;
+                case 4: path_products<4>(ct, j, p); break;
+                case 5: path_products<5>(ct, j, p); break;
+                case 6: path_products<6>(ct, j, p); break;
+                case 7: path_products<7>(ct, j, p); break;
+                case 8: path_products<8>(ct, j, p); break;
+                case 9: path_products<9>(ct, j, p); break;
+                case 10: path_products<10>(ct, j, p); break;
+                case 11: path_products<11>(ct, j, p); break;
+                case 12: path_products<12>(ct, j, p); break;
+                default:
+#pragma unroll
+                    for (int u = 0; u < kMixTokens; ++u) {
+                        if (!ct[u]) continue;
+                        float q = 1.0f;
+                        for (int m = 0; m < depth; ++m) {
+                            const float cv = ct[u][(1 << m) - 1 + (j >> (depth - m))];
+                            q *= ((j >> (depth - m - 1)) & 1) ? cv : 1.0f - cv;
+                        }
+                        p[u] = q;
+                    }
             }
-            mix[t * nl + j] = p;
-            if (mix_user) mix_user[t * nl + j] = p;
         }
-        hp[t * ld_hp + hidden + j] = __float2bfloat16_rn(p);
+#pragma unroll
+        for (int u = 0; u < kMixTokens; ++u) {
+            const int64_t t = t0 + u;
+            if (t >= B) break;
+            if (j < nl) {
+                mix[t * nl + j] = p[u];
+                if (mix_user) mix_user[t * nl + j] = p[u];
+            }
+            hp[t * ld_hp + hidden + j] = __float2bfloat16_rn(p[u]);
+        }
     }
 }
 
