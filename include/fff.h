@@ -179,7 +179,9 @@ fff_status_t fff_destroy(fff_handle_t h);
  * allocate nothing.  Allocates and synchronises.  The workspace is a few
  * int32 per token, plus, on the tensor-core path, a table of per-leaf token
  * lists of 2^depth * max_B int32 (only while that is at most 1 GiB; larger
- * layers run a bucketing kernel instead), of which a forward touches B entries. */
+ * layers run a bucketing kernel instead), of which a forward touches B entries;
+ * trees whose descent runs as two tensor-core stages add a table of per-node
+ * lists between the stages (at most 256 * max_B int32, same rule). */
 fff_status_t fff_reserve(fff_handle_t h, int64_t max_B);
 
 /* Pin the handle to one kernel family (FFF_PATH_*).  FFF_ERR_UNSUPPORTED if
@@ -194,7 +196,8 @@ typedef enum {
     FFF_TUNE_TCGEN05_GROUPED = 1, /* later descent stages on tcgen05 when their groups fill 128-row tiles (0: mma.sync) */
     FFF_TUNE_TCGEN05_LEAF = 2,    /* leaf evaluation on tcgen05 (0: mma.sync kernel) */
     FFF_TUNE_CTA_PAIRS = 3,       /* first descent stage with 128 or 256 nodes on pairs of CTAs (0: single CTAs) */
-    FFF_TUNE_DIRECT_LISTS = 4,    /* the last descent stage files tokens under their leaves (0: bucketing kernel) */
+    FFF_TUNE_DIRECT_LISTS = 4,    /* descent stages file the tokens under the nodes / leaves they reach, for the kernel
+                                     that follows (0: bucketing kernels) */
     FFF_TUNE_FUSED_SMALL = 5,     /* small trees with thin leaves in one launch: descent, grid barrier, leaf evaluation
                                      by groups of 32 hidden neurons kept in shared memory (0: descent, bucketing and
                                      leaf kernels).  Taken by default by layers without a tensor-core leaf path */

@@ -72,6 +72,13 @@ struct fff_handle_s {
     float* g_b1 = nullptr;
     unsigned char* g_w2 = nullptr;
     bool slots_no_pos2 = false;        // the stage that files the tokens does not end at the leaves: no second copy of its positions
+    // direct lists between the first and the second descent stage (two-stage trees): per node of the first stage's last
+    // level a list of the tokens that reached it, filled by the first stage and read by the grouped second stage
+    int32_t* ws_nslots = nullptr;      // [2^k0][nslot_cap]
+    int32_t* ws_ncursor = nullptr;     // [kUGMaxBins] counts (zero between forwards) + [1] finished-CTA counter
+    int64_t nslot_cap = 0;
+    bool ncursor_dirty = false;
+    bool nslots_here = false;          // the stage being launched files its tokens under the nodes it reaches
     fff::Tile* ws_tiles = nullptr;
 
     // workspace
@@ -263,7 +270,7 @@ void release(fff_handle_s* h) {
     dfree(h->fs_w1g); dfree(h->fs_b1g); dfree(h->fs_w2g); dfree(h->fs_b2f);
     dfree(h->w1codes); dfree(h->w2codes); dfree(h->scale1); dfree(h->scale2);
     dfree(h->tr_w2t); dfree(h->tr_c); dfree(h->tr_mix); dfree(h->tr_entpart); dfree(h->tr_hp);
-    dfree(h->w1img); dfree(h->b1img); dfree(h->w2img); dfree(h->w2uimg); dfree(h->ws_sched); dfree(h->ws_tiles); dfree(h->ws_rank); dfree(h->ws_rank8); dfree(h->ws_counts8); dfree(h->ws_blocksum); dfree(h->ws_matrix); dfree(h->ws_slots); dfree(h->ws_cursor);
+    dfree(h->w1img); dfree(h->b1img); dfree(h->w2img); dfree(h->w2uimg); dfree(h->ws_sched); dfree(h->ws_tiles); dfree(h->ws_rank); dfree(h->ws_rank8); dfree(h->ws_counts8); dfree(h->ws_blocksum); dfree(h->ws_matrix); dfree(h->ws_slots); dfree(h->ws_cursor); dfree(h->ws_nslots); dfree(h->ws_ncursor);
     if (h->copy_in) cudaStreamDestroy(h->copy_in);
     if (h->copy_out) cudaStreamDestroy(h->copy_out);
     for (int i = 0; i < fff_handle_s::kMaxHostChunks; ++i) {
@@ -330,8 +337,9 @@ fff_status_t grow_workspace(fff_handle_s* h, int64_t B) {
     if (B <= h->cap_B) return FFF_OK;
     if (cudaDeviceSynchronize() != cudaSuccess) return cudaGetLastError(), FFF_ERR_CUDA;
     dfree(h->ws_leaf); dfree(h->ws_perm); dfree(h->ws_perm2); dfree(h->ws_tiles); dfree(h->ws_rank); dfree(h->ws_pos[0]);
-    dfree(h->ws_rank8); dfree(h->ws_counts8); dfree(h->ws_blocksum); dfree(h->ws_slots); dfree(h->ws_cursor);
-    h->ws_slots = h->ws_cursor = nullptr;
+    dfree(h->ws_rank8); dfree(h->ws_counts8); dfree(h->ws_blocksum); dfree(h->ws_slots); dfree(h->ws_cursor); dfree(h->ws_nslots);
+    dfree(h->ws_ncursor);
+    h->ws_slots = h->ws_cursor = h->ws_nslots = h->ws_ncursor = nullptr;
     h->slot_cap = 0;
     h->ws_rank8 = h->ws_counts8 = nullptr;
     h->ws_blocksum = nullptr;
@@ -364,6 +372,15 @@ fff_status_t grow_workspace(fff_handle_s* h, int64_t B) {
         if ((s = clone((void**)&h->ws_cursor, nullptr, sizeof(int32_t) * (size_t)h->n_leaves)) != FFF_OK) return s;
         h->slot_cap = B;
         h->cursor_dirty = false;
+    }
+    // node lists for trees whose descent runs as two tcgen05 stages (a forward decides: the stages it runs depend on B):
+    // [nodes of the first stage][B]
+    if (h->ustages.size() >= 2 && h->ustages[0].umma && h->ustages[1].umma && (1 << h->ustages[0].k) <= fff::kUGMaxBins &&
+        ((size_t)B << h->ustages[0].k) * sizeof(int32_t) <= kMaxSlotBytes) {
+        if ((s = dmalloc((void**)&h->ws_nslots, sizeof(int32_t) * ((size_t)B << h->ustages[0].k))) != FFF_OK) return s;
+        if ((s = clone((void**)&h->ws_ncursor, nullptr, sizeof(int32_t) * (fff::kUGMaxBins + 1))) != FFF_OK) return s;
+        h->nslot_cap = B;
+        h->ncursor_dirty = false;
     }
     h->cap_B = B;
     return FFF_OK;
@@ -560,6 +577,12 @@ struct SlotArgs {
 };
 SlotArgs slot_args(const fff_handle_s* h, const int32_t* pos_out) {
     SlotArgs a;
+    if (h->nslots_here) {              // the lists between the first and the second stage
+        a.cursor = h->ws_ncursor;
+        a.slots = h->ws_nslots;
+        a.cap = (int)h->nslot_cap;
+        return a;
+    }
     if (!h->slots_here) return a;
     a.pos2 = pos_out == h->ws_leaf || h->slots_no_pos2 ? nullptr : h->ws_leaf;
     a.cursor = h->ws_cursor;
@@ -588,7 +611,7 @@ fff_status_t launch_descent_umma(fff_handle_s* h, const fff_handle_s::DenseStage
     if (!make_x_tensor_map(&tm, x, B, h->D, fff::kUM)) return FFF_ERR_CUDA;
     const int64_t n_tiles = (B + fff::kUM - 1) / fff::kUM;
     const int64_t grid = balanced_grid(h->sm_count, n_tiles);
-    const bool ranked = sg.k >= 4 && h->ws_rank8 && h->ws_counts8;      // also rank the tokens for the bucketing that follows
+    const bool ranked = !h->nslots_here && sg.k >= 4 && h->ws_rank8 && h->ws_counts8;      // also rank the tokens for the bucketing that follows
     int32_t* sums = nullptr;
     if (blocksum_for_descent(h, B, ranked, st, &sums) != FFF_OK) return FFF_ERR_CUDA;
     const SlotArgs sl = slot_args(h, pos_out);
@@ -615,7 +638,7 @@ fff_status_t launch_descent_umma_pair(fff_handle_s* h, const fff_handle_s::Dense
     if (!make_x_tensor_map(&tw, sg.wimg, (int64_t)(h->D / fff::kUKB) * NP, fff::kUKB, NP / 2, false)) return FFF_ERR_CUDA;
     const int64_t n_pairs = ((B + fff::kUM - 1) / fff::kUM + 1) / 2;
     const int64_t grid = 2 * balanced_grid(h->sm_count / 2, n_pairs);
-    const bool ranked = sg.k >= 4 && h->ws_rank8 && h->ws_counts8;
+    const bool ranked = !h->nslots_here && sg.k >= 4 && h->ws_rank8 && h->ws_counts8;
     int32_t* sums = nullptr;
     if (blocksum_for_descent(h, B, ranked, st, &sums) != FFF_OK) return FFF_ERR_CUDA;
     const SlotArgs sl = slot_args(h, pos_out);
@@ -647,6 +670,7 @@ fff_status_t run_descent_umma(fff_handle_s* h, const fff_handle_s::DenseStage& s
 template <int NP>
 fff_status_t launch_descent_umma_grouped(fff_handle_s* h, const fff_handle_s::DenseStage& sg, const void* x, const int32_t* perm,
                                          int32_t* pos_out, int64_t B, cudaStream_t st) {
+    const bool node_lists = perm == h->ws_nslots && h->ws_nslots != nullptr;      // tiles from the node counts, not from ws_tiles
     using L = fff::DescentUmmaGroupedLayout<NP>;
     const int stages = std::min((int)fff::kUmmaMaxStages, (kSmemBudget - L::smem_bytes(0)) / L::kStageBytes);
     if (stages < 2) return FFF_ERR_UNSUPPORTED;
@@ -659,7 +683,8 @@ fff_status_t launch_descent_umma_grouped(fff_handle_s* h, const fff_handle_s::De
     const SlotArgs sl = slot_args(h, pos_out);
     if (launch_chain(h, fff::k_descent_umma_grouped<NP>, (unsigned)grid, fff::kUGThreads, (size_t)L::smem_bytes(stages), st, 1, tm,
                      perm, (const fff::Tile*)h->ws_tiles, n_tiles, (const __nv_bfloat16*)sg.wimg, (const float*)sg.bimg, pos_out,
-                     sl.pos2, sl.cursor, sl.slots, sl.cap, h->D, sg.k, stages, h->d_status) != cudaSuccess)
+                     sl.pos2, sl.cursor, sl.slots, sl.cap, h->D, sg.k, stages, h->d_status, node_lists ? h->ws_ncursor : (int32_t*)nullptr,
+                     1 << sg.L0, (int)h->nslot_cap) != cudaSuccess)
         return cudaGetLastError(), FFF_ERR_CUDA;
     return launched(h, st, "tree_descent_umma_grouped");
 }
@@ -727,11 +752,23 @@ fff_status_t run_descent(fff_handle_s* h, const void* x, int32_t* leaf_out, Coar
     const int32_t* pos = nullptr;
     Coarse prev;
     const auto& plan = stage_plan(h);
+    // Two tcgen05 stages and nobody downstream who would refine the node bucketing: the first stage files the tokens
+    // under the nodes it reaches and the second derives its tiles from the counts; no bucketing launch in between.
+    const bool node_lists = n_dense == 2 && &plan == &h->ustages && plan[0].umma && plan[1].umma && h->ws_nslots &&
+                            B <= h->nslot_cap && h->tune[FFF_TUNE_DIRECT_LISTS] && h->tune[FFF_TUNE_TCGEN05_GROUPED] &&
+                            (B >> plan[1].L0) >= 64 && (coarse == nullptr || defer_tail != nullptr);
+    if (node_lists) {
+        if (h->ncursor_dirty &&
+            cudaMemsetAsync(h->ws_ncursor, 0, sizeof(int32_t) * (fff::kUGMaxBins + 1), st) != cudaSuccess)
+            return cudaGetLastError(), FFF_ERR_CUDA;
+        h->ncursor_dirty = true;
+        h->blocksum_wanted = false;
+    }
     for (int i = 0; i < n_dense; ++i) {
         const auto& sg = plan[i];
         // later stages: the tcgen05 kernel on 128-row tiles when the groups fill them reasonably, else mma.sync on 64-row tiles
         const bool grouped_umma = i > 0 && sg.umma && h->tune[FFF_TUNE_TCGEN05_GROUPED] && (B >> sg.L0) >= 64;
-        if (i > 0) {
+        if (i > 0 && !node_lists) {
             // bucket by the node reached so far; buffers alternate so that the previous level stays readable
             int32_t* perm_out = (i & 1) ? h->ws_perm2 : h->ws_perm;
             int32_t* off_out = h->ws_offsets2[i & 1];
@@ -746,11 +783,14 @@ fff_status_t run_descent(fff_handle_s* h, const void* x, int32_t* leaf_out, Coar
         const bool last = level + sg.k == h->depth;
         int32_t* out = last ? leaf_out : h->ws_pos[i & 1];
         h->slots_here = h->slots_now && last;
+        h->nslots_here = node_lists && i == 0;
         s = i == 0 && sg.umma ? run_descent_umma(h, sg, x, out, B, st)
-            : grouped_umma    ? run_descent_umma_grouped(h, sg, x, prev.perm, out, B, st)
+            : grouped_umma    ? run_descent_umma_grouped(h, sg, x, node_lists ? h->ws_nslots : prev.perm, out, B, st)
                               : run_descent_mma(h, sg, x, prev.perm, i > 0, out, B, st);
         h->slots_here = false;
+        h->nslots_here = false;
         if (s != FFF_OK) return s;
+        if (node_lists && i == 1) h->ncursor_dirty = false;       // its last CTA clears the counts
         level += sg.k;
         pos = out;
     }

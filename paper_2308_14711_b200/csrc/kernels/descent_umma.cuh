@@ -495,6 +495,7 @@ k_descent_umma_pair(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
 constexpr int kUGGatherWarps = 4;
 constexpr int kUGThreads = (kUmmaEpilogueWarps + 1 + kUGGatherWarps) * 32;
 constexpr int kUGSub = 2;                                  // K-blocks per ring stage
+constexpr int kUGMaxBins = 256;                            // nodes of the first stage's last level (direct lists)
 
 template <int NP> struct DescentUmmaGroupedLayout {
     static_assert(NP == 16 || NP == 32 || NP == 64, "accumulator width");
@@ -505,18 +506,24 @@ template <int NP> struct DescentUmmaGroupedLayout {
     static constexpr int kStageBytes = kXStageBytes + kWStageBytes;          // a multiple of 1024
     static constexpr int kBarrierBytes = 256;
     static constexpr int kTmemCols = 2 * NP < 64 ? 64 : 2 * NP;              // two accumulators; the epilogue always loads 32 columns
-    static constexpr int smem_bytes(int stages) { return 1024 + stages * kStageBytes + kBarrierBytes + 2 * NP * 4; }
+    static constexpr int kListBytes = (2 * kUGMaxBins + 1 + 16) * 4;          // direct lists: counts, tile prefix, warp sums
+    static constexpr int smem_bytes(int stages) { return 1024 + stages * kStageBytes + kBarrierBytes + 2 * NP * 4 + kListBytes; }
 };
 
 // wimg: [group][D / 64][NP rows][64 columns] swizzled, bimg: [group][NP] float32 (k_pack_nodes).
 // pos_out2 / cursor / slots / cap (optional): as in the first stage (slot_tokens).
+// node_counts (optional, n_bins <= kUGMaxBins): instead of a tile list and a permutation, the lists the first stage
+// filled directly (slot_tokens): perm[bin * node_cap + i], i < node_counts[bin], are the tokens that reached node
+// `bin`.  Every CTA then derives the tiles itself (tile t of the launch = the (t - tiles before its bin)-th run of
+// 128 entries of that bin's list), which saves the node bucketing launch in between.  node_counts[kUGMaxBins] counts
+// the CTAs that have finished; the last one clears the counts and that word for the next call.
 template <int NP>
 __global__ void __launch_bounds__(kUGThreads, 1)
 k_descent_umma_grouped(const __grid_constant__ CUtensorMap tmap_x, const int32_t* __restrict__ perm,
                        const Tile* __restrict__ tiles, int n_tiles_total, const __nv_bfloat16* __restrict__ wimg,
                        const float* __restrict__ bimg, int32_t* __restrict__ pos_out, int32_t* __restrict__ pos_out2,
                        int32_t* __restrict__ cursor, int32_t* __restrict__ slots, int cap, int D, int k, int kStages,
-                       int* __restrict__ status)
+                       int* __restrict__ status, int32_t* __restrict__ node_counts, int n_bins, int node_cap)
 {
     using L = DescentUmmaGroupedLayout<NP>;
     extern __shared__ unsigned char smem_raw[];
@@ -527,6 +534,9 @@ k_descent_umma_grouped(const __grid_constant__ CUtensorMap tmap_x, const int32_t
     uint64_t* acc_empty = acc_full + 2;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
     float* bias = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(full) + L::kBarrierBytes);     // [2][NP]
+    int* s_cnt = reinterpret_cast<int*>(bias + 2 * NP);    // [kUGMaxBins] tokens per node (direct lists)
+    int* s_tpre = s_cnt + kUGMaxBins;                      // [kUGMaxBins + 1] tiles before each node
+    int* s_wsum = s_tpre + kUGMaxBins + 1;                 // [16]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int KB = D / (kUKB * kUGSub);                    // ring stages per tile
@@ -554,6 +564,45 @@ k_descent_umma_grouped(const __grid_constant__ CUtensorMap tmap_x, const int32_t
     pdl_wait();
     const uint32_t tmem_base = *tmem_slot;
 
+    // direct lists: tiles per node and their running sum, by every CTA for itself (n_bins <= 256 <= threads)
+    if (node_counts) {
+        const int tid = threadIdx.x;
+        const int c = tid < n_bins ? node_counts[tid] : 0;
+        const int t = (c + kUM - 1) / kUM;
+        int incl = t;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(kFullMask, incl, o);
+            if (lane >= o) incl += v;
+        }
+        if (tid < kUGMaxBins) s_cnt[tid] = c;
+        if (lane == 31) s_wsum[warp] = incl;
+        __syncthreads();
+        int before = 0;
+        for (int w = 0; w < warp; ++w) before += s_wsum[w];
+        if (tid < n_bins) s_tpre[tid + 1] = before + incl;
+        if (tid == 0) s_tpre[0] = 0;
+        __syncthreads();
+        n_tiles_total = s_tpre[n_bins];
+    }
+    // tile `idx` of the launch
+    auto tile_at = [&](int idx) {
+        if (!node_counts) return tiles[idx];
+        int lo = 0, hi = n_bins;                              // s_tpre[lo] <= idx < s_tpre[hi]
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (s_tpre[mid] <= idx) lo = mid;
+            else hi = mid;
+        }
+        const int local = idx - s_tpre[lo];
+        Tile tl;
+        tl.bin = lo;
+        tl.start = lo * node_cap + local * kUM;
+        tl.rows = min(kUM, s_cnt[lo] - local * kUM);
+        tl.pad = 0;
+        return tl;
+    };
+
     bool timed_out = false;
     if (warp > 4) {
         // ------------------------------------------------------------------ row gathers (+ weight copies)
@@ -561,7 +610,7 @@ k_descent_umma_grouped(const __grid_constant__ CUtensorMap tmap_x, const int32_t
         int stage = 0;
         uint32_t phase = 0;
         for (int tile = blockIdx.x; tile < n_tiles_total; tile += gridDim.x) {
-            const Tile tl = tiles[tile];
+            const Tile tl = tile_at(tile);
             if (tl.rows <= 0) continue;
             const int total_groups = (tl.rows + 3) >> 2;
             const int groups = max((total_groups - gw + kUGGatherWarps - 1) / kUGGatherWarps, 0);
@@ -599,7 +648,7 @@ k_descent_umma_grouped(const __grid_constant__ CUtensorMap tmap_x, const int32_t
         uint32_t phase = 0;
         int it = 0;
         for (int tile = blockIdx.x; tile < n_tiles_total; tile += gridDim.x) {
-            if (tiles[tile].rows <= 0) continue;
+            if (tile_at(tile).rows <= 0) continue;
             const int a = it & 1;
             if (!timed_out && !ptx::mbar_wait(acc_empty + a, ((it >> 1) & 1) ^ 1)) timed_out = true;
             ptx::tc_fence_after_sync();
@@ -628,7 +677,7 @@ k_descent_umma_grouped(const __grid_constant__ CUtensorMap tmap_x, const int32_t
         // ------------------------------------------------------------------ epilogue: one token per thread
         int it = 0;
         for (int tile = blockIdx.x; tile < n_tiles_total; tile += gridDim.x) {
-            const Tile tl = tiles[tile];
+            const Tile tl = tile_at(tile);
             if (tl.rows <= 0) continue;
             const int a = it & 1;
             const int row = warp * 32 + lane;
@@ -680,6 +729,20 @@ k_descent_umma_grouped(const __grid_constant__ CUtensorMap tmap_x, const int32_t
     if (warp == 4) {
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, L::kTmemCols);
+    }
+    // the last CTA to finish rearms the direct lists' counts (every CTA has read them long ago: before its first tile)
+    if (node_counts && warp == 0) {
+        int is_last = 0;
+        if (lane == 0) {
+            __threadfence();
+            is_last = atomicAdd(node_counts + kUGMaxBins, 1) == (int)gridDim.x - 1 ? 1 : 0;
+        }
+        is_last = __shfl_sync(kFullMask, is_last, 0);
+        if (is_last) {
+            for (int b = lane; b < n_bins; b += 32) node_counts[b] = 0;
+            if (lane == 0) node_counts[kUGMaxBins] = 0;
+            __threadfence();
+        }
     }
 }
 

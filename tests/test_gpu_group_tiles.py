@@ -56,7 +56,7 @@ def test_grouped_tiles_match_the_oracle(cfg):
     layer.set_tuning("group_tiles", False)
     y3, leaf3 = layer.forward_infer(x)
     torch.cuda.synchronize()
-    assert layer.last_launch_count() >= 4          # two descent stages, node bucketing, leaf kernel
+    assert layer.last_launch_count() >= 3          # two descent stages and the leaf kernel
     np.testing.assert_array_equal(leaf3.cpu().numpy(), leaf_ref)
     util.check_outputs(y3, y_ref, "bf16")
     layer.close()
@@ -70,7 +70,7 @@ def test_too_few_tokens_per_node_keep_one_leaf_per_tile():
     layer = util.make_layer(case)
     y, leaf = layer.forward_infer(util.to_device(case.x, "bf16"))
     torch.cuda.synchronize()
-    assert layer.last_launch_count() >= 4
+    assert layer.last_launch_count() >= 3
     np.testing.assert_array_equal(leaf.cpu().numpy(), leaf_ref)
     util.check_outputs(y, y_ref, "bf16")
     layer.set_tuning("group_tiles", False)

@@ -360,9 +360,10 @@ def test_warp_kernels_changing_batch_sizes(routing, path, launches):
 
 
 def test_two_stage_descent_without_leaf_bucketing_kernel():
-    """Ten levels as two tensor-core stages in front of the tensor-core leaf kernel: a node bucketing between the
-    stages, then the second stage files the tokens under their leaves itself: four launches, no leaf bucketing
-    kernel.  The descent entry point alone is three launches and must leave nothing behind for the next forward."""
+    """Ten levels as two tensor-core stages in front of the tensor-core leaf kernel: the first stage files the tokens
+    under the nodes it reaches, the second derives its tiles from those lists and files the tokens under their leaves:
+    three launches, no bucketing kernel at all.  The descent entry point alone is two launches and must leave nothing
+    behind for the next forward.  With the direct lists switched off the two bucketing kernels are back."""
     cfg = wl.FFFConfig("bf16_d10_direct", 128, 64, 10, 16, "gelu", "bf16", 20000, "clusters")
     case = util.make_case(cfg, seed=8)
     y_ref, leaf_ref = orc.forward_i(case.net, case.x, threads=util.ORACLE_THREADS)
@@ -371,7 +372,7 @@ def test_two_stage_descent_without_leaf_bucketing_kernel():
     for B in (cfg.B, 17000, cfg.B):
         y, leaf = layer.forward_infer(x[:B])
         torch.cuda.synchronize()
-        assert layer.last_launch_count() == 4
+        assert layer.last_launch_count() == 3
         np.testing.assert_array_equal(leaf.cpu().numpy(), leaf_ref[:B])
         util.check_outputs(y, y_ref[:B], "bf16")
         off, perm = layer.last_bucketing(B)
@@ -379,7 +380,13 @@ def test_two_stage_descent_without_leaf_bucketing_kernel():
         np.testing.assert_array_equal(off.cpu().numpy(), off_b)
         np.testing.assert_array_equal(perm.cpu().numpy(), perm_b)
         np.testing.assert_array_equal(layer.tree_descent(x[:B]).cpu().numpy(), leaf_ref[:B])
-        assert layer.last_launch_count() == 3
+        assert layer.last_launch_count() == 2
+    layer.set_tuning("direct_lists", False)
+    y, leaf = layer.forward_infer(x)
+    torch.cuda.synchronize()
+    assert layer.last_launch_count() == 5          # stage, node bucketing, stage, leaf bucketing, leaf kernel
+    np.testing.assert_array_equal(leaf.cpu().numpy(), leaf_ref)
+    util.check_outputs(y, y_ref, "bf16")
     assert layer.last_status() == 0
     layer.close()
 
@@ -489,7 +496,8 @@ def test_every_tuning_switch_off_gives_the_same_results(switch):
         np.testing.assert_array_equal(off.cpu().numpy(), off_ref)
         np.testing.assert_array_equal(perm.cpu().numpy(), perm_ref)
         if switch == "direct_lists":
-            assert layer.last_launch_count() == launches_on + 1      # the leaf bucketing kernel is back
+            # the leaf bucketing kernel is back, and between two descent stages the node bucketing too
+            assert layer.last_launch_count() == launches_on + (2 if cfg.depth > 8 else 1)
         layer.set_tuning(switch, True)
         y_back, _ = layer.forward_infer(x)
         assert torch.equal(y_back, y_on)
