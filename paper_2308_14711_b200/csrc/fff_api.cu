@@ -755,7 +755,8 @@ fff_status_t run_descent(fff_handle_s* h, const void* x, int32_t* leaf_out, Coar
     // Two tcgen05 stages and nobody downstream who would refine the node bucketing: the first stage files the tokens
     // under the nodes it reaches and the second derives its tiles from the counts; no bucketing launch in between.
     const bool node_lists = n_dense == 2 && &plan == &h->ustages && plan[0].umma && plan[1].umma && h->ws_nslots &&
-                            B <= h->nslot_cap && h->tune[FFF_TUNE_DIRECT_LISTS] && h->tune[FFF_TUNE_TCGEN05_GROUPED] &&
+                            B <= h->nslot_cap && (h->nslot_cap << plan[0].k) <= INT32_MAX &&      // (a tile's start is an int)
+                            h->tune[FFF_TUNE_DIRECT_LISTS] && h->tune[FFF_TUNE_TCGEN05_GROUPED] &&
                             (B >> plan[1].L0) >= 64 && (coarse == nullptr || defer_tail != nullptr);
     if (node_lists) {
         if (h->ncursor_dirty &&

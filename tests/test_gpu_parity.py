@@ -391,6 +391,22 @@ def test_two_stage_descent_without_leaf_bucketing_kernel():
     layer.close()
 
 
+def test_two_stage_descent_on_a_large_ragged_batch():
+    """The node lists between the stages with many tiles per node, a ragged last tile in every list and skewed
+    routing (some nodes empty, some with thousands of tokens): leaf indices bit-exact, outputs within tolerance."""
+    for x_kind, B in (("normal", 200001), ("clusters", 150003)):
+        cfg = wl.FFFConfig("bf16_d10_large", 128, 64, 10, 16, "relu", "bf16", B, x_kind)
+        case = util.make_case(cfg, seed=12)
+        y_ref, leaf_ref = orc.forward_i(case.net, case.x, threads=util.ORACLE_THREADS)
+        layer = util.make_layer(case)
+        y, leaf = layer.forward_infer(util.to_device(case.x, "bf16"))
+        torch.cuda.synchronize()
+        assert layer.last_launch_count() == 3 and layer.last_status() == 0
+        np.testing.assert_array_equal(leaf.cpu().numpy(), leaf_ref)
+        util.check_outputs(y, y_ref, "bf16")
+        layer.close()
+
+
 def test_leaf_lists_too_large_fall_back_to_the_bucketing_kernel():
     """2048 leaves x 140 000 tokens x 4 bytes is more than the table of per-leaf lists may take (1 GiB): the forward
     then buckets by leaf with a kernel again (five launches) and reports that stable bucketing directly."""
